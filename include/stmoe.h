@@ -1,0 +1,191 @@
+/*
+ * stmoe.h — C ABI of the B200 (sm_100a) decode-time MoE layer step with the
+ * spatio-temporal expert predictor of ST-MoE.
+ *
+ * One layer step = gating network (RMSNorm, router GEMV, softmax, top-K;
+ * Section 2) -> verification + table update (Algorithm 3) and prediction of
+ * the next layer's experts (Algorithm 2, Eq. 1) -> miss loading and prefetch
+ * of predicted experts from a pinned host store into fixed HBM slots
+ * (Sections 4.1, 4.3.4) -> routed SwiGLU expert FFNs, probability-weighted
+ * sum (Section 2) and the residual update of the stack harness.
+ *
+ * Conventions
+ *   - Every function returns STMOE_OK (0) or a negative STMOE_ERR_* code; no
+ *     exception, abort or output crosses this boundary.
+ *   - "device" pointers are CUDA global memory of the device that was current
+ *     in stmoe_create; "host" pointers are ordinary or pinned host memory.
+ *   - load_* calls copy what they are given; the caller keeps its buffers.
+ *     The library owns its weight storage, pinned host store, slot cache,
+ *     copy stream, events and scratch.
+ *   - cuda_stream arguments are cudaStream_t handles passed as void*.
+ *   - There is no CPU fallback: without a CUDA device every call fails.
+ */
+#ifndef STMOE_H
+#define STMOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define STMOE_OK 0
+#define STMOE_ERR_BAD_ARG (-1)
+#define STMOE_ERR_OOM (-2)
+#define STMOE_ERR_CUDA (-3)
+#define STMOE_ERR_TIMEOUT (-4)
+#define STMOE_ERR_STATE (-5)
+#define STMOE_ERR_UNIMPLEMENTED (-6)
+
+/* weight_dtype */
+#define STMOE_F32 0
+#define STMOE_BF16 1
+#define STMOE_FP8_E4M3 2 /* e4m3 codes + one bf16 scale per output channel */
+
+/* predictor_mode: which sources feed Algorithm 2 (tables evolve identically) */
+#define STMOE_PRED_OFF 0
+#define STMOE_PRED_TEMPORAL 1 /* history table only            */
+#define STMOE_PRED_SPATIAL 2  /* cross-layer table only        */
+#define STMOE_PRED_ST 3       /* both, combined as in Eq. 1    */
+
+/* flags */
+#define STMOE_FLAG_RENORM_TOPK 1 /* divide the K gate weights by their sum (off: Section 2 uses
+                                    the plain softmax probabilities) */
+
+/* per-sequence result flags of a layer step */
+#define STMOE_TOKEN_NEAR_TIE 1u /* K-th and (K+1)-th router logit closer than 1e-4 */
+
+typedef struct stmoe stmoe_t;
+
+typedef struct {
+    int32_t n_layers;
+    int32_t n_experts;      /* routed experts per layer, <= 256 (8-bit ids in the CCT) */
+    int32_t top_k;          /* K of the gating network = candidates per CCT row, <= 32 */
+    int32_t n_shared;       /* always-on experts per layer (weight 1, not predicted)   */
+    int32_t hidden;         /* H, multiple of 16                                       */
+    int32_t inter;          /* I, multiple of 16                                       */
+    int32_t max_batch;      /* sequences decoded together, <= 64                       */
+    int32_t weight_dtype;   /* expert weights; the router is fp32 for STMOE_F32, else bf16 */
+    int64_t cache_slots;    /* 0: all experts resident in HBM; else number of HBM expert
+                               slots (>= max_batch*top_k), experts live in pinned host memory */
+    int32_t profile_tokens; /* P of Algorithm 1: decode steps spent counting co-activations */
+    int32_t predictor_mode;
+    int32_t flags;
+    int32_t prefetch_limit; /* max prefetch copies issued per layer step, 0 = no limit */
+    float rms_eps;
+    float residual_scale;   /* r in h' = h + r * MoE(RMSNorm(h))                       */
+} stmoe_config_t;
+
+typedef struct {
+    int64_t decode_steps;     /* completed decode steps (one per pass over all layers)   */
+    int64_t runtime_steps;    /* (layer, sequence) steps after profiling                  */
+    int64_t routed;           /* experts routed in those steps                            */
+    int64_t predicted;        /* experts predicted for those steps                        */
+    int64_t hits;             /* routed experts that were in the predicted set            */
+    int64_t near_ties;        /* sequences flagged STMOE_TOKEN_NEAR_TIE (all steps)       */
+    int64_t cache_hits;       /* routed experts found in an HBM slot                      */
+    int64_t cache_misses;     /* routed experts demand-loaded from the host store         */
+    int64_t prefetch_issued;
+    int64_t prefetch_useful;  /* prefetched experts used before eviction                  */
+    int64_t prefetch_wasted;  /* prefetched experts evicted unused                        */
+    int64_t prefetch_dropped; /* predictions not prefetched (no slot / over the limit)    */
+    int64_t prefetch_resident;/* predictions already in a slot                            */
+    int64_t h2d_bytes_demand;
+    int64_t h2d_bytes_prefetch;
+    double transfer_ms;       /* device time of all host->HBM expert copies               */
+    double exposed_ms;        /* time the compute stream waited for such copies           */
+} stmoe_stats_t;
+
+/* Create a stack for the current CUDA device.  Allocates weight storage (HBM
+ * for resident stacks, pinned host memory plus cache_slots HBM slots
+ * otherwise), predictor tables (Co, CCT per adjacent layer pair, HT per layer
+ * and sequence) and scratch.  *out is NULL on failure. */
+int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out);
+int stmoe_destroy(stmoe_t *s);
+const char *stmoe_strerror(int code);
+
+/* Router matrix of one layer, [E][H] row-major (w_j of Section 2 in row j), fp32 for
+ * STMOE_F32 stacks and bf16 otherwise.  w: host or device.  Synchronous. */
+int stmoe_load_router(stmoe_t *s, int layer, const void *w);
+
+/* Weights of experts first_expert .. first_expert+count-1 of one layer (is_shared: the
+ * always-on experts).  gate, up: [count][I][H]; down: [count][H][I]; row-major in
+ * weight_dtype.  scales (fp8 only, else NULL): [count][2I+H] bf16 = gate rows, up rows,
+ * down rows.  Pointers may be host or device.  Synchronous. */
+int stmoe_load_experts(stmoe_t *s, int layer, int first_expert, int count, const void *gate,
+                       const void *up, const void *down, const void *scales, int is_shared);
+
+/* One layer step for `batch` sequences.  Layers must be called in order 0..L-1 for each
+ * decode step (else STMOE_ERR_STATE).
+ *   h_in, h_out    device fp32 [batch][H]; may alias
+ *   routed_ids     device int32 [batch][K], ascending ids            (NULL: not returned)
+ *   routed_w       device fp32  [batch][K], gate weights              (NULL: not returned)
+ *   predicted_ids  device int32 [batch][max_pred], ascending ids of the prefetch set for
+ *                  layer+1 (after the last layer: layer 0 of the next decode step), padded
+ *                  with -1; max_pred = stmoe_max_predicted()          (NULL: not returned)
+ *   n_predicted    device int32 [batch]                              (NULL: not returned)
+ *   flags          device uint32 [batch], STMOE_TOKEN_*               (NULL: not returned)
+ * Resident stacks: the call only enqueues work on cuda_stream.  Stacks with cache_slots > 0:
+ * the call waits on the host (bounded, STMOE_ERR_TIMEOUT) for this layer's routing, issues
+ * demand and prefetch copies on the library's copy stream and fences them with events.
+ * Prediction never changes routing or output (Section 4.3.4). */
+int stmoe_decode_step(stmoe_t *s, int layer, int batch, const float *h_in, float *h_out,
+                      int32_t *routed_ids, float *routed_w, int32_t *predicted_ids,
+                      int32_t *n_predicted, uint32_t *flags, void *cuda_stream);
+
+/* All layers of one decode step: h_out = stack(h_in).  The per-layer outputs are as in
+ * stmoe_decode_step with a leading [n_layers] dimension; any of them may be NULL. */
+int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out,
+                       int32_t *routed_ids, float *routed_w, int32_t *predicted_ids,
+                       int32_t *n_predicted, uint32_t *flags, void *cuda_stream);
+
+int stmoe_max_predicted(const stmoe_t *s); /* min(E, K*K+K) */
+
+/* Counters and timings; synchronises the device. */
+int stmoe_stats(stmoe_t *s, stmoe_stats_t *out);
+
+/* Predictor tables as a canonical image: 8 int32 {magic 0x53544D50, version 1, L, E, K, B, P,
+ * built}, int64 decode steps, Co u32 [L-1][E][E], CCT ids u8 [L-1][E][K], CCT confidences u8
+ * [L-1][E][K], HT i16 [B][L][K] (-1 = empty).  buf == NULL: only *bytes is set.  Host buffer.
+ * Synchronises the device.  import restores such an image between decode steps. */
+int stmoe_export_state(stmoe_t *s, void *buf, size_t *bytes);
+int stmoe_import_state(stmoe_t *s, const void *buf, size_t bytes);
+
+/* tags[slot] = layer*E+expert held by each HBM slot, -1 if empty (host int32 [cache_slots]). */
+int stmoe_export_cache_tags(stmoe_t *s, int32_t *tags, int64_t n);
+
+/* ---- single kernels behind the step, exposed for testing and reuse -------------------- */
+
+/* Gating network of Section 2 for `batch` tokens: x = RMSNorm(h), z = W_r x, s = softmax(z),
+ * top-K by logit (ties: lower id), ids ascending, w = s[ids].  All pointers device.
+ * wr_dtype: STMOE_F32 or STMOE_BF16.  logits: fp32 [batch*E + batch]; receives the logits
+ * [batch][E] followed by the per-sequence factors 1/sqrt(mean(h^2)+eps). */
+int stmoe_router_topk(const float *h, const void *w_router, int wr_dtype, int batch, int n_experts,
+                      int hidden, int top_k, float rms_eps, int renorm, float *logits,
+                      int32_t *ids, float *w, uint32_t *flags, void *cuda_stream);
+
+/* Predictor only (Algorithms 1-3 on the stack's tables) driven by given routing:
+ * routed_ids device int32 [batch][K] ascending.  Same ordering rules and outputs as
+ * stmoe_decode_step; used to replay routing traces. */
+int stmoe_predictor_step(stmoe_t *s, int layer, int batch, const int32_t *routed_ids,
+                         int32_t *predicted_ids, int32_t *n_predicted, void *cuda_stream);
+
+/* Routed SwiGLU expert FFN, weighted sum and residual for given routing:
+ *   h_out[b] = h[b] + r * sum_k w[b][k] * W_d^e ( silu(W_g^e x_b) * (W_u^e x_b) ),
+ *   x_b = h[b] * inv_rms[b],  e = ids[b][k].
+ * experts: device array of n_experts expert images, each `stmoe_expert_image_bytes` long:
+ * gate [I][H], up [I][H], down [H][I], then (fp8) bf16 scales [2I+H].
+ * scratch: device, stmoe_moe_ffn_scratch_bytes(batch, top_k, hidden, inter) bytes,
+ * 256-byte aligned; contents need not be initialised. */
+size_t stmoe_expert_image_bytes(int hidden, int inter, int weight_dtype);
+size_t stmoe_moe_ffn_scratch_bytes(int batch, int top_k, int hidden, int inter);
+int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t *ids, const float *w,
+                  const void *experts, int weight_dtype, int batch, int n_experts, int top_k,
+                  int hidden, int inter, float residual_scale, float *h_out, void *scratch,
+                  size_t scratch_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STMOE_H */

@@ -1,0 +1,943 @@
+// Host runtime and C ABI of the decode-time MoE layer step: weight storage, predictor
+// tables, the HBM slot cache with its copy stream and event fences, kernel launches.
+#include "../../include/stmoe.h"
+
+#include <chrono>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <new>
+#include <set>
+#include <utility>
+#include <vector>
+
+#include "device_utils.cuh"
+#include "ffn.cuh"
+#include "predictor.cuh"
+#include "router.cuh"
+
+using namespace stmoe_dev;
+
+#define CU_TRY(expr)                                  \
+    do {                                              \
+        cudaError_t e_ = (expr);                      \
+        if (e_ != cudaSuccess) {                      \
+            (void)cudaGetLastError();                 \
+            return e_ == cudaErrorMemoryAllocation ? STMOE_ERR_OOM : STMOE_ERR_CUDA; \
+        }                                             \
+    } while (0)
+#define ST_TRY(expr)            \
+    do {                        \
+        int r_ = (expr);        \
+        if (r_ != STMOE_OK) return r_; \
+    } while (0)
+
+namespace {
+
+constexpr uint32_t kStateMagic = 0x53544D50;
+constexpr int kWaitTimeoutMs = 20000;
+
+inline int dtype_bytes(int dt) { return dt == STMOE_F32 ? 4 : dt == STMOE_BF16 ? 2 : 1; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t image_bytes(int H, int I, int dt)
+{
+    size_t n = 3 * (size_t)H * I * dtype_bytes(dt);
+    if (dt == STMOE_FP8_E4M3) n += 2 * (size_t)(2 * I + H);
+    return round_up(n, 256);
+}
+
+// ---- kernel dispatch -------------------------------------------------------------------
+// MTMAX = 1: every work-list entry holds one token.  MTMAX = 4: entries of 1..4 tokens; the
+// kernel is instantiated for 4 and clamps (extra token columns recompute the last token).
+struct FfnPlan {
+    int grid_gate_up = 0, grid_down = 0;
+};
+
+template <int DT, int MT> struct Shape;
+template <int DT> struct Shape<DT, 1> { static constexpr int RG = 4, UG = 2, RD = 8, UD = 2; };
+template <int DT> struct Shape<DT, 4> { static constexpr int RG = 2, UG = 2, RD = 4, UD = 2; };
+
+template <int DT, int MT> void launch_gate_up(const FfnArgs &a, int grid, cudaStream_t st)
+{
+    gate_up_kernel<DT, Shape<DT, MT>::RG, MT, Shape<DT, MT>::UG><<<grid, kFfnThreads, 0, st>>>(a);
+}
+template <int DT, int MT> void launch_down(const FfnArgs &a, int grid, cudaStream_t st)
+{
+    down_kernel<DT, Shape<DT, MT>::RD, MT, Shape<DT, MT>::UD><<<grid, kFfnThreads, 0, st>>>(a);
+}
+template <int DT, int MT> int occupancy_gate_up()
+{
+    int n = 0;
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        &n, gate_up_kernel<DT, Shape<DT, MT>::RG, MT, Shape<DT, MT>::UG>, kFfnThreads, 0);
+    return n;
+}
+template <int DT, int MT> int occupancy_down()
+{
+    int n = 0;
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        &n, down_kernel<DT, Shape<DT, MT>::RD, MT, Shape<DT, MT>::UD>, kFfnThreads, 0);
+    return n;
+}
+
+#define DISPATCH_DT_MT(dt, mt, FN, ...)                      \
+    do {                                                     \
+        if ((dt) == STMOE_F32) {                             \
+            if ((mt) == 1) FN<0, 1>(__VA_ARGS__); else FN<0, 4>(__VA_ARGS__); \
+        } else if ((dt) == STMOE_BF16) {                     \
+            if ((mt) == 1) FN<1, 1>(__VA_ARGS__); else FN<1, 4>(__VA_ARGS__); \
+        } else {                                             \
+            if ((mt) == 1) FN<2, 1>(__VA_ARGS__); else FN<2, 4>(__VA_ARGS__); \
+        }                                                    \
+    } while (0)
+
+int occ_gate_up(int dt, int mt)
+{
+    int n = 0;
+#define OCC_G(DT, MT) n = occupancy_gate_up<DT, MT>()
+    if (dt == STMOE_F32) { if (mt == 1) OCC_G(0, 1); else OCC_G(0, 4); }
+    else if (dt == STMOE_BF16) { if (mt == 1) OCC_G(1, 1); else OCC_G(1, 4); }
+    else { if (mt == 1) OCC_G(2, 1); else OCC_G(2, 4); }
+#undef OCC_G
+    return n;
+}
+int occ_down(int dt, int mt)
+{
+    int n = 0;
+#define OCC_D(DT, MT) n = occupancy_down<DT, MT>()
+    if (dt == STMOE_F32) { if (mt == 1) OCC_D(0, 1); else OCC_D(0, 4); }
+    else if (dt == STMOE_BF16) { if (mt == 1) OCC_D(1, 1); else OCC_D(1, 4); }
+    else { if (mt == 1) OCC_D(2, 1); else OCC_D(2, 4); }
+#undef OCC_D
+    return n;
+}
+
+int sm_count()
+{
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    return n > 0 ? n : 148;
+}
+
+FfnPlan make_plan(int dt, int mt)
+{
+    FfnPlan p;
+    const int sms = sm_count();
+    p.grid_gate_up = sms * std::max(1, std::min(occ_gate_up(dt, mt), 4));
+    p.grid_down = sms * std::max(1, std::min(occ_down(dt, mt), 4));
+    return p;
+}
+
+void launch_router_logits(int rdt, const float *h, const void *W, int B, int E, int H, float eps,
+                          float *inv_rms, float *logits, cudaStream_t st)
+{
+    const int grid = (E + kRouterWarps - 1) / kRouterWarps;
+    if (rdt == STMOE_F32)
+        router_logits_kernel<0><<<grid, kRouterWarps * kWarp, 0, st>>>(h, (const uint8_t *)W, B, E, H, eps,
+                                                                      inv_rms, logits);
+    else
+        router_logits_kernel<1><<<grid, kRouterWarps * kWarp, 0, st>>>(h, (const uint8_t *)W, B, E, H, eps,
+                                                                      inv_rms, logits);
+}
+
+// ---- device work-list storage ----------------------------------------------------------
+struct WorkListMem {
+    int *base = nullptr;
+    WorkList wl{};
+    int alloc(int pairs)
+    {
+        CU_TRY(cudaMalloc(&base, sizeof(int) * (size_t)(4 + 5 * pairs)));
+        bind(base, pairs);
+        return STMOE_OK;
+    }
+    void bind(int *p, int pairs)
+    {
+        wl.n_groups = p;
+        wl.g_expert = p + 4;
+        wl.g_start = p + 4 + pairs;
+        wl.g_count = p + 4 + 2 * pairs;
+        wl.pair_token = p + 4 + 3 * pairs;
+        wl.pair_slot = p + 4 + 4 * pairs;
+    }
+    void release()
+    {
+        if (base) cudaFree(base);
+        base = nullptr;
+    }
+};
+
+// ---- host-side slot cache (verification, miss loading, prefetch; Sections 4.1, 4.3.4) ---
+// LRU on a clock that ticks once per layer step, lowest slot on equal stamps, empty slots
+// (stamp -1) first.  Kept in an ordered set so a victim is found without scanning all slots.
+struct SlotCache {
+    int64_t S = 0, clock = 0;
+    int E = 0;
+    std::vector<int32_t> slot_of, tag;
+    std::vector<int64_t> stamp;
+    std::vector<uint8_t> pf_unused, guard;
+    std::set<std::pair<int64_t, int32_t>> order;  // (stamp, slot)
+    std::vector<int32_t> guarded;
+    int64_t hits = 0, misses = 0, pf_issued = 0, pf_useful = 0, pf_wasted = 0, pf_dropped = 0,
+            pf_resident = 0;
+
+    void init(int64_t slots, int L, int experts)
+    {
+        S = slots, E = experts;
+        slot_of.assign((size_t)L * E, -1);
+        tag.assign((size_t)S, -1);
+        stamp.assign((size_t)S, -1);
+        pf_unused.assign((size_t)S, 0);
+        guard.assign((size_t)S, 0);
+        for (int32_t s = 0; s < S; ++s) order.insert({-1, s});
+    }
+    void protect(int32_t s)
+    {
+        if (!guard[s]) guard[s] = 1, guarded.push_back(s);
+    }
+    void unprotect_all()
+    {
+        for (int32_t s : guarded) guard[s] = 0;
+        guarded.clear();
+    }
+    void touch(int32_t s)
+    {
+        order.erase({stamp[s], s});
+        stamp[s] = clock;
+        order.insert({stamp[s], s});
+    }
+    int32_t victim() const
+    {
+        for (const auto &it : order)
+            if (!guard[it.second]) return it.second;
+        return -1;
+    }
+    void place(int32_t s, int32_t key, bool by_prefetch)
+    {
+        if (tag[s] >= 0) {
+            slot_of[tag[s]] = -1;
+            if (pf_unused[s]) ++pf_wasted;
+        }
+        tag[s] = key, slot_of[key] = s;
+        pf_unused[s] = by_prefetch;
+        touch(s);
+    }
+};
+
+struct TimedSpan {
+    cudaEvent_t a, b;
+    int kind;  // 0 transfer, 1 exposed wait
+};
+
+}  // namespace
+
+struct stmoe {
+    stmoe_config_t cfg{};
+    int rdt = 0;          // router dtype
+    int KS = 0;           // K + n_shared
+    int max_pred = 0;
+    size_t img_bytes = 0;
+    int next_layer = 0;
+    int64_t host_t = 0;
+    bool built = false;
+
+    uint8_t *d_router = nullptr;    // [L][E][H]
+    uint8_t *d_resident = nullptr;  // [L][E] images (resident stacks)
+    uint8_t *d_shared = nullptr;    // [L][n_shared] images
+    uint8_t *h_store = nullptr;     // pinned [L][E] images (offloaded stacks)
+    uint8_t *d_slots = nullptr;     // [S] images
+    const uint8_t **d_blob_table = nullptr;  // [L][E+n_shared] (resident) or [E+n_shared] (per step)
+    const uint8_t **h_blob_table = nullptr;  // pinned staging of one step's table
+
+    PredState pst{};
+    float *d_inv = nullptr, *d_logits = nullptr, *d_w = nullptr, *d_act = nullptr, *d_part = nullptr;
+    int32_t *d_ids = nullptr;   // [L][B][K] routing of the current decode step
+    int32_t *d_queue = nullptr; // [1 + 2E]
+    int32_t *h_ids = nullptr, *h_queue = nullptr;  // pinned mirrors
+    WorkListMem wlm;
+    FfnPlan plan1, plan4;
+
+    SlotCache cache;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_route = nullptr;
+    std::vector<cudaEvent_t> slot_ready;  // last copy into each slot
+    std::vector<uint8_t> slot_pending;
+    std::deque<TimedSpan> spans;
+    std::vector<cudaEvent_t> free_events;
+    double transfer_ms = 0, exposed_ms = 0;
+    int64_t bytes_demand = 0, bytes_prefetch = 0;
+};
+
+namespace {
+
+bool offloaded(const stmoe *s) { return s->cfg.cache_slots > 0; }
+
+int get_event(stmoe *s, cudaEvent_t *ev)
+{
+    if (!s->free_events.empty()) {
+        *ev = s->free_events.back();
+        s->free_events.pop_back();
+        return STMOE_OK;
+    }
+    CU_TRY(cudaEventCreate(ev));
+    return STMOE_OK;
+}
+
+void harvest_spans(stmoe *s, bool all)
+{
+    while (!s->spans.empty()) {
+        TimedSpan &sp = s->spans.front();
+        if (all)
+            cudaEventSynchronize(sp.b);
+        else if (cudaEventQuery(sp.b) != cudaSuccess) {
+            (void)cudaGetLastError();
+            break;
+        }
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, sp.a, sp.b) == cudaSuccess) (sp.kind == 0 ? s->transfer_ms : s->exposed_ms) += ms;
+        s->free_events.push_back(sp.a);
+        s->free_events.push_back(sp.b);
+        s->spans.pop_front();
+    }
+}
+
+uint8_t *image_ptr(stmoe *s, int layer, int expert, bool shared)
+{
+    const stmoe_config_t &c = s->cfg;
+    if (shared) return s->d_shared + ((size_t)layer * c.n_shared + expert) * s->img_bytes;
+    if (offloaded(s)) return s->h_store + ((size_t)layer * c.n_experts + expert) * s->img_bytes;
+    return s->d_resident + ((size_t)layer * c.n_experts + expert) * s->img_bytes;
+}
+
+int launch_predictor(stmoe *s, int layer, int batch, const int32_t *cur, const int32_t *prev,
+                     int32_t *pred_ids, int32_t *n_pred, bool want_queue, cudaStream_t st)
+{
+    const stmoe_config_t &c = s->cfg;
+    PredArgs a{};
+    a.st = s->pst;
+    a.L = c.n_layers, a.E = c.n_experts, a.K = c.top_k, a.P = c.profile_tokens;
+    a.mode = c.predictor_mode, a.layer = layer, a.B = batch;
+    a.cur = cur, a.prev = prev;
+    a.pred_ids = pred_ids, a.n_pred = n_pred, a.max_pred = s->max_pred;
+    a.queue = want_queue ? s->d_queue : nullptr;
+    predictor_step_kernel<<<1, 256, 0, st>>>(a);
+    if (layer == c.n_layers - 1) {
+        if (!s->built && s->host_t == c.profile_tokens - 1) {
+            const int rows = (c.n_layers - 1) * c.n_experts;
+            if (rows > 0)
+                cct_build_kernel<<<(rows + 7) / 8, 256, 0, st>>>(s->pst, c.n_layers, c.n_experts, c.top_k);
+            s->built = true;
+        }
+        s->host_t += 1;
+    }
+    CU_TRY(cudaGetLastError());
+    return STMOE_OK;
+}
+
+// Verification, miss loading and prefetch for one layer step of an offloaded stack.
+int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
+{
+    const stmoe_config_t &c = s->cfg;
+    const int E = c.n_experts, K = c.top_k, L = c.n_layers;
+    const int next = (layer + 1) % L;
+    SlotCache &ch = s->cache;
+
+    // this layer's routing and the prefetch queue, on the host (bounded wait)
+    CU_TRY(cudaMemcpyAsync(s->h_ids, s->d_ids + (size_t)layer * c.max_batch * K, sizeof(int32_t) * batch * K,
+                           cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaMemcpyAsync(s->h_queue, s->d_queue, sizeof(int32_t) * (1 + 2 * E), cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaEventRecord(s->ev_route, st));
+    const auto t0 = std::chrono::steady_clock::now();
+    for (;;) {
+        const cudaError_t q = cudaEventQuery(s->ev_route);
+        if (q == cudaSuccess) break;
+        if (q != cudaErrorNotReady) {
+            (void)cudaGetLastError();
+            return STMOE_ERR_CUDA;
+        }
+        if (std::chrono::steady_clock::now() - t0 > std::chrono::milliseconds(kWaitTimeoutMs))
+            return STMOE_ERR_TIMEOUT;
+    }
+    harvest_spans(s, false);
+
+    std::vector<uint8_t> routed(E, 0);
+    for (int i = 0; i < batch * K; ++i) routed[s->h_ids[i]] = 1;
+
+    // verify: hits and demand loads (ascending expert id)
+    ch.unprotect_all();
+    for (int e = 0; e < E; ++e)
+        if (routed[e] && ch.slot_of[(size_t)layer * E + e] >= 0) ch.protect(ch.slot_of[(size_t)layer * E + e]);
+    std::vector<cudaEvent_t> wait_on;
+    bool any_copy = false;
+    cudaEvent_t span_a = nullptr, span_b = nullptr;
+    auto begin_copies = [&]() -> int {
+        if (any_copy) return STMOE_OK;
+        ST_TRY(get_event(s, &span_a));
+        ST_TRY(get_event(s, &span_b));
+        CU_TRY(cudaEventRecord(span_a, s->copy_stream));
+        any_copy = true;
+        return STMOE_OK;
+    };
+    auto copy_into = [&](int32_t slot, int lyr, int e) -> int {
+        ST_TRY(begin_copies());
+        CU_TRY(cudaMemcpyAsync(s->d_slots + (size_t)slot * s->img_bytes, image_ptr(s, lyr, e, false),
+                               s->img_bytes, cudaMemcpyHostToDevice, s->copy_stream));
+        CU_TRY(cudaEventRecord(s->slot_ready[slot], s->copy_stream));
+        s->slot_pending[slot] = 1;
+        return STMOE_OK;
+    };
+    for (int e = 0; e < E; ++e) {
+        if (!routed[e]) continue;
+        const int32_t key = layer * E + e;
+        int32_t slot = ch.slot_of[key];
+        if (slot >= 0) {
+            ++ch.hits;
+            if (ch.pf_unused[slot]) ++ch.pf_useful, ch.pf_unused[slot] = 0;
+            ch.touch(slot);
+        } else {
+            slot = ch.victim();
+            if (slot < 0) return STMOE_ERR_STATE;
+            ++ch.misses;
+            ch.place(slot, key, false);
+            ch.protect(slot);
+            ST_TRY(copy_into(slot, layer, e));
+            s->bytes_demand += (int64_t)s->img_bytes;
+        }
+        if (s->slot_pending[slot]) {
+            if (cudaEventQuery(s->slot_ready[slot]) != cudaSuccess) {
+                (void)cudaGetLastError();
+                wait_on.push_back(s->slot_ready[slot]);
+            }
+            s->slot_pending[slot] = 0;  // later steps on this stream are ordered behind the wait
+        }
+        s->h_blob_table[e] = s->d_slots + (size_t)slot * s->img_bytes;
+    }
+    for (int i = 0; i < c.n_shared; ++i) s->h_blob_table[E + i] = image_ptr(s, layer, i, true);
+    CU_TRY(cudaMemcpyAsync(s->d_blob_table, s->h_blob_table, sizeof(void *) * (E + c.n_shared),
+                           cudaMemcpyHostToDevice, st));
+    if (!wait_on.empty()) {
+        // event-fenced handoff: the FFN kernels of this step start only after the copies into
+        // the slots they read have landed; the time they wait is the exposed transfer time
+        TimedSpan w{};
+        w.kind = 1;
+        ST_TRY(get_event(s, &w.a));
+        ST_TRY(get_event(s, &w.b));
+        CU_TRY(cudaEventRecord(w.a, st));
+        for (cudaEvent_t e : wait_on) CU_TRY(cudaStreamWaitEvent(st, e, 0));
+        CU_TRY(cudaEventRecord(w.b, st));
+        s->spans.push_back(w);
+    }
+
+    // prefetch the queued experts of the next layer (priority order)
+    const int nq = s->h_queue[0];
+    for (int i = 0; i < nq; ++i) {
+        const int32_t sl = ch.slot_of[(size_t)next * E + s->h_queue[1 + i]];
+        if (sl >= 0) ch.protect(sl);
+    }
+    int issued = 0;
+    for (int i = 0; i < nq; ++i) {
+        const int f = s->h_queue[1 + i];
+        const int32_t key = next * E + f;
+        if (ch.slot_of[key] >= 0) {
+            ++ch.pf_resident;
+            continue;
+        }
+        const int32_t slot = (c.prefetch_limit > 0 && issued >= c.prefetch_limit) ? -1 : ch.victim();
+        if (slot < 0) {
+            ++ch.pf_dropped;
+            continue;
+        }
+        ch.place(slot, key, true);
+        ch.protect(slot);
+        ++ch.pf_issued, ++issued;
+        ST_TRY(copy_into(slot, next, f));
+        s->bytes_prefetch += (int64_t)s->img_bytes;
+    }
+    if (any_copy) {
+        CU_TRY(cudaEventRecord(span_b, s->copy_stream));
+        s->spans.push_back(TimedSpan{span_a, span_b, 0});
+    }
+    ch.clock += 1;
+    return STMOE_OK;
+}
+
+int run_ffn(int dt, int mt, const FfnPlan &plan, const FfnArgs &fa, const float *w, int B, int K,
+            int n_shared, float rscale, float *h_out, cudaStream_t st)
+{
+    DISPATCH_DT_MT(dt, mt, launch_gate_up, fa, plan.grid_gate_up, st);
+    DISPATCH_DT_MT(dt, mt, launch_down, fa, plan.grid_down, st);
+    const int n = B * fa.H;
+    combine_kernel<<<std::min((n + 255) / 256, 4096), 256, 0, st>>>(fa.h, fa.part, w, B, fa.H, K, n_shared,
+                                                                   rscale, h_out);
+    CU_TRY(cudaGetLastError());
+    return STMOE_OK;
+}
+
+int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, int32_t *routed_ids,
+               float *routed_w, int32_t *predicted_ids, int32_t *n_predicted, uint32_t *flags,
+               cudaStream_t st)
+{
+    const stmoe_config_t &c = s->cfg;
+    const int E = c.n_experts, K = c.top_k, H = c.hidden;
+    const int mt = batch == 1 ? 1 : 4;
+    int32_t *ids = s->d_ids + (size_t)layer * c.max_batch * K;
+    const int32_t *prev = layer > 0 ? s->d_ids + (size_t)(layer - 1) * c.max_batch * K : nullptr;
+
+    launch_router_logits(s->rdt, h_in, s->d_router + (size_t)layer * E * H * dtype_bytes(s->rdt), batch, E, H,
+                         c.rms_eps, s->d_inv, s->d_logits, st);
+    TopkArgs ta{};
+    ta.logits = s->d_logits;
+    ta.B = batch, ta.E = E, ta.K = K, ta.n_shared = c.n_shared, ta.mt = mt;
+    ta.renorm = (c.flags & STMOE_FLAG_RENORM_TOPK) ? 1 : 0;
+    ta.ids = ids, ta.w = s->d_w;
+    ta.ids_out = routed_ids, ta.w_out = routed_w, ta.flags_out = flags;
+    ta.near_tie_counter = s->pst.stats + 4;
+    ta.wl = s->wlm.wl;
+    topk_group_kernel<<<1, 256, 0, st>>>(ta);
+    CU_TRY(cudaGetLastError());
+    ST_TRY(launch_predictor(s, layer, batch, ids, prev, predicted_ids, n_predicted, offloaded(s), st));
+
+    FfnArgs fa{};
+    fa.h = h_in, fa.inv_rms = s->d_inv, fa.wl = s->wlm.wl;
+    fa.act = s->d_act, fa.part = s->d_part, fa.H = H, fa.I = c.inter, fa.E = E;
+    if (offloaded(s)) {
+        ST_TRY(cache_step(s, layer, batch, st));
+        fa.blob = s->d_blob_table;
+    } else {
+        fa.blob = s->d_blob_table + (size_t)layer * (E + c.n_shared);
+    }
+    return run_ffn(c.weight_dtype, mt, mt == 1 ? s->plan1 : s->plan4, fa, s->d_w, batch, K, c.n_shared,
+                   c.residual_scale, h_out, st);
+}
+
+size_t state_bytes(const stmoe_config_t &c)
+{
+    const size_t pairs = c.n_layers > 1 ? c.n_layers - 1 : 0;
+    return 40 + pairs * c.n_experts * c.n_experts * 4 + 2 * pairs * c.n_experts * c.top_k +
+           (size_t)c.max_batch * c.n_layers * c.top_k * 2;
+}
+
+}  // namespace
+
+// ============================================================================== C ABI
+extern "C" {
+
+const char *stmoe_strerror(int code)
+{
+    switch (code) {
+    case STMOE_OK: return "ok";
+    case STMOE_ERR_BAD_ARG: return "bad argument";
+    case STMOE_ERR_OOM: return "out of memory";
+    case STMOE_ERR_CUDA: return "CUDA error";
+    case STMOE_ERR_TIMEOUT: return "timed out waiting for the device";
+    case STMOE_ERR_STATE: return "call out of order or inconsistent state";
+    case STMOE_ERR_UNIMPLEMENTED: return "not implemented";
+    default: return "unknown error";
+    }
+}
+
+int stmoe_destroy(stmoe_t *s)
+{
+    if (!s) return STMOE_OK;
+    cudaDeviceSynchronize();
+    harvest_spans(s, true);
+    for (cudaEvent_t e : s->free_events) cudaEventDestroy(e);
+    for (cudaEvent_t e : s->slot_ready) cudaEventDestroy(e);
+    if (s->ev_route) cudaEventDestroy(s->ev_route);
+    if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
+    void *dev[] = {s->d_router, s->d_resident, s->d_shared, s->d_slots, (void *)s->d_blob_table,
+                   s->pst.Co, s->pst.cct_id, s->pst.cct_conf, s->pst.HT, s->pst.t, s->pst.pred_mask,
+                   s->pst.pred_valid, s->pst.stats, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
+                   s->d_ids, s->d_queue};
+    for (void *p : dev)
+        if (p) cudaFree(p);
+    s->wlm.release();
+    void *host[] = {s->h_store, (void *)s->h_blob_table, s->h_ids, s->h_queue};
+    for (void *p : host)
+        if (p) cudaFreeHost(p);
+    (void)cudaGetLastError();
+    delete s;
+    return STMOE_OK;
+}
+
+int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
+{
+    if (!out) return STMOE_ERR_BAD_ARG;
+    *out = nullptr;
+    if (!cfg) return STMOE_ERR_BAD_ARG;
+    const stmoe_config_t &c = *cfg;
+    if (c.n_layers < 1 || c.n_experts < 1 || c.n_experts > kMaxExperts || c.top_k < 1 || c.top_k > kMaxTopK ||
+        c.top_k > c.n_experts || c.n_shared < 0 || c.n_shared > 8 || c.hidden < 16 || c.hidden % 16 ||
+        c.inter < 16 || c.inter % 16 || c.max_batch < 1 || c.max_batch > kMaxBatch ||
+        c.weight_dtype < STMOE_F32 || c.weight_dtype > STMOE_FP8_E4M3 || c.cache_slots < 0 ||
+        c.profile_tokens < 0 || c.predictor_mode < 0 || c.predictor_mode > 3 || c.prefetch_limit < 0 ||
+        (c.cache_slots > 0 && c.cache_slots < (int64_t)c.max_batch * c.top_k) ||
+        c.cache_slots > (int64_t)c.n_layers * c.n_experts)
+        return STMOE_ERR_BAD_ARG;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+        (void)cudaGetLastError();
+        return STMOE_ERR_CUDA;
+    }
+    stmoe *s = new (std::nothrow) stmoe();
+    if (!s) return STMOE_ERR_OOM;
+    s->cfg = c;
+    s->rdt = c.weight_dtype == STMOE_F32 ? STMOE_F32 : STMOE_BF16;
+    s->KS = c.top_k + c.n_shared;
+    s->max_pred = std::min(c.n_experts, c.top_k * c.top_k + c.top_k);
+    s->img_bytes = image_bytes(c.hidden, c.inter, c.weight_dtype);
+    const int L = c.n_layers, E = c.n_experts, K = c.top_k, B = c.max_batch, H = c.hidden, I = c.inter;
+    const size_t pairs = L > 1 ? L - 1 : 0;
+
+    auto fail = [&](int code) {
+        stmoe_destroy(s);
+        return code;
+    };
+#define CR_TRY(expr)                                                                       \
+    do {                                                                                   \
+        cudaError_t e_ = (expr);                                                           \
+        if (e_ != cudaSuccess) {                                                           \
+            (void)cudaGetLastError();                                                      \
+            return fail(e_ == cudaErrorMemoryAllocation ? STMOE_ERR_OOM : STMOE_ERR_CUDA); \
+        }                                                                                  \
+    } while (0)
+
+    CR_TRY(cudaMalloc(&s->d_router, (size_t)L * E * H * dtype_bytes(s->rdt)));
+    if (c.n_shared) CR_TRY(cudaMalloc(&s->d_shared, (size_t)L * c.n_shared * s->img_bytes));
+    if (c.cache_slots > 0) {
+        CR_TRY(cudaHostAlloc(&s->h_store, (size_t)L * E * s->img_bytes, cudaHostAllocDefault));
+        CR_TRY(cudaMalloc(&s->d_slots, (size_t)c.cache_slots * s->img_bytes));
+        CR_TRY(cudaMalloc(&s->d_blob_table, sizeof(void *) * (E + c.n_shared)));
+        CR_TRY(cudaHostAlloc(&s->h_blob_table, sizeof(void *) * (E + c.n_shared), cudaHostAllocDefault));
+        CR_TRY(cudaHostAlloc(&s->h_ids, sizeof(int32_t) * B * K, cudaHostAllocDefault));
+        CR_TRY(cudaHostAlloc(&s->h_queue, sizeof(int32_t) * (1 + 2 * E), cudaHostAllocDefault));
+        CR_TRY(cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking));
+        CR_TRY(cudaEventCreateWithFlags(&s->ev_route, cudaEventDisableTiming));
+        s->cache.init(c.cache_slots, L, E);
+        s->slot_ready.resize((size_t)c.cache_slots);
+        s->slot_pending.assign((size_t)c.cache_slots, 0);
+        for (auto &e : s->slot_ready) CR_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    } else {
+        CR_TRY(cudaMalloc(&s->d_resident, (size_t)L * E * s->img_bytes));
+        std::vector<const uint8_t *> tab((size_t)L * (E + c.n_shared));
+        for (int l = 0; l < L; ++l) {
+            for (int e = 0; e < E; ++e) tab[(size_t)l * (E + c.n_shared) + e] = image_ptr(s, l, e, false);
+            for (int i = 0; i < c.n_shared; ++i) tab[(size_t)l * (E + c.n_shared) + E + i] = image_ptr(s, l, i, true);
+        }
+        CR_TRY(cudaMalloc(&s->d_blob_table, sizeof(void *) * tab.size()));
+        CR_TRY(cudaMemcpy(s->d_blob_table, tab.data(), sizeof(void *) * tab.size(), cudaMemcpyHostToDevice));
+    }
+    CR_TRY(cudaMalloc(&s->pst.Co, std::max<size_t>(pairs * E * E * 4, 4)));
+    CR_TRY(cudaMalloc(&s->pst.cct_id, std::max<size_t>(pairs * E * K, 4)));
+    CR_TRY(cudaMalloc(&s->pst.cct_conf, std::max<size_t>(pairs * E * K, 4)));
+    CR_TRY(cudaMalloc(&s->pst.HT, (size_t)B * L * K * 2));
+    CR_TRY(cudaMalloc(&s->pst.t, 16));
+    CR_TRY(cudaMalloc(&s->pst.pred_mask, (size_t)B * 8 * 4));
+    CR_TRY(cudaMalloc(&s->pst.pred_valid, (size_t)B * 4));
+    CR_TRY(cudaMalloc(&s->pst.stats, 8 * 8));
+    CR_TRY(cudaMemset(s->pst.Co, 0, std::max<size_t>(pairs * E * E * 4, 4)));
+    CR_TRY(cudaMemset(s->pst.cct_id, 0, std::max<size_t>(pairs * E * K, 4)));
+    CR_TRY(cudaMemset(s->pst.cct_conf, 0, std::max<size_t>(pairs * E * K, 4)));
+    CR_TRY(cudaMemset(s->pst.HT, 0xff, (size_t)B * L * K * 2));
+    CR_TRY(cudaMemset(s->pst.t, 0, 16));
+    CR_TRY(cudaMemset(s->pst.pred_mask, 0, (size_t)B * 8 * 4));
+    CR_TRY(cudaMemset(s->pst.pred_valid, 0, (size_t)B * 4));
+    CR_TRY(cudaMemset(s->pst.stats, 0, 8 * 8));
+    CR_TRY(cudaMalloc(&s->d_inv, sizeof(float) * B));
+    CR_TRY(cudaMalloc(&s->d_logits, sizeof(float) * B * E));
+    CR_TRY(cudaMalloc(&s->d_w, sizeof(float) * B * K));
+    CR_TRY(cudaMalloc(&s->d_act, sizeof(float) * (size_t)B * s->KS * I));
+    CR_TRY(cudaMalloc(&s->d_part, sizeof(float) * (size_t)B * s->KS * H));
+    CR_TRY(cudaMalloc(&s->d_ids, sizeof(int32_t) * (size_t)L * B * K));
+    CR_TRY(cudaMalloc(&s->d_queue, sizeof(int32_t) * (1 + 2 * E)));
+    CR_TRY(cudaMemset(s->d_queue, 0, sizeof(int32_t) * (1 + 2 * E)));
+    if (s->wlm.alloc(B * s->KS) != STMOE_OK) return fail(STMOE_ERR_OOM);
+    s->plan1 = make_plan(c.weight_dtype, 1);
+    s->plan4 = make_plan(c.weight_dtype, 4);
+    if (c.profile_tokens == 0 && L > 1) {
+        const int rows = (L - 1) * E;
+        cct_build_kernel<<<(rows + 7) / 8, 256>>>(s->pst, L, E, K);
+        CR_TRY(cudaGetLastError());
+    }
+    s->built = c.profile_tokens == 0;
+    CR_TRY(cudaDeviceSynchronize());
+#undef CR_TRY
+    *out = s;
+    return STMOE_OK;
+}
+
+int stmoe_max_predicted(const stmoe_t *s) { return s ? s->max_pred : STMOE_ERR_BAD_ARG; }
+
+int stmoe_load_router(stmoe_t *s, int layer, const void *w)
+{
+    if (!s || !w || layer < 0 || layer >= s->cfg.n_layers) return STMOE_ERR_BAD_ARG;
+    const size_t n = (size_t)s->cfg.n_experts * s->cfg.hidden * dtype_bytes(s->rdt);
+    CU_TRY(cudaMemcpy(s->d_router + (size_t)layer * n, w, n, cudaMemcpyDefault));
+    return STMOE_OK;
+}
+
+int stmoe_load_experts(stmoe_t *s, int layer, int first_expert, int count, const void *gate, const void *up,
+                       const void *down, const void *scales, int is_shared)
+{
+    if (!s || !gate || !up || !down || layer < 0 || layer >= s->cfg.n_layers || first_expert < 0 || count < 1)
+        return STMOE_ERR_BAD_ARG;
+    const stmoe_config_t &c = s->cfg;
+    if (first_expert + count > (is_shared ? c.n_shared : c.n_experts)) return STMOE_ERR_BAD_ARG;
+    if ((c.weight_dtype == STMOE_FP8_E4M3) != (scales != nullptr)) return STMOE_ERR_BAD_ARG;
+    const int wb = dtype_bytes(c.weight_dtype);
+    const size_t mat = (size_t)c.hidden * c.inter * wb, sc = 2 * (size_t)(2 * c.inter + c.hidden);
+    for (int i = 0; i < count; ++i) {
+        uint8_t *img = image_ptr(s, layer, first_expert + i, is_shared != 0);
+        CU_TRY(cudaMemcpy(img + image_gate(c.hidden, c.inter, wb), (const uint8_t *)gate + i * mat, mat, cudaMemcpyDefault));
+        CU_TRY(cudaMemcpy(img + image_up(c.hidden, c.inter, wb), (const uint8_t *)up + i * mat, mat, cudaMemcpyDefault));
+        CU_TRY(cudaMemcpy(img + image_down(c.hidden, c.inter, wb), (const uint8_t *)down + i * mat, mat, cudaMemcpyDefault));
+        if (scales)
+            CU_TRY(cudaMemcpy(img + image_scales(c.hidden, c.inter, wb), (const uint8_t *)scales + i * sc, sc, cudaMemcpyDefault));
+    }
+    return STMOE_OK;
+}
+
+int stmoe_decode_step(stmoe_t *s, int layer, int batch, const float *h_in, float *h_out, int32_t *routed_ids,
+                      float *routed_w, int32_t *predicted_ids, int32_t *n_predicted, uint32_t *flags,
+                      void *cuda_stream)
+{
+    if (!s || !h_in || !h_out || batch < 1 || batch > s->cfg.max_batch || layer < 0 || layer >= s->cfg.n_layers)
+        return STMOE_ERR_BAD_ARG;
+    if (layer != s->next_layer) return STMOE_ERR_STATE;
+    const int rc = layer_step(s, layer, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted,
+                              flags, (cudaStream_t)cuda_stream);
+    if (rc == STMOE_OK) s->next_layer = (layer + 1) % s->cfg.n_layers;
+    return rc;
+}
+
+int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, int32_t *routed_ids,
+                       float *routed_w, int32_t *predicted_ids, int32_t *n_predicted, uint32_t *flags,
+                       void *cuda_stream)
+{
+    if (!s || !h_in || !h_out || batch < 1 || batch > s->cfg.max_batch) return STMOE_ERR_BAD_ARG;
+    if (s->next_layer != 0) return STMOE_ERR_STATE;
+    const int K = s->cfg.top_k;
+    for (int l = 0; l < s->cfg.n_layers; ++l) {
+        const size_t o = (size_t)l * batch;
+        ST_TRY(layer_step(s, l, batch, l == 0 ? h_in : h_out, h_out, routed_ids ? routed_ids + o * K : nullptr,
+                          routed_w ? routed_w + o * K : nullptr,
+                          predicted_ids ? predicted_ids + o * s->max_pred : nullptr,
+                          n_predicted ? n_predicted + o : nullptr, flags ? flags + o : nullptr,
+                          (cudaStream_t)cuda_stream));
+    }
+    return STMOE_OK;
+}
+
+int stmoe_stats(stmoe_t *s, stmoe_stats_t *out)
+{
+    if (!s || !out) return STMOE_ERR_BAD_ARG;
+    CU_TRY(cudaDeviceSynchronize());
+    harvest_spans(s, true);
+    unsigned long long st[8];
+    long long t[2];
+    CU_TRY(cudaMemcpy(st, s->pst.stats, sizeof(st), cudaMemcpyDeviceToHost));
+    CU_TRY(cudaMemcpy(t, s->pst.t, sizeof(t), cudaMemcpyDeviceToHost));
+    memset(out, 0, sizeof(*out));
+    out->decode_steps = t[0];
+    out->runtime_steps = (int64_t)st[0], out->routed = (int64_t)st[1];
+    out->predicted = (int64_t)st[2], out->hits = (int64_t)st[3], out->near_ties = (int64_t)st[4];
+    const SlotCache &ch = s->cache;
+    out->cache_hits = ch.hits, out->cache_misses = ch.misses;
+    out->prefetch_issued = ch.pf_issued, out->prefetch_useful = ch.pf_useful;
+    out->prefetch_wasted = ch.pf_wasted, out->prefetch_dropped = ch.pf_dropped;
+    out->prefetch_resident = ch.pf_resident;
+    out->h2d_bytes_demand = s->bytes_demand, out->h2d_bytes_prefetch = s->bytes_prefetch;
+    out->transfer_ms = s->transfer_ms, out->exposed_ms = s->exposed_ms;
+    return STMOE_OK;
+}
+
+int stmoe_export_state(stmoe_t *s, void *buf, size_t *bytes)
+{
+    if (!s || !bytes) return STMOE_ERR_BAD_ARG;
+    const stmoe_config_t &c = s->cfg;
+    const size_t need = state_bytes(c);
+    if (!buf) {
+        *bytes = need;
+        return STMOE_OK;
+    }
+    if (*bytes < need) return STMOE_ERR_BAD_ARG;
+    *bytes = need;
+    CU_TRY(cudaDeviceSynchronize());
+    const size_t pairs = c.n_layers > 1 ? c.n_layers - 1 : 0;
+    uint8_t *o = (uint8_t *)buf;
+    const int32_t hdr[8] = {(int32_t)kStateMagic, 1, c.n_layers, c.n_experts, c.top_k, c.max_batch,
+                            c.profile_tokens, s->built ? 1 : 0};
+    memcpy(o, hdr, 32), o += 32;
+    CU_TRY(cudaMemcpy(o, s->pst.t, 8, cudaMemcpyDeviceToHost));
+    o += 8;
+    const size_t n_co = pairs * c.n_experts * c.n_experts * 4, n_cct = pairs * c.n_experts * c.top_k;
+    if (n_co) CU_TRY(cudaMemcpy(o, s->pst.Co, n_co, cudaMemcpyDeviceToHost));
+    o += n_co;
+    if (n_cct) CU_TRY(cudaMemcpy(o, s->pst.cct_id, n_cct, cudaMemcpyDeviceToHost));
+    o += n_cct;
+    if (n_cct) CU_TRY(cudaMemcpy(o, s->pst.cct_conf, n_cct, cudaMemcpyDeviceToHost));
+    o += n_cct;
+    CU_TRY(cudaMemcpy(o, s->pst.HT, (size_t)c.max_batch * c.n_layers * c.top_k * 2, cudaMemcpyDeviceToHost));
+    return STMOE_OK;
+}
+
+int stmoe_import_state(stmoe_t *s, const void *buf, size_t bytes)
+{
+    if (!s || !buf) return STMOE_ERR_BAD_ARG;
+    const stmoe_config_t &c = s->cfg;
+    if (bytes != state_bytes(c)) return STMOE_ERR_BAD_ARG;
+    if (s->next_layer != 0) return STMOE_ERR_STATE;
+    const uint8_t *o = (const uint8_t *)buf;
+    int32_t hdr[8];
+    memcpy(hdr, o, 32), o += 32;
+    if ((uint32_t)hdr[0] != kStateMagic || hdr[1] != 1 || hdr[2] != c.n_layers || hdr[3] != c.n_experts ||
+        hdr[4] != c.top_k || hdr[5] != c.max_batch || hdr[6] != c.profile_tokens)
+        return STMOE_ERR_BAD_ARG;
+    CU_TRY(cudaDeviceSynchronize());
+    long long t = 0;
+    memcpy(&t, o, 8);
+    CU_TRY(cudaMemcpy(s->pst.t, o, 8, cudaMemcpyHostToDevice));
+    o += 8;
+    const size_t pairs = c.n_layers > 1 ? c.n_layers - 1 : 0;
+    const size_t n_co = pairs * c.n_experts * c.n_experts * 4, n_cct = pairs * c.n_experts * c.top_k;
+    if (n_co) CU_TRY(cudaMemcpy(s->pst.Co, o, n_co, cudaMemcpyHostToDevice));
+    o += n_co;
+    if (n_cct) CU_TRY(cudaMemcpy(s->pst.cct_id, o, n_cct, cudaMemcpyHostToDevice));
+    o += n_cct;
+    if (n_cct) CU_TRY(cudaMemcpy(s->pst.cct_conf, o, n_cct, cudaMemcpyHostToDevice));
+    o += n_cct;
+    CU_TRY(cudaMemcpy(s->pst.HT, o, (size_t)c.max_batch * c.n_layers * c.top_k * 2, cudaMemcpyHostToDevice));
+    CU_TRY(cudaMemset(s->pst.pred_valid, 0, (size_t)c.max_batch * 4));
+    s->host_t = t;
+    s->built = hdr[7] != 0;
+    return STMOE_OK;
+}
+
+int stmoe_export_cache_tags(stmoe_t *s, int32_t *tags, int64_t n)
+{
+    if (!s || !tags || n != s->cfg.cache_slots || n == 0) return STMOE_ERR_BAD_ARG;
+    memcpy(tags, s->cache.tag.data(), sizeof(int32_t) * (size_t)n);
+    return STMOE_OK;
+}
+
+int stmoe_router_topk(const float *h, const void *w_router, int wr_dtype, int batch, int n_experts, int hidden,
+                      int top_k, float rms_eps, int renorm, float *logits, int32_t *ids, float *w,
+                      uint32_t *flags, void *cuda_stream)
+{
+    if (!h || !w_router || !logits || !ids || !w || batch < 1 || batch > kMaxBatch || n_experts < 1 ||
+        n_experts > kMaxExperts || top_k < 1 || top_k > kMaxTopK || top_k > n_experts || hidden < 16 ||
+        hidden % 16 || (wr_dtype != STMOE_F32 && wr_dtype != STMOE_BF16))
+        return STMOE_ERR_BAD_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    float *inv = logits + (size_t)batch * n_experts;  // tail of the caller's buffer
+    launch_router_logits(wr_dtype, h, w_router, batch, n_experts, hidden, rms_eps, inv, logits, st);
+    TopkArgs ta{};
+    ta.logits = logits;
+    ta.B = batch, ta.E = n_experts, ta.K = top_k, ta.mt = 1, ta.renorm = renorm;
+    ta.ids = ids, ta.w = w, ta.flags_out = flags;
+    topk_group_kernel<<<1, 256, 0, st>>>(ta);
+    CU_TRY(cudaGetLastError());
+    return STMOE_OK;
+}
+
+int stmoe_predictor_step(stmoe_t *s, int layer, int batch, const int32_t *routed_ids, int32_t *predicted_ids,
+                         int32_t *n_predicted, void *cuda_stream)
+{
+    if (!s || !routed_ids || batch < 1 || batch > s->cfg.max_batch || layer < 0 || layer >= s->cfg.n_layers)
+        return STMOE_ERR_BAD_ARG;
+    if (layer != s->next_layer) return STMOE_ERR_STATE;
+    const stmoe_config_t &c = s->cfg;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int32_t *ids = s->d_ids + (size_t)layer * c.max_batch * c.top_k;
+    const int32_t *prev = layer > 0 ? s->d_ids + (size_t)(layer - 1) * c.max_batch * c.top_k : nullptr;
+    CU_TRY(cudaMemcpyAsync(ids, routed_ids, sizeof(int32_t) * batch * c.top_k, cudaMemcpyDeviceToDevice, st));
+    ST_TRY(launch_predictor(s, layer, batch, ids, prev, predicted_ids, n_predicted, true, st));
+    s->next_layer = (layer + 1) % c.n_layers;
+    return STMOE_OK;
+}
+
+size_t stmoe_expert_image_bytes(int hidden, int inter, int weight_dtype)
+{
+    return image_bytes(hidden, inter, weight_dtype);
+}
+
+// scratch layout: work list | blob table | act | part
+static size_t ffn_scratch_layout(int B, int K, int H, int I, int E, size_t *o_tab, size_t *o_act, size_t *o_part)
+{
+    size_t o = round_up(sizeof(int) * (size_t)(4 + 5 * B * K), 256);
+    *o_tab = o, o += round_up(sizeof(void *) * (size_t)E, 256);
+    *o_act = o, o += round_up(sizeof(float) * (size_t)B * K * I, 256);
+    *o_part = o, o += round_up(sizeof(float) * (size_t)B * K * H, 256);
+    return o;
+}
+
+size_t stmoe_moe_ffn_scratch_bytes(int batch, int top_k, int hidden, int inter)
+{
+    size_t a, b, c;
+    return ffn_scratch_layout(batch, top_k, hidden, inter, kMaxExperts, &a, &b, &c);
+}
+
+}  // extern "C"
+
+namespace {
+
+// fills the work list and the expert-image table of a stand-alone FFN call from given routing
+__global__ void __launch_bounds__(256)
+group_given_ids_kernel(const int32_t *ids, int B, int E, int K, int mt, WorkList wl, const uint8_t *experts,
+                       size_t img_bytes, const uint8_t **table)
+{
+    __shared__ int s_g[kMaxExperts + 1], s_p[kMaxExperts + 1];
+    const int e = threadIdx.x;
+    int cnt = 0;
+    if (e < E)
+        for (int i = 0; i < B * K; ++i) cnt += (ids[i] == e);
+    s_g[e + 1] = (cnt + mt - 1) / mt, s_p[e + 1] = cnt;
+    if (e == 0) s_g[0] = s_p[0] = 0;
+    if (e < E) table[e] = experts + (size_t)e * img_bytes;
+    __syncthreads();
+    if (e == 0)
+        for (int i = 1; i <= kMaxExperts; ++i) s_g[i] += s_g[i - 1], s_p[i] += s_p[i - 1];
+    __syncthreads();
+    if (e < E && cnt > 0) {
+        for (int t = 0, g = s_g[e]; t < cnt; t += mt, ++g)
+            wl.g_expert[g] = e, wl.g_start[g] = s_p[e] + t, wl.g_count[g] = min(mt, cnt - t);
+        int n = 0;
+        for (int i = 0; i < B * K; ++i)
+            if (ids[i] == e) wl.pair_token[s_p[e] + n] = i / K, wl.pair_slot[s_p[e] + n] = i, ++n;
+    }
+    if (e == 0) *wl.n_groups = s_g[kMaxExperts];
+}
+
+}  // namespace
+
+extern "C" int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t *ids, const float *w,
+                             const void *experts, int weight_dtype, int batch, int n_experts, int top_k,
+                             int hidden, int inter, float residual_scale, float *h_out, void *scratch,
+                             size_t scratch_bytes, void *cuda_stream)
+{
+    if (!h || !ids || !w || !experts || !h_out || !scratch || batch < 1 || batch > kMaxBatch || n_experts < 1 ||
+        n_experts > kMaxExperts || top_k < 1 || top_k > kMaxTopK || top_k > n_experts || hidden < 16 ||
+        hidden % 16 || inter < 16 || inter % 16 || weight_dtype < STMOE_F32 || weight_dtype > STMOE_FP8_E4M3 ||
+        ((uintptr_t)scratch & 255))
+        return STMOE_ERR_BAD_ARG;
+    size_t o_tab, o_act, o_part;
+    if (scratch_bytes < ffn_scratch_layout(batch, top_k, hidden, inter, kMaxExperts, &o_tab, &o_act, &o_part))
+        return STMOE_ERR_BAD_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    uint8_t *sc = (uint8_t *)scratch;
+    WorkListMem wlm;
+    wlm.bind((int *)sc, batch * top_k);
+    const int mt = batch == 1 ? 1 : 4;
+    const uint8_t **table = (const uint8_t **)(sc + o_tab);
+    group_given_ids_kernel<<<1, 256, 0, st>>>(ids, batch, n_experts, top_k, mt, wlm.wl, (const uint8_t *)experts,
+                                             image_bytes(hidden, inter, weight_dtype), table);
+    FfnArgs fa{};
+    fa.h = h, fa.inv_rms = inv_rms, fa.wl = wlm.wl, fa.blob = table;
+    fa.act = (float *)(sc + o_act), fa.part = (float *)(sc + o_part);
+    fa.H = hidden, fa.I = inter, fa.E = n_experts;
+    static FfnPlan plans[3][2];
+    FfnPlan &plan = plans[weight_dtype][mt == 1 ? 0 : 1];
+    if (plan.grid_down == 0) plan = make_plan(weight_dtype, mt);
+    return run_ffn(weight_dtype, mt, plan, fa, w, batch, top_k, 0, residual_scale, h_out, st);
+}

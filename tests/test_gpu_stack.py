@@ -1,0 +1,135 @@
+"""GPU parity of the whole layer step on seeded stacks: teacher-forced layer outputs,
+predictor replay on the GPU's own routing, free-running decode, cache bookkeeping."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2606_15453_b200 as P
+from datagen import stacks
+from helpers import Pair, check_layer
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _teacher_forced(cfg, B, tokens, mode="st", prefetch_limit=0, flags=0):
+    """Feed both sides the oracle's hidden state at every (token, layer)."""
+    pr = Pair(cfg, B, mode=mode, prefetch_limit=prefetch_limit, flags=flags)
+    x = stacks.token_inputs(cfg, B, tokens).numpy()
+    replay = O.Predictor(cfg.n_layers, cfg.n_experts, cfg.top_k, B, cfg.profile_tokens, mode)
+    cache = O.CacheModel(cfg.cache_slots, cfg.n_layers, cfg.n_experts) if cfg.cache_slots else None
+    skipped = 0
+    for t in range(tokens):
+        h = x[t]
+        for l in range(cfg.n_layers):
+            o = pr.oracle.layer_step(l, h)
+            g = pr.gpu_step(l, h)
+            skipped += check_layer(cfg, g, o, h, where=f"t={t} l={l}")
+            # predictor replay: the oracle's tables driven by the GPU's routing, bit-exact
+            rp = replay.step(l, g["ids"])
+            assert g["n_pred"].tolist() == rp["n_pred"].tolist(), (t, l)
+            assert (g["pred_ids"] == rp["pred_ids"]).all(), (t, l)
+            if cache is not None:
+                cache.step(l, np.unique(g["ids"]), (l + 1) % cfg.n_layers, rp["queue_ids"],
+                           prefetch_limit)
+            h = o["h_out"]
+    assert pr.stack.export_state() == replay.export()
+    st, so = pr.stack.stats(), replay.stats()
+    assert (st["runtime_steps"], st["routed"], st["predicted"], st["hits"]) == \
+        (so["steps"], so["routed"], so["predicted"], so["hits"])
+    if cache is not None:
+        sc = cache.stats()
+        assert (st["cache_hits"], st["cache_misses"], st["prefetch_issued"], st["prefetch_useful"],
+                st["prefetch_wasted"], st["prefetch_dropped"], st["prefetch_resident"]) == \
+            (sc["hits"], sc["misses"], sc["pf_issued"], sc["pf_useful"], sc["pf_wasted"],
+             sc["pf_dropped"], sc["pf_resident"])
+        assert (pr.stack.export_cache_tags().numpy() == cache.tags()).all()
+        assert st["h2d_bytes_demand"] == sc["misses"] * P.expert_image_bytes(cfg.hidden, cfg.inter, cfg.dtype)
+    pr.close()
+    return skipped, st
+
+
+def test_c0_full_teacher_forced():
+    cfg = stacks.CONFIGS["C0"]
+    skipped, st = _teacher_forced(cfg, 1, cfg.tokens)
+    assert skipped <= 3
+    assert st["decode_steps"] == cfg.tokens and st["hits"] > 0
+
+
+def test_c0_free_running_and_routing_independent_of_predictor():
+    """Both sides run their own residual stream; outputs and routing are the same with the
+    predictor on or off (prediction never alters routing)."""
+    cfg = stacks.CONFIGS["C0"]
+    x = stacks.token_inputs(cfg, 1, cfg.tokens)
+    outs = {}
+    for mode in ("st", "off"):
+        pr = Pair(cfg, 1, mode=mode, oracle=(mode == "st"))
+        L, K = cfg.n_layers, cfg.top_k
+        ids = torch.empty(L, 1, K, dtype=torch.int32, device=DEV)
+        ho = torch.empty(1, cfg.hidden, device=DEV)
+        all_ids, all_h, first_div = [], [], None
+        for t in range(cfg.tokens):
+            pr.stack.decode_token(x[t].to(DEV), ho, routed_ids=ids)
+            torch.cuda.synchronize()
+            all_ids.append(ids.cpu().numpy().copy()), all_h.append(ho.cpu().numpy().copy())
+            if mode == "st" and first_div is None:
+                h_o, per = pr.oracle.decode_token(x[t].numpy())
+                o_ids = np.stack([r["ids"] for r in per])
+                ties = sum(int(r["ties"].sum()) for r in per)
+                if (o_ids != all_ids[-1]).any():
+                    assert ties > 0, f"routing diverged at token {t} without a near tie"
+                    first_div = t
+                else:
+                    assert np.abs(all_h[-1] - h_o).max() / np.abs(h_o).max() < 1e-4
+        outs[mode] = (np.stack(all_ids), np.stack(all_h))
+        pr.close()
+    assert (outs["st"][0] == outs["off"][0]).all() and (outs["st"][1] == outs["off"][1]).all()
+
+
+@pytest.mark.parametrize("name,B,kw,tokens", [
+    ("C1", 1, dict(n_layers=2, profile_tokens=2), 4),
+    ("C1", 4, dict(n_layers=2, profile_tokens=1), 3),
+    ("C2", 1, dict(n_layers=3, profile_tokens=2), 5),
+    ("C2", 8, dict(n_layers=2, profile_tokens=1), 3),
+    ("C3", 1, dict(n_layers=3, profile_tokens=2, cache_slots=96), 6),
+    ("C3", 16, dict(n_layers=2, profile_tokens=1, cache_slots=160), 3),
+    ("C4", 1, dict(n_layers=2, profile_tokens=1, cache_slots=64), 3),
+    ("C4", 32, dict(n_layers=2, profile_tokens=1, cache_slots=256, hidden=1024, inter=768), 2),
+])
+def test_config_shapes_teacher_forced(name, B, kw, tokens):
+    """The benchmark shapes (full H/I, fewer layers) incl. shared experts, offload and fp8."""
+    cfg = stacks.CONFIGS[name].scaled(**kw)
+    _teacher_forced(cfg, B, tokens, prefetch_limit=8 if cfg.cache_slots else 0)
+
+
+def test_ragged_shapes_and_modes():
+    cfg = stacks.CONFIGS["C0"].scaled(n_layers=3, n_experts=12, top_k=3, hidden=272, inter=176,
+                                      n_shared=1, profile_tokens=2, dtype="bf16")
+    for mode in ("temporal", "spatial"):
+        _teacher_forced(cfg, 5, 6, mode=mode)
+    _teacher_forced(cfg.scaled(n_layers=1, n_experts=4, top_k=4, n_shared=0), 2, 4)
+    _teacher_forced(cfg, 3, 4, flags=P.FLAG_RENORM_TOPK)
+
+
+def test_tiny_cache_thrashes_but_stays_correct():
+    cfg = stacks.CONFIGS["C0"].scaled(n_layers=3, n_experts=16, top_k=2, hidden=128, inter=256,
+                                      profile_tokens=3, dtype="bf16", cache_slots=4)
+    _, st = _teacher_forced(cfg, 2, 12)
+    assert st["cache_misses"] > 0 and st["transfer_ms"] > 0
+    _, st = _teacher_forced(cfg.scaled(cache_slots=48), 2, 12, prefetch_limit=2)
+    assert st["prefetch_issued"] > 0
+
+
+def test_argument_and_state_errors():
+    with pytest.raises(P.StmoeError):
+        P.Stack(2, 8, 2, 100, 64)                       # H not a multiple of 16
+    with pytest.raises(P.StmoeError):
+        P.Stack(2, 8, 2, 64, 64, cache_slots=1)         # fewer slots than routed experts
+    s = P.Stack(2, 8, 2, 64, 64, dtype="f32")
+    h = torch.zeros(1, 64, device=DEV)
+    with pytest.raises(P.StmoeError):
+        s.decode_step(1, h, h)                          # layer 0 is due
+    with pytest.raises(P.StmoeError):
+        s.decode_step(0, torch.zeros(2, 64, device=DEV), torch.zeros(2, 64, device=DEV))  # batch > max
+    s.close()
