@@ -95,6 +95,10 @@ typedef struct {
     int64_t h2d_bytes_prefetch;
     double transfer_ms;       /* device time of all host->HBM expert copies               */
     double exposed_ms;        /* time the compute stream waited for such copies           */
+    int64_t kernel_launches;  /* kernels launched by layer steps since creation           */
+    int64_t timed_ffn_launches; /* layer steps whose FFN kernels were timed (see below)   */
+    double gate_up_ms;        /* summed device time of the timed gate/up kernels          */
+    double down_ms;           /* summed device time of the timed down kernels             */
 } stmoe_stats_t;
 
 /* Create a stack for the current CUDA device.  Allocates weight storage (HBM
@@ -141,6 +145,10 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out,
                        int32_t *n_predicted, uint32_t *flags, void *cuda_stream);
 
 int stmoe_max_predicted(const stmoe_t *s); /* min(E, K*K+K) */
+
+/* on != 0: bracket the two expert-FFN kernels of every following layer step with CUDA events
+ * on the caller's stream; their summed durations appear in stmoe_stats.  Off by default. */
+int stmoe_set_kernel_timing(stmoe_t *s, int on);
 
 /* Counters and timings; synchronises the device. */
 int stmoe_stats(stmoe_t *s, stmoe_stats_t *out);

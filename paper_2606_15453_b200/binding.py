@@ -36,7 +36,8 @@ class Stats(C.Structure):
         "decode_steps", "runtime_steps", "routed", "predicted", "hits", "near_ties", "cache_hits",
         "cache_misses", "prefetch_issued", "prefetch_useful", "prefetch_wasted", "prefetch_dropped",
         "prefetch_resident", "h2d_bytes_demand", "h2d_bytes_prefetch")] + \
-        [("transfer_ms", C.c_double), ("exposed_ms", C.c_double)]
+        [("transfer_ms", C.c_double), ("exposed_ms", C.c_double), ("kernel_launches", C.c_int64),
+         ("timed_ffn_launches", C.c_int64), ("gate_up_ms", C.c_double), ("down_ms", C.c_double)]
 
 
 _lib = None
@@ -59,6 +60,7 @@ def lib():
         L.stmoe_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.stmoe_decode_token.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.stmoe_max_predicted.argtypes = [vp]
+        L.stmoe_set_kernel_timing.argtypes = [vp, i32]
         L.stmoe_stats.argtypes = [vp, C.POINTER(Stats)]
         L.stmoe_export_state.argtypes = [vp, vp, C.POINTER(sz)]
         L.stmoe_import_state.argtypes = [vp, vp, sz]
@@ -159,6 +161,9 @@ class Stack:
         _check(lib().stmoe_predictor_step(self._h, layer, routed_ids.shape[0],
                                           _dev(routed_ids, torch.int32), _ptr(predicted_ids),
                                           _ptr(n_predicted), _stream(stream)), "stmoe_predictor_step")
+
+    def set_kernel_timing(self, on: bool) -> None:
+        _check(lib().stmoe_set_kernel_timing(self._h, int(on)), "stmoe_set_kernel_timing")
 
     def stats(self) -> dict:
         st = Stats()

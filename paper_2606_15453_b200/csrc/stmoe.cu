@@ -227,7 +227,7 @@ struct SlotCache {
 
 struct TimedSpan {
     cudaEvent_t a, b;
-    int kind;  // 0 transfer, 1 exposed wait
+    int kind;  // 0 transfer, 1 exposed wait, 2 gate/up kernel, 3 down kernel
 };
 
 }  // namespace
@@ -265,7 +265,9 @@ struct stmoe {
     std::vector<uint8_t> slot_pending;
     std::deque<TimedSpan> spans;
     std::vector<cudaEvent_t> free_events;
-    double transfer_ms = 0, exposed_ms = 0;
+    double transfer_ms = 0, exposed_ms = 0, gate_up_ms = 0, down_ms = 0;
+    int64_t launches = 0, timed_ffn = 0;
+    bool time_kernels = false;
     int64_t bytes_demand = 0, bytes_prefetch = 0;
 };
 
@@ -295,9 +297,12 @@ void harvest_spans(stmoe *s, bool all)
             break;
         }
         float ms = 0.f;
-        if (cudaEventElapsedTime(&ms, sp.a, sp.b) == cudaSuccess) (sp.kind == 0 ? s->transfer_ms : s->exposed_ms) += ms;
+        if (cudaEventElapsedTime(&ms, sp.a, sp.b) == cudaSuccess) {
+            double *acc[4] = {&s->transfer_ms, &s->exposed_ms, &s->gate_up_ms, &s->down_ms};
+            *acc[sp.kind] += ms;
+        }
         s->free_events.push_back(sp.a);
-        s->free_events.push_back(sp.b);
+        if (sp.kind != 2) s->free_events.push_back(sp.b);  // a gate/up span's end event starts the down span
         s->spans.pop_front();
     }
 }
@@ -322,11 +327,13 @@ int launch_predictor(stmoe *s, int layer, int batch, const int32_t *cur, const i
     a.pred_ids = pred_ids, a.n_pred = n_pred, a.max_pred = s->max_pred;
     a.queue = want_queue ? s->d_queue : nullptr;
     predictor_step_kernel<<<1, 256, 0, st>>>(a);
+    s->launches += 1;
     if (layer == c.n_layers - 1) {
         if (!s->built && s->host_t == c.profile_tokens - 1) {
             const int rows = (c.n_layers - 1) * c.n_experts;
             if (rows > 0)
                 cct_build_kernel<<<(rows + 7) / 8, 256, 0, st>>>(s->pst, c.n_layers, c.n_experts, c.top_k);
+            s->launches += rows > 0;
             s->built = true;
         }
         s->host_t += 1;
@@ -462,11 +469,27 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
     return STMOE_OK;
 }
 
-int run_ffn(int dt, int mt, const FfnPlan &plan, const FfnArgs &fa, const float *w, int B, int K,
+int run_ffn(stmoe *s, int dt, int mt, const FfnPlan &plan, const FfnArgs &fa, const float *w, int B, int K,
             int n_shared, float rscale, float *h_out, cudaStream_t st)
 {
+    cudaEvent_t e0 = nullptr, e1 = nullptr, e2 = nullptr;
+    const bool timed = s && s->time_kernels;
+    if (timed) {
+        ST_TRY(get_event(s, &e0));
+        ST_TRY(get_event(s, &e1));
+        ST_TRY(get_event(s, &e2));
+        CU_TRY(cudaEventRecord(e0, st));
+    }
     DISPATCH_DT_MT(dt, mt, launch_gate_up, fa, plan.grid_gate_up, st);
+    if (timed) CU_TRY(cudaEventRecord(e1, st));
     DISPATCH_DT_MT(dt, mt, launch_down, fa, plan.grid_down, st);
+    if (timed) {
+        CU_TRY(cudaEventRecord(e2, st));
+        s->spans.push_back(TimedSpan{e0, e1, 2});
+        s->spans.push_back(TimedSpan{e1, e2, 3});
+        s->timed_ffn += 1;
+    }
+    if (s) s->launches += 3;
     const int n = B * fa.H;
     combine_kernel<<<std::min((n + 255) / 256, 4096), 256, 0, st>>>(fa.h, fa.part, w, B, fa.H, K, n_shared,
                                                                    rscale, h_out);
@@ -507,7 +530,8 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
     } else {
         fa.blob = s->d_blob_table + (size_t)layer * (E + c.n_shared);
     }
-    return run_ffn(c.weight_dtype, mt, mt == 1 ? s->plan1 : s->plan4, fa, s->d_w, batch, K, c.n_shared,
+    s->launches += 2;
+    return run_ffn(s, c.weight_dtype, mt, mt == 1 ? s->plan1 : s->plan4, fa, s->d_w, batch, K, c.n_shared,
                    c.residual_scale, h_out, st);
 }
 
@@ -669,6 +693,13 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
 
 int stmoe_max_predicted(const stmoe_t *s) { return s ? s->max_pred : STMOE_ERR_BAD_ARG; }
 
+int stmoe_set_kernel_timing(stmoe_t *s, int on)
+{
+    if (!s) return STMOE_ERR_BAD_ARG;
+    s->time_kernels = on != 0;
+    return STMOE_OK;
+}
+
 int stmoe_load_router(stmoe_t *s, int layer, const void *w)
 {
     if (!s || !w || layer < 0 || layer >= s->cfg.n_layers) return STMOE_ERR_BAD_ARG;
@@ -749,6 +780,8 @@ int stmoe_stats(stmoe_t *s, stmoe_stats_t *out)
     out->prefetch_resident = ch.pf_resident;
     out->h2d_bytes_demand = s->bytes_demand, out->h2d_bytes_prefetch = s->bytes_prefetch;
     out->transfer_ms = s->transfer_ms, out->exposed_ms = s->exposed_ms;
+    out->kernel_launches = s->launches, out->timed_ffn_launches = s->timed_ffn;
+    out->gate_up_ms = s->gate_up_ms, out->down_ms = s->down_ms;
     return STMOE_OK;
 }
 
@@ -939,5 +972,5 @@ extern "C" int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t
     static FfnPlan plans[3][2];
     FfnPlan &plan = plans[weight_dtype][mt == 1 ? 0 : 1];
     if (plan.grid_down == 0) plan = make_plan(weight_dtype, mt);
-    return run_ffn(weight_dtype, mt, plan, fa, w, batch, top_k, 0, residual_scale, h_out, st);
+    return run_ffn(nullptr, weight_dtype, mt, plan, fa, w, batch, top_k, 0, residual_scale, h_out, st);
 }
