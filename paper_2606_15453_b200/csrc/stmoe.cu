@@ -40,6 +40,10 @@ constexpr int kWaitTimeoutMs = 20000;
 inline int dtype_bytes(int dt) { return dt == STMOE_F32 ? 4 : dt == STMOE_BF16 ? 2 : 1; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// the down projection's rows are cut into segments of at most 16 KB so that the last block a
+// warp claims stays short
+int down_splits(int I, int dt) { return (int)((((size_t)I * dtype_bytes(dt)) + 16383) / 16384); }
+
 size_t image_bytes(int H, int I, int dt)
 {
     size_t n = 3 * (size_t)H * I * dtype_bytes(dt);
@@ -55,8 +59,9 @@ struct FfnPlan {
 };
 
 template <int DT, int MT> struct Shape;
-template <int DT> struct Shape<DT, 1> { static constexpr int RG = 4, UG = 2, RD = 8, UD = 2; };
+template <int DT> struct Shape<DT, 1> { static constexpr int RG = 2, UG = 4, RD = 4, UD = 4; };
 template <int DT> struct Shape<DT, 4> { static constexpr int RG = 2, UG = 2, RD = 4, UD = 2; };
+template <> struct Shape<2, 4> { static constexpr int RG = 2, UG = 1, RD = 2, UD = 2; };
 
 template <int DT, int MT> void launch_gate_up(const FfnArgs &a, int grid, cudaStream_t st)
 {
@@ -125,8 +130,8 @@ FfnPlan make_plan(int dt, int mt)
 {
     FfnPlan p;
     const int sms = sm_count();
-    p.grid_gate_up = sms * std::max(1, std::min(occ_gate_up(dt, mt), 4));
-    p.grid_down = sms * std::max(1, std::min(occ_down(dt, mt), 4));
+    p.grid_gate_up = sms * std::max(1, std::min(occ_gate_up(dt, mt), 1));
+    p.grid_down = sms * std::max(1, std::min(occ_down(dt, mt), 1));
     return p;
 }
 
@@ -237,6 +242,7 @@ struct stmoe {
     int rdt = 0;          // router dtype
     int KS = 0;           // K + n_shared
     int max_pred = 0;
+    int S = 1;            // column splits of the down projection
     size_t img_bytes = 0;
     int next_layer = 0;
     int64_t host_t = 0;
@@ -492,7 +498,7 @@ int run_ffn(stmoe *s, int dt, int mt, const FfnPlan &plan, const FfnArgs &fa, co
     if (s) s->launches += 3;
     const int n = B * fa.H;
     combine_kernel<<<std::min((n + 255) / 256, 4096), 256, 0, st>>>(fa.h, fa.part, w, B, fa.H, K, n_shared,
-                                                                   rscale, h_out);
+                                                                   fa.S, rscale, h_out);
     CU_TRY(cudaGetLastError());
     return STMOE_OK;
 }
@@ -523,7 +529,7 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
 
     FfnArgs fa{};
     fa.h = h_in, fa.inv_rms = s->d_inv, fa.wl = s->wlm.wl;
-    fa.act = s->d_act, fa.part = s->d_part, fa.H = H, fa.I = c.inter, fa.E = E;
+    fa.act = s->d_act, fa.part = s->d_part, fa.H = H, fa.I = c.inter, fa.E = E, fa.S = s->S;
     if (offloaded(s)) {
         ST_TRY(cache_step(s, layer, batch, st));
         fa.blob = s->d_blob_table;
@@ -611,6 +617,7 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
     s->KS = c.top_k + c.n_shared;
     s->max_pred = std::min(c.n_experts, c.top_k * c.top_k + c.top_k);
     s->img_bytes = image_bytes(c.hidden, c.inter, c.weight_dtype);
+    s->S = down_splits(c.inter, c.weight_dtype);
     const int L = c.n_layers, E = c.n_experts, K = c.top_k, B = c.max_batch, H = c.hidden, I = c.inter;
     const size_t pairs = L > 1 ? L - 1 : 0;
 
@@ -672,7 +679,7 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
     CR_TRY(cudaMalloc(&s->d_logits, sizeof(float) * B * E));
     CR_TRY(cudaMalloc(&s->d_w, sizeof(float) * B * K));
     CR_TRY(cudaMalloc(&s->d_act, sizeof(float) * (size_t)B * s->KS * I));
-    CR_TRY(cudaMalloc(&s->d_part, sizeof(float) * (size_t)B * s->KS * H));
+    CR_TRY(cudaMalloc(&s->d_part, sizeof(float) * (size_t)B * s->KS * s->S * H));
     CR_TRY(cudaMalloc(&s->d_ids, sizeof(int32_t) * (size_t)L * B * K));
     CR_TRY(cudaMalloc(&s->d_queue, sizeof(int32_t) * (1 + 2 * E)));
     CR_TRY(cudaMemset(s->d_queue, 0, sizeof(int32_t) * (1 + 2 * E)));
@@ -896,19 +903,19 @@ size_t stmoe_expert_image_bytes(int hidden, int inter, int weight_dtype)
 }
 
 // scratch layout: work list | blob table | act | part
-static size_t ffn_scratch_layout(int B, int K, int H, int I, int E, size_t *o_tab, size_t *o_act, size_t *o_part)
+static size_t ffn_scratch_layout(int B, int K, int H, int I, int E, int S, size_t *o_tab, size_t *o_act, size_t *o_part)
 {
     size_t o = round_up(sizeof(int) * (size_t)(4 + 5 * B * K), 256);
     *o_tab = o, o += round_up(sizeof(void *) * (size_t)E, 256);
     *o_act = o, o += round_up(sizeof(float) * (size_t)B * K * I, 256);
-    *o_part = o, o += round_up(sizeof(float) * (size_t)B * K * H, 256);
+    *o_part = o, o += round_up(sizeof(float) * (size_t)B * K * S * H, 256);
     return o;
 }
 
 size_t stmoe_moe_ffn_scratch_bytes(int batch, int top_k, int hidden, int inter)
 {
     size_t a, b, c;
-    return ffn_scratch_layout(batch, top_k, hidden, inter, kMaxExperts, &a, &b, &c);
+    return ffn_scratch_layout(batch, top_k, hidden, inter, kMaxExperts, down_splits(inter, STMOE_F32), &a, &b, &c);
 }
 
 }  // extern "C"
@@ -955,7 +962,8 @@ extern "C" int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t
         ((uintptr_t)scratch & 255))
         return STMOE_ERR_BAD_ARG;
     size_t o_tab, o_act, o_part;
-    if (scratch_bytes < ffn_scratch_layout(batch, top_k, hidden, inter, kMaxExperts, &o_tab, &o_act, &o_part))
+    const int S = down_splits(inter, weight_dtype);
+    if (scratch_bytes < ffn_scratch_layout(batch, top_k, hidden, inter, kMaxExperts, down_splits(inter, STMOE_F32), &o_tab, &o_act, &o_part))
         return STMOE_ERR_BAD_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     uint8_t *sc = (uint8_t *)scratch;
@@ -968,7 +976,7 @@ extern "C" int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t
     FfnArgs fa{};
     fa.h = h, fa.inv_rms = inv_rms, fa.wl = wlm.wl, fa.blob = table;
     fa.act = (float *)(sc + o_act), fa.part = (float *)(sc + o_part);
-    fa.H = hidden, fa.I = inter, fa.E = n_experts;
+    fa.H = hidden, fa.I = inter, fa.E = n_experts, fa.S = S;
     static FfnPlan plans[3][2];
     FfnPlan &plan = plans[weight_dtype][mt == 1 ? 0 : 1];
     if (plan.grid_down == 0) plan = make_plan(weight_dtype, mt);
