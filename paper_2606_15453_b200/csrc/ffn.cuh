@@ -27,7 +27,15 @@ struct FfnArgs {
     float *part;             // [B*(K+n_shared)][S][H]
     int H, I, E;
     int S;                   // column splits of the down projection
+    // fused weighted sum + residual (done by whichever warp completes a 32-row tile last)
+    const float *w;          // [B][K] gate weights
+    float *h_out;            // [B][H]
+    unsigned *tile_done;     // [ceil(H/32)] rows finished per tile, zero between launches
+    int B, K, n_shared;
+    float residual_scale;
 };
+
+constexpr int kTileRows = 32;
 
 // Layout of one expert image.
 __host__ __device__ inline size_t image_gate(int, int, int) { return 0; }
@@ -216,32 +224,44 @@ __global__ void __launch_bounds__(kFfnThreads, 1) down_kernel(FfnArgs a)
                         a.part[((size_t)slot[t] * S + s) * H + r0 + r] = v;
                     }
                 }
+            // publish the rows; the warp that completes a tile sums it up (fixed order)
+            __threadfence();
+            __syncwarp();
+            const int want_per_row = *a.wl.n_groups * S;
+            for (int rr = r0; rr < r0 + nrows;) {
+                const int tile = rr / kTileRows;
+                const int n = min(r0 + nrows, (tile + 1) * kTileRows) - rr;
+                const int tile_rows = min(kTileRows, H - tile * kTileRows);
+                unsigned prev = 0;
+                if (lane == 0) prev = atomicAdd(a.tile_done + tile, (unsigned)n);
+                prev = __shfl_sync(kFull, prev, 0);
+                if (prev + n == (unsigned)(want_per_row * tile_rows)) {
+                    __threadfence();
+                    if (lane == 0) a.tile_done[tile] = 0u;
+                    const int c = tile * kTileRows + lane;
+                    if (lane < tile_rows) {
+                        const int KS = a.K + a.n_shared;
+                        for (int b = 0; b < a.B; ++b) {
+                            float y = 0.f;
+                            for (int q = 0; q < a.n_shared; ++q) {
+                                float p = 0.f;
+                                for (int z = 0; z < S; ++z)
+                                    p += __ldcg(a.part + (((size_t)b * KS + a.K + q) * S + z) * H + c);
+                                y += p;
+                            }
+                            for (int k = 0; k < a.K; ++k) {
+                                float p = 0.f;
+                                for (int z = 0; z < S; ++z)
+                                    p += __ldcg(a.part + (((size_t)b * KS + k) * S + z) * H + c);
+                                y = fmaf(a.w[b * a.K + k], p, y);
+                            }
+                            a.h_out[(size_t)b * H + c] = fmaf(a.residual_scale, y, a.h[(size_t)b * H + c]);
+                        }
+                    }
+                }
+                rr += n;
+            }
         }
-    }
-}
-
-// h_out[b][i] = h[b][i] + r * ( sum_shared part + sum_k w[b][k] * part ), fixed order; the
-// column splits of each partial are summed first, also in index order.
-__global__ void __launch_bounds__(256)
-combine_kernel(const float *__restrict__ h, const float *__restrict__ part, const float *__restrict__ w,
-               int B, int H, int K, int n_shared, int S, float residual_scale, float *__restrict__ h_out)
-{
-    const int KS = K + n_shared;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)B * H;
-         i += (size_t)gridDim.x * blockDim.x) {
-        const int b = (int)(i / H), c = (int)(i % H);
-        float y = 0.f;
-        for (int s = 0; s < n_shared; ++s) {
-            float p = 0.f;
-            for (int q = 0; q < S; ++q) p += part[(((size_t)b * KS + K + s) * S + q) * H + c];
-            y += p;
-        }
-        for (int k = 0; k < K; ++k) {
-            float p = 0.f;
-            for (int q = 0; q < S; ++q) p += part[(((size_t)b * KS + k) * S + q) * H + c];
-            y = fmaf(w[b * K + k], p, y);
-        }
-        h_out[i] = fmaf(residual_scale, y, h[i]);
     }
 }
 

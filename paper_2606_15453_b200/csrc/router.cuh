@@ -92,138 +92,264 @@ struct TopkArgs {
     WorkList wl;      // wl.n_groups == nullptr: no grouping
 };
 
-// softmax + top-K (K rounds of warp arg-max on (logit, lower id first) keys, one more round
-// for the K-th/(K+1)-th gap), then grouping by expert.  One CTA, one warp per sequence.
-__global__ void __launch_bounds__(256) topk_group_kernel(TopkArgs a)
+constexpr int kVpl = kMaxExperts / kWarp;  // logits held per lane
+
+// softmax + top-K for one sequence, by one warp.  Lane l holds the logits of experts
+// l, l+32, ... in z[].  K rounds of warp arg-max on (logit, lower id first) keys, one more
+// round for the K-th/(K+1)-th gap; ids are emitted in ascending order with w = softmax(z)[id].
+__device__ __forceinline__ void route_token(const float (&z)[kVpl], float *s_zrow, int *s_ids_row,
+                                            const TopkArgs &a, int b, int lane)
 {
-    constexpr int NW = 8, VPL = kMaxExperts / kWarp;
-    __shared__ float s_z[NW][kMaxExperts];
-    __shared__ int s_ids[kMaxBatch * kMaxTopK];
-    __shared__ int s_scan_g[kMaxExperts + 1], s_scan_p[kMaxExperts + 1];
-    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
     const int E = a.E, K = a.K;
-
-    for (int b = warp; b < a.B; b += NW) {
-        float z[VPL];
-        float m = -INFINITY;
+    float m = -INFINITY;
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) {
+    for (int v = 0; v < kVpl; ++v) {
+        const int j = v * kWarp + lane;
+        if (j < E) s_zrow[j] = z[v];
+        m = fmaxf(m, z[v]);
+    }
+    m = warp_max(m);
+    float sum = 0.f;
+#pragma unroll
+    for (int v = 0; v < kVpl; ++v)
+        if (v * kWarp + lane < E) sum += expf(z[v] - m);
+    sum = warp_sum(sum);
+    __syncwarp();
+
+    uint32_t taken = 0;  // bit v: my value v is selected
+    float kth = 0.f, gap = INFINITY;
+    for (int r = 0; r <= K && r < E; ++r) {
+        unsigned long long best = 0;
+#pragma unroll
+        for (int v = 0; v < kVpl; ++v) {
             const int j = v * kWarp + lane;
-            z[v] = j < E ? a.logits[(size_t)b * E + j] : -INFINITY;
-            if (j < E) s_z[warp][j] = z[v];
-            m = fmaxf(m, z[v]);
-        }
-        m = warp_max(m);
-        float sum = 0.f;
-#pragma unroll
-        for (int v = 0; v < VPL; ++v)
-            if (v * kWarp + lane < E) sum += expf(z[v] - m);
-        sum = warp_sum(sum);
-        __syncwarp();
-
-        uint32_t taken = 0;  // bit v: my value v is selected
-        float kth = 0.f, gap = INFINITY;
-        for (int r = 0; r <= K && r < E; ++r) {
-            unsigned long long best = 0;
-#pragma unroll
-            for (int v = 0; v < VPL; ++v) {
-                const int j = v * kWarp + lane;
-                if (j < E && !((taken >> v) & 1u)) {
-                    const unsigned long long key =
-                        ((unsigned long long)float_key(z[v]) << 32) | (uint32_t)(0xffffffffu - j);
-                    best = key > best ? key : best;
-                }
-            }
-            best = warp_max_u64(best);
-            const int j = (int)(0xffffffffu - (uint32_t)best);
-            if (r < K) {
-                if (j % kWarp == lane) taken |= 1u << (j / kWarp);
-                kth = s_z[warp][j];
-            } else {
-                gap = kth - s_z[warp][j];
+            if (j < E && !((taken >> v) & 1u)) {
+                const unsigned long long key =
+                    ((unsigned long long)float_key(z[v]) << 32) | (uint32_t)(0xffffffffu - j);
+                best = key > best ? key : best;
             }
         }
-
-        float sel = 0.f;
-#pragma unroll
-        for (int v = 0; v < VPL; ++v)
-            if ((taken >> v) & 1u) sel += expf(z[v] - m);
-        sel = warp_sum(sel);
-        const float denom = a.renorm ? sel : sum;
-        int base = 0;
-#pragma unroll
-        for (int v = 0; v < VPL; ++v) {
-            const unsigned msk = __ballot_sync(kFull, (taken >> v) & 1u);
-            if ((taken >> v) & 1u) {
-                const int pos = base + __popc(msk & ((1u << lane) - 1u));
-                const int j = v * kWarp + lane;
-                const float p = expf(z[v] - m) / denom;
-                a.ids[(size_t)b * K + pos] = j;
-                a.w[(size_t)b * K + pos] = p;
-                s_ids[b * K + pos] = j;
-                if (a.ids_out) a.ids_out[(size_t)b * K + pos] = j;
-                if (a.w_out) a.w_out[(size_t)b * K + pos] = p;
-            }
-            base += __popc(msk);
-        }
-        if (lane == 0) {
-            const uint32_t f = gap < 1e-4f ? 1u : 0u;
-            if (a.flags_out) a.flags_out[b] = f;
-            if (f && a.near_tie_counter) atomicAdd(a.near_tie_counter, 1ull);
+        best = warp_max_u64(best);
+        const int j = (int)(0xffffffffu - (uint32_t)best);
+        if (r < K) {
+            if (j % kWarp == lane) taken |= 1u << (j / kWarp);
+            kth = s_zrow[j];
+        } else {
+            gap = kth - s_zrow[j];
         }
     }
-    if (a.wl.n_groups == nullptr) return;
-    __syncthreads();
 
-    // grouping: thread e owns expert e
-    const int e = threadIdx.x, KS = K + a.n_shared, mt = a.mt;
+    float sel = 0.f;
+#pragma unroll
+    for (int v = 0; v < kVpl; ++v)
+        if ((taken >> v) & 1u) sel += expf(z[v] - m);
+    sel = warp_sum(sel);
+    const float denom = a.renorm ? sel : sum;
+    int base = 0;
+#pragma unroll
+    for (int v = 0; v < kVpl; ++v) {
+        const unsigned msk = __ballot_sync(kFull, (taken >> v) & 1u);
+        if ((taken >> v) & 1u) {
+            const int pos = base + __popc(msk & ((1u << lane) - 1u));
+            const int j = v * kWarp + lane;
+            const float p = expf(z[v] - m) / denom;
+            a.ids[(size_t)b * K + pos] = j;
+            a.w[(size_t)b * K + pos] = p;
+            s_ids_row[pos] = j;
+            if (a.ids_out) a.ids_out[(size_t)b * K + pos] = j;
+            if (a.w_out) a.w_out[(size_t)b * K + pos] = p;
+        }
+        base += __popc(msk);
+    }
+    if (lane == 0) {
+        const uint32_t f = gap < 1e-4f ? 1u : 0u;
+        if (a.flags_out) a.flags_out[b] = f;
+        if (f && a.near_tie_counter) atomicAdd(a.near_tie_counter, 1ull);
+    }
+    __syncwarp();
+}
+
+// Grouping of the batch's routed pairs by expert (256 threads, thread e owns expert e):
+// entries of at most mt tokens in ascending expert order, then the shared experts.
+// s_ids: [B*K] routed ids; s_scan: 2*(kMaxExperts+1) ints of scratch.
+__device__ __forceinline__ void group_tokens(const int *s_ids, int *s_scan, int B, int E, int K, int n_shared,
+                                             int mt, const WorkList &wl)
+{
+    int *s_g = s_scan, *s_p = s_scan + kMaxExperts + 1;
+    const int e = threadIdx.x, KS = K + n_shared, lane = e % kWarp, warp = e / kWarp;
     int cnt = 0;
     if (e < E)
-        for (int i = 0; i < a.B * K; ++i) cnt += (s_ids[i] == e);
-    if (e < kMaxExperts) {
-        s_scan_g[e + 1] = (cnt + mt - 1) / mt;
-        s_scan_p[e + 1] = cnt;
+        for (int i = 0; i < B * K; ++i) cnt += (s_ids[i] == e);
+    // exclusive scans of (entries, pairs) over the 256 experts
+    int g_inc = (cnt + mt - 1) / mt, p_inc = cnt;
+#pragma unroll
+    for (int o = 1; o < kWarp; o <<= 1) {
+        const int tg = __shfl_up_sync(kFull, g_inc, o), tp = __shfl_up_sync(kFull, p_inc, o);
+        if (lane >= o) g_inc += tg, p_inc += tp;
     }
-    if (e == 0) s_scan_g[0] = s_scan_p[0] = 0;
+    if (lane == kWarp - 1) s_g[warp] = g_inc, s_p[warp] = p_inc;
     __syncthreads();
-    if (threadIdx.x == 0)
-        for (int i = 1; i <= kMaxExperts; ++i) {
-            s_scan_g[i] += s_scan_g[i - 1];
-            s_scan_p[i] += s_scan_p[i - 1];
-        }
-    __syncthreads();
+    int g0 = g_inc - (cnt + mt - 1) / mt, p0 = p_inc - cnt, g_all = 0;
+    for (int wi = 0; wi < kMaxExperts / kWarp; ++wi) {
+        if (wi < warp) g0 += s_g[wi], p0 += s_p[wi];
+        g_all += s_g[wi];
+    }
     if (e < E && cnt > 0) {
-        const int g0 = s_scan_g[e], p0 = s_scan_p[e];
         for (int t = 0, g = g0; t < cnt; t += mt, ++g) {
-            a.wl.g_expert[g] = e;
-            a.wl.g_start[g] = p0 + t;
-            a.wl.g_count[g] = min(mt, cnt - t);
+            wl.g_expert[g] = e;
+            wl.g_start[g] = p0 + t;
+            wl.g_count[g] = min(mt, cnt - t);
         }
         int n = 0;
-        for (int i = 0; i < a.B * K; ++i)
+        for (int i = 0; i < B * K; ++i)
             if (s_ids[i] == e) {
-                const int b = i / K, k = i % K;
-                a.wl.pair_token[p0 + n] = b;
-                a.wl.pair_slot[p0 + n] = b * KS + k;
+                wl.pair_token[p0 + n] = i / K;
+                wl.pair_slot[p0 + n] = (i / K) * KS + i % K;
                 ++n;
             }
     }
-    const int routed_groups = s_scan_g[kMaxExperts];
-    const int tiles = (a.B + mt - 1) / mt;
-    if (e < a.n_shared) {
-        const int p0 = a.B * K + e * a.B;
+    const int tiles = (B + mt - 1) / mt;
+    if (e < n_shared) {
+        const int ps = B * K + e * B;
         for (int t = 0; t < tiles; ++t) {
-            const int g = routed_groups + e * tiles + t;
-            a.wl.g_expert[g] = E + e;
-            a.wl.g_start[g] = p0 + t * mt;
-            a.wl.g_count[g] = min(mt, a.B - t * mt);
+            const int g = g_all + e * tiles + t;
+            wl.g_expert[g] = E + e;
+            wl.g_start[g] = ps + t * mt;
+            wl.g_count[g] = min(mt, B - t * mt);
         }
-        for (int b = 0; b < a.B; ++b) {
-            a.wl.pair_token[p0 + b] = b;
-            a.wl.pair_slot[p0 + b] = b * KS + K + e;
+        for (int b = 0; b < B; ++b) {
+            wl.pair_token[ps + b] = b;
+            wl.pair_slot[ps + b] = b * KS + K + e;
         }
     }
-    if (threadIdx.x == 0) *a.wl.n_groups = routed_groups + a.n_shared * tiles;
+    if (threadIdx.x == 0) *wl.n_groups = g_all + n_shared * tiles;
+}
+
+// Stand-alone softmax/top-K/grouping over ready logits.  One CTA, one warp per sequence.
+__global__ void __launch_bounds__(256) topk_group_kernel(TopkArgs a)
+{
+    constexpr int NW = 8;
+    __shared__ float s_z[NW][kMaxExperts];
+    __shared__ int s_ids[kMaxBatch * kMaxTopK];
+    __shared__ int s_scan[2 * (kMaxExperts + 1)];
+    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
+    for (int b = warp; b < a.B; b += NW) {
+        float z[kVpl];
+#pragma unroll
+        for (int v = 0; v < kVpl; ++v) {
+            const int j = v * kWarp + lane;
+            z[v] = j < a.E ? a.logits[(size_t)b * a.E + j] : -INFINITY;
+        }
+        route_token(z, s_z[warp], s_ids + b * a.K, a, b, lane);
+    }
+    if (a.wl.n_groups == nullptr) return;
+    __syncthreads();
+    group_tokens(s_ids, s_scan, a.B, a.E, a.K, a.n_shared, a.mt, a.wl);
+}
+
+// ---- the whole gating network in one launch -------------------------------------------------
+// Split-K router GEMV over many CTAs (one warp per (expert row, column chunk), all of its
+// loads issued up front), partial logits and partial sums of squares to global memory; the
+// CTA that arrives last (arrival counter, no waiting) sums them in a fixed order, applies the
+// RMSNorm factor and runs softmax / top-K / grouping.
+constexpr int kRouterUnroll = 4;
+
+struct RouterArgs {
+    const float *h;      // [B][H]
+    const uint8_t *W;    // [E][H]
+    int H;
+    float eps;
+    float *part;         // [C][B][E] partial logits, C = column chunks
+    float *ss_part;      // [C][B] partial sums of squares
+    unsigned *arrivals;  // [1], zero between launches
+    float *inv_rms;      // [B]
+    float *logits_out;   // optional [B][E]
+    TopkArgs tk;         // tk.logits unused
+};
+
+template <int DT> __host__ __device__ constexpr int router_chunk_cols()
+{
+    return kWarp * Fmt<DT>::kEpl * kRouterUnroll;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(256) router_fused_kernel(RouterArgs a)
+{
+    constexpr int EPL = Fmt<DT>::kEpl, BYTES = Fmt<DT>::kBytes, CH = router_chunk_cols<DT>(), NW = 8;
+    __shared__ float s_z[NW][kMaxExperts];
+    __shared__ int s_ids[kMaxBatch * kMaxTopK];
+    __shared__ int s_scan[2 * (kMaxExperts + 1)];
+    __shared__ int s_last;
+    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
+    const int B = a.tk.B, E = a.tk.E, H = a.H;
+    const int C = (H + CH - 1) / CH;
+
+    const int task = blockIdx.x * NW + warp;
+    if (task < E * C) {
+        const int j = task / C, c = task % C;
+        const uint8_t *row = a.W + (size_t)j * H * BYTES;
+        float wf[kRouterUnroll][EPL];
+#pragma unroll
+        for (int u = 0; u < kRouterUnroll; ++u) {
+            const int k = c * CH + (u * kWarp + lane) * EPL;
+            if (k < H) {
+                Fmt<DT>::unpack(ld_stream16(row + (size_t)k * BYTES), wf[u]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) wf[u][e] = 0.f;
+            }
+        }
+        for (int b = 0; b < B; ++b) {
+            float acc = 0.f, ss = 0.f;
+#pragma unroll
+            for (int u = 0; u < kRouterUnroll; ++u) {
+                const int k = c * CH + (u * kWarp + lane) * EPL;
+                if (k < H) {
+#pragma unroll
+                    for (int e = 0; e < EPL; e += 4) {
+                        const float4 v = ld_f4(a.h + (size_t)b * H + k + e);
+                        acc = fmaf(wf[u][e], v.x, acc), acc = fmaf(wf[u][e + 1], v.y, acc);
+                        acc = fmaf(wf[u][e + 2], v.z, acc), acc = fmaf(wf[u][e + 3], v.w, acc);
+                        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+                    }
+                }
+            }
+            acc = warp_sum(acc);
+            if (j == 0) ss = warp_sum(ss);
+            if (lane == 0) {
+                a.part[((size_t)c * B + b) * E + j] = acc;
+                if (j == 0) a.ss_part[c * B + b] = ss;
+            }
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(a.arrivals, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (threadIdx.x == 0) *a.arrivals = 0u;
+
+    for (int b = warp; b < B; b += NW) {
+        float ss = 0.f;
+        for (int c = 0; c < C; ++c) ss += __ldcg(a.ss_part + c * B + b);
+        const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
+        if (lane == 0) a.inv_rms[b] = inv;
+        float z[kVpl];
+#pragma unroll
+        for (int v = 0; v < kVpl; ++v) {
+            const int j = v * kWarp + lane;
+            float s = 0.f;
+            if (j < E)
+                for (int c = 0; c < C; ++c) s += __ldcg(a.part + ((size_t)c * B + b) * E + j);
+            z[v] = j < E ? s * inv : -INFINITY;
+            if (j < E && a.logits_out) a.logits_out[(size_t)b * E + j] = z[v];
+        }
+        route_token(z, s_z[warp], s_ids + b * a.tk.K, a.tk, b, lane);
+    }
+    if (a.tk.wl.n_groups == nullptr) return;
+    __syncthreads();
+    group_tokens(s_ids, s_scan, B, E, a.tk.K, a.tk.n_shared, a.tk.mt, a.tk.wl);
 }
 
 }  // namespace stmoe_dev

@@ -257,12 +257,25 @@ struct stmoe {
     const uint8_t **h_blob_table = nullptr;  // pinned staging of one step's table
 
     PredState pst{};
+    float *d_rpart = nullptr, *d_sspart = nullptr;
+    unsigned *d_arrivals = nullptr, *d_tile_done = nullptr;
     float *d_inv = nullptr, *d_logits = nullptr, *d_w = nullptr, *d_act = nullptr, *d_part = nullptr;
     int32_t *d_ids = nullptr;   // [L][B][K] routing of the current decode step
     int32_t *d_queue = nullptr; // [1 + 2E]
     int32_t *h_ids = nullptr, *h_queue = nullptr;  // pinned mirrors
     WorkListMem wlm;
     FfnPlan plan1, plan4;
+
+    cudaStream_t side_stream = nullptr;   // predictor kernels of resident stacks
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    bool side_pending = false;
+    // one decode step of a resident stack captured as a CUDA graph, replayed while the
+    // caller keeps passing the same buffers
+    cudaGraphExec_t graph_exec = nullptr;
+    const void *graph_key[9] = {};
+    int64_t graph_launches = 0;
+    int graph_captures = 0;
+    bool graph_off = false;
 
     SlotCache cache;
     cudaStream_t copy_stream = nullptr;
@@ -475,8 +488,7 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
     return STMOE_OK;
 }
 
-int run_ffn(stmoe *s, int dt, int mt, const FfnPlan &plan, const FfnArgs &fa, const float *w, int B, int K,
-            int n_shared, float rscale, float *h_out, cudaStream_t st)
+int run_ffn(stmoe *s, int dt, int mt, const FfnPlan &plan, const FfnArgs &fa, cudaStream_t st)
 {
     cudaEvent_t e0 = nullptr, e1 = nullptr, e2 = nullptr;
     const bool timed = s && s->time_kernels;
@@ -495,10 +507,7 @@ int run_ffn(stmoe *s, int dt, int mt, const FfnPlan &plan, const FfnArgs &fa, co
         s->spans.push_back(TimedSpan{e1, e2, 3});
         s->timed_ffn += 1;
     }
-    if (s) s->launches += 3;
-    const int n = B * fa.H;
-    combine_kernel<<<std::min((n + 255) / 256, 4096), 256, 0, st>>>(fa.h, fa.part, w, B, fa.H, K, n_shared,
-                                                                   fa.S, rscale, h_out);
+    if (s) s->launches += 2;
     CU_TRY(cudaGetLastError());
     return STMOE_OK;
 }
@@ -513,32 +522,72 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
     int32_t *ids = s->d_ids + (size_t)layer * c.max_batch * K;
     const int32_t *prev = layer > 0 ? s->d_ids + (size_t)(layer - 1) * c.max_batch * K : nullptr;
 
-    launch_router_logits(s->rdt, h_in, s->d_router + (size_t)layer * E * H * dtype_bytes(s->rdt), batch, E, H,
-                         c.rms_eps, s->d_inv, s->d_logits, st);
-    TopkArgs ta{};
-    ta.logits = s->d_logits;
+    RouterArgs ra{};
+    ra.h = h_in, ra.W = s->d_router + (size_t)layer * E * H * dtype_bytes(s->rdt), ra.H = H, ra.eps = c.rms_eps;
+    ra.part = s->d_rpart, ra.ss_part = s->d_sspart, ra.arrivals = s->d_arrivals, ra.inv_rms = s->d_inv;
+    TopkArgs &ta = ra.tk;
     ta.B = batch, ta.E = E, ta.K = K, ta.n_shared = c.n_shared, ta.mt = mt;
     ta.renorm = (c.flags & STMOE_FLAG_RENORM_TOPK) ? 1 : 0;
     ta.ids = ids, ta.w = s->d_w;
     ta.ids_out = routed_ids, ta.w_out = routed_w, ta.flags_out = flags;
     ta.near_tie_counter = s->pst.stats + 4;
     ta.wl = s->wlm.wl;
-    topk_group_kernel<<<1, 256, 0, st>>>(ta);
+    if (s->rdt == STMOE_F32) {
+        const int C = (H + router_chunk_cols<0>() - 1) / router_chunk_cols<0>();
+        router_fused_kernel<0><<<(E * C + 7) / 8, 256, 0, st>>>(ra);
+    } else {
+        const int C = (H + router_chunk_cols<1>() - 1) / router_chunk_cols<1>();
+        router_fused_kernel<1><<<(E * C + 7) / 8, 256, 0, st>>>(ra);
+    }
     CU_TRY(cudaGetLastError());
-    ST_TRY(launch_predictor(s, layer, batch, ids, prev, predicted_ids, n_predicted, offloaded(s), st));
+    if (offloaded(s))  // the host needs the prefetch queue before it can issue copies
+        ST_TRY(launch_predictor(s, layer, batch, ids, prev, predicted_ids, n_predicted, true, st));
 
     FfnArgs fa{};
     fa.h = h_in, fa.inv_rms = s->d_inv, fa.wl = s->wlm.wl;
     fa.act = s->d_act, fa.part = s->d_part, fa.H = H, fa.I = c.inter, fa.E = E, fa.S = s->S;
+    fa.w = s->d_w, fa.h_out = h_out, fa.tile_done = s->d_tile_done;
+    fa.B = batch, fa.K = K, fa.n_shared = c.n_shared, fa.residual_scale = c.residual_scale;
     if (offloaded(s)) {
         ST_TRY(cache_step(s, layer, batch, st));
         fa.blob = s->d_blob_table;
     } else {
         fa.blob = s->d_blob_table + (size_t)layer * (E + c.n_shared);
     }
-    s->launches += 2;
-    return run_ffn(s, c.weight_dtype, mt, mt == 1 ? s->plan1 : s->plan4, fa, s->d_w, batch, K, c.n_shared,
-                   c.residual_scale, h_out, st);
+    s->launches += 1;
+    ST_TRY(run_ffn(s, c.weight_dtype, mt, mt == 1 ? s->plan1 : s->plan4, fa, st));
+    if (!offloaded(s)) {
+        // resident: nothing in the step depends on the predictor, so it runs on a side stream
+        // once the FFN kernels (which fill every SM) are done, beside the next layer's router
+        CU_TRY(cudaEventRecord(s->ev_fork, st));
+        CU_TRY(cudaStreamWaitEvent(s->side_stream, s->ev_fork, 0));
+        ST_TRY(launch_predictor(s, layer, batch, ids, prev, predicted_ids, n_predicted, false, s->side_stream));
+        s->side_pending = true;
+    }
+    return STMOE_OK;
+}
+
+int join_side(stmoe *s, cudaStream_t st)
+{
+    if (!s->side_pending) return STMOE_OK;
+    CU_TRY(cudaEventRecord(s->ev_join, s->side_stream));
+    CU_TRY(cudaStreamWaitEvent(st, s->ev_join, 0));
+    s->side_pending = false;
+    return STMOE_OK;
+}
+
+int token_eager(stmoe *s, int batch, const float *h_in, float *h_out, int32_t *routed_ids, float *routed_w,
+                int32_t *predicted_ids, int32_t *n_predicted, uint32_t *flags, cudaStream_t st)
+{
+    const int K = s->cfg.top_k;
+    for (int l = 0; l < s->cfg.n_layers; ++l) {
+        const size_t o = (size_t)l * batch;
+        ST_TRY(layer_step(s, l, batch, l == 0 ? h_in : h_out, h_out, routed_ids ? routed_ids + o * K : nullptr,
+                          routed_w ? routed_w + o * K : nullptr,
+                          predicted_ids ? predicted_ids + o * s->max_pred : nullptr,
+                          n_predicted ? n_predicted + o : nullptr, flags ? flags + o : nullptr, st));
+    }
+    return join_side(s, st);
 }
 
 size_t state_bytes(const stmoe_config_t &c)
@@ -575,10 +624,14 @@ int stmoe_destroy(stmoe_t *s)
     for (cudaEvent_t e : s->free_events) cudaEventDestroy(e);
     for (cudaEvent_t e : s->slot_ready) cudaEventDestroy(e);
     if (s->ev_route) cudaEventDestroy(s->ev_route);
+    if (s->graph_exec) cudaGraphExecDestroy(s->graph_exec);
+    if (s->ev_fork) cudaEventDestroy(s->ev_fork);
+    if (s->ev_join) cudaEventDestroy(s->ev_join);
+    if (s->side_stream) cudaStreamDestroy(s->side_stream);
     if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
     void *dev[] = {s->d_router, s->d_resident, s->d_shared, s->d_slots, (void *)s->d_blob_table,
                    s->pst.Co, s->pst.cct_id, s->pst.cct_conf, s->pst.HT, s->pst.t, s->pst.pred_mask,
-                   s->pst.pred_valid, s->pst.stats, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
+                   s->pst.pred_valid, s->pst.stats, s->d_rpart, s->d_sspart, s->d_arrivals, s->d_tile_done, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
                    s->d_ids, s->d_queue};
     for (void *p : dev)
         if (p) cudaFree(p);
@@ -635,6 +688,9 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
     } while (0)
 
     CR_TRY(cudaMalloc(&s->d_router, (size_t)L * E * H * dtype_bytes(s->rdt)));
+    CR_TRY(cudaStreamCreateWithFlags(&s->side_stream, cudaStreamNonBlocking));
+    CR_TRY(cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming));
+    CR_TRY(cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming));
     if (c.n_shared) CR_TRY(cudaMalloc(&s->d_shared, (size_t)L * c.n_shared * s->img_bytes));
     if (c.cache_slots > 0) {
         CR_TRY(cudaHostAlloc(&s->h_store, (size_t)L * E * s->img_bytes, cudaHostAllocDefault));
@@ -677,6 +733,16 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
     CR_TRY(cudaMemset(s->pst.stats, 0, 8 * 8));
     CR_TRY(cudaMalloc(&s->d_inv, sizeof(float) * B));
     CR_TRY(cudaMalloc(&s->d_logits, sizeof(float) * B * E));
+    {
+        const int ch = s->rdt == STMOE_F32 ? router_chunk_cols<0>() : router_chunk_cols<1>();
+        const int C = (H + ch - 1) / ch;
+        CR_TRY(cudaMalloc(&s->d_rpart, sizeof(float) * (size_t)C * B * E));
+        CR_TRY(cudaMalloc(&s->d_sspart, sizeof(float) * (size_t)C * B));
+        CR_TRY(cudaMalloc(&s->d_arrivals, 16));
+        CR_TRY(cudaMemset(s->d_arrivals, 0, 16));
+        CR_TRY(cudaMalloc(&s->d_tile_done, sizeof(unsigned) * ((H + kTileRows - 1) / kTileRows)));
+        CR_TRY(cudaMemset(s->d_tile_done, 0, sizeof(unsigned) * ((H + kTileRows - 1) / kTileRows)));
+    }
     CR_TRY(cudaMalloc(&s->d_w, sizeof(float) * B * K));
     CR_TRY(cudaMalloc(&s->d_act, sizeof(float) * (size_t)B * s->KS * I));
     CR_TRY(cudaMalloc(&s->d_part, sizeof(float) * (size_t)B * s->KS * s->S * H));
@@ -743,8 +809,9 @@ int stmoe_decode_step(stmoe_t *s, int layer, int batch, const float *h_in, float
     if (!s || !h_in || !h_out || batch < 1 || batch > s->cfg.max_batch || layer < 0 || layer >= s->cfg.n_layers)
         return STMOE_ERR_BAD_ARG;
     if (layer != s->next_layer) return STMOE_ERR_STATE;
-    const int rc = layer_step(s, layer, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted,
-                              flags, (cudaStream_t)cuda_stream);
+    int rc = layer_step(s, layer, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted,
+                        flags, (cudaStream_t)cuda_stream);
+    if (rc == STMOE_OK) rc = join_side(s, (cudaStream_t)cuda_stream);
     if (rc == STMOE_OK) s->next_layer = (layer + 1) % s->cfg.n_layers;
     return rc;
 }
@@ -755,15 +822,51 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, i
 {
     if (!s || !h_in || !h_out || batch < 1 || batch > s->cfg.max_batch) return STMOE_ERR_BAD_ARG;
     if (s->next_layer != 0) return STMOE_ERR_STATE;
-    const int K = s->cfg.top_k;
-    for (int l = 0; l < s->cfg.n_layers; ++l) {
-        const size_t o = (size_t)l * batch;
-        ST_TRY(layer_step(s, l, batch, l == 0 ? h_in : h_out, h_out, routed_ids ? routed_ids + o * K : nullptr,
-                          routed_w ? routed_w + o * K : nullptr,
-                          predicted_ids ? predicted_ids + o * s->max_pred : nullptr,
-                          n_predicted ? n_predicted + o : nullptr, flags ? flags + o : nullptr,
-                          (cudaStream_t)cuda_stream));
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const stmoe_config_t &c = s->cfg;
+    const bool build_due = !s->built && s->host_t == c.profile_tokens - 1;
+    if (offloaded(s) || s->time_kernels || s->graph_off || build_due)
+        return token_eager(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
+
+    const void *key[9] = {(const void *)(intptr_t)batch, h_in, h_out, routed_ids, routed_w, predicted_ids,
+                          n_predicted, flags, st};
+    if (s->graph_exec && memcmp(key, s->graph_key, sizeof(key)) == 0) {
+        CU_TRY(cudaGraphLaunch(s->graph_exec, st));
+        s->host_t += 1;
+        s->launches += s->graph_launches;
+        return STMOE_OK;
     }
+    if (s->graph_captures >= 16) {  // the caller keeps changing buffers: stop re-capturing
+        s->graph_off = true;
+        return token_eager(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
+    }
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        (void)cudaGetLastError();  // e.g. the legacy default stream cannot be captured
+        s->graph_off = true;
+        return token_eager(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
+    }
+    const int64_t before = s->launches;
+    const int rc = token_eager(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+    if (rc != STMOE_OK || ce != cudaSuccess || !graph) {
+        (void)cudaGetLastError();
+        if (graph) cudaGraphDestroy(graph);
+        s->graph_off = true;
+        return rc != STMOE_OK ? rc : STMOE_ERR_CUDA;
+    }
+    if (s->graph_exec) cudaGraphExecDestroy(s->graph_exec), s->graph_exec = nullptr;
+    const cudaError_t ie = cudaGraphInstantiate(&s->graph_exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ie != cudaSuccess) {
+        (void)cudaGetLastError();
+        s->graph_exec = nullptr, s->graph_off = true;
+        return STMOE_ERR_CUDA;
+    }
+    memcpy(s->graph_key, key, sizeof(key));
+    s->graph_launches = s->launches - before;
+    s->graph_captures += 1;
+    CU_TRY(cudaGraphLaunch(s->graph_exec, st));
     return STMOE_OK;
 }
 
@@ -903,19 +1006,21 @@ size_t stmoe_expert_image_bytes(int hidden, int inter, int weight_dtype)
 }
 
 // scratch layout: work list | blob table | act | part
-static size_t ffn_scratch_layout(int B, int K, int H, int I, int E, int S, size_t *o_tab, size_t *o_act, size_t *o_part)
+static size_t ffn_scratch_layout(int B, int K, int H, int I, int E, int S, size_t *o_tab, size_t *o_act, size_t *o_part,
+                                 size_t *o_tiles)
 {
     size_t o = round_up(sizeof(int) * (size_t)(4 + 5 * B * K), 256);
     *o_tab = o, o += round_up(sizeof(void *) * (size_t)E, 256);
     *o_act = o, o += round_up(sizeof(float) * (size_t)B * K * I, 256);
     *o_part = o, o += round_up(sizeof(float) * (size_t)B * K * S * H, 256);
+    *o_tiles = o, o += round_up(sizeof(unsigned) * (size_t)((H + kTileRows - 1) / kTileRows), 256);
     return o;
 }
 
 size_t stmoe_moe_ffn_scratch_bytes(int batch, int top_k, int hidden, int inter)
 {
-    size_t a, b, c;
-    return ffn_scratch_layout(batch, top_k, hidden, inter, kMaxExperts, down_splits(inter, STMOE_F32), &a, &b, &c);
+    size_t a, b, c, d;
+    return ffn_scratch_layout(batch, top_k, hidden, inter, kMaxExperts, down_splits(inter, STMOE_F32), &a, &b, &c, &d);
 }
 
 }  // extern "C"
@@ -925,8 +1030,9 @@ namespace {
 // fills the work list and the expert-image table of a stand-alone FFN call from given routing
 __global__ void __launch_bounds__(256)
 group_given_ids_kernel(const int32_t *ids, int B, int E, int K, int mt, WorkList wl, const uint8_t *experts,
-                       size_t img_bytes, const uint8_t **table)
+                       size_t img_bytes, const uint8_t **table, unsigned *tile_done, int n_tiles)
 {
+    for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) tile_done[i] = 0u;
     __shared__ int s_g[kMaxExperts + 1], s_p[kMaxExperts + 1];
     const int e = threadIdx.x;
     int cnt = 0;
@@ -961,9 +1067,9 @@ extern "C" int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t
         hidden % 16 || inter < 16 || inter % 16 || weight_dtype < STMOE_F32 || weight_dtype > STMOE_FP8_E4M3 ||
         ((uintptr_t)scratch & 255))
         return STMOE_ERR_BAD_ARG;
-    size_t o_tab, o_act, o_part;
+    size_t o_tab, o_act, o_part, o_tiles;
     const int S = down_splits(inter, weight_dtype);
-    if (scratch_bytes < ffn_scratch_layout(batch, top_k, hidden, inter, kMaxExperts, down_splits(inter, STMOE_F32), &o_tab, &o_act, &o_part))
+    if (scratch_bytes < ffn_scratch_layout(batch, top_k, hidden, inter, kMaxExperts, down_splits(inter, STMOE_F32), &o_tab, &o_act, &o_part, &o_tiles))
         return STMOE_ERR_BAD_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     uint8_t *sc = (uint8_t *)scratch;
@@ -972,13 +1078,16 @@ extern "C" int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t
     const int mt = batch == 1 ? 1 : 4;
     const uint8_t **table = (const uint8_t **)(sc + o_tab);
     group_given_ids_kernel<<<1, 256, 0, st>>>(ids, batch, n_experts, top_k, mt, wlm.wl, (const uint8_t *)experts,
-                                             image_bytes(hidden, inter, weight_dtype), table);
+                                             image_bytes(hidden, inter, weight_dtype), table,
+                                             (unsigned *)(sc + o_tiles), (hidden + kTileRows - 1) / kTileRows);
     FfnArgs fa{};
     fa.h = h, fa.inv_rms = inv_rms, fa.wl = wlm.wl, fa.blob = table;
     fa.act = (float *)(sc + o_act), fa.part = (float *)(sc + o_part);
     fa.H = hidden, fa.I = inter, fa.E = n_experts, fa.S = S;
+    fa.w = w, fa.h_out = h_out, fa.tile_done = (unsigned *)(sc + o_tiles);
+    fa.B = batch, fa.K = top_k, fa.n_shared = 0, fa.residual_scale = residual_scale;
     static FfnPlan plans[3][2];
     FfnPlan &plan = plans[weight_dtype][mt == 1 ? 0 : 1];
     if (plan.grid_down == 0) plan = make_plan(weight_dtype, mt);
-    return run_ffn(nullptr, weight_dtype, mt, plan, fa, w, batch, top_k, 0, residual_scale, h_out, st);
+    return run_ffn(nullptr, weight_dtype, mt, plan, fa, st);
 }

@@ -121,6 +121,38 @@ def test_tiny_cache_thrashes_but_stays_correct():
     assert st["prefetch_issued"] > 0
 
 
+def test_graph_replay_matches_eager_decode():
+    """decode_token on a capturable stream replays a CUDA graph; on the default stream it
+    launches kernel by kernel.  Outputs, routing, predictions and tables must be identical."""
+    cfg = stacks.CONFIGS["C2"].scaled(n_layers=3, hidden=512, inter=352, n_experts=16, top_k=3,
+                                      profile_tokens=3)
+    B, T = 4, 10
+    x = stacks.token_inputs(cfg, B, T).to(DEV)
+    results = []
+    for use_graph in (False, True):
+        pr = Pair(cfg, B, oracle=False)
+        L, K = cfg.n_layers, cfg.top_k
+        ids = torch.empty(L, B, K, dtype=torch.int32, device=DEV)
+        pred = torch.empty(L, B, pr.stack.max_pred, dtype=torch.int32, device=DEV)
+        h_in, ho = torch.empty(B, cfg.hidden, device=DEV), torch.empty(B, cfg.hidden, device=DEV)
+        stream = torch.cuda.Stream() if use_graph else torch.cuda.current_stream()
+        rec = []
+        with torch.cuda.stream(stream):
+            for t in range(T):
+                h_in.copy_(x[t])
+                pr.stack.decode_token(h_in, ho, ids, None, pred, None, stream=stream)
+                stream.synchronize()
+                rec.append((ho.cpu().clone(), ids.cpu().clone(), pred.cpu().clone()))
+        results.append((rec, pr.stack.export_state(), pr.stack.stats()))
+        pr.close()
+    (ra, sa, ta), (rb, sb, tb) = results
+    for a, b in zip(ra, rb):
+        assert all(torch.equal(u, v) for u, v in zip(a, b))
+    assert sa == sb
+    for k in ("runtime_steps", "routed", "predicted", "hits", "decode_steps", "kernel_launches"):
+        assert ta[k] == tb[k], k
+
+
 def test_argument_and_state_errors():
     with pytest.raises(P.StmoeError):
         P.Stack(2, 8, 2, 100, 64)                       # H not a multiple of 16
