@@ -15,7 +15,10 @@
 
 namespace stmoe_dev {
 
-constexpr int kFfnThreads = 512;
+#ifndef STMOE_FFN_THREADS
+#define STMOE_FFN_THREADS 512  // one CTA of 16 warps per SM
+#endif
+constexpr int kFfnThreads = STMOE_FFN_THREADS;
 constexpr int kFfnWarps = kFfnThreads / kWarp;
 
 struct FfnArgs {

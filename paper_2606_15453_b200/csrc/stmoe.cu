@@ -32,6 +32,18 @@ using namespace stmoe_dev;
         if (r_ != STMOE_OK) return r_; \
     } while (0)
 
+// Tile shapes of the batch-1 FFN kernels (rows per block, loads in flight per row) and the
+// longest row segment of the down projection; overridable for tuning builds.
+#ifndef STMOE_RG1
+#define STMOE_RG1 2
+#define STMOE_UG1 4
+#define STMOE_RD1 8
+#define STMOE_UD1 2
+#endif
+#ifndef STMOE_SEG_BYTES
+#define STMOE_SEG_BYTES 16384
+#endif
+
 namespace {
 
 constexpr uint32_t kStateMagic = 0x53544D50;
@@ -42,7 +54,10 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // the down projection's rows are cut into segments of at most 16 KB so that the last block a
 // warp claims stays short
-int down_splits(int I, int dt) { return (int)((((size_t)I * dtype_bytes(dt)) + 16383) / 16384); }
+int down_splits(int I, int dt)
+{
+    return (int)((((size_t)I * dtype_bytes(dt)) + STMOE_SEG_BYTES - 1) / STMOE_SEG_BYTES);
+}
 
 size_t image_bytes(int H, int I, int dt)
 {
@@ -59,7 +74,9 @@ struct FfnPlan {
 };
 
 template <int DT, int MT> struct Shape;
-template <int DT> struct Shape<DT, 1> { static constexpr int RG = 2, UG = 4, RD = 4, UD = 4; };
+template <int DT> struct Shape<DT, 1> {
+    static constexpr int RG = STMOE_RG1, UG = STMOE_UG1, RD = STMOE_RD1, UD = STMOE_UD1;
+};
 template <int DT> struct Shape<DT, 4> { static constexpr int RG = 2, UG = 2, RD = 4, UD = 2; };
 template <> struct Shape<2, 4> { static constexpr int RG = 2, UG = 1, RD = 2, UD = 2; };
 
