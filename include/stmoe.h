@@ -37,6 +37,7 @@ extern "C" {
 #define STMOE_ERR_TIMEOUT (-4)
 #define STMOE_ERR_STATE (-5)
 #define STMOE_ERR_UNIMPLEMENTED (-6)
+#define STMOE_ERR_TOO_LARGE (-7)
 
 /* weight_dtype */
 #define STMOE_F32 0
@@ -192,6 +193,26 @@ int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t *ids, cons
                   const void *experts, int weight_dtype, int batch, int n_experts, int top_k,
                   int hidden, int inter, float residual_scale, float *h_out, void *scratch,
                   size_t scratch_bytes, void *cuda_stream);
+
+/* stmoe_moe_ffn without a scratch argument and without any allocation (the paper has no
+ * counterpart; this serves hosts, not the method).  For callers that must not allocate device
+ * memory once they are running: serving loops where cudaMalloc could stall the device or fail
+ * because a framework already owns all of HBM, and plug-in hosts that forbid allocator calls.
+ * The work list, activations and partial sums live in an 8 MiB area built into the library
+ * image; each GPU that loads the library holds those 8 MiB until the process exits.
+ *   - Same arguments, layout and results as stmoe_moe_ffn; inputs and outputs stay with the
+ *     caller.  Calls no cudaMalloc/cudaFree or other allocating routine.
+ *   - Returns STMOE_ERR_TOO_LARGE when stmoe_moe_ffn_scratch_bytes(batch, top_k, hidden, inter)
+ *     exceeds 8 MiB (for example batch 64, top_k 8, hidden 4096, inter 14336).
+ *   - The first call on each device looks up the area's device address (with that device
+ *     current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one area, which keeps whatever the last call left; the
+ *     call clears the counters that must start at zero itself.  Two calls whose kernels can
+ *     overlap on the GPU (different streams, no ordering between them) race on it: order
+ *     them, or use stmoe_moe_ffn with separate scratch buffers. */
+int stmoe_moe_ffn_static(const float *h, const float *inv_rms, const int32_t *ids, const float *w,
+                         const void *experts, int weight_dtype, int batch, int n_experts, int top_k,
+                         int hidden, int inter, float residual_scale, float *h_out, void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -72,6 +72,7 @@ def lib():
         L.stmoe_moe_ffn_scratch_bytes.restype = sz
         L.stmoe_moe_ffn_scratch_bytes.argtypes = [i32, i32, i32, i32]
         L.stmoe_moe_ffn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, vp, vp, sz, vp]
+        L.stmoe_moe_ffn_static.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, vp, vp]
         _lib = L
     return _lib
 
@@ -220,4 +221,17 @@ def moe_ffn(h, inv_rms, ids, w, experts, dtype, n_experts, hidden, inter, residu
               _dev(experts), DTYPE[dtype], B, n_experts, K, hidden, inter, residual_scale,
               _dev(h_out, torch.float32), _dev(scratch), scratch.numel() * scratch.element_size(),
               _stream(stream)), entry)
+    return h_out
+
+
+def moe_ffn_static(h, inv_rms, ids, w, experts, dtype, n_experts, hidden, inter, residual_scale, h_out,
+                   stream=None):
+    """stmoe_moe_ffn_static: the same computation as moe_ffn for callers that must not allocate
+    device memory; scratch is an 8 MiB area inside the library, shared by every call on the
+    device (order calls that could overlap).  Raises StmoeError when the problem needs more."""
+    B, K = ids.shape
+    _check(lib().stmoe_moe_ffn_static(_dev(h, torch.float32), _ptr(inv_rms), _dev(ids, torch.int32),
+                                      _dev(w, torch.float32), _dev(experts), DTYPE[dtype], B, n_experts, K,
+                                      hidden, inter, residual_scale, _dev(h_out, torch.float32),
+                                      _stream(stream)), "stmoe_moe_ffn_static")
     return h_out

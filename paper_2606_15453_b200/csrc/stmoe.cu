@@ -629,6 +629,7 @@ const char *stmoe_strerror(int code)
     case STMOE_ERR_TIMEOUT: return "timed out waiting for the device";
     case STMOE_ERR_STATE: return "call out of order or inconsistent state";
     case STMOE_ERR_UNIMPLEMENTED: return "not implemented";
+    case STMOE_ERR_TOO_LARGE: return "problem exceeds the capacity of the built-in scratch area";
     default: return "unknown error";
     }
 }
@@ -1107,4 +1108,34 @@ extern "C" int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t
     FfnPlan &plan = plans[weight_dtype][mt == 1 ? 0 : 1];
     if (plan.grid_down == 0) plan = make_plan(weight_dtype, mt);
     return run_ffn(nullptr, weight_dtype, mt, plan, fa, st);
+}
+
+// ---- allocation-free variant of stmoe_moe_ffn ---------------------------------------------
+// Scratch for callers that may not allocate device memory lives in this library image: every
+// GPU that loads the library holds these bytes until the process exits.
+#define STMOE_STATIC_SCRATCH_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[STMOE_STATIC_SCRATCH_BYTES];
+// Device address of g_static_scratch per device ordinal.  In host code the array's name is
+// only a handle for the runtime, never a pointer a kernel may use, so the address is looked
+// up once per device with that device current.
+static void *g_static_scratch_ptr[64] = {};
+
+extern "C" int stmoe_moe_ffn_static(const float *h, const float *inv_rms, const int32_t *ids, const float *w,
+                                    const void *experts, int weight_dtype, int batch, int n_experts, int top_k,
+                                    int hidden, int inter, float residual_scale, float *h_out, void *cuda_stream)
+{
+    if (batch < 1 || top_k < 1 || hidden < 16 || inter < 16) return STMOE_ERR_BAD_ARG;
+    if (stmoe_moe_ffn_scratch_bytes(batch, top_k, hidden, inter) > (size_t)STMOE_STATIC_SCRATCH_BYTES)
+        return STMOE_ERR_TOO_LARGE;
+    int dev = -1;
+    CU_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return STMOE_ERR_BAD_ARG;
+    if (!g_static_scratch_ptr[dev]) {
+        void *p = nullptr;
+        CU_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+        g_static_scratch_ptr[dev] = p;
+    }
+    return stmoe_moe_ffn(h, inv_rms, ids, w, experts, weight_dtype, batch, n_experts, top_k, hidden, inter,
+                         residual_scale, h_out, g_static_scratch_ptr[dev], (size_t)STMOE_STATIC_SCRATCH_BYTES,
+                         cuda_stream);
 }
