@@ -32,8 +32,9 @@ from datagen import stacks  # noqa: E402
 
 METRIC, UNIT = "decode_tokens_per_s", "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate/up launch at this workload, from the
-# ncu capture summarised under profiles/ (None until captured).
-NCU_TRAFFIC_BYTES = {"C1": None}
+# ncu capture summarised in profiles/ffn_kernels_c1_2layers_ncu_full.md (taken on a 2-layer stack
+# of the same shape: one launch does the same work there, so no scaling is applied).
+NCU_TRAFFIC_BYTES = {"C1": 469797888 + 3237120}
 
 
 def measured_peaks():
@@ -314,6 +315,7 @@ def main():
                      "algorithmic_bytes_per_launch": gate_up_bytes, "us_per_launch": gu_ms * 1e3,
                      "down_kernel": {"achieved": (gate_up_bytes / 2) / (dn_ms * 1e-3) / 1e9 if dn_ms else None,
                                      "us_per_launch": dn_ms * 1e3},
+                     "router_kernel": {"us_per_launch": s2["router_ms"] / max(n_ffn, 1) * 1e3},
                      "whole_step": {"bytes_per_token": statistics.mean(step_bytes) / batch,
                                     "achieved": step_gbs, "frac": step_gbs / peak,
                                     "frac_of_8000": step_gbs / 8000.0}},

@@ -100,6 +100,7 @@ typedef struct {
     int64_t timed_ffn_launches; /* layer steps whose FFN kernels were timed (see below)   */
     double gate_up_ms;        /* summed device time of the timed gate/up kernels          */
     double down_ms;           /* summed device time of the timed down kernels             */
+    double router_ms;         /* summed device time of the timed router kernels           */
 } stmoe_stats_t;
 
 /* Create a stack for the current CUDA device.  Allocates weight storage (HBM
@@ -147,8 +148,9 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out,
 
 int stmoe_max_predicted(const stmoe_t *s); /* min(E, K*K+K) */
 
-/* on != 0: bracket the two expert-FFN kernels of every following layer step with CUDA events
- * on the caller's stream; their summed durations appear in stmoe_stats.  Off by default. */
+/* on != 0: bracket the expert-FFN kernels of every following layer step with CUDA events
+ * on the caller's stream (the router kernel too); their summed durations appear in stmoe_stats.
+ * Off by default. */
 int stmoe_set_kernel_timing(stmoe_t *s, int on);
 
 /* Counters and timings; synchronises the device. */

@@ -37,7 +37,8 @@ class Stats(C.Structure):
         "cache_misses", "prefetch_issued", "prefetch_useful", "prefetch_wasted", "prefetch_dropped",
         "prefetch_resident", "h2d_bytes_demand", "h2d_bytes_prefetch")] + \
         [("transfer_ms", C.c_double), ("exposed_ms", C.c_double), ("kernel_launches", C.c_int64),
-         ("timed_ffn_launches", C.c_int64), ("gate_up_ms", C.c_double), ("down_ms", C.c_double)]
+         ("timed_ffn_launches", C.c_int64), ("gate_up_ms", C.c_double), ("down_ms", C.c_double),
+         ("router_ms", C.c_double)]
 
 
 _lib = None

@@ -95,56 +95,58 @@ struct TopkArgs {
 constexpr int kVpl = kMaxExperts / kWarp;  // logits held per lane
 
 // softmax + top-K for one sequence, by one warp.  Lane l holds the logits of experts
-// l, l+32, ... in z[].  K rounds of warp arg-max on (logit, lower id first) keys, one more
-// round for the K-th/(K+1)-th gap; ids are emitted in ascending order with w = softmax(z)[id].
-__device__ __forceinline__ void route_token(const float (&z)[kVpl], float *s_zrow, int *s_ids_row,
-                                            const TopkArgs &a, int b, int lane)
+// l, l+32, ... in z[].  K rounds of warp arg-max (hardware redux on order-preserving 32-bit
+// keys, then redux-min over the tied ids so the lower id wins), one more round for the
+// K-th/(K+1)-th gap; ids are emitted in ascending order with w = softmax(z)[id].
+__device__ __forceinline__ void route_token(const float (&z)[kVpl], float *, int *s_ids_row, const TopkArgs &a,
+                                            int b, int lane)
 {
     const int E = a.E, K = a.K;
     float m = -INFINITY;
+    uint32_t key[kVpl];
 #pragma unroll
     for (int v = 0; v < kVpl; ++v) {
-        const int j = v * kWarp + lane;
-        if (j < E) s_zrow[j] = z[v];
         m = fmaxf(m, z[v]);
+        key[v] = (v * kWarp + lane < E) ? float_key(z[v]) : 0u;  // 0 never wins: real keys are > 0
     }
     m = warp_max(m);
-    float sum = 0.f;
+    float ex[kVpl], sum = 0.f;
 #pragma unroll
-    for (int v = 0; v < kVpl; ++v)
-        if (v * kWarp + lane < E) sum += expf(z[v] - m);
+    for (int v = 0; v < kVpl; ++v) {
+        ex[v] = (v * kWarp + lane < E) ? expf(z[v] - m) : 0.f;
+        sum += ex[v];
+    }
     sum = warp_sum(sum);
-    __syncwarp();
 
     uint32_t taken = 0;  // bit v: my value v is selected
     float kth = 0.f, gap = INFINITY;
     for (int r = 0; r <= K && r < E; ++r) {
-        unsigned long long best = 0;
+        uint32_t best = 0;
+        int best_v = 0;
 #pragma unroll
-        for (int v = 0; v < kVpl; ++v) {
-            const int j = v * kWarp + lane;
-            if (j < E && !((taken >> v) & 1u)) {
-                const unsigned long long key =
-                    ((unsigned long long)float_key(z[v]) << 32) | (uint32_t)(0xffffffffu - j);
-                best = key > best ? key : best;
-            }
-        }
-        best = warp_max_u64(best);
-        const int j = (int)(0xffffffffu - (uint32_t)best);
+        for (int v = 0; v < kVpl; ++v)
+            if (!((taken >> v) & 1u) && key[v] > best) best = key[v], best_v = v;  // first max = lowest id
+        const uint32_t top = __reduce_max_sync(kFull, best);
+        const uint32_t cand = (best == top && best != 0u) ? (uint32_t)(best_v * kWarp + lane) : 0xffffffffu;
+        const int j = (int)__reduce_min_sync(kFull, cand);
+        float zj = 0.f;
+#pragma unroll
+        for (int v = 0; v < kVpl; ++v)
+            if (v == best_v) zj = z[v];
+        zj = __shfl_sync(kFull, zj, j % kWarp);
         if (r < K) {
             if (j % kWarp == lane) taken |= 1u << (j / kWarp);
-            kth = s_zrow[j];
+            kth = zj;
         } else {
-            gap = kth - s_zrow[j];
+            gap = kth - zj;
         }
     }
 
     float sel = 0.f;
 #pragma unroll
     for (int v = 0; v < kVpl; ++v)
-        if ((taken >> v) & 1u) sel += expf(z[v] - m);
-    sel = warp_sum(sel);
-    const float denom = a.renorm ? sel : sum;
+        if ((taken >> v) & 1u) sel += ex[v];
+    sel = a.renorm ? warp_sum(sel) : sum;
     int base = 0;
 #pragma unroll
     for (int v = 0; v < kVpl; ++v) {
@@ -152,7 +154,7 @@ __device__ __forceinline__ void route_token(const float (&z)[kVpl], float *s_zro
         if ((taken >> v) & 1u) {
             const int pos = base + __popc(msk & ((1u << lane) - 1u));
             const int j = v * kWarp + lane;
-            const float p = expf(z[v] - m) / denom;
+            const float p = ex[v] / sel;
             a.ids[(size_t)b * K + pos] = j;
             a.w[(size_t)b * K + pos] = p;
             s_ids_row[pos] = j;

@@ -249,7 +249,7 @@ struct SlotCache {
 
 struct TimedSpan {
     cudaEvent_t a, b;
-    int kind;  // 0 transfer, 1 exposed wait, 2 gate/up kernel, 3 down kernel
+    int kind;  // 0 transfer, 1 exposed wait, 2 gate/up kernel, 3 down kernel, 4 router kernel
 };
 
 }  // namespace
@@ -301,7 +301,7 @@ struct stmoe {
     std::vector<uint8_t> slot_pending;
     std::deque<TimedSpan> spans;
     std::vector<cudaEvent_t> free_events;
-    double transfer_ms = 0, exposed_ms = 0, gate_up_ms = 0, down_ms = 0;
+    double transfer_ms = 0, exposed_ms = 0, gate_up_ms = 0, down_ms = 0, router_ms = 0;
     int64_t launches = 0, timed_ffn = 0;
     bool time_kernels = false;
     int64_t bytes_demand = 0, bytes_prefetch = 0;
@@ -334,7 +334,7 @@ void harvest_spans(stmoe *s, bool all)
         }
         float ms = 0.f;
         if (cudaEventElapsedTime(&ms, sp.a, sp.b) == cudaSuccess) {
-            double *acc[4] = {&s->transfer_ms, &s->exposed_ms, &s->gate_up_ms, &s->down_ms};
+            double *acc[5] = {&s->transfer_ms, &s->exposed_ms, &s->gate_up_ms, &s->down_ms, &s->router_ms};
             *acc[sp.kind] += ms;
         }
         s->free_events.push_back(sp.a);
@@ -539,6 +539,12 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
     int32_t *ids = s->d_ids + (size_t)layer * c.max_batch * K;
     const int32_t *prev = layer > 0 ? s->d_ids + (size_t)(layer - 1) * c.max_batch * K : nullptr;
 
+    cudaEvent_t er0 = nullptr, er1 = nullptr;
+    if (s->time_kernels) {
+        ST_TRY(get_event(s, &er0));
+        ST_TRY(get_event(s, &er1));
+        CU_TRY(cudaEventRecord(er0, st));
+    }
     RouterArgs ra{};
     ra.h = h_in, ra.W = s->d_router + (size_t)layer * E * H * dtype_bytes(s->rdt), ra.H = H, ra.eps = c.rms_eps;
     ra.part = s->d_rpart, ra.ss_part = s->d_sspart, ra.arrivals = s->d_arrivals, ra.inv_rms = s->d_inv;
@@ -557,6 +563,10 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
         router_fused_kernel<1><<<(E * C + 7) / 8, 256, 0, st>>>(ra);
     }
     CU_TRY(cudaGetLastError());
+    if (s->time_kernels) {
+        CU_TRY(cudaEventRecord(er1, st));
+        s->spans.push_back(TimedSpan{er0, er1, 4});
+    }
     if (offloaded(s))  // the host needs the prefetch queue before it can issue copies
         ST_TRY(launch_predictor(s, layer, batch, ids, prev, predicted_ids, n_predicted, true, st));
 
@@ -909,7 +919,7 @@ int stmoe_stats(stmoe_t *s, stmoe_stats_t *out)
     out->h2d_bytes_demand = s->bytes_demand, out->h2d_bytes_prefetch = s->bytes_prefetch;
     out->transfer_ms = s->transfer_ms, out->exposed_ms = s->exposed_ms;
     out->kernel_launches = s->launches, out->timed_ffn_launches = s->timed_ffn;
-    out->gate_up_ms = s->gate_up_ms, out->down_ms = s->down_ms;
+    out->gate_up_ms = s->gate_up_ms, out->down_ms = s->down_ms, out->router_ms = s->router_ms;
     return STMOE_OK;
 }
 
