@@ -19,6 +19,18 @@ namespace stmoe_dev {
 #define STMOE_FFN_THREADS 512  // one CTA of 16 warps per SM
 #endif
 constexpr int kFfnThreads = STMOE_FFN_THREADS;
+
+// Tile shapes of the one-token code path (rows per block, loads in flight per row) and the
+// longest row segment of the down projection; overridable for tuning builds.
+#ifndef STMOE_RG1
+#define STMOE_RG1 2
+#define STMOE_UG1 4
+#define STMOE_RD1 8
+#define STMOE_UD1 2
+#endif
+#ifndef STMOE_SEG_BYTES
+#define STMOE_SEG_BYTES 16384
+#endif
 constexpr int kFfnWarps = kFfnThreads / kWarp;
 
 struct FfnArgs {
@@ -112,158 +124,225 @@ struct BlockTickets {
     }
 };
 
+// Fused weighted sum + residual.  Called by a whole warp after it has stored the partial sums
+// of rows [r0, r0+nrows) of one (entry, segment): the rows are counted per 32-row tile, and the
+// warp whose count completes a tile (want_per_row contributions for each of its rows) sums
+// the tile over segments, shared experts and routed experts in a fixed order:
+//   h_out[b][c] = h[b][c] + r * ( sum_shared part + sum_k w[b][k] * part ).
+// No waiting is involved; the counter is left at zero for the next launch.
+__device__ __forceinline__ void finish_rows(const FfnArgs &a, int r0, int nrows, int want_per_row, int S, int lane)
+{
+    const int H = a.H;
+    __threadfence();
+    __syncwarp();
+    for (int rr = r0; rr < r0 + nrows;) {
+        const int tile = rr / kTileRows;
+        const int n = min(r0 + nrows, (tile + 1) * kTileRows) - rr;
+        const int tile_rows = min(kTileRows, H - tile * kTileRows);
+        unsigned prev = 0;
+        if (lane == 0) prev = atomicAdd(a.tile_done + tile, (unsigned)n);
+        prev = __shfl_sync(kFull, prev, 0);
+        if (prev + n == (unsigned)(want_per_row * tile_rows)) {
+            __threadfence();
+            if (lane == 0) a.tile_done[tile] = 0u;
+            const int c = tile * kTileRows + lane;
+            if (lane < tile_rows) {
+                const int KS = a.K + a.n_shared;
+                for (int b = 0; b < a.B; ++b) {
+                    float y = 0.f;
+                    for (int q = 0; q < a.n_shared; ++q) {
+                        float p = 0.f;
+                        for (int z = 0; z < S; ++z) p += __ldcg(a.part + (((size_t)b * KS + a.K + q) * S + z) * H + c);
+                        y += p;
+                    }
+                    for (int k = 0; k < a.K; ++k) {
+                        float p = 0.f;
+                        for (int z = 0; z < S; ++z) p += __ldcg(a.part + (((size_t)b * KS + k) * S + z) * H + c);
+                        y = fmaf(a.w[b * a.K + k], p, y);
+                    }
+                    a.h_out[(size_t)b * H + c] = fmaf(a.residual_scale, y, a.h[(size_t)b * H + c]);
+                }
+            }
+        }
+        rr += n;
+    }
+}
+
+// What a warp needs to know about a work-list entry, kept in registers across the blocks it
+// claims: consecutive blocks nearly always belong to the same entry, and looking the entry up
+// costs two dependent trips to L2 before the first weight load can be issued.
+template <int MT> struct Entry {
+    int g = -1, cnt = 0;
+    const uint8_t *img = nullptr;
+    int tok[MT], slot[MT];
+    float inv[MT];
+    __device__ __forceinline__ void load(const FfnArgs &a, int g_new)
+    {
+        if (g_new == g) return;
+        g = g_new;
+        img = a.blob[a.wl.g_expert[g]];
+        const int start = a.wl.g_start[g];
+        cnt = a.wl.g_count[g];
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+            const int p = start + min(t, cnt - 1);
+            tok[t] = a.wl.pair_token[p], slot[t] = a.wl.pair_slot[p];
+            inv[t] = a.inv_rms ? a.inv_rms[tok[t]] : 1.f;
+        }
+    }
+};
+
+// One block of the gate/up projection: rows [r0, r0+nrows) (nrows <= R) of work-list entry g.
 // act[slot][i] = silu(g_i) * u_i,  g = W_g x, u = W_u x,  x = h * inv_rms  (folded into g, u)
-template <int DT, int R, int MT, int U>
-__global__ void __launch_bounds__(kFfnThreads, 1) gate_up_kernel(FfnArgs a)
+template <int DT, int R, int MT, int U, int MTE>
+__device__ __forceinline__ void gate_up_block(const FfnArgs &a, const Entry<MTE> &en, int r0, int nrows, int lane)
 {
     constexpr int BYTES = Fmt<DT>::kBytes;
-    __shared__ int s_next;
-    const int lane = threadIdx.x % kWarp;
     const int H = a.H, I = a.I;
     const size_t row_bytes = (size_t)H * BYTES;
+    const int cnt = en.cnt;
+    const uint8_t *img = en.img;
+    const uint8_t *rowp[2][R];
+    const float *xp[MT];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        rowp[0][r] = img + image_gate(H, I, BYTES) + (size_t)(r0 + r) * row_bytes;
+        rowp[1][r] = img + image_up(H, I, BYTES) + (size_t)(r0 + r) * row_bytes;
+    }
+#pragma unroll
+    for (int t = 0; t < MT; ++t) xp[t] = a.h + (size_t)en.tok[t] * H;
+    float acc[2][R][MT];
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int t = 0; t < MT; ++t) acc[m][r][t] = 0.f;
+    gemv_rows<DT, 2, R, MT, U>(rowp, nrows, xp, H, lane, acc);
+
+    const uint16_t *sc = reinterpret_cast<const uint16_t *>(img + image_scales(H, I, BYTES));
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+            float gv = warp_sum(acc[0][r][t]), uv = warp_sum(acc[1][r][t]);
+            if (lane == (r * MT + t) % kWarp && r < nrows && t < cnt) {
+                gv *= en.inv[t], uv *= en.inv[t];
+                if (DT == 2) {
+                    gv *= bf16_to_f32(sc[r0 + r]);
+                    uv *= bf16_to_f32(sc[I + r0 + r]);
+                }
+                a.act[(size_t)en.slot[t] * I + r0 + r] = gv / (1.f + expf(-gv)) * uv;
+            }
+        }
+}
+
+// Tile shapes: R rows per block and U loads in flight per row, for entries of one token (the
+// batch-1 shape, widest loads) and for entries of up to four tokens.
+template <int DT> struct TileShape {
+    static constexpr int RG1 = STMOE_RG1, UG1 = STMOE_UG1, RD1 = STMOE_RD1, UD1 = STMOE_UD1;
+    static constexpr int RG4 = 2, UG4 = DT == 2 ? 1 : 2, RD4 = DT == 2 ? 2 : 4, UD4 = 2;
+};
+
+// Work-list entries are walked in claims of RG1 rows; an entry that holds one token takes the
+// one-token code path even in the multi-token kernel (MTMAX = 4), so a batch whose sequences
+// mostly route to different experts streams as fast as batch 1.
+template <int DT, int MTMAX>
+__global__ void __launch_bounds__(kFfnThreads, 1) gate_up_kernel(FfnArgs a)
+{
+    using TS = TileShape<DT>;
+    constexpr int RC = TS::RG1;
+    __shared__ int s_next;
+    const int lane = threadIdx.x % kWarp;
+    const int I = a.I;
     BlockTickets tk;
     tk.init(*a.wl.n_groups * I, &s_next);
+    Entry<MTMAX> en;
 
-    for (int u0 = tk.claim(&s_next, R, lane); u0 < tk.last; u0 = tk.claim(&s_next, R, lane)) {
-        const int uend = min(u0 + R, tk.last);
+    for (int u0 = tk.claim(&s_next, RC, lane); u0 < tk.last; u0 = tk.claim(&s_next, RC, lane)) {
+        const int uend = min(u0 + RC, tk.last);
         for (int u = u0; u < uend;) {
             const int g = u / I, r0 = u % I;
             const int nrows = min(uend - u, I - r0);
             u += nrows;
-            const int ex = a.wl.g_expert[g], start = a.wl.g_start[g], cnt = a.wl.g_count[g];
-            const uint8_t *img = a.blob[ex];
-            const uint8_t *rowp[2][R];
-            const float *xp[MT];
-            int tok[MT], slot[MT];
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                rowp[0][r] = img + image_gate(H, I, BYTES) + (size_t)(r0 + r) * row_bytes;
-                rowp[1][r] = img + image_up(H, I, BYTES) + (size_t)(r0 + r) * row_bytes;
+            en.load(a, g);
+            if (MTMAX == 1 || en.cnt == 1) {
+                gate_up_block<DT, TS::RG1, 1, TS::UG1>(a, en, r0, nrows, lane);
+            } else {
+                for (int q = 0; q < nrows; q += TS::RG4)
+                    gate_up_block<DT, TS::RG4, MTMAX, TS::UG4>(a, en, r0 + q, min(TS::RG4, nrows - q), lane);
             }
-#pragma unroll
-            for (int t = 0; t < MT; ++t) {
-                const int p = start + min(t, cnt - 1);
-                tok[t] = a.wl.pair_token[p], slot[t] = a.wl.pair_slot[p];
-                xp[t] = a.h + (size_t)tok[t] * H;
-            }
-            float acc[2][R][MT];
-#pragma unroll
-            for (int m = 0; m < 2; ++m)
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-#pragma unroll
-                    for (int t = 0; t < MT; ++t) acc[m][r][t] = 0.f;
-            gemv_rows<DT, 2, R, MT, U>(rowp, nrows, xp, H, lane, acc);
-
-            const uint16_t *sc = reinterpret_cast<const uint16_t *>(img + image_scales(H, I, BYTES));
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-#pragma unroll
-                for (int t = 0; t < MT; ++t) {
-                    float gv = warp_sum(acc[0][r][t]), uv = warp_sum(acc[1][r][t]);
-                    if (lane == (r * MT + t) % kWarp && r < nrows && t < cnt) {
-                        const float inv = a.inv_rms ? a.inv_rms[tok[t]] : 1.f;
-                        gv *= inv, uv *= inv;
-                        if (DT == 2) {
-                            gv *= bf16_to_f32(sc[r0 + r]);
-                            uv *= bf16_to_f32(sc[I + r0 + r]);
-                        }
-                        a.act[(size_t)slot[t] * I + r0 + r] = gv / (1.f + expf(-gv)) * uv;
-                    }
-                }
         }
     }
 }
 
+// One block of the down projection: rows [r0, r0+nrows) of segment s of entry g.
 // part[slot][s][h] = sum over the columns of split s of W_d[h][col] * act[slot][col]
-template <int DT, int R, int MT, int U>
+template <int DT, int R, int MT, int U, int MTE>
+__device__ __forceinline__ void down_block(const FfnArgs &a, const Entry<MTE> &en, int s, int seg, int r0, int nrows,
+                                           int lane)
+{
+    constexpr int BYTES = Fmt<DT>::kBytes;
+    const int H = a.H, I = a.I, S = a.S;
+    const size_t row_bytes = (size_t)I * BYTES;
+    const int c0 = s * seg, ncols = min(seg, I - c0);
+    const int cnt = en.cnt;
+    const uint8_t *img = en.img;
+    const uint8_t *rowp[1][R];
+    const float *xp[MT];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+        rowp[0][r] = img + image_down(H, I, BYTES) + (size_t)(r0 + r) * row_bytes + (size_t)c0 * BYTES;
+#pragma unroll
+    for (int t = 0; t < MT; ++t) xp[t] = a.act + (size_t)en.slot[t] * I + c0;
+    float acc[1][R][MT];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int t = 0; t < MT; ++t) acc[0][r][t] = 0.f;
+    if (ncols > 0) gemv_rows<DT, 1, R, MT, U>(rowp, nrows, xp, ncols, lane, acc);
+
+    const uint16_t *sc = reinterpret_cast<const uint16_t *>(img + image_scales(H, I, BYTES));
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+            float v = warp_sum(acc[0][r][t]);
+            if (lane == (r * MT + t) % kWarp && r < nrows && t < cnt) {
+                if (DT == 2) v *= bf16_to_f32(sc[2 * I + r0 + r]);
+                a.part[((size_t)en.slot[t] * S + s) * H + r0 + r] = v;
+            }
+        }
+}
+
+template <int DT, int MTMAX>
 __global__ void __launch_bounds__(kFfnThreads, 1) down_kernel(FfnArgs a)
 {
-    constexpr int BYTES = Fmt<DT>::kBytes, EPL = Fmt<DT>::kEpl;
+    using TS = TileShape<DT>;
+    constexpr int EPL = Fmt<DT>::kEpl, RC = TS::RD1;
     __shared__ int s_next;
     const int lane = threadIdx.x % kWarp;
     const int H = a.H, I = a.I, S = a.S;
-    const size_t row_bytes = (size_t)I * BYTES;
     // columns of one split, a multiple of one warp-wide load
     const int seg = ((I + S - 1) / S + kWarp * EPL - 1) / (kWarp * EPL) * (kWarp * EPL);
     BlockTickets tk;
     tk.init(*a.wl.n_groups * S * H, &s_next);
+    Entry<MTMAX> en;
 
-    for (int u0 = tk.claim(&s_next, R, lane); u0 < tk.last; u0 = tk.claim(&s_next, R, lane)) {
-        const int uend = min(u0 + R, tk.last);
+    for (int u0 = tk.claim(&s_next, RC, lane); u0 < tk.last; u0 = tk.claim(&s_next, RC, lane)) {
+        const int uend = min(u0 + RC, tk.last);
         for (int u = u0; u < uend;) {
             const int g = u / (S * H), s = (u / H) % S, r0 = u % H;
             const int nrows = min(uend - u, H - r0);
             u += nrows;
-            const int c0 = s * seg, ncols = min(seg, I - c0);
-            const int ex = a.wl.g_expert[g], start = a.wl.g_start[g], cnt = a.wl.g_count[g];
-            const uint8_t *img = a.blob[ex];
-            const uint8_t *rowp[1][R];
-            const float *xp[MT];
-            int slot[MT];
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-                rowp[0][r] = img + image_down(H, I, BYTES) + (size_t)(r0 + r) * row_bytes + (size_t)c0 * BYTES;
-#pragma unroll
-            for (int t = 0; t < MT; ++t) {
-                slot[t] = a.wl.pair_slot[start + min(t, cnt - 1)];
-                xp[t] = a.act + (size_t)slot[t] * I + c0;
+            en.load(a, g);
+            if (MTMAX == 1 || en.cnt == 1) {
+                down_block<DT, TS::RD1, 1, TS::UD1>(a, en, s, seg, r0, nrows, lane);
+            } else {
+                for (int q = 0; q < nrows; q += TS::RD4)
+                    down_block<DT, TS::RD4, MTMAX, TS::UD4>(a, en, s, seg, r0 + q, min(TS::RD4, nrows - q), lane);
             }
-            float acc[1][R][MT];
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-#pragma unroll
-                for (int t = 0; t < MT; ++t) acc[0][r][t] = 0.f;
-            if (ncols > 0) gemv_rows<DT, 1, R, MT, U>(rowp, nrows, xp, ncols, lane, acc);
-
-            const uint16_t *sc = reinterpret_cast<const uint16_t *>(img + image_scales(H, I, BYTES));
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-#pragma unroll
-                for (int t = 0; t < MT; ++t) {
-                    float v = warp_sum(acc[0][r][t]);
-                    if (lane == (r * MT + t) % kWarp && r < nrows && t < cnt) {
-                        if (DT == 2) v *= bf16_to_f32(sc[2 * I + r0 + r]);
-                        a.part[((size_t)slot[t] * S + s) * H + r0 + r] = v;
-                    }
-                }
-            // publish the rows; the warp that completes a tile sums it up (fixed order)
-            __threadfence();
-            __syncwarp();
-            const int want_per_row = *a.wl.n_groups * S;
-            for (int rr = r0; rr < r0 + nrows;) {
-                const int tile = rr / kTileRows;
-                const int n = min(r0 + nrows, (tile + 1) * kTileRows) - rr;
-                const int tile_rows = min(kTileRows, H - tile * kTileRows);
-                unsigned prev = 0;
-                if (lane == 0) prev = atomicAdd(a.tile_done + tile, (unsigned)n);
-                prev = __shfl_sync(kFull, prev, 0);
-                if (prev + n == (unsigned)(want_per_row * tile_rows)) {
-                    __threadfence();
-                    if (lane == 0) a.tile_done[tile] = 0u;
-                    const int c = tile * kTileRows + lane;
-                    if (lane < tile_rows) {
-                        const int KS = a.K + a.n_shared;
-                        for (int b = 0; b < a.B; ++b) {
-                            float y = 0.f;
-                            for (int q = 0; q < a.n_shared; ++q) {
-                                float p = 0.f;
-                                for (int z = 0; z < S; ++z)
-                                    p += __ldcg(a.part + (((size_t)b * KS + a.K + q) * S + z) * H + c);
-                                y += p;
-                            }
-                            for (int k = 0; k < a.K; ++k) {
-                                float p = 0.f;
-                                for (int z = 0; z < S; ++z)
-                                    p += __ldcg(a.part + (((size_t)b * KS + k) * S + z) * H + c);
-                                y = fmaf(a.w[b * a.K + k], p, y);
-                            }
-                            a.h_out[(size_t)b * H + c] = fmaf(a.residual_scale, y, a.h[(size_t)b * H + c]);
-                        }
-                    }
-                }
-                rr += n;
-            }
+            finish_rows(a, r0, nrows, *a.wl.n_groups * S, S, lane);
         }
     }
 }

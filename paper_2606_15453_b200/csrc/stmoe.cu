@@ -32,18 +32,6 @@ using namespace stmoe_dev;
         if (r_ != STMOE_OK) return r_; \
     } while (0)
 
-// Tile shapes of the batch-1 FFN kernels (rows per block, loads in flight per row) and the
-// longest row segment of the down projection; overridable for tuning builds.
-#ifndef STMOE_RG1
-#define STMOE_RG1 2
-#define STMOE_UG1 4
-#define STMOE_RD1 8
-#define STMOE_UD1 2
-#endif
-#ifndef STMOE_SEG_BYTES
-#define STMOE_SEG_BYTES 16384
-#endif
-
 namespace {
 
 constexpr uint32_t kStateMagic = 0x53544D50;
@@ -73,33 +61,24 @@ struct FfnPlan {
     int grid_gate_up = 0, grid_down = 0;
 };
 
-template <int DT, int MT> struct Shape;
-template <int DT> struct Shape<DT, 1> {
-    static constexpr int RG = STMOE_RG1, UG = STMOE_UG1, RD = STMOE_RD1, UD = STMOE_UD1;
-};
-template <int DT> struct Shape<DT, 4> { static constexpr int RG = 2, UG = 2, RD = 4, UD = 2; };
-template <> struct Shape<2, 4> { static constexpr int RG = 2, UG = 1, RD = 2, UD = 2; };
-
 template <int DT, int MT> void launch_gate_up(const FfnArgs &a, int grid, cudaStream_t st)
 {
-    gate_up_kernel<DT, Shape<DT, MT>::RG, MT, Shape<DT, MT>::UG><<<grid, kFfnThreads, 0, st>>>(a);
+    gate_up_kernel<DT, MT><<<grid, kFfnThreads, 0, st>>>(a);
 }
 template <int DT, int MT> void launch_down(const FfnArgs &a, int grid, cudaStream_t st)
 {
-    down_kernel<DT, Shape<DT, MT>::RD, MT, Shape<DT, MT>::UD><<<grid, kFfnThreads, 0, st>>>(a);
+    down_kernel<DT, MT><<<grid, kFfnThreads, 0, st>>>(a);
 }
 template <int DT, int MT> int occupancy_gate_up()
 {
     int n = 0;
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-        &n, gate_up_kernel<DT, Shape<DT, MT>::RG, MT, Shape<DT, MT>::UG>, kFfnThreads, 0);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, gate_up_kernel<DT, MT>, kFfnThreads, 0);
     return n;
 }
 template <int DT, int MT> int occupancy_down()
 {
     int n = 0;
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-        &n, down_kernel<DT, Shape<DT, MT>::RD, MT, Shape<DT, MT>::UD>, kFfnThreads, 0);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, down_kernel<DT, MT>, kFfnThreads, 0);
     return n;
 }
 
