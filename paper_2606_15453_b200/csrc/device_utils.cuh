@@ -21,6 +21,15 @@ __device__ __forceinline__ uint4 ld_stream16(const void *p)
     return v;
 }
 
+// Programmatic dependent launch.  pdl_wait: block until the kernel launched before this one
+// in the stream has completed and its writes are visible (returns at once when the launch was
+// an ordinary one).  pdl_launch_dependents: allow the next kernel in the stream, if it was
+// launched with programmatic serialization, to start occupying SMs as this grid's CTAs retire.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 __device__ __forceinline__ float4 ld_f4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
 
 __device__ __forceinline__ float bf16_to_f32(uint16_t v) { return __uint_as_float((uint32_t)v << 16); }

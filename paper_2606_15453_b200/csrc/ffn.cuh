@@ -255,6 +255,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) gate_up_kernel(FfnArgs a)
     __shared__ int s_next;
     const int lane = threadIdx.x % kWarp;
     const int I = a.I;
+    pdl_launch_dependents();  // the down kernel may move in behind the CTAs of this grid
     BlockTickets tk;
     tk.init(*a.wl.n_groups * I, &s_next);
     Entry<MTMAX> en;
@@ -325,11 +326,28 @@ __global__ void __launch_bounds__(kFfnThreads, 1) down_kernel(FfnArgs a)
     const int H = a.H, I = a.I, S = a.S;
     // columns of one split, a multiple of one warp-wide load
     const int seg = ((I + S - 1) / S + kWarp * EPL - 1) / (kWarp * EPL) * (kWarp * EPL);
+    // Launched with programmatic serialization behind the gate/up kernel: the work list is
+    // older than that kernel, so the first claim can be made and its weight rows pulled into L2
+    // while gate/up is still finishing; only the activations have to wait.
+    pdl_launch_dependents();
     BlockTickets tk;
     tk.init(*a.wl.n_groups * S * H, &s_next);
     Entry<MTMAX> en;
+    int u0 = tk.claim(&s_next, RC, lane);
+    if (u0 < tk.last) {
+        const int g = u0 / (S * H), s = (u0 / H) % S, r0 = u0 % H;
+        en.load(a, g);
+        const int n = min(min(RC, tk.last - u0), H - r0);
+        const size_t row_bytes = (size_t)I * Fmt<DT>::kBytes;
+        // just what the first load step of each row needs
+        const int seg_bytes = min(min(seg, I - s * seg) * Fmt<DT>::kBytes, TS::UD1 * kWarp * 16);
+        const uint8_t *base = en.img + image_down(H, I, Fmt<DT>::kBytes) + (size_t)s * seg * Fmt<DT>::kBytes;
+        for (int r = 0; r < n; ++r)
+            for (int o = lane * 128; o < seg_bytes; o += kWarp * 128) prefetch_l2(base + (size_t)(r0 + r) * row_bytes + o);
+    }
+    pdl_wait();
 
-    for (int u0 = tk.claim(&s_next, RC, lane); u0 < tk.last; u0 = tk.claim(&s_next, RC, lane)) {
+    for (; u0 < tk.last; u0 = tk.claim(&s_next, RC, lane)) {
         const int uend = min(u0 + RC, tk.last);
         for (int u = u0; u < uend;) {
             const int g = u / (S * H), s = (u / H) % S, r0 = u % H;

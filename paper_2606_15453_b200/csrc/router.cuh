@@ -301,6 +301,7 @@ __global__ void __launch_bounds__(256) router_fused_kernel(RouterArgs a)
                 for (int e = 0; e < EPL; ++e) wf[u][e] = 0.f;
             }
         }
+        pdl_wait();  // the router weights above do not depend on the previous kernel; h does
         for (int b = 0; b < B; ++b) {
             float acc = 0.f, ss = 0.f;
 #pragma unroll
@@ -324,6 +325,7 @@ __global__ void __launch_bounds__(256) router_fused_kernel(RouterArgs a)
             }
         }
     }
+    pdl_wait();  // warps without a task: nothing below may run ahead of the previous kernel either
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) s_last = (atomicAdd(a.arrivals, 1u) == gridDim.x - 1);

@@ -61,13 +61,26 @@ struct FfnPlan {
     int grid_gate_up = 0, grid_down = 0;
 };
 
+// Launch with the programmatic-stream-serialization attribute: the kernel may start before the
+// previous kernel in the stream has finished and orders itself with griddepcontrol.wait.
+template <typename Arg> void launch_pdl(void (*kernel)(Arg), int grid, int block, cudaStream_t st, const Arg &arg)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid), cfg.blockDim = dim3(block), cfg.dynamicSmemBytes = 0, cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at, cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, arg);
+}
+
 template <int DT, int MT> void launch_gate_up(const FfnArgs &a, int grid, cudaStream_t st)
 {
     gate_up_kernel<DT, MT><<<grid, kFfnThreads, 0, st>>>(a);
 }
 template <int DT, int MT> void launch_down(const FfnArgs &a, int grid, cudaStream_t st)
 {
-    down_kernel<DT, MT><<<grid, kFfnThreads, 0, st>>>(a);
+    launch_pdl(down_kernel<DT, MT>, grid, kFfnThreads, st, a);
 }
 template <int DT, int MT> int occupancy_gate_up()
 {
@@ -536,10 +549,16 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
     ta.wl = s->wlm.wl;
     if (s->rdt == STMOE_F32) {
         const int C = (H + router_chunk_cols<0>() - 1) / router_chunk_cols<0>();
-        router_fused_kernel<0><<<(E * C + 7) / 8, 256, 0, st>>>(ra);
+        if (layer > 0 && !offloaded(s))
+            launch_pdl(router_fused_kernel<0>, (E * C + 7) / 8, 256, st, ra);
+        else
+            router_fused_kernel<0><<<(E * C + 7) / 8, 256, 0, st>>>(ra);
     } else {
         const int C = (H + router_chunk_cols<1>() - 1) / router_chunk_cols<1>();
-        router_fused_kernel<1><<<(E * C + 7) / 8, 256, 0, st>>>(ra);
+        if (layer > 0 && !offloaded(s))
+            launch_pdl(router_fused_kernel<1>, (E * C + 7) / 8, 256, st, ra);
+        else
+            router_fused_kernel<1><<<(E * C + 7) / 8, 256, 0, st>>>(ra);
     }
     CU_TRY(cudaGetLastError());
     if (s->time_kernels) {
