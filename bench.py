@@ -87,9 +87,9 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
-def load_stack(cfg, batch, dev):
+def load_stack(cfg, batch, dev, **kw):
     import paper_2606_15453_b200 as P
-    st = P.Stack.from_config(cfg, max_batch=batch)
+    st = P.Stack.from_config(cfg, max_batch=batch, **kw)
     for l, w in enumerate(stacks.router_weights(cfg)):
         st.load_router(l, w)
     for l in range(cfg.n_layers):
@@ -184,6 +184,8 @@ def main():
     ap.add_argument("--ref-layers", type=int, default=2)
     ap.add_argument("--cpu-sample-layers", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--prefetch-limit", type=int, default=0, help="offloaded stacks: copies per layer step")
+    ap.add_argument("--mode", default="st", choices=["off", "temporal", "spatial", "st"])
     args = ap.parse_args()
 
     cfg = stacks.CONFIGS[args.workload]
@@ -207,7 +209,7 @@ def main():
 
     import paper_2606_15453_b200 as P
     P.build()
-    st = load_stack(cfg, batch, dev)                    # every rank holds a full replica
+    st = load_stack(cfg, batch, dev, prefetch_limit=args.prefetch_limit, mode=args.mode)  # a full replica per rank
     L, K, H = cfg.n_layers, cfg.top_k, cfg.hidden
     n_tok = cfg.profile_tokens + args.warmup + args.steps
     x_host = stacks.token_inputs(cfg, batch, n_tok).pin_memory()
@@ -323,9 +325,18 @@ def main():
                       "precision": run["hits"] / max(run["predicted"], 1),
                       "mean_predicted": run["predicted"] / max(run["runtime_steps"], 1),
                       "near_ties": run["near_ties"]},
-        "cache": {"hits": run["cache_hits"], "misses": run["cache_misses"],
+        "cache": {"slots": cfg.cache_slots, "hits": run["cache_hits"], "misses": run["cache_misses"],
+                  "hit_rate": run["cache_hits"] / max(run["cache_hits"] + run["cache_misses"], 1),
+                  "prefetch_issued": s1["prefetch_issued"] - s0["prefetch_issued"],
+                  "prefetch_useful": s1["prefetch_useful"] - s0["prefetch_useful"],
+                  "prefetch_wasted": s1["prefetch_wasted"] - s0["prefetch_wasted"],
+                  "h2d_gb": (s1["h2d_bytes_demand"] + s1["h2d_bytes_prefetch"]
+                             - s0["h2d_bytes_demand"] - s0["h2d_bytes_prefetch"]) / 1e9,
                   "transfer_ms": s1["transfer_ms"] - s0["transfer_ms"],
-                  "exposed_ms": s1["exposed_ms"] - s0["exposed_ms"]},
+                  "exposed_ms": s1["exposed_ms"] - s0["exposed_ms"],
+                  "hidden_frac": 1.0 - (s1["exposed_ms"] - s0["exposed_ms"])
+                  / max(s1["transfer_ms"] - s0["transfer_ms"], 1e-9),
+                  "prefetch_limit": args.prefetch_limit, "mode": args.mode},
     }
     if world == 1 and not args.no_cpu_baseline:
         st.close()

@@ -54,6 +54,9 @@ extern "C" {
 #define STMOE_FLAG_RENORM_TOPK 1 /* divide the K gate weights by their sum (off: Section 2 uses
                                     the plain softmax probabilities) */
 
+#define STMOE_FLAG_NO_PERSISTENT 2 /* resident stacks: decode steps as per-layer kernels (replayed as a
+                                      CUDA graph) instead of the single persistent kernel */
+
 /* per-sequence result flags of a layer step */
 #define STMOE_TOKEN_NEAR_TIE 1u /* K-th and (K+1)-th router logit closer than 1e-4 */
 
@@ -141,7 +144,10 @@ int stmoe_decode_step(stmoe_t *s, int layer, int batch, const float *h_in, float
                       int32_t *n_predicted, uint32_t *flags, void *cuda_stream);
 
 /* All layers of one decode step: h_out = stack(h_in).  The per-layer outputs are as in
- * stmoe_decode_step with a leading [n_layers] dimension; any of them may be NULL. */
+ * stmoe_decode_step with a leading [n_layers] dimension; any of them may be NULL.  Resident
+ * stacks run the whole step as one persistent cooperative kernel (one CTA per SM, bounded grid
+ * barriers between the phases of a layer; a barrier that times out makes stmoe_stats return
+ * STMOE_ERR_TIMEOUT). */
 int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out,
                        int32_t *routed_ids, float *routed_w, int32_t *predicted_ids,
                        int32_t *n_predicted, uint32_t *flags, void *cuda_stream);

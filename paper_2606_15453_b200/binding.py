@@ -17,6 +17,7 @@ from . import build as _build
 DTYPE = {"f32": 0, "bf16": 1, "fp8": 2}
 MODE = {"off": 0, "temporal": 1, "spatial": 2, "st": 3}
 FLAG_RENORM_TOPK = 1
+FLAG_NO_PERSISTENT = 2
 
 
 class StmoeError(RuntimeError):

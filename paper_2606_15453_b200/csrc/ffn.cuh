@@ -247,20 +247,26 @@ template <int DT> struct TileShape {
 // Work-list entries are walked in claims of RG1 rows; an entry that holds one token takes the
 // one-token code path even in the multi-token kernel (MTMAX = 4), so a batch whose sequences
 // mostly route to different experts streams as fast as batch 1.
-template <int DT, int MTMAX>
-__global__ void __launch_bounds__(kFfnThreads, 1) gate_up_kernel(FfnArgs a)
+struct NoSideWork {
+    __device__ void operator()() const {}
+};
+
+// The rows of the gate/up projection this CTA owns.  side() runs once per warp after the
+// ticket counter is set up and before the warp starts claiming blocks (the persistent kernel
+// parks the predictor there on one warp).
+template <int DT, int MTMAX, typename Side = NoSideWork>
+__device__ __forceinline__ void gate_up_phase(const FfnArgs &a, int *s_next, Side side = Side())
 {
     using TS = TileShape<DT>;
     constexpr int RC = TS::RG1;
-    __shared__ int s_next;
     const int lane = threadIdx.x % kWarp;
     const int I = a.I;
-    pdl_launch_dependents();  // the down kernel may move in behind the CTAs of this grid
     BlockTickets tk;
-    tk.init(*a.wl.n_groups * I, &s_next);
+    tk.init(*a.wl.n_groups * I, s_next);
+    side();
     Entry<MTMAX> en;
 
-    for (int u0 = tk.claim(&s_next, RC, lane); u0 < tk.last; u0 = tk.claim(&s_next, RC, lane)) {
+    for (int u0 = tk.claim(s_next, RC, lane); u0 < tk.last; u0 = tk.claim(s_next, RC, lane)) {
         const int uend = min(u0 + RC, tk.last);
         for (int u = u0; u < uend;) {
             const int g = u / I, r0 = u % I;
@@ -275,6 +281,17 @@ __global__ void __launch_bounds__(kFfnThreads, 1) gate_up_kernel(FfnArgs a)
             }
         }
     }
+}
+
+// Work-list entries are walked in claims of RG1 rows; an entry that holds one token takes the
+// one-token code path even in the multi-token kernel (MTMAX = 4), so a batch whose sequences
+// mostly route to different experts streams as fast as batch 1.
+template <int DT, int MTMAX>
+__global__ void __launch_bounds__(kFfnThreads, 1) gate_up_kernel(FfnArgs a)
+{
+    __shared__ int s_next;
+    pdl_launch_dependents();  // the down kernel may move in behind the CTAs of this grid
+    gate_up_phase<DT, MTMAX>(a, &s_next);
 }
 
 // One block of the down projection: rows [r0, r0+nrows) of segment s of entry g.
@@ -316,38 +333,40 @@ __device__ __forceinline__ void down_block(const FfnArgs &a, const Entry<MTE> &e
         }
 }
 
-template <int DT, int MTMAX>
-__global__ void __launch_bounds__(kFfnThreads, 1) down_kernel(FfnArgs a)
+// The rows of the down projection this CTA owns.  kPdl: the stand-alone kernel is launched
+// with programmatic serialization behind the gate/up kernel; the work list is older than that
+// kernel, so the first claim can be made and the start of its weight rows pulled into L2 while
+// gate/up is still finishing; only the activations have to wait.
+template <int DT, int MTMAX, bool kPdl>
+__device__ __forceinline__ void down_phase(const FfnArgs &a, int *s_next)
 {
     using TS = TileShape<DT>;
     constexpr int EPL = Fmt<DT>::kEpl, RC = TS::RD1;
-    __shared__ int s_next;
     const int lane = threadIdx.x % kWarp;
     const int H = a.H, I = a.I, S = a.S;
     // columns of one split, a multiple of one warp-wide load
     const int seg = ((I + S - 1) / S + kWarp * EPL - 1) / (kWarp * EPL) * (kWarp * EPL);
-    // Launched with programmatic serialization behind the gate/up kernel: the work list is
-    // older than that kernel, so the first claim can be made and its weight rows pulled into L2
-    // while gate/up is still finishing; only the activations have to wait.
-    pdl_launch_dependents();
     BlockTickets tk;
-    tk.init(*a.wl.n_groups * S * H, &s_next);
+    tk.init(*a.wl.n_groups * S * H, s_next);
     Entry<MTMAX> en;
-    int u0 = tk.claim(&s_next, RC, lane);
-    if (u0 < tk.last) {
-        const int g = u0 / (S * H), s = (u0 / H) % S, r0 = u0 % H;
-        en.load(a, g);
-        const int n = min(min(RC, tk.last - u0), H - r0);
-        const size_t row_bytes = (size_t)I * Fmt<DT>::kBytes;
-        // just what the first load step of each row needs
-        const int seg_bytes = min(min(seg, I - s * seg) * Fmt<DT>::kBytes, TS::UD1 * kWarp * 16);
-        const uint8_t *base = en.img + image_down(H, I, Fmt<DT>::kBytes) + (size_t)s * seg * Fmt<DT>::kBytes;
-        for (int r = 0; r < n; ++r)
-            for (int o = lane * 128; o < seg_bytes; o += kWarp * 128) prefetch_l2(base + (size_t)(r0 + r) * row_bytes + o);
+    int u0 = tk.claim(s_next, RC, lane);
+    if (kPdl) {
+        if (u0 < tk.last) {
+            const int g = u0 / (S * H), s = (u0 / H) % S, r0 = u0 % H;
+            en.load(a, g);
+            const int n = min(min(RC, tk.last - u0), H - r0);
+            const size_t row_bytes = (size_t)I * Fmt<DT>::kBytes;
+            // just what the first load step of each row needs
+            const int seg_bytes = min(min(seg, I - s * seg) * Fmt<DT>::kBytes, TS::UD1 * kWarp * 16);
+            const uint8_t *base = en.img + image_down(H, I, Fmt<DT>::kBytes) + (size_t)s * seg * Fmt<DT>::kBytes;
+            for (int r = 0; r < n; ++r)
+                for (int o = lane * 128; o < seg_bytes; o += kWarp * 128)
+                    prefetch_l2(base + (size_t)(r0 + r) * row_bytes + o);
+        }
+        pdl_wait();
     }
-    pdl_wait();
 
-    for (; u0 < tk.last; u0 = tk.claim(&s_next, RC, lane)) {
+    for (; u0 < tk.last; u0 = tk.claim(s_next, RC, lane)) {
         const int uend = min(u0 + RC, tk.last);
         for (int u = u0; u < uend;) {
             const int g = u / (S * H), s = (u / H) % S, r0 = u % H;
@@ -363,6 +382,14 @@ __global__ void __launch_bounds__(kFfnThreads, 1) down_kernel(FfnArgs a)
             finish_rows(a, r0, nrows, *a.wl.n_groups * S, S, lane);
         }
     }
+}
+
+template <int DT, int MTMAX>
+__global__ void __launch_bounds__(kFfnThreads, 1) down_kernel(FfnArgs a)
+{
+    __shared__ int s_next;
+    pdl_launch_dependents();  // the next layer's router may move in behind this grid
+    down_phase<DT, MTMAX, true>(a, &s_next);
 }
 
 }  // namespace stmoe_dev

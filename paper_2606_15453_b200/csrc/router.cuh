@@ -190,7 +190,7 @@ __device__ __forceinline__ void group_tokens(const int *s_ids, int *s_scan, int 
         if (lane >= o) g_inc += tg, p_inc += tp;
     }
     if (lane == kWarp - 1) s_g[warp] = g_inc, s_p[warp] = p_inc;
-    __syncthreads();
+    asm volatile("bar.sync 2, 256;" ::: "memory");  // the 256 grouping threads only
     int g0 = g_inc - (cnt + mt - 1) / mt, p0 = p_inc - cnt, g_all = 0;
     for (int wi = 0; wi < kMaxExperts / kWarp; ++wi) {
         if (wi < warp) g0 += s_g[wi], p0 += s_p[wi];
@@ -231,7 +231,6 @@ __device__ __forceinline__ void group_tokens(const int *s_ids, int *s_scan, int 
 __global__ void __launch_bounds__(256) topk_group_kernel(TopkArgs a)
 {
     constexpr int NW = 8;
-    __shared__ float s_z[NW][kMaxExperts];
     __shared__ int s_ids[kMaxBatch * kMaxTopK];
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
     const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
@@ -242,7 +241,7 @@ __global__ void __launch_bounds__(256) topk_group_kernel(TopkArgs a)
             const int j = v * kWarp + lane;
             z[v] = j < a.E ? a.logits[(size_t)b * a.E + j] : -INFINITY;
         }
-        route_token(z, s_z[warp], s_ids + b * a.K, a, b, lane);
+        route_token(z, nullptr, s_ids + b * a.K, a, b, lane);
     }
     if (a.wl.n_groups == nullptr) return;
     __syncthreads();
@@ -274,67 +273,64 @@ template <int DT> __host__ __device__ constexpr int router_chunk_cols()
     return kWarp * Fmt<DT>::kEpl * kRouterUnroll;
 }
 
-template <int DT>
-__global__ void __launch_bounds__(256) router_fused_kernel(RouterArgs a)
+// One split-K task: partial logits of expert row j over column chunk c for every sequence
+// (and, for j == 0, the partial sums of squares of that chunk).  kPdl: wait for the previous
+// kernel between loading the (independent) router weights and reading h.
+template <int DT, bool kPdl>
+__device__ __forceinline__ void router_task(const RouterArgs &a, int task, int lane)
 {
-    constexpr int EPL = Fmt<DT>::kEpl, BYTES = Fmt<DT>::kBytes, CH = router_chunk_cols<DT>(), NW = 8;
-    __shared__ float s_z[NW][kMaxExperts];
-    __shared__ int s_ids[kMaxBatch * kMaxTopK];
-    __shared__ int s_scan[2 * (kMaxExperts + 1)];
-    __shared__ int s_last;
-    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
+    constexpr int EPL = Fmt<DT>::kEpl, BYTES = Fmt<DT>::kBytes, CH = router_chunk_cols<DT>();
     const int B = a.tk.B, E = a.tk.E, H = a.H;
     const int C = (H + CH - 1) / CH;
-
-    const int task = blockIdx.x * NW + warp;
-    if (task < E * C) {
-        const int j = task / C, c = task % C;
-        const uint8_t *row = a.W + (size_t)j * H * BYTES;
-        float wf[kRouterUnroll][EPL];
+    const int j = task / C, c = task % C;
+    const uint8_t *row = a.W + (size_t)j * H * BYTES;
+    float wf[kRouterUnroll][EPL];
+#pragma unroll
+    for (int u = 0; u < kRouterUnroll; ++u) {
+        const int k = c * CH + (u * kWarp + lane) * EPL;
+        if (k < H) {
+            Fmt<DT>::unpack(ld_stream16(row + (size_t)k * BYTES), wf[u]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) wf[u][e] = 0.f;
+        }
+    }
+    if (kPdl) pdl_wait();  // the router weights above do not depend on the previous kernel; h does
+    for (int b = 0; b < B; ++b) {
+        float acc = 0.f, ss = 0.f;
 #pragma unroll
         for (int u = 0; u < kRouterUnroll; ++u) {
             const int k = c * CH + (u * kWarp + lane) * EPL;
             if (k < H) {
-                Fmt<DT>::unpack(ld_stream16(row + (size_t)k * BYTES), wf[u]);
-            } else {
 #pragma unroll
-                for (int e = 0; e < EPL; ++e) wf[u][e] = 0.f;
-            }
-        }
-        pdl_wait();  // the router weights above do not depend on the previous kernel; h does
-        for (int b = 0; b < B; ++b) {
-            float acc = 0.f, ss = 0.f;
-#pragma unroll
-            for (int u = 0; u < kRouterUnroll; ++u) {
-                const int k = c * CH + (u * kWarp + lane) * EPL;
-                if (k < H) {
-#pragma unroll
-                    for (int e = 0; e < EPL; e += 4) {
-                        const float4 v = ld_f4(a.h + (size_t)b * H + k + e);
-                        acc = fmaf(wf[u][e], v.x, acc), acc = fmaf(wf[u][e + 1], v.y, acc);
-                        acc = fmaf(wf[u][e + 2], v.z, acc), acc = fmaf(wf[u][e + 3], v.w, acc);
-                        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-                    }
+                for (int e = 0; e < EPL; e += 4) {
+                    const float4 v = ld_f4(a.h + (size_t)b * H + k + e);
+                    acc = fmaf(wf[u][e], v.x, acc), acc = fmaf(wf[u][e + 1], v.y, acc);
+                    acc = fmaf(wf[u][e + 2], v.z, acc), acc = fmaf(wf[u][e + 3], v.w, acc);
+                    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
                 }
             }
-            acc = warp_sum(acc);
-            if (j == 0) ss = warp_sum(ss);
-            if (lane == 0) {
-                a.part[((size_t)c * B + b) * E + j] = acc;
-                if (j == 0) a.ss_part[c * B + b] = ss;
-            }
+        }
+        acc = warp_sum(acc);
+        if (j == 0) ss = warp_sum(ss);
+        if (lane == 0) {
+            a.part[((size_t)c * B + b) * E + j] = acc;
+            if (j == 0) a.ss_part[c * B + b] = ss;
         }
     }
-    pdl_wait();  // warps without a task: nothing below may run ahead of the previous kernel either
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = (atomicAdd(a.arrivals, 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    if (threadIdx.x == 0) *a.arrivals = 0u;
+}
 
-    for (int b = warp; b < B; b += NW) {
+// Sum the split-K partials in a fixed order, apply the RMSNorm factor, softmax/top-K every
+// sequence (one warp each, nw warps) and group the batch by expert.  Needs all 256+ threads
+// of the CTA for the grouping; s_ids [B*K], s_scan [2*(kMaxExperts+1)].
+template <int DT>
+__device__ __forceinline__ void router_finalize(const RouterArgs &a, int *s_ids, int *s_scan, int nw)
+{
+    constexpr int CH = router_chunk_cols<DT>();
+    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
+    const int B = a.tk.B, E = a.tk.E, H = a.H;
+    const int C = (H + CH - 1) / CH;
+    for (int b = warp; b < B; b += nw) {
         float ss = 0.f;
         for (int c = 0; c < C; ++c) ss += __ldcg(a.ss_part + c * B + b);
         const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
@@ -349,11 +345,33 @@ __global__ void __launch_bounds__(256) router_fused_kernel(RouterArgs a)
             z[v] = j < E ? s * inv : -INFINITY;
             if (j < E && a.logits_out) a.logits_out[(size_t)b * E + j] = z[v];
         }
-        route_token(z, s_z[warp], s_ids + b * a.tk.K, a.tk, b, lane);
+        route_token(z, nullptr, s_ids + b * a.tk.K, a.tk, b, lane);
     }
     if (a.tk.wl.n_groups == nullptr) return;
     __syncthreads();
-    group_tokens(s_ids, s_scan, B, E, a.tk.K, a.tk.n_shared, a.tk.mt, a.tk.wl);
+    if (threadIdx.x < 256) group_tokens(s_ids, s_scan, B, E, a.tk.K, a.tk.n_shared, a.tk.mt, a.tk.wl);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(256) router_fused_kernel(RouterArgs a)
+{
+    constexpr int CH = router_chunk_cols<DT>(), NW = 8;
+    __shared__ int s_ids[kMaxBatch * kMaxTopK];
+    __shared__ int s_scan[2 * (kMaxExperts + 1)];
+    __shared__ int s_last;
+    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
+    const int C = (a.H + CH - 1) / CH;
+    const int task = blockIdx.x * NW + warp;
+    if (task < a.tk.E * C) router_task<DT, true>(a, task, lane);
+    pdl_wait();  // warps without a task: nothing below may run ahead of the previous kernel either
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(a.arrivals, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (threadIdx.x == 0) *a.arrivals = 0u;
+    router_finalize<DT>(a, s_ids, s_scan, NW);
 }
 
 }  // namespace stmoe_dev

@@ -15,6 +15,7 @@
 #include "ffn.cuh"
 #include "predictor.cuh"
 #include "router.cuh"
+#include "token_kernel.cuh"
 
 using namespace stmoe_dev;
 
@@ -126,6 +127,18 @@ int occ_down(int dt, int mt)
 #undef OCC_D
     return n;
 }
+
+template <int DT, int MT> void *token_kernel_ptr(int rdt)
+{
+    return rdt == STMOE_F32 ? (void *)decode_token_kernel<DT, 0, MT> : (void *)decode_token_kernel<DT, 1, MT>;
+}
+void *token_kernel(int dt, int rdt, int mt)
+{
+    if (dt == STMOE_F32) return mt == 1 ? token_kernel_ptr<0, 1>(rdt) : token_kernel_ptr<0, 4>(rdt);
+    if (dt == STMOE_BF16) return mt == 1 ? token_kernel_ptr<1, 1>(rdt) : token_kernel_ptr<1, 4>(rdt);
+    return mt == 1 ? token_kernel_ptr<2, 1>(rdt) : token_kernel_ptr<2, 4>(rdt);
+}
+size_t token_smem(int B, int K, int n_shared) { return sizeof(int) * (size_t)(4 + 5 * B * (K + n_shared) + 3 * B * K); }
 
 int sm_count()
 {
@@ -252,6 +265,7 @@ struct stmoe {
     int KS = 0;           // K + n_shared
     int max_pred = 0;
     int S = 1;            // column splits of the down projection
+    unsigned *d_err = nullptr;  // set by a kernel whose bounded wait ran out
     size_t img_bytes = 0;
     int next_layer = 0;
     int64_t host_t = 0;
@@ -285,6 +299,12 @@ struct stmoe {
     int64_t graph_launches = 0;
     int graph_captures = 0;
     bool graph_off = false;
+
+    // persistent one-kernel decode step of resident stacks (token_kernel.cuh)
+    bool persistent = false;
+    int persistent_grid = 0;
+    float *d_hbuf = nullptr, *d_rpart_all = nullptr, *d_sspart_all = nullptr, *d_act_all = nullptr, *d_part_all = nullptr;
+    unsigned *d_tiles_all = nullptr, *d_barrier = nullptr;
 
     SlotCache cache;
     cudaStream_t copy_stream = nullptr;
@@ -615,6 +635,40 @@ int token_eager(stmoe *s, int batch, const float *h_in, float *h_out, int32_t *r
     return join_side(s, st);
 }
 
+int token_persistent(stmoe *s, int batch, const float *h_in, float *h_out, int32_t *routed_ids, float *routed_w,
+                     int32_t *predicted_ids, int32_t *n_predicted, uint32_t *flags, cudaStream_t st)
+{
+    const stmoe_config_t &c = s->cfg;
+    TokenArgs a{};
+    a.L = c.n_layers, a.B = batch, a.E = c.n_experts, a.K = c.top_k, a.n_shared = c.n_shared;
+    a.H = c.hidden, a.I = c.inter, a.S = s->S, a.mt = batch == 1 ? 1 : 4;
+    a.renorm = (c.flags & STMOE_FLAG_RENORM_TOPK) ? 1 : 0;
+    a.eps = c.rms_eps, a.residual_scale = c.residual_scale;
+    a.h_in = h_in, a.h_out = h_out, a.hbuf = s->d_hbuf;
+    a.router = s->d_router, a.blob = s->d_blob_table;
+    a.rpart = s->d_rpart_all, a.sspart = s->d_sspart_all, a.act = s->d_act_all, a.part = s->d_part_all;
+    a.tile_done = s->d_tiles_all;
+    a.ids_all = s->d_ids, a.Bmax = c.max_batch;
+    a.ids_out = routed_ids, a.w_out = routed_w, a.flags_out = flags;
+    a.pred_ids = predicted_ids, a.n_pred = n_predicted, a.max_pred = s->max_pred;
+    a.pst = s->pst, a.P = c.profile_tokens, a.mode = c.predictor_mode;
+    a.barrier = s->d_barrier, a.err = s->d_err;
+    CU_TRY(cudaMemsetAsync(s->d_barrier, 0, 4, st));
+    void *args[] = {&a};
+    CU_TRY(cudaLaunchCooperativeKernel(token_kernel(c.weight_dtype, s->rdt, a.mt), dim3(s->persistent_grid),
+                                       dim3(kFfnThreads), args, token_smem(batch, c.top_k, c.n_shared), st));
+    s->launches += 1;
+    if (!s->built && s->host_t == c.profile_tokens - 1) {
+        const int rows = (c.n_layers - 1) * c.n_experts;
+        if (rows > 0) cct_build_kernel<<<(rows + 7) / 8, 256, 0, st>>>(s->pst, c.n_layers, c.n_experts, c.top_k);
+        s->launches += rows > 0;
+        s->built = true;
+        CU_TRY(cudaGetLastError());
+    }
+    s->host_t += 1;
+    return STMOE_OK;
+}
+
 size_t state_bytes(const stmoe_config_t &c)
 {
     const size_t pairs = c.n_layers > 1 ? c.n_layers - 1 : 0;
@@ -657,7 +711,8 @@ int stmoe_destroy(stmoe_t *s)
     if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
     void *dev[] = {s->d_router, s->d_resident, s->d_shared, s->d_slots, (void *)s->d_blob_table,
                    s->pst.Co, s->pst.cct_id, s->pst.cct_conf, s->pst.HT, s->pst.t, s->pst.pred_mask,
-                   s->pst.pred_valid, s->pst.stats, s->d_rpart, s->d_sspart, s->d_arrivals, s->d_tile_done, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
+                   s->pst.pred_valid, s->pst.stats, s->d_rpart, s->d_sspart, s->d_arrivals, s->d_tile_done, s->d_hbuf, s->d_rpart_all, s->d_sspart_all,
+                   s->d_act_all, s->d_part_all, s->d_tiles_all, s->d_barrier, s->d_err, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
                    s->d_ids, s->d_queue};
     for (void *p : dev)
         if (p) cudaFree(p);
@@ -778,6 +833,36 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
     if (s->wlm.alloc(B * s->KS) != STMOE_OK) return fail(STMOE_ERR_OOM);
     s->plan1 = make_plan(c.weight_dtype, 1);
     s->plan4 = make_plan(c.weight_dtype, 4);
+    if (c.cache_slots == 0 && !(c.flags & STMOE_FLAG_NO_PERSISTENT)) {
+        int dev = 0, coop = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+        const size_t smem = token_smem(B, K, c.n_shared);
+        bool ok = coop != 0 && smem <= 64 * 1024;
+        for (int mt = 1; ok && mt <= 4; mt += 3) {
+            void *k = token_kernel(c.weight_dtype, s->rdt, mt);
+            int occ = 0;
+            ok = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess &&
+                 cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kFfnThreads, smem) == cudaSuccess && occ >= 1;
+        }
+        (void)cudaGetLastError();
+        if (ok) {
+            const int ch = s->rdt == STMOE_F32 ? router_chunk_cols<0>() : router_chunk_cols<1>();
+            const size_t C = (H + ch - 1) / ch, tiles = (H + kTileRows - 1) / kTileRows, pairs = (size_t)B * s->KS;
+            CR_TRY(cudaMalloc(&s->d_hbuf, sizeof(float) * (size_t)(L + 1) * B * H));
+            CR_TRY(cudaMalloc(&s->d_rpart_all, sizeof(float) * L * C * B * E));
+            CR_TRY(cudaMalloc(&s->d_sspart_all, sizeof(float) * L * C * B));
+            CR_TRY(cudaMalloc(&s->d_act_all, sizeof(float) * L * pairs * I));
+            CR_TRY(cudaMalloc(&s->d_part_all, sizeof(float) * L * pairs * s->S * H));
+            CR_TRY(cudaMalloc(&s->d_tiles_all, sizeof(unsigned) * L * tiles));
+            CR_TRY(cudaMemset(s->d_tiles_all, 0, sizeof(unsigned) * L * tiles));
+            CR_TRY(cudaMalloc(&s->d_barrier, 16));
+            CR_TRY(cudaMalloc(&s->d_err, 16));
+            CR_TRY(cudaMemset(s->d_err, 0, 16));
+            s->persistent = true;
+            s->persistent_grid = sm_count();
+        }
+    }
     if (c.profile_tokens == 0 && L > 1) {
         const int rows = (L - 1) * E;
         cct_build_kernel<<<(rows + 7) / 8, 256>>>(s->pst, L, E, K);
@@ -851,6 +936,8 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, i
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const stmoe_config_t &c = s->cfg;
     const bool build_due = !s->built && s->host_t == c.profile_tokens - 1;
+    if (s->persistent && !s->time_kernels)
+        return token_persistent(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
     if (offloaded(s) || s->time_kernels || s->graph_off || build_due)
         return token_eager(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
 
@@ -901,6 +988,11 @@ int stmoe_stats(stmoe_t *s, stmoe_stats_t *out)
     if (!s || !out) return STMOE_ERR_BAD_ARG;
     CU_TRY(cudaDeviceSynchronize());
     harvest_spans(s, true);
+    if (s->d_err) {
+        unsigned err = 0;
+        CU_TRY(cudaMemcpy(&err, s->d_err, 4, cudaMemcpyDeviceToHost));
+        if (err) return STMOE_ERR_TIMEOUT;
+    }
     unsigned long long st[8];
     long long t[2];
     CU_TRY(cudaMemcpy(st, s->pst.stats, sizeof(st), cudaMemcpyDeviceToHost));
@@ -1147,3 +1239,11 @@ extern "C" int stmoe_moe_ffn_static(const float *h, const float *inv_rms, const 
                          residual_scale, h_out, g_static_scratch_ptr[dev], (size_t)STMOE_STATIC_SCRATCH_BYTES,
                          cuda_stream);
 }
+
+#ifdef STMOE_DBG_PHASES
+extern "C" int stmoe_dbg_phases(unsigned long long *out, int n)
+{
+    cudaDeviceSynchronize();
+    return cudaMemcpyFromSymbol(out, g_dbg_phases, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -3;
+}
+#endif

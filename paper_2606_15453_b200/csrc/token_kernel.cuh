@@ -1,0 +1,279 @@
+// One decode step of a resident stack as a single persistent kernel.
+//
+// One 512-thread CTA per SM, launched cooperatively (all CTAs resident), walks the layers:
+//   R   split-K router GEMV tasks dealt over all warps of the grid        -> grid barrier
+//   T   every CTA sums the partial logits and runs softmax / top-K / grouping for the whole
+//       batch itself (redundantly: cheaper than one CTA doing it while 147 wait, and the work
+//       list then lives in shared memory); CTA 0 also writes the step's outputs
+//   GU  gate/up projection over this CTA's share of the rows              -> grid barrier
+//   D   down projection + fused weighted sum / residual                   -> grid barrier
+// so a layer costs three grid barriers (about a microsecond each) instead of three kernel
+// launches with their launch latency, ramp-up and drain.  The predictor (Algorithms 1-3) runs
+// on one warp of the last CTA beside the GU phase of the same layer.
+//
+// Coherence: data that other SMs produce inside this launch is either read past L1
+// (ld.global.cg: router partials, down-projection partials) or lives at an address that is
+// unique to the layer (hidden state, activations), so a line can never be in an SM's L1 before
+// its producer has written it and a grid barrier has been passed.
+// Grid barrier: one monotonically increasing counter; every wait is bounded and a timeout
+// raises an error word that makes all later barriers fall through, so the kernel always ends.
+#pragma once
+#include "device_utils.cuh"
+#include "ffn.cuh"
+#include "predictor.cuh"
+#include "router.cuh"
+
+namespace stmoe_dev {
+
+constexpr int kBarrierSpinLimit = 1 << 22;
+
+#ifdef STMOE_DBG_PHASES
+__device__ unsigned long long g_dbg_phases[8192];
+__device__ __forceinline__ void dbg_stamp(int idx)
+{
+    if (threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        if (blockIdx.x == 0 && idx < 2048) g_dbg_phases[idx] = t;
+        if (idx >= 16 && idx < 24) g_dbg_phases[4096 + blockIdx.x * 8 + (idx - 16)] = t;  // layer 2, every CTA
+    }
+}
+#define DBG_STAMP(i) dbg_stamp(i)
+#else
+#define DBG_STAMP(i)
+#endif
+
+struct TokenArgs {
+    int L, B, E, K, n_shared, H, I, S, mt, renorm;
+    float eps, residual_scale;
+    const float *h_in;              // [B][H]
+    float *h_out;                   // [B][H]
+    float *hbuf;                    // [L][B][H]   input of layers 1..L-1 lives in hbuf[l]
+    const uint8_t *router;          // [L][E][H]
+    const uint8_t *const *blob;     // [L][E+n_shared]
+    float *rpart, *sspart;          // [L][C][B][E], [L][C][B]
+    float *act, *part;              // [L][B*KS][I], [L][B*KS][S][H]
+    unsigned *tile_done;            // [L][ceil(H/32)]
+    int32_t *ids_all;               // [L][Bmax][K] library copy of the routing
+    int Bmax;
+    int32_t *ids_out;               // optional [L][B][K]
+    float *w_out;                   // optional [L][B][K]
+    uint32_t *flags_out;            // optional [L][B]
+    int32_t *pred_ids;              // optional [L][B][max_pred]
+    int32_t *n_pred;                // optional [L][B]
+    int max_pred;
+    PredState pst;
+    int P, mode;
+    unsigned *barrier;              // [1] zero at launch
+    unsigned *err;                  // [1]
+};
+
+// Algorithms 1-3 for one layer step on a single warp (same arithmetic and order as
+// predictor_step_kernel; rows are updated in place in global memory, which only this warp
+// touches during the launch).  cur/prev: routing of this and the previous layer [B][K].
+__device__ __forceinline__ void predictor_step_warp(const TokenArgs &a, int layer, const int *cur, const int *prev,
+                                                    int *s_score, int lane)
+{
+    const int E = a.E, K = a.K, L = a.L, B = a.B;
+    const PredState &st = a.pst;
+    const long long t = *st.t;
+    const bool runtime = t >= a.P;
+    const bool last_profiling = (!runtime) && t == a.P - 1 && layer == L - 1;
+    if (runtime) {
+        for (int b = 0; b < B; ++b) {
+            const bool valid = st.pred_valid[b] != 0;
+            int np = 0, nh = 0;
+            if (valid) {
+                if (lane < 8) np = __popc(st.pred_mask[b * 8 + lane]);
+                if (lane < K) {
+                    const int f = cur[b * K + lane];
+                    nh = (st.pred_mask[b * 8 + (f >> 5)] >> (f & 31)) & 1u;
+                }
+            }
+            np = __reduce_add_sync(kFull, np);
+            nh = __reduce_add_sync(kFull, nh);
+            if (lane == 0) {
+                atomicAdd(&st.stats[0], 1ull);
+                atomicAdd(&st.stats[1], (unsigned long long)K);
+                atomicAdd(&st.stats[2], (unsigned long long)np);
+                atomicAdd(&st.stats[3], (unsigned long long)nh);
+            }
+        }
+        if (layer > 0) {
+            uint8_t *gid = st.cct_id + (size_t)(layer - 1) * E * K;
+            uint8_t *gcf = st.cct_conf + (size_t)(layer - 1) * E * K;
+            for (int b = 0; b < B; ++b)
+                for (int k = 0; k < K; ++k) {
+                    const int e = prev[b * K + k];
+                    update_row(gid + e * K, gcf + e * K, K, cur + b * K, lane);
+                    __syncwarp();
+                }
+        }
+    } else if (layer > 0) {
+        uint32_t *Co = st.Co + (size_t)(layer - 1) * E * E;
+        for (int i = lane; i < B * K * K; i += kWarp) {
+            const int b = i / (K * K), r = i % (K * K);
+            atomicAdd(&Co[(size_t)prev[b * K + r / K] * E + cur[b * K + r % K]], 1u);
+        }
+    }
+    __syncwarp();
+
+    const bool predict_now = runtime || last_profiling;
+    const int next = (layer + 1) % L;
+    const bool spatial = predict_now && (a.mode & 2) && layer < L - 1;
+    const bool temporal = predict_now && (a.mode & 1);
+    int32_t *pred_ids = a.pred_ids ? a.pred_ids + (size_t)layer * B * a.max_pred : nullptr;
+    int32_t *n_pred = a.n_pred ? a.n_pred + (size_t)layer * B : nullptr;
+    for (int b = 0; b < B; ++b) {
+        for (int f = lane; f < kMaxExperts; f += kWarp) s_score[f] = 0;
+        __syncwarp();
+        if (spatial) {
+            const uint8_t *cid = st.cct_id + (size_t)layer * E * K;
+            const uint8_t *ccf = st.cct_conf + (size_t)layer * E * K;
+            for (int k = 0; k < K; ++k) {
+                const int e = cur[b * K + k];
+                if (lane < K) s_score[cid[e * K + lane]] += ccf[e * K + lane];
+                __syncwarp();
+            }
+        }
+        if (temporal) {
+            if (lane < K) {
+                const int hte = st.HT[((size_t)b * L + next) * K + lane];
+                if (hte >= 0) s_score[hte] += kThreshold;
+            }
+            __syncwarp();
+        }
+        int count = 0;
+        for (int w = 0; w < kMaxExperts / kWarp; ++w) {
+            const int f = w * kWarp + lane;
+            const bool in = f < E && s_score[f] >= kThreshold;
+            const unsigned msk = __ballot_sync(kFull, in);
+            if (lane == 0) st.pred_mask[b * 8 + w] = msk;
+            if (in) {
+                const int pos = count + __popc(msk & ((1u << lane) - 1u));
+                if (pred_ids && pos < a.max_pred) pred_ids[(size_t)b * a.max_pred + pos] = f;
+            }
+            count += __popc(msk);
+        }
+        if (pred_ids)
+            for (int i = count + lane; i < a.max_pred; i += kWarp) pred_ids[(size_t)b * a.max_pred + i] = -1;
+        if (lane == 0) {
+            st.pred_valid[b] = predict_now ? 1u : 0u;
+            if (n_pred) n_pred[b] = count;
+        }
+        __syncwarp();
+    }
+    for (int i = lane; i < B * K; i += kWarp) {
+        const int b = i / K, k = i % K;
+        st.HT[((size_t)b * L + layer) * K + k] = (int16_t)cur[b * K + k];
+    }
+    __syncwarp();
+    if (lane == 0 && layer == L - 1) *st.t = t + 1;
+}
+
+// Bounded grid barrier on a monotonically increasing counter.
+__device__ __forceinline__ void grid_barrier(unsigned *counter, unsigned *err, unsigned &target, volatile int *s_dead,
+                                             int dbg_idx = -1)
+{
+    target += gridDim.x;
+    __syncthreads();
+    if (dbg_idx >= 0) DBG_STAMP(dbg_idx);
+    if (threadIdx.x == 0 && !*s_dead) {
+        __threadfence();
+        atomicAdd(counter, 1u);
+        int spins = 0;
+        for (;;) {
+            unsigned seen;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+            if (seen >= target) break;
+            if (++spins > kBarrierSpinLimit || *((volatile unsigned *)err)) {
+                *err = 1u;
+                *s_dead = 1;
+                break;
+            }
+        }
+        __threadfence();
+    }
+    __syncthreads();
+}
+
+template <int DT, int RDT, int MTMAX>
+__global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs a)
+{
+    constexpr int CH = router_chunk_cols<RDT>(), NW = kFfnThreads / kWarp;
+    extern __shared__ __align__(16) int dyn[];  // work list | ids | prev ids | gate weights
+    __shared__ int s_scan[2 * (kMaxExperts + 1)];
+    __shared__ int s_score[kMaxExperts];
+    __shared__ float s_inv[kMaxBatch];
+    __shared__ int s_next, s_dead;
+    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
+    const int L = a.L, B = a.B, E = a.E, K = a.K, H = a.H, I = a.I, S = a.S;
+    const int KS = K + a.n_shared, pairs = B * KS;
+    const int C = (H + CH - 1) / CH, tiles = (H + kTileRows - 1) / kTileRows;
+
+    WorkList wl;
+    wl.n_groups = dyn, wl.g_expert = dyn + 4, wl.g_start = dyn + 4 + pairs, wl.g_count = dyn + 4 + 2 * pairs;
+    wl.pair_token = dyn + 4 + 3 * pairs, wl.pair_slot = dyn + 4 + 4 * pairs;
+    int *s_ids = dyn + 4 + 5 * pairs;
+    int *s_prev = s_ids + B * K;
+    float *s_w = reinterpret_cast<float *>(s_prev + B * K);
+    if (threadIdx.x == 0) s_dead = 0;
+    unsigned target = 0;
+    const bool lead = blockIdx.x == 0;
+    const bool pred_cta = blockIdx.x == gridDim.x - 1;
+
+    for (int l = 0; l < L; ++l) {
+        const float *h = l == 0 ? a.h_in : a.hbuf + (size_t)l * B * H;
+        float *h_next = l == L - 1 ? a.h_out : a.hbuf + (size_t)(l + 1) * B * H;
+
+        // ---- R: split-K router GEMV -------------------------------------------------------
+        RouterArgs ra;
+        ra.h = h, ra.W = a.router + (size_t)l * E * H * Fmt<RDT>::kBytes, ra.H = H, ra.eps = a.eps;
+        ra.part = a.rpart + (size_t)l * C * B * E, ra.ss_part = a.sspart + (size_t)l * C * B;
+        ra.arrivals = nullptr, ra.inv_rms = s_inv, ra.logits_out = nullptr;
+        TopkArgs &tk = ra.tk;
+        tk.logits = nullptr, tk.B = B, tk.E = E, tk.K = K, tk.n_shared = a.n_shared, tk.mt = a.mt, tk.renorm = a.renorm;
+        tk.ids = s_ids, tk.w = s_w;
+        tk.ids_out = (lead && a.ids_out) ? a.ids_out + (size_t)l * B * K : nullptr;
+        tk.w_out = (lead && a.w_out) ? a.w_out + (size_t)l * B * K : nullptr;
+        tk.flags_out = (lead && a.flags_out) ? a.flags_out + (size_t)l * B : nullptr;
+        tk.near_tie_counter = lead ? a.pst.stats + 4 : nullptr;
+        tk.wl = wl;
+        DBG_STAMP(l * 8 + 0);
+        {
+            const int task = warp * gridDim.x + blockIdx.x;  // spread the tasks over the SMs first
+            if (task < E * C) router_task<RDT, false>(ra, task, lane);
+        }
+        grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 1);
+        DBG_STAMP(l * 8 + 2);
+
+        // ---- T: softmax / top-K / grouping, redundantly per CTA ---------------------------
+        router_finalize<RDT>(ra, s_ids, s_scan, NW);
+        __syncthreads();
+        if (lead)
+            for (int i = threadIdx.x; i < B * K; i += blockDim.x)
+                a.ids_all[(size_t)l * a.Bmax * K + i] = s_ids[i];
+
+        DBG_STAMP(l * 8 + 3);
+        // ---- GU (+ the predictor on one warp of the last CTA) -----------------------------
+        FfnArgs fa;
+        fa.h = h, fa.inv_rms = s_inv, fa.wl = wl, fa.blob = a.blob + (size_t)l * (E + a.n_shared);
+        fa.act = a.act + (size_t)l * pairs * I, fa.part = a.part + (size_t)l * pairs * S * H;
+        fa.H = H, fa.I = I, fa.E = E, fa.S = S;
+        fa.w = s_w, fa.h_out = h_next, fa.tile_done = a.tile_done + (size_t)l * tiles;
+        fa.B = B, fa.K = K, fa.n_shared = a.n_shared, fa.residual_scale = a.residual_scale;
+        gate_up_phase<DT, MTMAX>(fa, &s_next, [&]() {
+            if (pred_cta && warp == NW - 1) predictor_step_warp(a, l, s_ids, s_prev, s_score, lane);
+        });
+        grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 4);
+        DBG_STAMP(l * 8 + 5);
+
+        // ---- D ---------------------------------------------------------------------------
+        down_phase<DT, MTMAX, false>(fa, &s_next);
+        for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
+        grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 6);
+        DBG_STAMP(l * 8 + 7);
+    }
+}
+
+}  // namespace stmoe_dev

@@ -121,36 +121,44 @@ def test_tiny_cache_thrashes_but_stays_correct():
     assert st["prefetch_issued"] > 0
 
 
-def test_graph_replay_matches_eager_decode():
-    """decode_token on a capturable stream replays a CUDA graph; on the default stream it
-    launches kernel by kernel.  Outputs, routing, predictions and tables must be identical."""
+@pytest.mark.parametrize("B", [1, 4])
+def test_decode_token_paths_agree(B):
+    """decode_token has three execution paths for a resident stack: the persistent one-kernel
+    step (default), per-layer kernels replayed as a CUDA graph (capturable stream), and per-layer
+    kernels launched one by one (default stream).  Outputs, routing, predictions, tables and
+    counters must be identical, bit for bit."""
     cfg = stacks.CONFIGS["C2"].scaled(n_layers=3, hidden=512, inter=352, n_experts=16, top_k=3,
                                       profile_tokens=3)
-    B, T = 4, 10
+    T = 10
     x = stacks.token_inputs(cfg, B, T).to(DEV)
     results = []
-    for use_graph in (False, True):
-        pr = Pair(cfg, B, oracle=False)
+    for path in ("persistent", "graph", "eager"):
+        pr = Pair(cfg, B, oracle=False, flags=0 if path == "persistent" else P.FLAG_NO_PERSISTENT)
         L, K = cfg.n_layers, cfg.top_k
         ids = torch.empty(L, B, K, dtype=torch.int32, device=DEV)
+        w = torch.empty(L, B, K, dtype=torch.float32, device=DEV)
         pred = torch.empty(L, B, pr.stack.max_pred, dtype=torch.int32, device=DEV)
+        npred = torch.empty(L, B, dtype=torch.int32, device=DEV)
         h_in, ho = torch.empty(B, cfg.hidden, device=DEV), torch.empty(B, cfg.hidden, device=DEV)
-        stream = torch.cuda.Stream() if use_graph else torch.cuda.current_stream()
+        stream = torch.cuda.Stream() if path == "graph" else torch.cuda.current_stream()
         rec = []
         with torch.cuda.stream(stream):
             for t in range(T):
                 h_in.copy_(x[t])
-                pr.stack.decode_token(h_in, ho, ids, None, pred, None, stream=stream)
+                pr.stack.decode_token(h_in, ho, ids, w, pred, npred, stream=stream)
                 stream.synchronize()
-                rec.append((ho.cpu().clone(), ids.cpu().clone(), pred.cpu().clone()))
+                rec.append((ho.cpu().clone(), ids.cpu().clone(), w.cpu().clone(), pred.cpu().clone(),
+                            npred.cpu().clone()))
         results.append((rec, pr.stack.export_state(), pr.stack.stats()))
         pr.close()
-    (ra, sa, ta), (rb, sb, tb) = results
-    for a, b in zip(ra, rb):
-        assert all(torch.equal(u, v) for u, v in zip(a, b))
-    assert sa == sb
-    for k in ("runtime_steps", "routed", "predicted", "hits", "decode_steps", "kernel_launches"):
-        assert ta[k] == tb[k], k
+    ref_rec, ref_state, ref_stats = results[0]
+    for rec, state, st in results[1:]:
+        for a, b in zip(ref_rec, rec):
+            assert all(torch.equal(u, v) for u, v in zip(a, b))
+        assert state == ref_state
+        for k in ("runtime_steps", "routed", "predicted", "hits", "decode_steps", "near_ties"):
+            assert st[k] == ref_stats[k], k
+    assert ref_stats["kernel_launches"] < results[1][2]["kernel_launches"]
 
 
 def test_argument_and_state_errors():
