@@ -31,10 +31,11 @@ sys.path.insert(0, ROOT)
 from datagen import stacks  # noqa: E402
 
 METRIC, UNIT = "decode_tokens_per_s", "tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one gate/up launch at this workload, from the
-# ncu capture summarised in profiles/ffn_kernels_c1_2layers_ncu_full.md (taken on a 2-layer stack
-# of the same shape: one launch does the same work there, so no scaling is applied).
-NCU_TRAFFIC_BYTES = {"C1": 469797888 + 3237120}
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_token_kernel launch, from the ncu
+# capture summarised in profiles/decode_token_kernel_c1_2layers_ncu_full.md.  The capture ran a
+# 2-layer stack of the same shape (1409.598 MB read + 4.767 MB written); traffic grows in
+# proportion to the layer count, so the full launch is that figure x layers / 2.
+NCU_TRAFFIC_BYTES_PER_LAYER = {"C1": (1409598000 + 4766976) / 2}
 
 
 def measured_peaks():
@@ -297,6 +298,8 @@ def main():
     run = {k: s1[k] - s0[k] for k in ("runtime_steps", "routed", "predicted", "hits", "near_ties",
                                       "cache_hits", "cache_misses", "kernel_launches")}
     step_gbs = statistics.mean(step_bytes) / (ms / args.steps * 1e-3) / 1e9
+    persistent = cfg.cache_slots == 0          # resident stacks: one kernel launch per decode step
+    per_layer = NCU_TRAFFIC_BYTES_PER_LAYER.get(args.workload) if batch == 1 else None
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -310,14 +313,22 @@ def main():
                 "h2d_bytes_per_step": batch * H * 4,
                 "d2h_bytes_per_step": batch * H * 4 + L * batch * K * 4},
         "gpu_launches": run["kernel_launches"],
-        "roofline": {"bound": "hbm", "kernel": "gate_up_kernel", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm",
+                     "kernel": "decode_token_kernel" if persistent else "gate_up_kernel",
+                     "achieved": step_gbs if persistent else achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s",
-                     "frac": achieved / peak if achieved else None,
-                     "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                     "algorithmic_bytes_per_launch": gate_up_bytes, "us_per_launch": gu_ms * 1e3,
-                     "down_kernel": {"achieved": (gate_up_bytes / 2) / (dn_ms * 1e-3) / 1e9 if dn_ms else None,
-                                     "us_per_launch": dn_ms * 1e3},
-                     "router_kernel": {"us_per_launch": s2["router_ms"] / max(n_ffn, 1) * 1e3},
+                     "frac": (step_gbs if persistent else achieved or 0.0) / peak,
+                     "frac_of_8000": (step_gbs if persistent else achieved or 0.0) / 8000.0,
+                     "traffic": per_layer * L if (persistent and per_layer) else None,
+                     "algorithmic_bytes_per_launch": statistics.mean(step_bytes) if persistent else gate_up_bytes,
+                     "us_per_launch": ms / args.steps * 1e3 if persistent else gu_ms * 1e3,
+                     "per_layer_kernels": {
+                         "note": "second pass over the same steps as per-layer kernels, events around each",
+                         "gate_up": {"achieved": achieved, "us_per_launch": gu_ms * 1e3,
+                                     "algorithmic_bytes_per_launch": gate_up_bytes},
+                         "down": {"achieved": (gate_up_bytes / 2) / (dn_ms * 1e-3) / 1e9 if dn_ms else None,
+                                  "us_per_launch": dn_ms * 1e3},
+                         "router": {"us_per_launch": s2["router_ms"] / max(n_ffn, 1) * 1e3}},
                      "whole_step": {"bytes_per_token": statistics.mean(step_bytes) / batch,
                                     "achieved": step_gbs, "frac": step_gbs / peak,
                                     "frac_of_8000": step_gbs / 8000.0}},
