@@ -183,7 +183,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling runs)")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--ref-layers", type=int, default=2)
-    ap.add_argument("--cpu-sample-layers", type=int, default=8)
+    ap.add_argument("--cpu-sample-layers", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefetch-limit", type=int, default=0, help="offloaded stacks: copies per layer step")
     ap.add_argument("--mode", default="st", choices=["off", "temporal", "spatial", "st"])
