@@ -106,20 +106,75 @@ __device__ __forceinline__ void gemv_rows(const uint8_t *(&rowp)[NMAT][R], int n
     }
 }
 
-// Hands out the CTA's share [first, last) of `total` units in blocks of R to its warps.
+// Cost of streaming one row for a work-list entry, in units of a one-token row: the
+// multi-token code path keeps fewer loads in flight and does more arithmetic per byte, and
+// measures about twice as slow per row.
+constexpr int kMultiTokenRowCost = 2;
+
+// Hands out the CTA's share [first, last) of the rows (rpe per work-list entry) in blocks of R
+// to its warps.  The shares are equal in cost, not in rows: with kWeighted, rows of entries that
+// hold more than one token count kMultiTokenRowCost times, so a CTA that gets them gets fewer.
+// s_tk: three ints of shared memory (ticket, first, last).
 struct BlockTickets {
     int first, last;
-    __device__ void init(int total, int *s_next)
+
+    // row index at which the cumulative cost reaches `target` (warp 0, all lanes)
+    static __device__ int row_at_cost(const WorkList &wl, int n_groups, int rpe, long long target, int lane)
     {
-        first = (int)((long long)total * blockIdx.x / gridDim.x);
-        last = (int)((long long)total * (blockIdx.x + 1) / gridDim.x);
-        if (threadIdx.x == 0) *s_next = first;
-        __syncthreads();
+        long long base = 0;  // cost of the entries before the chunk being scanned
+        for (int g0 = 0; g0 < n_groups; g0 += kWarp) {
+            const int g = g0 + lane;
+            const int w = g < n_groups ? (wl.g_count[g] > 1 ? kMultiTokenRowCost : 1) : 0;
+            int incl = w;
+#pragma unroll
+            for (int o = 1; o < kWarp; o <<= 1) {
+                const int t = __shfl_up_sync(kFull, incl, o);
+                if (lane >= o) incl += t;
+            }
+            const long long end = base + (long long)incl * rpe;        // cost up to and including g
+            const long long beg = end - (long long)w * rpe;
+            const unsigned hit = __ballot_sync(kFull, w > 0 && target >= beg && target < end);
+            if (hit) {
+                const int src = __ffs(hit) - 1;
+                const long long b = __shfl_sync(kFull, beg, src);
+                const int ws = __shfl_sync(kFull, w, src);
+                return (g0 + src) * rpe + (int)((target - b) / ws);
+            }
+            base = __shfl_sync(kFull, end, kWarp - 1);
+        }
+        return n_groups * rpe;
     }
-    __device__ int claim(int *s_next, int R, int lane) const
+
+    template <bool kWeighted> __device__ void init(const WorkList &wl, int rpe, int *s_tk)
+    {
+        const int n_groups = *wl.n_groups;
+        if (!kWeighted) {
+            const int total = n_groups * rpe;
+            first = (int)((long long)total * blockIdx.x / gridDim.x);
+            last = (int)((long long)total * (blockIdx.x + 1) / gridDim.x);
+            if (threadIdx.x == 0) s_tk[0] = first;
+            __syncthreads();
+            return;
+        }
+        if (threadIdx.x < kWarp) {
+            const int lane = threadIdx.x;
+            long long cost = 0;
+            for (int g = lane; g < n_groups; g += kWarp) cost += wl.g_count[g] > 1 ? kMultiTokenRowCost : 1;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) cost += __shfl_xor_sync(kFull, cost, o);
+            cost *= rpe;
+            const int f = row_at_cost(wl, n_groups, rpe, cost * blockIdx.x / gridDim.x, lane);
+            const int l = blockIdx.x + 1 == gridDim.x ? n_groups * rpe
+                                                      : row_at_cost(wl, n_groups, rpe, cost * (blockIdx.x + 1) / gridDim.x, lane);
+            if (lane == 0) s_tk[0] = f, s_tk[1] = f, s_tk[2] = l;
+        }
+        __syncthreads();
+        first = s_tk[1], last = s_tk[2];
+    }
+    __device__ int claim(int *s_tk, int R, int lane) const
     {
         int u = 0;
-        if (lane == 0) u = atomicAdd(s_next, R);
+        if (lane == 0) u = atomicAdd(s_tk, R);
         return __shfl_sync(kFull, u, 0);
     }
 };
@@ -262,7 +317,7 @@ __device__ __forceinline__ void gate_up_phase(const FfnArgs &a, int *s_next, Sid
     const int lane = threadIdx.x % kWarp;
     const int I = a.I;
     BlockTickets tk;
-    tk.init(*a.wl.n_groups * I, s_next);
+    tk.init<(MTMAX > 1)>(a.wl, I, s_next);
     side();
     Entry<MTMAX> en;
 
@@ -289,9 +344,9 @@ __device__ __forceinline__ void gate_up_phase(const FfnArgs &a, int *s_next, Sid
 template <int DT, int MTMAX>
 __global__ void __launch_bounds__(kFfnThreads, 1) gate_up_kernel(FfnArgs a)
 {
-    __shared__ int s_next;
+    __shared__ int s_next[3];
     pdl_launch_dependents();  // the down kernel may move in behind the CTAs of this grid
-    gate_up_phase<DT, MTMAX>(a, &s_next);
+    gate_up_phase<DT, MTMAX>(a, s_next);
 }
 
 // One block of the down projection: rows [r0, r0+nrows) of segment s of entry g.
@@ -347,7 +402,7 @@ __device__ __forceinline__ void down_phase(const FfnArgs &a, int *s_next)
     // columns of one split, a multiple of one warp-wide load
     const int seg = ((I + S - 1) / S + kWarp * EPL - 1) / (kWarp * EPL) * (kWarp * EPL);
     BlockTickets tk;
-    tk.init(*a.wl.n_groups * S * H, s_next);
+    tk.init<(MTMAX > 1)>(a.wl, S * H, s_next);
     Entry<MTMAX> en;
     int u0 = tk.claim(s_next, RC, lane);
     if (kPdl) {
@@ -387,9 +442,9 @@ __device__ __forceinline__ void down_phase(const FfnArgs &a, int *s_next)
 template <int DT, int MTMAX>
 __global__ void __launch_bounds__(kFfnThreads, 1) down_kernel(FfnArgs a)
 {
-    __shared__ int s_next;
+    __shared__ int s_next[3];
     pdl_launch_dependents();  // the next layer's router may move in behind this grid
-    down_phase<DT, MTMAX, true>(a, &s_next);
+    down_phase<DT, MTMAX, true>(a, s_next);
 }
 
 }  // namespace stmoe_dev

@@ -205,7 +205,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs 
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
     __shared__ int s_score[kMaxExperts];
     __shared__ float s_inv[kMaxBatch];
-    __shared__ int s_next, s_dead;
+    __shared__ int s_next[3], s_dead;
     const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
     const int L = a.L, B = a.B, E = a.E, K = a.K, H = a.H, I = a.I, S = a.S;
     const int KS = K + a.n_shared, pairs = B * KS;
@@ -262,14 +262,14 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs 
         fa.H = H, fa.I = I, fa.E = E, fa.S = S;
         fa.w = s_w, fa.h_out = h_next, fa.tile_done = a.tile_done + (size_t)l * tiles;
         fa.B = B, fa.K = K, fa.n_shared = a.n_shared, fa.residual_scale = a.residual_scale;
-        gate_up_phase<DT, MTMAX>(fa, &s_next, [&]() {
+        gate_up_phase<DT, MTMAX>(fa, s_next, [&]() {
             if (pred_cta && warp == NW - 1) predictor_step_warp(a, l, s_ids, s_prev, s_score, lane);
         });
         grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 4);
         DBG_STAMP(l * 8 + 5);
 
         // ---- D ---------------------------------------------------------------------------
-        down_phase<DT, MTMAX, false>(fa, &s_next);
+        down_phase<DT, MTMAX, false>(fa, s_next);
         for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
         grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 6);
         DBG_STAMP(l * 8 + 7);
