@@ -202,18 +202,31 @@ __device__ __forceinline__ void finish_rows(const FfnArgs &a, int r0, int nrows,
             if (lane == 0) a.tile_done[tile] = 0u;
             const int c = tile * kTileRows + lane;
             if (lane < tile_rows) {
-                const int KS = a.K + a.n_shared;
+                // terms in summation order: shared experts, then routed experts, segments
+                // innermost; the loads of eight terms are issued together (each is a trip to
+                // L2), the arithmetic keeps the fixed order
+                const int KS = a.K + a.n_shared, n_terms = KS * S;
                 for (int b = 0; b < a.B; ++b) {
-                    float y = 0.f;
-                    for (int q = 0; q < a.n_shared; ++q) {
-                        float p = 0.f;
-                        for (int z = 0; z < S; ++z) p += __ldcg(a.part + (((size_t)b * KS + a.K + q) * S + z) * H + c);
-                        y += p;
-                    }
-                    for (int k = 0; k < a.K; ++k) {
-                        float p = 0.f;
-                        for (int z = 0; z < S; ++z) p += __ldcg(a.part + (((size_t)b * KS + k) * S + z) * H + c);
-                        y = fmaf(a.w[b * a.K + k], p, y);
+                    float y = 0.f, p = 0.f;
+                    for (int t0 = 0; t0 < n_terms; t0 += 8) {
+                        float v[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int t = t0 + i, q = t / S, z = t % S;
+                            const int slot = q < a.n_shared ? a.K + q : q - a.n_shared;
+                            v[i] = t < n_terms ? __ldcg(a.part + (((size_t)b * KS + slot) * S + z) * H + c) : 0.f;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int t = t0 + i, q = t / S, z = t % S;
+                            if (t < n_terms) {
+                                p += v[i];
+                                if (z == S - 1) {
+                                    y = q < a.n_shared ? y + p : fmaf(a.w[b * a.K + q - a.n_shared], p, y);
+                                    p = 0.f;
+                                }
+                            }
+                        }
                     }
                     a.h_out[(size_t)b * H + c] = fmaf(a.residual_scale, y, a.h[(size_t)b * H + c]);
                 }
