@@ -187,12 +187,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefetch-limit", type=int, default=0, help="offloaded stacks: copies per layer step")
     ap.add_argument("--mode", default="st", choices=["off", "temporal", "spatial", "st"])
+    ap.add_argument("--resident", action="store_true", help="keep every expert in HBM (cache_slots = 0)")
     args = ap.parse_args()
 
     cfg = stacks.CONFIGS[args.workload]
     if args.layers:
         cfg = cfg.scaled(n_layers=args.layers,
                          cache_slots=min(cfg.cache_slots, args.layers * cfg.n_experts))
+    if args.resident:
+        cfg = cfg.scaled(cache_slots=0, name=cfg.name + "-resident")
     batch = args.batch
     if args.impl == "reference":
         return run_reference(args, cfg, batch)

@@ -177,6 +177,16 @@ __device__ __forceinline__ void route_token(const float (&z)[kVpl], float *, int
 __device__ __forceinline__ void group_tokens(const int *s_ids, int *s_scan, int B, int E, int K, int n_shared,
                                              int mt, const WorkList &wl)
 {
+    if (B == 1) {  // one sequence: its K experts (already ascending), then the shared ones
+        const int t = threadIdx.x;
+        if (t < K + n_shared) {
+            wl.g_expert[t] = t < K ? s_ids[t] : E + (t - K);
+            wl.g_start[t] = t, wl.g_count[t] = 1;
+            wl.pair_token[t] = 0, wl.pair_slot[t] = t;
+        }
+        if (t == 0) *wl.n_groups = K + n_shared;
+        return;
+    }
     int *s_g = s_scan, *s_p = s_scan + kMaxExperts + 1;
     const int e = threadIdx.x, KS = K + n_shared, lane = e % kWarp, warp = e / kWarp;
     int cnt = 0;
@@ -345,11 +355,15 @@ __device__ __forceinline__ void router_finalize(const RouterArgs &a, int *s_ids,
             z[v] = j < E ? s * inv : -INFINITY;
             if (j < E && a.logits_out) a.logits_out[(size_t)b * E + j] = z[v];
         }
+        if (b == 0) DBG_STAMP(2000);
         route_token(z, nullptr, s_ids + b * a.tk.K, a.tk, b, lane);
+        if (b == 0) DBG_STAMP(2001);
     }
     if (a.tk.wl.n_groups == nullptr) return;
     __syncthreads();
+    DBG_STAMP(2002);
     if (threadIdx.x < 256) group_tokens(s_ids, s_scan, B, E, a.tk.K, a.tk.n_shared, a.tk.mt, a.tk.wl);
+    DBG_STAMP(2003);
 }
 
 template <int DT>

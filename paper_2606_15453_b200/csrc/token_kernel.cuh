@@ -27,21 +27,6 @@ namespace stmoe_dev {
 
 constexpr int kBarrierSpinLimit = 1 << 22;
 
-#ifdef STMOE_DBG_PHASES
-__device__ unsigned long long g_dbg_phases[8192];
-__device__ __forceinline__ void dbg_stamp(int idx)
-{
-    if (threadIdx.x == 0) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-        if (blockIdx.x == 0 && idx < 2048) g_dbg_phases[idx] = t;
-        if (idx >= 16 && idx < 24) g_dbg_phases[4096 + blockIdx.x * 8 + (idx - 16)] = t;  // layer 2, every CTA
-    }
-}
-#define DBG_STAMP(i) dbg_stamp(i)
-#else
-#define DBG_STAMP(i)
-#endif
 
 struct TokenArgs {
     int L, B, E, K, n_shared, H, I, S, mt, renorm;
