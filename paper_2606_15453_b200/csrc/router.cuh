@@ -330,6 +330,81 @@ __device__ __forceinline__ void router_task(const RouterArgs &a, int task, int l
     }
 }
 
+// Gating of a single sequence by the first 256 threads of the CTA (thread j owns expert j):
+// the latency-critical batch-1 case, where one warp would walk K+1 arg-max rounds alone.
+// Every thread sums its own logit, the softmax statistics are two block reductions, and the
+// top-K is found by rank counting (rank_j = number of experts that beat j; ties: lower id
+// wins), which takes E comparisons per thread but no dependent rounds.  scratch: 320 ints.
+template <int DT>
+__device__ __forceinline__ void route_single_block(const RouterArgs &a, int *s_ids, int *scratch)
+{
+    constexpr int CH = router_chunk_cols<DT>();
+    const int j = threadIdx.x, lane = j % kWarp, warp = j / kWarp;
+    const int E = a.tk.E, K = a.tk.K, H = a.H;
+    const int C = (H + CH - 1) / CH;
+    uint32_t *s_key = reinterpret_cast<uint32_t *>(scratch);      // [256]
+    float *s_red = reinterpret_cast<float *>(scratch + 256);      // [8] max, [8] sum, [8] selected sum
+    float *s_pick = reinterpret_cast<float *>(scratch + 256 + 24); // [0] K-th logit, [1] (K+1)-th
+    int *s_cnt = scratch + 256 + 32;                              // [8] selected per warp
+    auto sync256 = []() { asm volatile("bar.sync 2, 256;" ::: "memory"); };
+
+    float ss = 0.f;
+    for (int c = 0; c < C; ++c) ss += __ldcg(a.ss_part + c);
+    const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
+    if (j == 0) a.inv_rms[0] = inv;
+    float z = -INFINITY;
+    if (j < E) {
+        float s = 0.f;
+        for (int c = 0; c < C; ++c) s += __ldcg(a.part + (size_t)c * E + j);
+        z = s * inv;
+        if (a.logits_out) a.logits_out[j] = z;
+    }
+    const uint32_t key = j < E ? float_key(z) : 0u;
+    s_key[j] = key;
+    const float wm = warp_max(z);
+    if (lane == 0) s_red[warp] = wm;
+    sync256();
+    float m = s_red[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) m = fmaxf(m, s_red[w]);
+    const float ex = j < E ? expf(z - m) : 0.f;
+    const float wsum = warp_sum(ex);
+    if (lane == 0) s_red[8 + warp] = wsum;
+
+    int rank = 0;
+    if (j < E)
+        for (int i = 0; i < E; ++i) {
+            const uint32_t k = s_key[i];
+            rank += (k > key) || (k == key && i < j);
+        }
+    const bool sel = j < E && rank < K;
+    if (j < E && rank == K - 1) s_pick[0] = z;
+    if (j < E && rank == K) s_pick[1] = z;
+    const unsigned msk = __ballot_sync(kFull, sel);
+    const float wsel = warp_sum(sel ? ex : 0.f);
+    if (lane == 0) s_cnt[warp] = __popc(msk), s_red[16 + warp] = wsel;
+    sync256();
+    float sum = 0.f, selsum = 0.f;
+    int pos = __popc(msk & ((1u << lane) - 1u));
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        sum += s_red[8 + w], selsum += s_red[16 + w];
+        if (w < warp) pos += s_cnt[w];
+    }
+    if (sel) {
+        const float p = ex / (a.tk.renorm ? selsum : sum);
+        a.tk.ids[pos] = j, a.tk.w[pos] = p, s_ids[pos] = j;
+        if (a.tk.ids_out) a.tk.ids_out[pos] = j;
+        if (a.tk.w_out) a.tk.w_out[pos] = p;
+    }
+    if (j == 0) {
+        const float gap = K < E ? s_pick[0] - s_pick[1] : INFINITY;
+        const uint32_t f = gap < 1e-4f ? 1u : 0u;
+        if (a.tk.flags_out) a.tk.flags_out[0] = f;
+        if (f && a.tk.near_tie_counter) atomicAdd(a.tk.near_tie_counter, 1ull);
+    }
+}
+
 // Sum the split-K partials in a fixed order, apply the RMSNorm factor, softmax/top-K every
 // sequence (one warp each, nw warps) and group the batch by expert.  Needs all 256+ threads
 // of the CTA for the grouping; s_ids [B*K], s_scan [2*(kMaxExperts+1)].
@@ -340,25 +415,28 @@ __device__ __forceinline__ void router_finalize(const RouterArgs &a, int *s_ids,
     const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
     const int B = a.tk.B, E = a.tk.E, H = a.H;
     const int C = (H + CH - 1) / CH;
-    for (int b = warp; b < B; b += nw) {
-        float ss = 0.f;
-        for (int c = 0; c < C; ++c) ss += __ldcg(a.ss_part + c * B + b);
-        const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
-        if (lane == 0) a.inv_rms[b] = inv;
-        float z[kVpl];
+    if (B == 1) {
+        if (threadIdx.x < 256) route_single_block<DT>(a, s_ids, s_scan);
+    } else {
+        for (int b = warp; b < B; b += nw) {
+            float ss = 0.f;
+            for (int c = 0; c < C; ++c) ss += __ldcg(a.ss_part + c * B + b);
+            const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
+            if (lane == 0) a.inv_rms[b] = inv;
+            float z[kVpl];
 #pragma unroll
-        for (int v = 0; v < kVpl; ++v) {
-            const int j = v * kWarp + lane;
-            float s = 0.f;
-            if (j < E)
-                for (int c = 0; c < C; ++c) s += __ldcg(a.part + ((size_t)c * B + b) * E + j);
-            z[v] = j < E ? s * inv : -INFINITY;
-            if (j < E && a.logits_out) a.logits_out[(size_t)b * E + j] = z[v];
+            for (int v = 0; v < kVpl; ++v) {
+                const int j = v * kWarp + lane;
+                float s = 0.f;
+                if (j < E)
+                    for (int c = 0; c < C; ++c) s += __ldcg(a.part + ((size_t)c * B + b) * E + j);
+                z[v] = j < E ? s * inv : -INFINITY;
+                if (j < E && a.logits_out) a.logits_out[(size_t)b * E + j] = z[v];
+            }
+            route_token(z, nullptr, s_ids + b * a.tk.K, a.tk, b, lane);
         }
-        if (b == 0) DBG_STAMP(2000);
-        route_token(z, nullptr, s_ids + b * a.tk.K, a.tk, b, lane);
-        if (b == 0) DBG_STAMP(2001);
     }
+    DBG_STAMP(2001);
     if (a.tk.wl.n_groups == nullptr) return;
     __syncthreads();
     DBG_STAMP(2002);
