@@ -838,7 +838,7 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
         const size_t smem = token_smem(B, K, c.n_shared);
-        bool ok = coop != 0 && smem <= 64 * 1024;
+        bool ok = coop != 0 && smem <= 160 * 1024;
         for (int mt = 1; ok && mt <= 4; mt += 3) {
             void *k = token_kernel(c.weight_dtype, s->rdt, mt);
             int occ = 0;

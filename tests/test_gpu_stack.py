@@ -121,15 +121,19 @@ def test_tiny_cache_thrashes_but_stays_correct():
     assert st["prefetch_issued"] > 0
 
 
-@pytest.mark.parametrize("B", [1, 4])
-def test_decode_token_paths_agree(B):
+@pytest.mark.parametrize("B,shape", [
+    (1, dict(hidden=512, inter=352, n_experts=16, top_k=3)),
+    (4, dict(hidden=512, inter=352, n_experts=16, top_k=3)),
+    (33, dict(hidden=272, inter=208, n_experts=256, top_k=8, n_shared=1)),     # maximum expert count
+    (64, dict(hidden=144, inter=96, n_experts=40, top_k=32, n_shared=0)),      # maximum batch and K
+])
+def test_decode_token_paths_agree(B, shape):
     """decode_token has three execution paths for a resident stack: the persistent one-kernel
     step (default), per-layer kernels replayed as a CUDA graph (capturable stream), and per-layer
     kernels launched one by one (default stream).  Outputs, routing, predictions, tables and
     counters must be identical, bit for bit."""
-    cfg = stacks.CONFIGS["C2"].scaled(n_layers=3, hidden=512, inter=352, n_experts=16, top_k=3,
-                                      profile_tokens=3)
-    T = 10
+    cfg = stacks.CONFIGS["C2"].scaled(n_layers=3, profile_tokens=3, **shape)
+    T = 10 if B <= 4 else 5
     x = stacks.token_inputs(cfg, B, T).to(DEV)
     results = []
     for path in ("persistent", "graph", "eager"):
