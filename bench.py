@@ -187,6 +187,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefetch-limit", type=int, default=0, help="offloaded stacks: copies per layer step")
     ap.add_argument("--mode", default="st", choices=["off", "temporal", "spatial", "st"])
+    ap.add_argument("--inter-layer-gap-us", type=float, default=0.0,
+                    help="idle the compute stream this long after every layer: a stand-in for the attention "
+                         "block the paper overlaps expert prefetch with (Section 4.3.4); 0 = pure MoE stack")
     ap.add_argument("--resident", action="store_true", help="keep every expert in HBM (cache_slots = 0)")
     args = ap.parse_args()
 
@@ -232,11 +235,21 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    gap_cycles = int(args.inter_layer_gap_us * 1965)      # torch.cuda._sleep spins on the SM clock
+
+    def decode(h_src):
+        h_in.copy_(h_src)
+        if gap_cycles <= 0:
+            st.decode_token(h_in, h_out, ids, None, pred, npred)
+            return
+        for l in range(L):                                # per-layer entry point + attention stand-in
+            st.decode_step(l, h_in if l == 0 else h_out, h_out, ids[l], None, pred[l], npred[l])
+            torch.cuda._sleep(gap_cycles)
+
     # set-up: the profiling phase of Algorithm 1, then warm-up
     t = 0
     for _ in range(cfg.profile_tokens + args.warmup):
-        h_in.copy_(x_dev[t])
-        st.decode_token(h_in, h_out, ids, None, pred, npred)
+        decode(x_dev[t])
         t += 1
     s0 = st.stats()
 
@@ -248,8 +261,7 @@ def main():
     ids_seen = []
     ev0.record(stream)
     for i in range(args.steps):
-        h_in.copy_(x_dev[t + i])
-        st.decode_token(h_in, h_out, ids, None, pred, npred)
+        decode(x_dev[t + i])
     ev1.record(stream)
     barrier()
     clocks = sampler.stop()
@@ -350,7 +362,8 @@ def main():
                   "exposed_ms": s1["exposed_ms"] - s0["exposed_ms"],
                   "hidden_frac": 1.0 - (s1["exposed_ms"] - s0["exposed_ms"])
                   / max(s1["transfer_ms"] - s0["transfer_ms"], 1e-9),
-                  "prefetch_limit": args.prefetch_limit, "mode": args.mode},
+                  "prefetch_limit": args.prefetch_limit, "mode": args.mode,
+                  "inter_layer_gap_us": args.inter_layer_gap_us},
     }
     if world == 1 and not args.no_cpu_baseline:
         st.close()
