@@ -348,14 +348,25 @@ __device__ __forceinline__ void route_single_block(const RouterArgs &a, int *s_i
     int *s_cnt = scratch + 256 + 32;                              // [8] selected per warp
     auto sync256 = []() { asm volatile("bar.sync 2, 256;" ::: "memory"); };
 
-    float ss = 0.f;
-    for (int c = 0; c < C; ++c) ss += __ldcg(a.ss_part + c);
+    // both sets of partials in one trip to L2 (at most 8 column chunks: H <= 8192 in bf16)
+    float sp[8], lp[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        sp[c] = c < C ? __ldcg(a.ss_part + c) : 0.f;
+        lp[c] = (c < C && j < E) ? __ldcg(a.part + (size_t)c * E + j) : 0.f;
+    }
+    float ss = 0.f, s = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+        if (c < C) ss += sp[c], s += lp[c];
+    for (int c = 8; c < C; ++c) {
+        ss += __ldcg(a.ss_part + c);
+        if (j < E) s += __ldcg(a.part + (size_t)c * E + j);
+    }
     const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
     if (j == 0) a.inv_rms[0] = inv;
     float z = -INFINITY;
     if (j < E) {
-        float s = 0.f;
-        for (int c = 0; c < C; ++c) s += __ldcg(a.part + (size_t)c * E + j);
         z = s * inv;
         if (a.logits_out) a.logits_out[j] = z;
     }
