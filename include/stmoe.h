@@ -222,6 +222,25 @@ int stmoe_moe_ffn_static(const float *h, const float *inv_rms, const int32_t *id
                          const void *experts, int weight_dtype, int batch, int n_experts, int top_k,
                          int hidden, int inter, float residual_scale, float *h_out, void *cuda_stream);
 
+/* One expert's SwiGLU FFN (Section 2: the expert network of a routed token) for m tokens that
+ * share the expert, as bf16 tensor-core GEMMs (tcgen05.mma, accumulators in tensor memory):
+ *   y[t] = W_d ( bf16( silu(W_g x_t) * (W_u x_t) ) ),  x_t = bf16( h[t] * inv_rms[t] ),
+ * products exact, sums in fp32.  This is the regime where the per-expert token count makes the
+ * FFN a real dense contraction; the decode step itself streams weights through the CUDA cores.
+ *   h        device fp32 [m][hidden]; inv_rms device fp32 [m] or NULL (= 1).
+ *   image    device, one STMOE_BF16 expert image (gate [I][H], up [I][H], down [H][I]).
+ *   y        device fp32 [m][hidden], overwritten.
+ *   flags    device uint32, caller-zeroed; set to 1 when a bounded wait inside a kernel ran out
+ *            (y is then undefined).
+ *   scratch  device, stmoe_expert_ffn_dense_scratch_bytes(m, hidden, inter) bytes, 256-byte
+ *            aligned, contents need not be initialised.
+ * m in 1..64; hidden and inter multiples of 64; else STMOE_ERR_BAD_ARG.  Asynchronous on
+ * cuda_stream. */
+size_t stmoe_expert_ffn_dense_scratch_bytes(int m, int hidden, int inter);
+int stmoe_expert_ffn_dense(const float *h, const float *inv_rms, const void *image, int m, int hidden,
+                           int inter, float *y, uint32_t *flags, void *scratch, size_t scratch_bytes,
+                           void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -75,6 +75,9 @@ def lib():
         L.stmoe_moe_ffn_scratch_bytes.argtypes = [i32, i32, i32, i32]
         L.stmoe_moe_ffn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, vp, vp, sz, vp]
         L.stmoe_moe_ffn_static.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, vp, vp]
+        L.stmoe_expert_ffn_dense_scratch_bytes.restype = sz
+        L.stmoe_expert_ffn_dense_scratch_bytes.argtypes = [i32, i32, i32]
+        L.stmoe_expert_ffn_dense.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -237,3 +240,18 @@ def moe_ffn_static(h, inv_rms, ids, w, experts, dtype, n_experts, hidden, inter,
                                       hidden, inter, residual_scale, _dev(h_out, torch.float32),
                                       _stream(stream)), "stmoe_moe_ffn_static")
     return h_out
+
+
+def expert_ffn_dense(h, inv_rms, image, hidden, inter, stream=None):
+    """stmoe_expert_ffn_dense: one bf16 expert's SwiGLU FFN for the m <= 64 tokens in h [m][hidden]
+    on the tensor cores.  Returns (y [m][hidden] fp32, flags uint32 tensor; non-zero = a bounded
+    wait inside a kernel ran out)."""
+    m = h.shape[0]
+    n = lib().stmoe_expert_ffn_dense_scratch_bytes(m, hidden, inter)
+    scratch = torch.empty(max(n, 256), dtype=torch.uint8, device=h.device)
+    y = torch.empty(m, hidden, dtype=torch.float32, device=h.device)
+    flags = torch.zeros(1, dtype=torch.int32, device=h.device)
+    _check(lib().stmoe_expert_ffn_dense(_dev(h, torch.float32), _ptr(inv_rms), _dev(image), m, hidden, inter,
+                                        _dev(y), _dev(flags), _dev(scratch), scratch.numel(), _stream(stream)),
+           "stmoe_expert_ffn_dense")
+    return y, flags

@@ -11,6 +11,7 @@
 #include <utility>
 #include <vector>
 
+#include "dense_ffn.cuh"
 #include "device_utils.cuh"
 #include "ffn.cuh"
 #include "predictor.cuh"
@@ -1238,6 +1239,60 @@ extern "C" int stmoe_moe_ffn_static(const float *h, const float *inv_rms, const 
     return stmoe_moe_ffn(h, inv_rms, ids, w, experts, weight_dtype, batch, n_experts, top_k, hidden, inter,
                          residual_scale, h_out, g_static_scratch_ptr[dev], (size_t)STMOE_STATIC_SCRATCH_BYTES,
                          cuda_stream);
+}
+
+// ---- tensor-core expert FFN for many tokens of one expert ------------------------------------
+static size_t dense_scratch_layout(int np, int H, int I, size_t *o_act)
+{
+    size_t o = round_up(sizeof(__nv_bfloat16) * (size_t)np * H, 256);
+    *o_act = o, o += round_up(sizeof(__nv_bfloat16) * (size_t)np * I, 256);
+    return o;
+}
+
+extern "C" size_t stmoe_expert_ffn_dense_scratch_bytes(int m, int hidden, int inter)
+{
+    if (m < 1 || m > kDenseMaxTokens || hidden < 1 || inter < 1) return 0;
+    size_t o_act;
+    return dense_scratch_layout((m + 15) / 16 * 16, hidden, inter, &o_act);
+}
+
+extern "C" int stmoe_expert_ffn_dense(const float *h, const float *inv_rms, const void *image, int m, int hidden,
+                                      int inter, float *y, uint32_t *flags, void *scratch, size_t scratch_bytes,
+                                      void *cuda_stream)
+{
+    if (!h || !image || !y || !flags || !scratch || m < 1 || m > kDenseMaxTokens || hidden < kDenseKStep ||
+        hidden % kDenseKStep || inter < kDenseKStep || inter % kDenseKStep || ((uintptr_t)scratch & 255) ||
+        ((uintptr_t)image & 15))
+        return STMOE_ERR_BAD_ARG;
+    const int np = (m + 15) / 16 * 16;
+    size_t o_act;
+    if (scratch_bytes < dense_scratch_layout(np, hidden, inter, &o_act)) return STMOE_ERR_BAD_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    __nv_bfloat16 *xb = (__nv_bfloat16 *)scratch, *act = (__nv_bfloat16 *)((uint8_t *)scratch + o_act);
+    const __nv_bfloat16 *img = (const __nv_bfloat16 *)image;
+    const int smem2 = kDenseStages * (2 * kDenseRows + np) * kDenseKStep * 2;
+    const int smem1 = kDenseStages * (kDenseRows + np) * kDenseKStep * 2;
+    static bool attr_set[64] = {};
+    int dev = -1;
+    CU_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return STMOE_ERR_BAD_ARG;
+    if (!attr_set[dev]) {
+        const int smem_max = kDenseStages * (2 * kDenseRows + kDenseMaxTokens) * kDenseKStep * 2;
+        CU_TRY(cudaFuncSetAttribute(dense_ffn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
+        CU_TRY(cudaFuncSetAttribute(dense_ffn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
+        attr_set[dev] = true;
+    }
+    dense_cast_kernel<<<148, 256, 0, st>>>(h, inv_rms, m, np, hidden, xb);
+    DenseArgs gu{};
+    gu.W0 = img, gu.W1 = img + (size_t)inter * hidden, gu.X = xb;
+    gu.rows = inter, gu.kd = hidden, gu.m = m, gu.np = np, gu.act_out = act, gu.err = flags;
+    dense_ffn_kernel<2><<<(inter + kDenseRows - 1) / kDenseRows, kDenseThreads, smem2, st>>>(gu);
+    DenseArgs dn{};
+    dn.W0 = img + 2 * (size_t)inter * hidden, dn.X = act;
+    dn.rows = hidden, dn.kd = inter, dn.m = m, dn.np = np, dn.y_out = y, dn.err = flags;
+    dense_ffn_kernel<1><<<(hidden + kDenseRows - 1) / kDenseRows, kDenseThreads, smem1, st>>>(dn);
+    CU_TRY(cudaGetLastError());
+    return STMOE_OK;
 }
 
 #ifdef STMOE_DBG_PHASES
