@@ -348,21 +348,20 @@ __device__ __forceinline__ void route_single_block(const RouterArgs &a, int *s_i
     int *s_cnt = scratch + 256 + 32;                              // [8] selected per warp
     auto sync256 = []() { asm volatile("bar.sync 2, 256;" ::: "memory"); };
 
-    // both sets of partials in one trip to L2 (at most 8 column chunks: H <= 8192 in bf16)
-    float sp[8], lp[8];
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        sp[c] = c < C ? __ldcg(a.ss_part + c) : 0.f;
-        lp[c] = (c < C && j < E) ? __ldcg(a.part + (size_t)c * E + j) : 0.f;
-    }
+    // Partials in one trip to L2.  The sums of squares are fetched one chunk per lane and summed
+    // across the warp: every CTA of a persistent grid reads these same few lines at the same
+    // moment, and the L2 slice that holds them serves the requests one by one.
     float ss = 0.f, s = 0.f;
+    for (int c = lane; c < C; c += kWarp) ss += __ldcg(a.ss_part + c);
+    for (int c0 = 0; c0 < C; c0 += 8) {
+        float lp[8];
 #pragma unroll
-    for (int c = 0; c < 8; ++c)
-        if (c < C) ss += sp[c], s += lp[c];
-    for (int c = 8; c < C; ++c) {
-        ss += __ldcg(a.ss_part + c);
-        if (j < E) s += __ldcg(a.part + (size_t)c * E + j);
+        for (int i = 0; i < 8; ++i) lp[i] = (c0 + i < C && j < E) ? __ldcg(a.part + (size_t)(c0 + i) * E + j) : 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (c0 + i < C) s += lp[i];
     }
+    ss = warp_sum(ss);
     const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
     if (j == 0) a.inv_rms[0] = inv;
     float z = -INFINITY;
@@ -431,7 +430,8 @@ __device__ __forceinline__ void router_finalize(const RouterArgs &a, int *s_ids,
     } else {
         for (int b = warp; b < B; b += nw) {
             float ss = 0.f;
-            for (int c = 0; c < C; ++c) ss += __ldcg(a.ss_part + c * B + b);
+            for (int c = lane; c < C; c += kWarp) ss += __ldcg(a.ss_part + c * B + b);
+            ss = warp_sum(ss);
             const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
             if (lane == 0) a.inv_rms[b] = inv;
             float z[kVpl];
