@@ -57,6 +57,11 @@ extern "C" {
 #define STMOE_FLAG_NO_PERSISTENT 2 /* resident stacks: decode steps as per-layer kernels (replayed as a
                                       CUDA graph) instead of the single persistent kernel */
 
+#define STMOE_FLAG_NO_DENSE 4 /* never use the tensor-core FFN kernels: by default resident bf16 stacks run
+                                decode steps of at least stmoe_set_dense_min_batch() sequences (default 4)
+                                with one work-list entry per expert on tcgen05 tiles, rounding the
+                                normalised hidden state and the gated activations to bf16 */
+
 /* per-sequence result flags of a layer step */
 #define STMOE_TOKEN_NEAR_TIE 1u /* K-th and (K+1)-th router logit closer than 1e-4 */
 
@@ -158,6 +163,10 @@ int stmoe_max_predicted(const stmoe_t *s); /* min(E, K*K+K) */
  * on the caller's stream (the router kernel too); their summed durations appear in stmoe_stats.
  * Off by default. */
 int stmoe_set_kernel_timing(stmoe_t *s, int on);
+
+/* Smallest batch that takes the tensor-core FFN path (see STMOE_FLAG_NO_DENSE); between decode
+ * steps.  min_batch < 2 or a stack without that path: STMOE_ERR_BAD_ARG. */
+int stmoe_set_dense_min_batch(stmoe_t *s, int min_batch);
 
 /* Counters and timings; synchronises the device. */
 int stmoe_stats(stmoe_t *s, stmoe_stats_t *out);

@@ -18,6 +18,7 @@ DTYPE = {"f32": 0, "bf16": 1, "fp8": 2}
 MODE = {"off": 0, "temporal": 1, "spatial": 2, "st": 3}
 FLAG_RENORM_TOPK = 1
 FLAG_NO_PERSISTENT = 2
+FLAG_NO_DENSE = 4
 
 
 class StmoeError(RuntimeError):
@@ -63,6 +64,7 @@ def lib():
         L.stmoe_decode_token.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.stmoe_max_predicted.argtypes = [vp]
         L.stmoe_set_kernel_timing.argtypes = [vp, i32]
+        L.stmoe_set_dense_min_batch.argtypes = [vp, i32]
         L.stmoe_stats.argtypes = [vp, C.POINTER(Stats)]
         L.stmoe_export_state.argtypes = [vp, vp, C.POINTER(sz)]
         L.stmoe_import_state.argtypes = [vp, vp, sz]
@@ -170,6 +172,9 @@ class Stack:
 
     def set_kernel_timing(self, on: bool) -> None:
         _check(lib().stmoe_set_kernel_timing(self._h, int(on)), "stmoe_set_kernel_timing")
+
+    def set_dense_min_batch(self, min_batch: int) -> None:
+        _check(lib().stmoe_set_dense_min_batch(self._h, int(min_batch)), "stmoe_set_dense_min_batch")
 
     def stats(self) -> dict:
         st = Stats()

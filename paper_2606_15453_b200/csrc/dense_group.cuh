@@ -1,0 +1,252 @@
+// Grouped expert FFN on the tensor cores for decode steps with several tokens per expert
+// (tcgen05.mma, accumulators in tensor memory, operands staged by TMA; sm_100a).
+//
+// The work list holds one entry per active expert (all of its tokens).  A task is one entry x
+// one tile of 128 weight rows (x one split of the reduction dimension for the down
+// projection); tasks are dealt round-robin over a persistent grid of one CTA per SM.  Weights
+// stay the streamed operand: the 128 weight rows are the MMA's M, the tokens its N (the batch
+// padded to a multiple of 16), and the CTA walks the reduction dimension 64 columns per stage.
+//   warp 0      one thread issues the TMA loads of a stage: the 128x64 weight tile(s) through a
+//               3-D tensor map over the expert store (column, row, image) and the Nx64
+//               activation tile, all in the 128-byte swizzled layout the MMA reads
+//   warp 1      one thread issues four K=16 tcgen05.mma per stage and matrix, frees the stage
+//               with tcgen05.commit and hands a finished accumulator to the epilogue; the warp
+//               also owns the tensor-memory allocation
+//   warps 2-5   epilogue: read the accumulator (two buffers, so the next task's MMAs overlap),
+//               apply SiLU(gate)*up or nothing, store the rows of the entry's tokens
+// Gate/up multiplies against the whole batch's activations (tensor work is free next to the
+// weight stream) and the epilogue keeps the entry's tokens.  The down projection multiplies
+// against the entry's own rows of the activation buffer, which are consecutive.
+// Every wait is bounded; a wait that runs out raises the error word and the kernel drains.
+#pragma once
+#include <cuda.h>
+
+#include "dense_ffn.cuh"
+
+namespace stmoe_dev {
+
+constexpr int kGroupThreads = 192;
+constexpr int kGroupTileBytes = kDenseRows * kDenseKStep * 2;     // 16 KB weight tile of a stage
+constexpr int kGroupActBytes = kDenseMaxTokens * kDenseKStep * 2; // 8 KB activation tile (64 tokens)
+constexpr int kGroupTmemCols = 256;                               // two accumulator buffers of 128 columns
+
+template <int NMAT> __host__ __device__ constexpr int group_stages() { return NMAT == 2 ? 5 : 8; }
+template <int NMAT> __host__ __device__ constexpr int group_stage_bytes() { return NMAT * kGroupTileBytes + kGroupActBytes; }
+template <int NMAT> __host__ __device__ constexpr int group_smem_bytes() { return group_stages<NMAT>() * group_stage_bytes<NMAT>() + 1024; }
+
+struct GroupArgs {
+    WorkList wl;
+    int E;                 // routed experts (entries with g_expert >= E are shared experts)
+    int img_routed0;       // image index of this layer's expert 0 in the store
+    int img_shared0;       // image index of this layer's shared expert 0
+    int rows;              // weight rows: I (gate/up) or H (down)
+    int kd;                // reduction length: H (gate/up) or I (down)
+    int np;                // batch padded to a multiple of 16 (MMA N and activation box rows)
+    int splits, seg;       // down: splits of the reduction dimension, columns per split (multiple of 64)
+    int KS;                // K + n_shared
+    __nv_bfloat16 *act;    // gate/up out, down in: [pairs][I]
+    float *part;           // down out: [B*KS][splits][H]
+    unsigned *err;
+};
+
+__device__ __forceinline__ void dmbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(dsmem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int c0, int c1, int c2, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dsmem_u32(dst)), "l"(map), "r"(dsmem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dsmem_u32(dst)), "l"(map), "r"(dsmem_u32(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
+// K-major operand tile in the 128-byte swizzled layout (rows of 128 bytes, 8-row groups 1024
+// bytes apart, tile base 1024-byte aligned); kstep = which 16-column slice of the 64.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr, int kstep)
+{
+    return (uint64_t)(((smem_addr + kstep * 32) >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ float tmem_ld1(uint32_t addr)
+{
+    uint32_t r;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(addr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    return __uint_as_float(r);
+}
+
+struct GroupTask {
+    int g, row0, k0, k1, z;
+};
+// task -> (entry, row tile, split); gate/up has one split
+__device__ __forceinline__ GroupTask group_task(const GroupArgs &a, int task)
+{
+    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
+    GroupTask t;
+    t.g = task / (tiles * a.splits);
+    const int r = task - t.g * tiles * a.splits;
+    t.row0 = (r / a.splits) * kDenseRows;
+    t.z = r % a.splits;
+    t.k0 = t.z * a.seg;
+    t.k1 = min(a.kd, t.k0 + a.seg);
+    return t;
+}
+
+// NMAT = 2: gate and up projections with the SiLU epilogue; NMAT = 1: down projection.
+template <int NMAT>
+__global__ void __launch_bounds__(kGroupThreads, 1)
+dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
+                   const __grid_constant__ CUtensorMap map_x, GroupArgs a)
+{
+    constexpr int NS = group_stages<NMAT>(), STAGE = group_stage_bytes<NMAT>();
+    extern __shared__ uint8_t dsm_raw[];
+    __shared__ uint64_t full[NS], empty[NS], tfull[2], tempty[2];
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_dead;
+    uint8_t *dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid / kWarp, lane = tid % kWarp;
+    const int np = a.np;
+    const int n_groups = *a.wl.n_groups;
+    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
+    const int n_tasks = n_groups * tiles * a.splits;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) dmbar_init(&full[s], 1), dmbar_init(&empty[s], 1);
+        for (int b = 0; b < 2; ++b) dmbar_init(&tfull[b], 1), dmbar_init(&tempty[b], 4);
+        s_dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dsmem_u32(&s_tmem)),
+                     "r"(kGroupTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s_tmem;
+
+    if (warp == 0) {
+        // ---- TMA producer -----------------------------------------------------------------------
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            int issued = 0;
+            for (int task = blockIdx.x; task < n_tasks && !s_dead; task += gridDim.x) {
+                const GroupTask t = group_task(a, task);
+                const int ge = a.wl.g_expert[t.g];
+                const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
+                const int xrow = NMAT == 2 ? 0 : a.wl.g_start[t.g];
+                for (int k = t.k0; k < t.k1; k += kDenseKStep) {
+                    if (!dmbar_wait(&empty[s], ph ^ 1u, &s_dead)) break;
+                    uint8_t *st = dsm + (size_t)s * STAGE;
+                    dmbar_expect_tx(&full[s], (uint32_t)(NMAT * kGroupTileBytes + np * kDenseKStep * 2));
+                    tma_load_3d(st, &map_w0, k, t.row0, img, &full[s]);
+                    if (NMAT == 2) tma_load_3d(st + kGroupTileBytes, &map_w1, k, t.row0, img, &full[s]);
+                    tma_load_2d(st + NMAT * kGroupTileBytes, &map_x, k, xrow, &full[s]);
+                    ++issued;
+                    if (++s == NS) s = 0, ph ^= 1u;
+                }
+            }
+            // every load that was issued has to land before the CTA may exit
+            for (int i = 0; i < min(issued, NS); ++i) {
+                if (s == 0) s = NS, ph ^= 1u;
+                --s;
+                dmbar_wait(&full[s], ph, &s_dead);
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issue ----------------------------------------------------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(np);
+            int s = 0, it = 0;
+            uint32_t ph = 0;
+            for (int task = blockIdx.x; task < n_tasks && !s_dead; task += gridDim.x, ++it) {
+                const GroupTask t = group_task(a, task);
+                const int ab = it & 1;
+                if (!dmbar_wait(&tempty[ab], (((uint32_t)it >> 1) & 1u) ^ 1u, &s_dead)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t acc = tmem + ab * 128;
+                bool first = true;
+                for (int k = t.k0; k < t.k1; k += kDenseKStep) {
+                    if (!dmbar_wait(&full[s], ph, &s_dead)) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t st = dsmem_u32(dsm + (size_t)s * STAGE);
+#pragma unroll
+                    for (int j = 0; j < kDenseKStep / 16; ++j) {
+                        const uint64_t bd = umma_desc_sw128(st + NMAT * kGroupTileBytes, j);
+#pragma unroll
+                        for (int mat = 0; mat < NMAT; ++mat)
+                            umma_bf16(acc + mat * 64, umma_desc_sw128(st + mat * kGroupTileBytes, j), bd, idesc,
+                                      !first || j > 0);
+                    }
+                    first = false;
+                    umma_commit(&empty[s]);
+                    if (++s == NS) s = 0, ph ^= 1u;
+                }
+                umma_commit(&tfull[ab]);
+            }
+        }
+    } else {
+        // ---- epilogue: thread = one weight row (TMEM lane) -------------------------------------
+        const int lg = warp % 4;  // the TMEM lane quarter this warp may read
+        int it = 0;
+        for (int task = blockIdx.x; task < n_tasks; task += gridDim.x, ++it) {
+            const GroupTask t = group_task(a, task);
+            const int ab = it & 1;
+            const int start = a.wl.g_start[t.g], count = a.wl.g_count[t.g];
+            const bool ok = dmbar_wait(&tfull[ab], ((uint32_t)it >> 1) & 1u, &s_dead);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t acc = tmem + ab * 128 + ((uint32_t)(lg * kWarp) << 16);
+            const int row = t.row0 + lg * kWarp + lane;
+            if (NMAT == 2) {
+                for (int i = 0; i < count; ++i) {
+                    const int tok = a.wl.pair_token[start + i];
+                    const float g = tmem_ld1(acc + tok), u = tmem_ld1(acc + 64 + tok);
+                    if (ok && row < a.rows)
+                        a.act[(size_t)(start + i) * a.rows + row] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
+                }
+            } else {
+                for (int i0 = 0; i0 < count; i0 += 8) {
+                    float y[8];
+                    tmem_ld8(acc + i0, y);
+                    if (ok && row < a.rows) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (i0 + i < count) {
+                                const int slot = a.wl.pair_slot[start + i0 + i];
+                                a.part[((size_t)slot * a.splits + t.z) * a.rows + row] = y[i];
+                            }
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) dmbar_arrive(&tempty[ab]);
+            if (!ok) break;
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kGroupTmemCols) : "memory");
+    }
+    if (tid == 0 && s_dead) *a.err = 1u;
+}
+
+// h_out[b][c] = h[b][c] + r * (weighted sum of the down projection's partial sums)
+__global__ void __launch_bounds__(256) dense_combine_kernel(FfnArgs a, int S)
+{
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < a.B * a.H; i += gridDim.x * blockDim.x)
+        a.h_out[i] = finish_value(a, i / a.H, i % a.H, S);
+}
+
+}  // namespace stmoe_dev

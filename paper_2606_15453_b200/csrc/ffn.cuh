@@ -179,12 +179,42 @@ struct BlockTickets {
     }
 };
 
+// Output element (sequence b, column c) of the layer from the down projection's partial sums,
+// in a fixed summation order: shared experts, then routed experts, segments innermost:
+//   h_out[b][c] = h[b][c] + r * ( sum_shared part + sum_k w[b][k] * part ).
+// The loads of eight terms are issued together (each is a trip to L2), the arithmetic keeps the
+// fixed order.
+__device__ __forceinline__ float finish_value(const FfnArgs &a, int b, int c, int S)
+{
+    const int H = a.H, KS = a.K + a.n_shared, n_terms = KS * S;
+    float y = 0.f, p = 0.f;
+    for (int t0 = 0; t0 < n_terms; t0 += 8) {
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int t = t0 + i, q = t / S, z = t % S;
+            const int slot = q < a.n_shared ? a.K + q : q - a.n_shared;
+            v[i] = t < n_terms ? __ldcg(a.part + (((size_t)b * KS + slot) * S + z) * H + c) : 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int t = t0 + i, q = t / S, z = t % S;
+            if (t < n_terms) {
+                p += v[i];
+                if (z == S - 1) {
+                    y = q < a.n_shared ? y + p : fmaf(a.w[b * a.K + q - a.n_shared], p, y);
+                    p = 0.f;
+                }
+            }
+        }
+    }
+    return fmaf(a.residual_scale, y, a.h[(size_t)b * H + c]);
+}
+
 // Fused weighted sum + residual.  Called by a whole warp after it has stored the partial sums
 // of rows [r0, r0+nrows) of one (entry, segment): the rows are counted per 32-row tile, and the
-// warp whose count completes a tile (want_per_row contributions for each of its rows) sums
-// the tile over segments, shared experts and routed experts in a fixed order:
-//   h_out[b][c] = h[b][c] + r * ( sum_shared part + sum_k w[b][k] * part ).
-// No waiting is involved; the counter is left at zero for the next launch.
+// warp whose count completes a tile (want_per_row contributions for each of its rows) computes
+// the tile's outputs.  No waiting is involved; the counter is left at zero for the next launch.
 __device__ __forceinline__ void finish_rows(const FfnArgs &a, int r0, int nrows, int want_per_row, int S, int lane)
 {
     const int H = a.H;
@@ -201,36 +231,8 @@ __device__ __forceinline__ void finish_rows(const FfnArgs &a, int r0, int nrows,
             __threadfence();
             if (lane == 0) a.tile_done[tile] = 0u;
             const int c = tile * kTileRows + lane;
-            if (lane < tile_rows) {
-                // terms in summation order: shared experts, then routed experts, segments
-                // innermost; the loads of eight terms are issued together (each is a trip to
-                // L2), the arithmetic keeps the fixed order
-                const int KS = a.K + a.n_shared, n_terms = KS * S;
-                for (int b = 0; b < a.B; ++b) {
-                    float y = 0.f, p = 0.f;
-                    for (int t0 = 0; t0 < n_terms; t0 += 8) {
-                        float v[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const int t = t0 + i, q = t / S, z = t % S;
-                            const int slot = q < a.n_shared ? a.K + q : q - a.n_shared;
-                            v[i] = t < n_terms ? __ldcg(a.part + (((size_t)b * KS + slot) * S + z) * H + c) : 0.f;
-                        }
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const int t = t0 + i, q = t / S, z = t % S;
-                            if (t < n_terms) {
-                                p += v[i];
-                                if (z == S - 1) {
-                                    y = q < a.n_shared ? y + p : fmaf(a.w[b * a.K + q - a.n_shared], p, y);
-                                    p = 0.f;
-                                }
-                            }
-                        }
-                    }
-                    a.h_out[(size_t)b * H + c] = fmaf(a.residual_scale, y, a.h[(size_t)b * H + c]);
-                }
-            }
+            if (lane < tile_rows)
+                for (int b = 0; b < a.B; ++b) a.h_out[(size_t)b * H + c] = finish_value(a, b, c, S);
         }
         rr += n;
     }

@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "dense_ffn.cuh"
+#include "dense_group.cuh"
 #include "device_utils.cuh"
 #include "ffn.cuh"
 #include "predictor.cuh"
@@ -307,6 +308,14 @@ struct stmoe {
     float *d_hbuf = nullptr, *d_rpart_all = nullptr, *d_sspart_all = nullptr, *d_act_all = nullptr, *d_part_all = nullptr;
     unsigned *d_tiles_all = nullptr, *d_barrier = nullptr;
 
+    // tensor-core path for batched steps of resident bf16 stacks (dense_group.cuh)
+    bool dense = false;
+    int dense_min_batch = 0;
+    CUtensorMap map_gate{}, map_up{}, map_down{}, map_x[4]{}, map_act[4]{};  // [np/16 - 1]
+    __nv_bfloat16 *d_xb = nullptr, *d_actb = nullptr;
+    float *d_part_dense = nullptr;
+    int dense_grid = 0;
+
     SlotCache cache;
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_route = nullptr;
@@ -518,6 +527,115 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
     return STMOE_OK;
 }
 
+// ---- tensor-core path (dense_group.cuh) ---------------------------------------------------
+constexpr int kDenseMinBatch = 4;
+constexpr int kDenseMaxSplits = 4;
+
+bool use_dense(const stmoe *s, int batch) { return s->dense && batch >= s->dense_min_batch; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 tensor of `rank` dimensions (dims[0] innermost, strides in bytes for dims 1..), boxes of
+// 64 columns x box_rows rows (x 1 image), 128-byte swizzle, zero fill outside
+int encode_map(EncodeTiledFn fn, CUtensorMap *m, void *base, int rank, const cuuint64_t *dims,
+               const cuuint64_t *strides, int box_rows)
+{
+    cuuint32_t box[3] = {(cuuint32_t)kDenseKStep, (cuuint32_t)box_rows, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
+               ? STMOE_OK
+               : STMOE_ERR_CUDA;
+}
+
+int dense_setup(stmoe *s)
+{
+    const stmoe_config_t &c = s->cfg;
+    const int L = c.n_layers, E = c.n_experts, B = c.max_batch, H = c.hidden, I = c.inter;
+    int dev = 0, major = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (major != 10) return STMOE_OK;  // tcgen05 kernels need sm_100: stay on the CUDA-core path
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr) != cudaSuccess || !sym) {
+        (void)cudaGetLastError();
+        return STMOE_OK;
+    }
+    EncodeTiledFn enc = (EncodeTiledFn)sym;
+    const size_t pairs = (size_t)B * s->KS;
+    CU_TRY(cudaMalloc(&s->d_xb, sizeof(__nv_bfloat16) * (size_t)kDenseMaxTokens * H));
+    CU_TRY(cudaMemset(s->d_xb, 0, sizeof(__nv_bfloat16) * (size_t)kDenseMaxTokens * H));
+    CU_TRY(cudaMalloc(&s->d_actb, sizeof(__nv_bfloat16) * (pairs + kDenseMaxTokens) * I));
+    CU_TRY(cudaMemset(s->d_actb, 0, sizeof(__nv_bfloat16) * (pairs + kDenseMaxTokens) * I));
+    CU_TRY(cudaMalloc(&s->d_part_dense, sizeof(float) * pairs * kDenseMaxSplits * H));
+    const cuuint64_t n_img = (cuuint64_t)L * (E + c.n_shared);
+    const cuuint64_t gd[3] = {(cuuint64_t)H, (cuuint64_t)I, n_img}, gs[2] = {(cuuint64_t)H * 2, s->img_bytes};
+    const cuuint64_t dd[3] = {(cuuint64_t)I, (cuuint64_t)H, n_img}, ds[2] = {(cuuint64_t)I * 2, s->img_bytes};
+    ST_TRY(encode_map(enc, &s->map_gate, s->d_resident, 3, gd, gs, kDenseRows));
+    ST_TRY(encode_map(enc, &s->map_up, s->d_resident + (size_t)I * H * 2, 3, gd, gs, kDenseRows));
+    ST_TRY(encode_map(enc, &s->map_down, s->d_resident + 2 * (size_t)I * H * 2, 3, dd, ds, kDenseRows));
+    for (int i = 0; i < 4; ++i) {
+        const cuuint64_t xd[2] = {(cuuint64_t)H, (cuuint64_t)kDenseMaxTokens}, xs[1] = {(cuuint64_t)H * 2};
+        const cuuint64_t ad[2] = {(cuuint64_t)I, (cuuint64_t)(pairs + kDenseMaxTokens)}, as[1] = {(cuuint64_t)I * 2};
+        ST_TRY(encode_map(enc, &s->map_x[i], s->d_xb, 2, xd, xs, 16 * (i + 1)));
+        ST_TRY(encode_map(enc, &s->map_act[i], s->d_actb, 2, ad, as, 16 * (i + 1)));
+    }
+    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, group_smem_bytes<2>()));
+    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, group_smem_bytes<1>()));
+    s->dense_grid = sm_count();
+    s->dense_min_batch = kDenseMinBatch;
+    s->dense = true;
+    return STMOE_OK;
+}
+
+// gate/up, down and the weighted sum of one layer step on the tensor-core kernels; the work
+// list (one entry per expert) and inv_rms come from the router kernel launched before
+int dense_ffn(stmoe *s, int layer, int batch, const FfnArgs &fa, cudaStream_t st)
+{
+    const stmoe_config_t &c = s->cfg;
+    const int E = c.n_experts, H = c.hidden, I = c.inter, np = (batch + 15) / 16 * 16;
+    cudaEvent_t e0 = nullptr, e1 = nullptr, e2 = nullptr;
+    const bool timed = s->time_kernels;
+    if (timed) {
+        ST_TRY(get_event(s, &e0));
+        ST_TRY(get_event(s, &e1));
+        ST_TRY(get_event(s, &e2));
+        CU_TRY(cudaEventRecord(e0, st));
+    }
+    dense_cast_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fa.h, fa.inv_rms, batch, batch, H, s->d_xb);
+    GroupArgs g{};
+    g.wl = fa.wl, g.E = E, g.img_routed0 = layer * E, g.img_shared0 = c.n_layers * E + layer * c.n_shared;
+    g.np = np, g.KS = s->KS, g.act = s->d_actb, g.part = s->d_part_dense, g.err = s->d_err;
+    g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kDenseKStep - 1) / kDenseKStep * kDenseKStep;
+    dense_group_kernel<2><<<s->dense_grid, kGroupThreads, group_smem_bytes<2>(), st>>>(s->map_gate, s->map_up,
+                                                                                      s->map_x[np / 16 - 1], g);
+    if (timed) CU_TRY(cudaEventRecord(e1, st));
+    // down: split the reduction dimension until there are a few tasks per SM
+    const int entries = std::min(E, batch * c.top_k) + c.n_shared, tiles = (H + kDenseRows - 1) / kDenseRows;
+    int splits = std::max(1, std::min(kDenseMaxSplits, (4 * s->dense_grid + entries * tiles - 1) / (entries * tiles)));
+    int seg = ((I + splits - 1) / splits + kDenseKStep - 1) / kDenseKStep * kDenseKStep;
+    splits = (I + seg - 1) / seg;  // no empty split
+    g.rows = H, g.kd = I, g.splits = splits, g.seg = seg;
+    dense_group_kernel<1><<<s->dense_grid, kGroupThreads, group_smem_bytes<1>(), st>>>(s->map_down, s->map_down,
+                                                                                      s->map_act[np / 16 - 1], g);
+    FfnArgs fc = fa;
+    fc.part = s->d_part_dense;
+    dense_combine_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fc, splits);
+    if (timed) {
+        CU_TRY(cudaEventRecord(e2, st));
+        s->spans.push_back(TimedSpan{e0, e1, 2});
+        s->spans.push_back(TimedSpan{e1, e2, 3});
+        s->timed_ffn += 1;
+    }
+    s->launches += 4;
+    CU_TRY(cudaGetLastError());
+    return STMOE_OK;
+}
+
 int run_ffn(stmoe *s, int dt, int mt, const FfnPlan &plan, const FfnArgs &fa, cudaStream_t st)
 {
     cudaEvent_t e0 = nullptr, e1 = nullptr, e2 = nullptr;
@@ -548,7 +666,8 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
 {
     const stmoe_config_t &c = s->cfg;
     const int E = c.n_experts, K = c.top_k, H = c.hidden;
-    const int mt = batch == 1 ? 1 : 4;
+    const bool dense = use_dense(s, batch);
+    const int mt = batch == 1 ? 1 : dense ? kDenseMaxTokens : 4;
     int32_t *ids = s->d_ids + (size_t)layer * c.max_batch * K;
     const int32_t *prev = layer > 0 ? s->d_ids + (size_t)(layer - 1) * c.max_batch * K : nullptr;
 
@@ -601,7 +720,10 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
         fa.blob = s->d_blob_table + (size_t)layer * (E + c.n_shared);
     }
     s->launches += 1;
-    ST_TRY(run_ffn(s, c.weight_dtype, mt, mt == 1 ? s->plan1 : s->plan4, fa, st));
+    if (dense)
+        ST_TRY(dense_ffn(s, layer, batch, fa, st));
+    else
+        ST_TRY(run_ffn(s, c.weight_dtype, mt, mt == 1 ? s->plan1 : s->plan4, fa, st));
     if (!offloaded(s)) {
         // resident: nothing in the step depends on the predictor, so it runs on a side stream
         // once the FFN kernels (which fill every SM) are done, beside the next layer's router
@@ -714,7 +836,8 @@ int stmoe_destroy(stmoe_t *s)
                    s->pst.Co, s->pst.cct_id, s->pst.cct_conf, s->pst.HT, s->pst.t, s->pst.pred_mask,
                    s->pst.pred_valid, s->pst.stats, s->d_rpart, s->d_sspart, s->d_arrivals, s->d_tile_done, s->d_hbuf, s->d_rpart_all, s->d_sspart_all,
                    s->d_act_all, s->d_part_all, s->d_tiles_all, s->d_barrier, s->d_err, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
-                   s->d_ids, s->d_queue};
+                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense};
+    if (s->d_shared && s->d_resident && s->d_shared > s->d_resident) dev[2] = nullptr;  // one allocation
     for (void *p : dev)
         if (p) cudaFree(p);
     s->wlm.release();
@@ -773,7 +896,7 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
     CR_TRY(cudaStreamCreateWithFlags(&s->side_stream, cudaStreamNonBlocking));
     CR_TRY(cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming));
     CR_TRY(cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming));
-    if (c.n_shared) CR_TRY(cudaMalloc(&s->d_shared, (size_t)L * c.n_shared * s->img_bytes));
+    if (c.n_shared && c.cache_slots > 0) CR_TRY(cudaMalloc(&s->d_shared, (size_t)L * c.n_shared * s->img_bytes));
     if (c.cache_slots > 0) {
         CR_TRY(cudaHostAlloc(&s->h_store, (size_t)L * E * s->img_bytes, cudaHostAllocDefault));
         CR_TRY(cudaMalloc(&s->d_slots, (size_t)c.cache_slots * s->img_bytes));
@@ -788,7 +911,10 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
         s->slot_pending.assign((size_t)c.cache_slots, 0);
         for (auto &e : s->slot_ready) CR_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
     } else {
-        CR_TRY(cudaMalloc(&s->d_resident, (size_t)L * E * s->img_bytes));
+        // routed images [L][E], then the shared ones [L][n_shared], in one allocation: one
+        // tensor map with the image index as its outermost coordinate covers both
+        CR_TRY(cudaMalloc(&s->d_resident, (size_t)L * (E + c.n_shared) * s->img_bytes));
+        if (c.n_shared) s->d_shared = s->d_resident + (size_t)L * E * s->img_bytes;
         std::vector<const uint8_t *> tab((size_t)L * (E + c.n_shared));
         for (int l = 0; l < L; ++l) {
             for (int e = 0; e < E; ++e) tab[(size_t)l * (E + c.n_shared) + e] = image_ptr(s, l, e, false);
@@ -813,6 +939,8 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
     CR_TRY(cudaMemset(s->pst.pred_mask, 0, (size_t)B * 8 * 4));
     CR_TRY(cudaMemset(s->pst.pred_valid, 0, (size_t)B * 4));
     CR_TRY(cudaMemset(s->pst.stats, 0, 8 * 8));
+    CR_TRY(cudaMalloc(&s->d_err, 16));
+    CR_TRY(cudaMemset(s->d_err, 0, 16));
     CR_TRY(cudaMalloc(&s->d_inv, sizeof(float) * B));
     CR_TRY(cudaMalloc(&s->d_logits, sizeof(float) * B * E));
     {
@@ -858,11 +986,13 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
             CR_TRY(cudaMalloc(&s->d_tiles_all, sizeof(unsigned) * L * tiles));
             CR_TRY(cudaMemset(s->d_tiles_all, 0, sizeof(unsigned) * L * tiles));
             CR_TRY(cudaMalloc(&s->d_barrier, 16));
-            CR_TRY(cudaMalloc(&s->d_err, 16));
-            CR_TRY(cudaMemset(s->d_err, 0, 16));
             s->persistent = true;
             s->persistent_grid = sm_count();
         }
+    }
+    if (c.cache_slots == 0 && c.weight_dtype == STMOE_BF16 && !(c.flags & STMOE_FLAG_NO_DENSE) && B >= 2) {
+        const int rc = dense_setup(s);
+        if (rc != STMOE_OK) return fail(rc);
     }
     if (c.profile_tokens == 0 && L > 1) {
         const int rows = (L - 1) * E;
@@ -882,6 +1012,13 @@ int stmoe_set_kernel_timing(stmoe_t *s, int on)
 {
     if (!s) return STMOE_ERR_BAD_ARG;
     s->time_kernels = on != 0;
+    return STMOE_OK;
+}
+
+int stmoe_set_dense_min_batch(stmoe_t *s, int min_batch)
+{
+    if (!s || !s->dense || min_batch < 2 || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
+    s->dense_min_batch = min_batch;
     return STMOE_OK;
 }
 
@@ -937,7 +1074,7 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, i
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const stmoe_config_t &c = s->cfg;
     const bool build_due = !s->built && s->host_t == c.profile_tokens - 1;
-    if (s->persistent && !s->time_kernels)
+    if (s->persistent && !s->time_kernels && !use_dense(s, batch))
         return token_persistent(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
     if (offloaded(s) || s->time_kernels || s->graph_off || build_due)
         return token_eager(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);

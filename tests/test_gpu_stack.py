@@ -137,7 +137,8 @@ def test_decode_token_paths_agree(B, shape):
     x = stacks.token_inputs(cfg, B, T).to(DEV)
     results = []
     for path in ("persistent", "graph", "eager"):
-        pr = Pair(cfg, B, oracle=False, flags=0 if path == "persistent" else P.FLAG_NO_PERSISTENT)
+        pr = Pair(cfg, B, oracle=False,
+                  flags=P.FLAG_NO_DENSE | (0 if path == "persistent" else P.FLAG_NO_PERSISTENT))
         L, K = cfg.n_layers, cfg.top_k
         ids = torch.empty(L, B, K, dtype=torch.int32, device=DEV)
         w = torch.empty(L, B, K, dtype=torch.float32, device=DEV)
