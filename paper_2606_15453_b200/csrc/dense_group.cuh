@@ -30,9 +30,19 @@ constexpr int kGroupTileBytes = kDenseRows * kDenseKStep * 2;     // 16 KB weigh
 constexpr int kGroupActBytes = kDenseMaxTokens * kDenseKStep * 2; // 8 KB activation tile (64 tokens)
 constexpr int kGroupTmemCols = 256;                               // two accumulator buffers of 128 columns
 
-template <int NMAT> __host__ __device__ constexpr int group_stages() { return NMAT == 2 ? 5 : 8; }
-template <int NMAT> __host__ __device__ constexpr int group_stage_bytes() { return NMAT * kGroupTileBytes + kGroupActBytes; }
-template <int NMAT> __host__ __device__ constexpr int group_smem_bytes() { return group_stages<NMAT>() * group_stage_bytes<NMAT>() + 1024; }
+constexpr int kGroupMaxStages = 12;
+constexpr int kGroupSmemBytes = 226 * 1024;                       // dynamic shared memory of a CTA (one per SM)
+// A stage holds NMAT weight tiles and np activation rows of 128 bytes (np a multiple of 16, so
+// every tile base stays 1024-byte aligned once rounded up); as many stages as fit.
+template <int NMAT> __host__ __device__ constexpr int group_stage_bytes(int np)
+{
+    return NMAT * kGroupTileBytes + (np * kDenseKStep * 2 + 1023) / 1024 * 1024;
+}
+template <int NMAT> __host__ __device__ constexpr int group_stages(int np)
+{
+    const int n = (kGroupSmemBytes - 1024) / group_stage_bytes<NMAT>(np);
+    return n < kGroupMaxStages ? n : kGroupMaxStages;
+}
 
 struct GroupArgs {
     WorkList wl;
@@ -105,14 +115,14 @@ __global__ void __launch_bounds__(kGroupThreads, 1)
 dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
                    const __grid_constant__ CUtensorMap map_x, GroupArgs a)
 {
-    constexpr int NS = group_stages<NMAT>(), STAGE = group_stage_bytes<NMAT>();
     extern __shared__ uint8_t dsm_raw[];
-    __shared__ uint64_t full[NS], empty[NS], tfull[2], tempty[2];
+    __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2];
     __shared__ uint32_t s_tmem;
     __shared__ int s_dead;
     uint8_t *dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, warp = tid / kWarp, lane = tid % kWarp;
     const int np = a.np;
+    const int NS = group_stages<NMAT>(np), STAGE = group_stage_bytes<NMAT>(np);
     const int n_groups = *a.wl.n_groups;
     const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
     const int n_tasks = n_groups * tiles * a.splits;

@@ -92,15 +92,17 @@ struct TopkArgs {
     WorkList wl;      // wl.n_groups == nullptr: no grouping
 };
 
-constexpr int kVpl = kMaxExperts / kWarp;  // logits held per lane
+constexpr int kVplMax = kMaxExperts / kWarp;  // logits held per lane at the maximum expert count
 
 // softmax + top-K for one sequence, by one warp.  Lane l holds the logits of experts
 // l, l+32, ... in z[].  K rounds of warp arg-max (hardware redux on order-preserving 32-bit
 // keys, then redux-min over the tied ids so the lower id wins), one more round for the
 // K-th/(K+1)-th gap; ids are emitted in ascending order with w = softmax(z)[id].
-__device__ __forceinline__ void route_token(const float (&z)[kVpl], float *, int *s_ids_row, const TopkArgs &a,
+template <int VPL>
+__device__ __forceinline__ void route_token(const float (&z)[VPL], float *, int *s_ids_row, const TopkArgs &a,
                                             int b, int lane)
 {
+    constexpr int kVpl = VPL;  // logits per lane: experts lane, lane+32, ... (E <= 32*VPL)
     const int E = a.E, K = a.K;
     float m = -INFINITY;
     uint32_t key[kVpl];
@@ -187,11 +189,18 @@ __device__ __forceinline__ void group_tokens(const int *s_ids, int *s_scan, int 
         if (t == 0) *wl.n_groups = K + n_shared;
         return;
     }
-    int *s_g = s_scan, *s_p = s_scan + kMaxExperts + 1;
+    // Thread e owns expert e for the counts and the entries; the pairs are placed by one thread
+    // each: a 64-bit token mask per expert gives a pair's position inside its entry (tokens
+    // ascending) without any thread walking the whole batch.
+    __shared__ unsigned long long s_mask[kMaxExperts];
+    int *s_g = s_scan, *s_p = s_scan + 8, *s_base = s_scan + 16;  // warp sums; first pair of each expert
     const int e = threadIdx.x, KS = K + n_shared, lane = e % kWarp, warp = e / kWarp;
-    int cnt = 0;
-    if (e < E)
-        for (int i = 0; i < B * K; ++i) cnt += (s_ids[i] == e);
+    auto sync256 = []() { asm volatile("bar.sync 2, 256;" ::: "memory"); };
+    s_mask[e] = 0ull;
+    sync256();
+    for (int i = e; i < B * K; i += 256) atomicOr(&s_mask[s_ids[i]], 1ull << (i / K));
+    sync256();
+    const int cnt = e < E ? __popcll(s_mask[e]) : 0;
     // exclusive scans of (entries, pairs) over the 256 experts
     int g_inc = (cnt + mt - 1) / mt, p_inc = cnt;
 #pragma unroll
@@ -200,39 +209,39 @@ __device__ __forceinline__ void group_tokens(const int *s_ids, int *s_scan, int 
         if (lane >= o) g_inc += tg, p_inc += tp;
     }
     if (lane == kWarp - 1) s_g[warp] = g_inc, s_p[warp] = p_inc;
-    asm volatile("bar.sync 2, 256;" ::: "memory");  // the 256 grouping threads only
+    sync256();
     int g0 = g_inc - (cnt + mt - 1) / mt, p0 = p_inc - cnt, g_all = 0;
     for (int wi = 0; wi < kMaxExperts / kWarp; ++wi) {
         if (wi < warp) g0 += s_g[wi], p0 += s_p[wi];
         g_all += s_g[wi];
     }
+    s_base[e] = p0;
+    sync256();
     if (e < E && cnt > 0) {
         for (int t = 0, g = g0; t < cnt; t += mt, ++g) {
             wl.g_expert[g] = e;
             wl.g_start[g] = p0 + t;
             wl.g_count[g] = min(mt, cnt - t);
         }
-        int n = 0;
-        for (int i = 0; i < B * K; ++i)
-            if (s_ids[i] == e) {
-                wl.pair_token[p0 + n] = i / K;
-                wl.pair_slot[p0 + n] = (i / K) * KS + i % K;
-                ++n;
-            }
+    }
+    for (int i = e; i < B * K; i += 256) {
+        const int x = s_ids[i], b = i / K;
+        const int p = s_base[x] + __popcll(s_mask[x] & ((1ull << b) - 1ull));
+        wl.pair_token[p] = b;
+        wl.pair_slot[p] = b * KS + i % K;
     }
     const int tiles = (B + mt - 1) / mt;
-    if (e < n_shared) {
-        const int ps = B * K + e * B;
-        for (int t = 0; t < tiles; ++t) {
-            const int g = g_all + e * tiles + t;
-            wl.g_expert[g] = E + e;
-            wl.g_start[g] = ps + t * mt;
-            wl.g_count[g] = min(mt, B - t * mt);
-        }
-        for (int b = 0; b < B; ++b) {
-            wl.pair_token[ps + b] = b;
-            wl.pair_slot[ps + b] = b * KS + K + e;
-        }
+    for (int i = e; i < n_shared * tiles; i += 256) {
+        const int sh = i / tiles, t = i % tiles;
+        const int g = g_all + i;
+        wl.g_expert[g] = E + sh;
+        wl.g_start[g] = B * K + sh * B + t * mt;
+        wl.g_count[g] = min(mt, B - t * mt);
+    }
+    for (int i = e; i < n_shared * B; i += 256) {
+        const int sh = i / B, b = i % B;
+        wl.pair_token[B * K + i] = b;
+        wl.pair_slot[B * K + i] = b * KS + K + sh;
     }
     if (threadIdx.x == 0) *wl.n_groups = g_all + n_shared * tiles;
 }
@@ -245,13 +254,13 @@ __global__ void __launch_bounds__(256) topk_group_kernel(TopkArgs a)
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
     const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
     for (int b = warp; b < a.B; b += NW) {
-        float z[kVpl];
+        float z[kVplMax];
 #pragma unroll
-        for (int v = 0; v < kVpl; ++v) {
+        for (int v = 0; v < kVplMax; ++v) {
             const int j = v * kWarp + lane;
             z[v] = j < a.E ? a.logits[(size_t)b * a.E + j] : -INFINITY;
         }
-        route_token(z, nullptr, s_ids + b * a.K, a, b, lane);
+        route_token<kVplMax>(z, nullptr, s_ids + b * a.K, a, b, lane);
     }
     if (a.wl.n_groups == nullptr) return;
     __syncthreads();
@@ -415,37 +424,51 @@ __device__ __forceinline__ void route_single_block(const RouterArgs &a, int *s_i
     }
 }
 
-// Sum the split-K partials in a fixed order, apply the RMSNorm factor, softmax/top-K every
-// sequence (one warp each, nw warps) and group the batch by expert.  Needs all 256+ threads
-// of the CTA for the grouping; s_ids [B*K], s_scan [2*(kMaxExperts+1)].
+// Sequences b = warp, warp + nw, ...: sum the split-K partials in a fixed order, apply the RMSNorm
+// factor, softmax / top-K by one warp each.  VPL = logits per lane (E <= 32*VPL).
+template <int VPL>
+__device__ __forceinline__ void finalize_tokens(const RouterArgs &a, int *s_ids, int nw, int C)
+{
+    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
+    const int B = a.tk.B, E = a.tk.E, H = a.H;
+    for (int b = warp; b < B; b += nw) {
+        float ss = 0.f;
+        for (int c = lane; c < C; c += kWarp) ss += __ldcg(a.ss_part + c * B + b);
+        ss = warp_sum(ss);
+        const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
+        if (lane == 0) a.inv_rms[b] = inv;
+        float z[VPL];
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            const int j = v * kWarp + lane;
+            float s = 0.f;
+            if (j < E)
+                for (int c = 0; c < C; ++c) s += __ldcg(a.part + ((size_t)c * B + b) * E + j);
+            z[v] = j < E ? s * inv : -INFINITY;
+            if (j < E && a.logits_out) a.logits_out[(size_t)b * E + j] = z[v];
+        }
+        route_token<VPL>(z, nullptr, s_ids + b * a.tk.K, a.tk, b, lane);
+    }
+}
+
+// Sum the split-K partials, softmax/top-K every sequence and group the batch by expert.  Needs
+// all 256+ threads of the CTA for the grouping; s_ids [B*K], s_scan [2*(kMaxExperts+1)].
 template <int DT>
 __device__ __forceinline__ void router_finalize(const RouterArgs &a, int *s_ids, int *s_scan, int nw)
 {
     constexpr int CH = router_chunk_cols<DT>();
-    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
     const int B = a.tk.B, E = a.tk.E, H = a.H;
     const int C = (H + CH - 1) / CH;
     if (B == 1) {
         if (threadIdx.x < 256) route_single_block<DT>(a, s_ids, s_scan);
+    } else if (E <= 32) {
+        finalize_tokens<1>(a, s_ids, nw, C);
+    } else if (E <= 64) {
+        finalize_tokens<2>(a, s_ids, nw, C);
+    } else if (E <= 128) {
+        finalize_tokens<4>(a, s_ids, nw, C);
     } else {
-        for (int b = warp; b < B; b += nw) {
-            float ss = 0.f;
-            for (int c = lane; c < C; c += kWarp) ss += __ldcg(a.ss_part + c * B + b);
-            ss = warp_sum(ss);
-            const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
-            if (lane == 0) a.inv_rms[b] = inv;
-            float z[kVpl];
-#pragma unroll
-            for (int v = 0; v < kVpl; ++v) {
-                const int j = v * kWarp + lane;
-                float s = 0.f;
-                if (j < E)
-                    for (int c = 0; c < C; ++c) s += __ldcg(a.part + ((size_t)c * B + b) * E + j);
-                z[v] = j < E ? s * inv : -INFINITY;
-                if (j < E && a.logits_out) a.logits_out[(size_t)b * E + j] = z[v];
-            }
-            route_token(z, nullptr, s_ids + b * a.tk.K, a.tk, b, lane);
-        }
+        finalize_tokens<kVplMax>(a, s_ids, nw, C);
     }
     DBG_STAMP(2001);
     if (a.tk.wl.n_groups == nullptr) return;

@@ -584,8 +584,8 @@ int dense_setup(stmoe *s)
         ST_TRY(encode_map(enc, &s->map_x[i], s->d_xb, 2, xd, xs, 16 * (i + 1)));
         ST_TRY(encode_map(enc, &s->map_act[i], s->d_actb, 2, ad, as, 16 * (i + 1)));
     }
-    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, group_smem_bytes<2>()));
-    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, group_smem_bytes<1>()));
+    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
+    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
     s->dense_grid = sm_count();
     s->dense_min_batch = kDenseMinBatch;
     s->dense = true;
@@ -611,7 +611,7 @@ int dense_ffn(stmoe *s, int layer, int batch, const FfnArgs &fa, cudaStream_t st
     g.wl = fa.wl, g.E = E, g.img_routed0 = layer * E, g.img_shared0 = c.n_layers * E + layer * c.n_shared;
     g.np = np, g.KS = s->KS, g.act = s->d_actb, g.part = s->d_part_dense, g.err = s->d_err;
     g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kDenseKStep - 1) / kDenseKStep * kDenseKStep;
-    dense_group_kernel<2><<<s->dense_grid, kGroupThreads, group_smem_bytes<2>(), st>>>(s->map_gate, s->map_up,
+    dense_group_kernel<2><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_gate, s->map_up,
                                                                                       s->map_x[np / 16 - 1], g);
     if (timed) CU_TRY(cudaEventRecord(e1, st));
     // down: split the reduction dimension until there are a few tasks per SM
@@ -620,7 +620,7 @@ int dense_ffn(stmoe *s, int layer, int batch, const FfnArgs &fa, cudaStream_t st
     int seg = ((I + splits - 1) / splits + kDenseKStep - 1) / kDenseKStep * kDenseKStep;
     splits = (I + seg - 1) / seg;  // no empty split
     g.rows = H, g.kd = I, g.splits = splits, g.seg = seg;
-    dense_group_kernel<1><<<s->dense_grid, kGroupThreads, group_smem_bytes<1>(), st>>>(s->map_down, s->map_down,
+    dense_group_kernel<1><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_down, s->map_down,
                                                                                       s->map_act[np / 16 - 1], g);
     FfnArgs fc = fa;
     fc.part = s->d_part_dense;
