@@ -14,8 +14,8 @@
 //               also owns the tensor-memory allocation
 //   warps 2-5   epilogue: read the accumulator (two buffers, so the next task's MMAs overlap),
 //               apply SiLU(gate)*up or nothing, store the rows of the entry's tokens
-// Gate/up multiplies against the whole batch's activations (tensor work is free next to the
-// weight stream) and the epilogue keeps the entry's tokens.  The down projection multiplies
+// Gate/up multiplies against the whole batch's hidden state in bf16 (tensor work is free next
+// to the weight stream); the epilogue keeps the entry's tokens and applies their RMSNorm factors.  The down projection multiplies
 // against the entry's own rows of the activation buffer, which are consecutive.
 // Every wait is bounded; a wait that runs out raises the error word and the kernel drains.
 #pragma once
@@ -54,6 +54,7 @@ struct GroupArgs {
     int np;                // batch padded to a multiple of 16 (MMA N and activation box rows)
     int splits, seg;       // down: splits of the reduction dimension, columns per split (multiple of 64)
     int KS;                // K + n_shared
+    const float *inv_rms;  // gate/up: RMSNorm factor per sequence, applied to the accumulators
     __nv_bfloat16 *act;    // gate/up out, down in: [pairs][I]
     float *part;           // down out: [B*KS][splits][H]
     unsigned *err;
@@ -220,7 +221,8 @@ dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_cons
             if (NMAT == 2) {
                 for (int i = 0; i < count; ++i) {
                     const int tok = a.wl.pair_token[start + i];
-                    const float g = tmem_ld1(acc + tok), u = tmem_ld1(acc + 64 + tok);
+                    const float inv = a.inv_rms[tok];  // W (inv * h) = inv * (W h)
+                    const float g = inv * tmem_ld1(acc + tok), u = inv * tmem_ld1(acc + 64 + tok);
                     if (ok && row < a.rows)
                         a.act[(size_t)(start + i) * a.rows + row] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
                 }
@@ -252,11 +254,15 @@ dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_cons
     if (tid == 0 && s_dead) *a.err = 1u;
 }
 
-// h_out[b][c] = h[b][c] + r * (weighted sum of the down projection's partial sums)
-__global__ void __launch_bounds__(256) dense_combine_kernel(FfnArgs a, int S)
+// h_out[b][c] = h[b][c] + r * (weighted sum of the down projection's partial sums); the bf16
+// copy is the next layer's gate/up operand
+__global__ void __launch_bounds__(256) dense_combine_kernel(FfnArgs a, int S, __nv_bfloat16 *xb)
 {
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < a.B * a.H; i += gridDim.x * blockDim.x)
-        a.h_out[i] = finish_value(a, i / a.H, i % a.H, S);
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < a.B * a.H; i += gridDim.x * blockDim.x) {
+        const float v = finish_value(a, i / a.H, i % a.H, S);
+        a.h_out[i] = v;
+        xb[i] = __float2bfloat16_rn(v);
+    }
 }
 
 }  // namespace stmoe_dev

@@ -272,14 +272,25 @@ __global__ void __launch_bounds__(256) topk_group_kernel(TopkArgs a)
 // loads issued up front), partial logits and partial sums of squares to global memory; the
 // CTA that arrives last (arrival counter, no waiting) sums them in a fixed order, applies the
 // RMSNorm factor and runs softmax / top-K / grouping.
-constexpr int kRouterUnroll = 4;
+// Column chunk of one task: 4 warp-wide 16-byte loads of weights for a single sequence (few,
+// long tasks: the phase is one trip to memory either way), 1 for a batch, where the warp also
+// has to fetch that chunk of every sequence's hidden state and short chunks keep all of those
+// loads in flight at once.
+template <int DT> __host__ __device__ constexpr int router_chunk_cols(int batch)
+{
+    return kWarp * Fmt<DT>::kEpl * (batch == 1 ? 4 : 1);
+}
+template <int DT> __host__ __device__ constexpr int router_chunks(int hidden, int batch)
+{
+    return (hidden + router_chunk_cols<DT>(batch) - 1) / router_chunk_cols<DT>(batch);
+}
 
 struct RouterArgs {
     const float *h;      // [B][H]
     const uint8_t *W;    // [E][H]
     int H;
     float eps;
-    float *part;         // [C][B][E] partial logits, C = column chunks
+    float *part;         // [C][B][E] partial logits, C = router_chunks(H, B) column chunks
     float *ss_part;      // [C][B] partial sums of squares
     unsigned *arrivals;  // [1], zero between launches
     float *inv_rms;      // [B]
@@ -287,25 +298,22 @@ struct RouterArgs {
     TopkArgs tk;         // tk.logits unused
 };
 
-template <int DT> __host__ __device__ constexpr int router_chunk_cols()
-{
-    return kWarp * Fmt<DT>::kEpl * kRouterUnroll;
-}
-
 // One split-K task: partial logits of expert row j over column chunk c for every sequence
-// (and, for j == 0, the partial sums of squares of that chunk).  kPdl: wait for the previous
-// kernel between loading the (independent) router weights and reading h.
-template <int DT, bool kPdl>
+// (and, for j == 0, the partial sums of squares of that chunk).  U = weight loads per lane
+// (4: single sequence, 1: batch).  kPdl: wait for the previous kernel between loading the
+// (independent) router weights and reading h.
+template <int DT, int U, bool kPdl>
 __device__ __forceinline__ void router_task(const RouterArgs &a, int task, int lane)
 {
-    constexpr int EPL = Fmt<DT>::kEpl, BYTES = Fmt<DT>::kBytes, CH = router_chunk_cols<DT>();
+    constexpr int EPL = Fmt<DT>::kEpl, BYTES = Fmt<DT>::kBytes, CH = kWarp * EPL * U;
+    constexpr int TB = U == 1 ? 8 : 1;  // sequences whose loads are issued together
     const int B = a.tk.B, E = a.tk.E, H = a.H;
     const int C = (H + CH - 1) / CH;
     const int j = task / C, c = task % C;
     const uint8_t *row = a.W + (size_t)j * H * BYTES;
-    float wf[kRouterUnroll][EPL];
+    float wf[U][EPL];
 #pragma unroll
-    for (int u = 0; u < kRouterUnroll; ++u) {
+    for (int u = 0; u < U; ++u) {
         const int k = c * CH + (u * kWarp + lane) * EPL;
         if (k < H) {
             Fmt<DT>::unpack(ld_stream16(row + (size_t)k * BYTES), wf[u]);
@@ -315,27 +323,52 @@ __device__ __forceinline__ void router_task(const RouterArgs &a, int task, int l
         }
     }
     if (kPdl) pdl_wait();  // the router weights above do not depend on the previous kernel; h does
-    for (int b = 0; b < B; ++b) {
-        float acc = 0.f, ss = 0.f;
+    for (int b0 = 0; b0 < B; b0 += TB) {
+        float4 hv[TB][U][EPL / 4];
 #pragma unroll
-        for (int u = 0; u < kRouterUnroll; ++u) {
-            const int k = c * CH + (u * kWarp + lane) * EPL;
-            if (k < H) {
+        for (int t = 0; t < TB; ++t)
 #pragma unroll
-                for (int e = 0; e < EPL; e += 4) {
-                    const float4 v = ld_f4(a.h + (size_t)b * H + k + e);
-                    acc = fmaf(wf[u][e], v.x, acc), acc = fmaf(wf[u][e + 1], v.y, acc);
-                    acc = fmaf(wf[u][e + 2], v.z, acc), acc = fmaf(wf[u][e + 3], v.w, acc);
+            for (int u = 0; u < U; ++u) {
+                const int k = c * CH + (u * kWarp + lane) * EPL;
+#pragma unroll
+                for (int e = 0; e < EPL / 4; ++e)
+                    hv[t][u][e] = (k < H && b0 + t < B) ? ld_f4(a.h + (size_t)(b0 + t) * H + k + 4 * e)
+                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+        for (int t = 0; t < TB; ++t) {
+            float acc = 0.f, ss = 0.f;
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int e = 0; e < EPL / 4; ++e) {
+                    const float4 v = hv[t][u][e];
+                    acc = fmaf(wf[u][4 * e], v.x, acc), acc = fmaf(wf[u][4 * e + 1], v.y, acc);
+                    acc = fmaf(wf[u][4 * e + 2], v.z, acc), acc = fmaf(wf[u][4 * e + 3], v.w, acc);
                     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
                 }
+            acc = warp_sum(acc);
+            if (j == 0) ss = warp_sum(ss);
+            if (lane == 0 && b0 + t < B) {
+                a.part[((size_t)c * B + b0 + t) * E + j] = acc;
+                if (j == 0) a.ss_part[c * B + b0 + t] = ss;
             }
         }
-        acc = warp_sum(acc);
-        if (j == 0) ss = warp_sum(ss);
-        if (lane == 0) {
-            a.part[((size_t)c * B + b) * E + j] = acc;
-            if (j == 0) a.ss_part[c * B + b] = ss;
-        }
+    }
+}
+
+// All split-K tasks of a layer's gating network, dealt over `n_warps` warps of which this is
+// number `w` (tasks w, w + n_warps, ...).
+template <int DT, bool kPdl>
+__device__ __forceinline__ void router_tasks(const RouterArgs &a, int w, int n_warps, int lane)
+{
+    const int B = a.tk.B;
+    const int n_tasks = a.tk.E * (B == 1 ? router_chunks<DT>(a.H, 1) : router_chunks<DT>(a.H, 2));
+    for (int task = w; task < n_tasks; task += n_warps) {
+        if (B == 1)
+            router_task<DT, 4, kPdl>(a, task, lane);
+        else
+            router_task<DT, 1, kPdl>(a, task, lane);
     }
 }
 
@@ -347,10 +380,9 @@ __device__ __forceinline__ void router_task(const RouterArgs &a, int task, int l
 template <int DT>
 __device__ __forceinline__ void route_single_block(const RouterArgs &a, int *s_ids, int *scratch)
 {
-    constexpr int CH = router_chunk_cols<DT>();
     const int j = threadIdx.x, lane = j % kWarp, warp = j / kWarp;
     const int E = a.tk.E, K = a.tk.K, H = a.H;
-    const int C = (H + CH - 1) / CH;
+    const int C = router_chunks<DT>(H, 1);
     uint32_t *s_key = reinterpret_cast<uint32_t *>(scratch);      // [256]
     float *s_red = reinterpret_cast<float *>(scratch + 256);      // [8] max, [8] sum, [8] selected sum
     float *s_pick = reinterpret_cast<float *>(scratch + 256 + 24); // [0] K-th logit, [1] (K+1)-th
@@ -456,9 +488,8 @@ __device__ __forceinline__ void finalize_tokens(const RouterArgs &a, int *s_ids,
 template <int DT>
 __device__ __forceinline__ void router_finalize(const RouterArgs &a, int *s_ids, int *s_scan, int nw)
 {
-    constexpr int CH = router_chunk_cols<DT>();
     const int B = a.tk.B, E = a.tk.E, H = a.H;
-    const int C = (H + CH - 1) / CH;
+    const int C = router_chunks<DT>(H, B);
     if (B == 1) {
         if (threadIdx.x < 256) route_single_block<DT>(a, s_ids, s_scan);
     } else if (E <= 32) {
@@ -481,14 +512,12 @@ __device__ __forceinline__ void router_finalize(const RouterArgs &a, int *s_ids,
 template <int DT>
 __global__ void __launch_bounds__(256) router_fused_kernel(RouterArgs a)
 {
-    constexpr int CH = router_chunk_cols<DT>(), NW = 8;
+    constexpr int NW = 8;
     __shared__ int s_ids[kMaxBatch * kMaxTopK];
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
     __shared__ int s_last;
     const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
-    const int C = (a.H + CH - 1) / CH;
-    const int task = blockIdx.x * NW + warp;
-    if (task < a.tk.E * C) router_task<DT, true>(a, task, lane);
+    router_tasks<DT, true>(a, blockIdx.x * NW + warp, gridDim.x * NW, lane);
     pdl_wait();  // warps without a task: nothing below may run ahead of the previous kernel either
     __threadfence();
     __syncthreads();

@@ -594,7 +594,8 @@ int dense_setup(stmoe *s)
 
 // gate/up, down and the weighted sum of one layer step on the tensor-core kernels; the work
 // list (one entry per expert) and inv_rms come from the router kernel launched before
-int dense_ffn(stmoe *s, int layer, int batch, const FfnArgs &fa, cudaStream_t st)
+// chained: h_in is the output of the previous layer's dense_ffn, whose bf16 copy is still in d_xb
+int dense_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, cudaStream_t st)
 {
     const stmoe_config_t &c = s->cfg;
     const int E = c.n_experts, H = c.hidden, I = c.inter, np = (batch + 15) / 16 * 16;
@@ -606,10 +607,13 @@ int dense_ffn(stmoe *s, int layer, int batch, const FfnArgs &fa, cudaStream_t st
         ST_TRY(get_event(s, &e2));
         CU_TRY(cudaEventRecord(e0, st));
     }
-    dense_cast_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fa.h, fa.inv_rms, batch, batch, H, s->d_xb);
+    if (!chained) {
+        dense_cast_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fa.h, nullptr, batch, batch, H, s->d_xb);
+        s->launches += 1;
+    }
     GroupArgs g{};
     g.wl = fa.wl, g.E = E, g.img_routed0 = layer * E, g.img_shared0 = c.n_layers * E + layer * c.n_shared;
-    g.np = np, g.KS = s->KS, g.act = s->d_actb, g.part = s->d_part_dense, g.err = s->d_err;
+    g.np = np, g.KS = s->KS, g.inv_rms = fa.inv_rms, g.act = s->d_actb, g.part = s->d_part_dense, g.err = s->d_err;
     g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kDenseKStep - 1) / kDenseKStep * kDenseKStep;
     dense_group_kernel<2><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_gate, s->map_up,
                                                                                       s->map_x[np / 16 - 1], g);
@@ -624,14 +628,14 @@ int dense_ffn(stmoe *s, int layer, int batch, const FfnArgs &fa, cudaStream_t st
                                                                                       s->map_act[np / 16 - 1], g);
     FfnArgs fc = fa;
     fc.part = s->d_part_dense;
-    dense_combine_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fc, splits);
+    dense_combine_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fc, splits, s->d_xb);
     if (timed) {
         CU_TRY(cudaEventRecord(e2, st));
         s->spans.push_back(TimedSpan{e0, e1, 2});
         s->spans.push_back(TimedSpan{e1, e2, 3});
         s->timed_ffn += 1;
     }
-    s->launches += 4;
+    s->launches += 3;
     CU_TRY(cudaGetLastError());
     return STMOE_OK;
 }
@@ -662,7 +666,7 @@ int run_ffn(stmoe *s, int dt, int mt, const FfnPlan &plan, const FfnArgs &fa, cu
 
 int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, int32_t *routed_ids,
                float *routed_w, int32_t *predicted_ids, int32_t *n_predicted, uint32_t *flags,
-               cudaStream_t st)
+               cudaStream_t st, bool chained = false)
 {
     const stmoe_config_t &c = s->cfg;
     const int E = c.n_experts, K = c.top_k, H = c.hidden;
@@ -687,18 +691,20 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
     ta.ids_out = routed_ids, ta.w_out = routed_w, ta.flags_out = flags;
     ta.near_tie_counter = s->pst.stats + 4;
     ta.wl = s->wlm.wl;
-    if (s->rdt == STMOE_F32) {
-        const int C = (H + router_chunk_cols<0>() - 1) / router_chunk_cols<0>();
-        if (layer > 0 && !offloaded(s))
-            launch_pdl(router_fused_kernel<0>, (E * C + 7) / 8, 256, st, ra);
-        else
-            router_fused_kernel<0><<<(E * C + 7) / 8, 256, 0, st>>>(ra);
-    } else {
-        const int C = (H + router_chunk_cols<1>() - 1) / router_chunk_cols<1>();
-        if (layer > 0 && !offloaded(s))
-            launch_pdl(router_fused_kernel<1>, (E * C + 7) / 8, 256, st, ra);
-        else
-            router_fused_kernel<1><<<(E * C + 7) / 8, 256, 0, st>>>(ra);
+    {
+        const int C = s->rdt == STMOE_F32 ? router_chunks<0>(H, batch) : router_chunks<1>(H, batch);
+        const int grid = std::min((E * C + 7) / 8, 2 * s->plan1.grid_gate_up);
+        if (s->rdt == STMOE_F32) {
+            if (layer > 0 && !offloaded(s))
+                launch_pdl(router_fused_kernel<0>, grid, 256, st, ra);
+            else
+                router_fused_kernel<0><<<grid, 256, 0, st>>>(ra);
+        } else {
+            if (layer > 0 && !offloaded(s))
+                launch_pdl(router_fused_kernel<1>, grid, 256, st, ra);
+            else
+                router_fused_kernel<1><<<grid, 256, 0, st>>>(ra);
+        }
     }
     CU_TRY(cudaGetLastError());
     if (s->time_kernels) {
@@ -721,7 +727,7 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
     }
     s->launches += 1;
     if (dense)
-        ST_TRY(dense_ffn(s, layer, batch, fa, st));
+        ST_TRY(dense_ffn(s, layer, batch, chained, fa, st));
     else
         ST_TRY(run_ffn(s, c.weight_dtype, mt, mt == 1 ? s->plan1 : s->plan4, fa, st));
     if (!offloaded(s)) {
@@ -753,7 +759,7 @@ int token_eager(stmoe *s, int batch, const float *h_in, float *h_out, int32_t *r
         ST_TRY(layer_step(s, l, batch, l == 0 ? h_in : h_out, h_out, routed_ids ? routed_ids + o * K : nullptr,
                           routed_w ? routed_w + o * K : nullptr,
                           predicted_ids ? predicted_ids + o * s->max_pred : nullptr,
-                          n_predicted ? n_predicted + o : nullptr, flags ? flags + o : nullptr, st));
+                          n_predicted ? n_predicted + o : nullptr, flags ? flags + o : nullptr, st, l > 0));
     }
     return join_side(s, st);
 }
@@ -944,8 +950,7 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
     CR_TRY(cudaMalloc(&s->d_inv, sizeof(float) * B));
     CR_TRY(cudaMalloc(&s->d_logits, sizeof(float) * B * E));
     {
-        const int ch = s->rdt == STMOE_F32 ? router_chunk_cols<0>() : router_chunk_cols<1>();
-        const int C = (H + ch - 1) / ch;
+        const int C = s->rdt == STMOE_F32 ? router_chunks<0>(H, 2) : router_chunks<1>(H, 2);  // the finer chunking
         CR_TRY(cudaMalloc(&s->d_rpart, sizeof(float) * (size_t)C * B * E));
         CR_TRY(cudaMalloc(&s->d_sspart, sizeof(float) * (size_t)C * B));
         CR_TRY(cudaMalloc(&s->d_arrivals, 16));
@@ -976,8 +981,7 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
         }
         (void)cudaGetLastError();
         if (ok) {
-            const int ch = s->rdt == STMOE_F32 ? router_chunk_cols<0>() : router_chunk_cols<1>();
-            const size_t C = (H + ch - 1) / ch, tiles = (H + kTileRows - 1) / kTileRows, pairs = (size_t)B * s->KS;
+            const size_t C = s->rdt == STMOE_F32 ? router_chunks<0>(H, 2) : router_chunks<1>(H, 2), tiles = (H + kTileRows - 1) / kTileRows, pairs = (size_t)B * s->KS;
             CR_TRY(cudaMalloc(&s->d_hbuf, sizeof(float) * (size_t)(L + 1) * B * H));
             CR_TRY(cudaMalloc(&s->d_rpart_all, sizeof(float) * L * C * B * E));
             CR_TRY(cudaMalloc(&s->d_sspart_all, sizeof(float) * L * C * B));

@@ -185,7 +185,7 @@ __device__ __forceinline__ void grid_barrier(unsigned *counter, unsigned *err, u
 template <int DT, int RDT, int MTMAX>
 __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs a)
 {
-    constexpr int CH = router_chunk_cols<RDT>(), NW = kFfnThreads / kWarp;
+    constexpr int NW = kFfnThreads / kWarp;
     extern __shared__ __align__(16) int dyn[];  // work list | ids | prev ids | gate weights
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
     __shared__ int s_score[kMaxExperts];
@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs 
     const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
     const int L = a.L, B = a.B, E = a.E, K = a.K, H = a.H, I = a.I, S = a.S;
     const int KS = K + a.n_shared, pairs = B * KS;
-    const int C = (H + CH - 1) / CH, tiles = (H + kTileRows - 1) / kTileRows;
+    const int C = router_chunks<RDT>(H, B), tiles = (H + kTileRows - 1) / kTileRows;
 
     WorkList wl;
     wl.n_groups = dyn, wl.g_expert = dyn + 4, wl.g_start = dyn + 4 + pairs, wl.g_count = dyn + 4 + 2 * pairs;
@@ -225,10 +225,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs 
         tk.near_tie_counter = lead ? a.pst.stats + 4 : nullptr;
         tk.wl = wl;
         DBG_STAMP(l * 8 + 0);
-        {
-            const int task = warp * gridDim.x + blockIdx.x;  // spread the tasks over the SMs first
-            if (task < E * C) router_task<RDT, false>(ra, task, lane);
-        }
+        router_tasks<RDT, false>(ra, warp * gridDim.x + blockIdx.x, NW * gridDim.x, lane);  // over the SMs first
         grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 1);
         DBG_STAMP(l * 8 + 2);
 
