@@ -614,14 +614,14 @@ int dense_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, c
     GroupArgs g{};
     g.wl = fa.wl, g.E = E, g.img_routed0 = layer * E, g.img_shared0 = c.n_layers * E + layer * c.n_shared;
     g.np = np, g.KS = s->KS, g.inv_rms = fa.inv_rms, g.act = s->d_actb, g.part = s->d_part_dense, g.err = s->d_err;
-    g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kDenseKStep - 1) / kDenseKStep * kDenseKStep;
+    g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + group_kstage<2>() - 1) / group_kstage<2>() * group_kstage<2>();
     dense_group_kernel<2><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_gate, s->map_up,
                                                                                       s->map_x[np / 16 - 1], g);
     if (timed) CU_TRY(cudaEventRecord(e1, st));
     // down: split the reduction dimension until there are a few tasks per SM
     const int entries = std::min(E, batch * c.top_k) + c.n_shared, tiles = (H + kDenseRows - 1) / kDenseRows;
     int splits = std::max(1, std::min(kDenseMaxSplits, (4 * s->dense_grid + entries * tiles - 1) / (entries * tiles)));
-    int seg = ((I + splits - 1) / splits + kDenseKStep - 1) / kDenseKStep * kDenseKStep;
+    int seg = ((I + splits - 1) / splits + group_kstage<1>() - 1) / group_kstage<1>() * group_kstage<1>();
     splits = (I + seg - 1) / seg;  // no empty split
     g.rows = H, g.kd = I, g.splits = splits, g.seg = seg;
     dense_group_kernel<1><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_down, s->map_down,
