@@ -123,30 +123,172 @@ __device__ __forceinline__ GroupTask group_task(const GroupArgs &a, int task)
     return t;
 }
 
-// NMAT = 2: gate and up projections with the SiLU epilogue; NMAT = 1: down projection.
+// Shared-memory ring of stages with its barriers, and the accumulator hand-off barriers.
+struct GroupRing {
+    uint8_t *dsm;                           // 1024-byte aligned
+    uint64_t *full, *empty, *tfull, *tempty;
+    int NS, slot;                           // stages, bytes per stage slot
+    uint32_t tmem;                          // base of the 256 accumulator columns
+    volatile int *dead;
+};
+struct RingPos {
+    int s = 0;
+    uint32_t ph = 0;
+};
+
+__device__ __forceinline__ void group_ring_init(const GroupRing &r)
+{
+    for (int s = 0; s < r.NS; ++s) dmbar_init(&r.full[s], 1), dmbar_init(&r.empty[s], 1);
+    for (int b = 0; b < 2; ++b) dmbar_init(&r.tfull[b], 1), dmbar_init(&r.tempty[b], 4);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+// One thread: issue the TMA loads of this CTA's tasks.  pos/issued carry on from earlier calls.
+// NMAT = 2: gate and up projections; NMAT = 1: down projection.
+template <int NMAT>
+__device__ __forceinline__ void group_produce(const CUtensorMap *map_w0, const CUtensorMap *map_w1,
+                                              const CUtensorMap *map_x, const GroupArgs &a, const GroupRing &r,
+                                              RingPos &pos, int &issued)
+{
+    constexpr int KB = group_kboxes<NMAT>(), KSTAGE = group_kstage<NMAT>();
+    const int np = a.np, box = NMAT * kGroupTileBytes + group_act_bytes(np);
+    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
+    const int n_tasks = *a.wl.n_groups * tiles * a.splits;
+    for (int task = blockIdx.x; task < n_tasks && !*r.dead; task += gridDim.x) {
+        const GroupTask t = group_task(a, task);
+        const int ge = a.wl.g_expert[t.g];
+        const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
+        const int xrow = NMAT == 2 ? 0 : a.wl.g_start[t.g];
+        for (int k = t.k0; k < t.k1; k += KSTAGE) {
+            if (!dmbar_wait(&r.empty[pos.s], pos.ph ^ 1u, r.dead)) return;
+            uint8_t *st = r.dsm + (size_t)pos.s * r.slot;
+            // boxes past the end of the reduction dimension are zero-filled and still count
+            dmbar_expect_tx(&r.full[pos.s], (uint32_t)(KB * (NMAT * kGroupTileBytes + np * kDenseKStep * 2)));
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb) {
+                uint8_t *sb = st + kb * box;
+                tma_load_3d(sb, map_w0, k + kb * kDenseKStep, t.row0, img, &r.full[pos.s]);
+                if (NMAT == 2) tma_load_3d(sb + kGroupTileBytes, map_w1, k + kb * kDenseKStep, t.row0, img, &r.full[pos.s]);
+                tma_load_2d(sb + NMAT * kGroupTileBytes, map_x, k + kb * kDenseKStep, xrow, &r.full[pos.s]);
+            }
+            ++issued;
+            if (++pos.s == r.NS) pos.s = 0, pos.ph ^= 1u;
+        }
+    }
+}
+
+// Every load that was issued has to land before the CTA may exit.
+__device__ __forceinline__ void group_drain(const GroupRing &r, RingPos pos, int issued)
+{
+    for (int i = 0; i < min(issued, r.NS); ++i) {
+        if (pos.s == 0) pos.s = r.NS, pos.ph ^= 1u;
+        --pos.s;
+        dmbar_wait(&r.full[pos.s], pos.ph, r.dead);
+    }
+}
+
+// One thread: issue the MMAs of this CTA's tasks.  `it` counts the CTA's tasks across calls
+// (accumulator buffer = it & 1).
+template <int NMAT>
+__device__ __forceinline__ void group_mma(const GroupArgs &a, const GroupRing &r, RingPos &pos, int &it)
+{
+    constexpr int KB = group_kboxes<NMAT>(), KSTAGE = group_kstage<NMAT>();
+    const int np = a.np, box = NMAT * kGroupTileBytes + group_act_bytes(np);
+    const uint32_t idesc = umma_idesc_bf16(np);
+    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
+    const int n_tasks = *a.wl.n_groups * tiles * a.splits;
+    for (int task = blockIdx.x; task < n_tasks && !*r.dead; task += gridDim.x, ++it) {
+        const GroupTask t = group_task(a, task);
+        const int ab = it & 1;
+        if (!dmbar_wait(&r.tempty[ab], (((uint32_t)it >> 1) & 1u) ^ 1u, r.dead)) return;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t acc = r.tmem + ab * 128;
+        bool first = true;
+        for (int k = t.k0; k < t.k1; k += KSTAGE) {
+            if (!dmbar_wait(&r.full[pos.s], pos.ph, r.dead)) return;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb) {
+                const uint32_t st = dsmem_u32(r.dsm + (size_t)pos.s * r.slot) + kb * box;
+#pragma unroll
+                for (int j = 0; j < kDenseKStep / 16; ++j) {
+                    const uint64_t bd = umma_desc_sw128(st + NMAT * kGroupTileBytes, j);
+#pragma unroll
+                    for (int mat = 0; mat < NMAT; ++mat)
+                        umma_bf16(acc + mat * 64, umma_desc_sw128(st + mat * kGroupTileBytes, j), bd, idesc,
+                                  !first || kb > 0 || j > 0);
+                }
+            }
+            first = false;
+            umma_commit(&r.empty[pos.s]);
+            if (++pos.s == r.NS) pos.s = 0, pos.ph ^= 1u;
+        }
+        umma_commit(&r.tfull[ab]);
+    }
+}
+
+// Four warps (lg = the TMEM lane quarter the warp may read = warp index % 4): thread = one
+// weight row.  `it` as in group_mma.
+template <int NMAT>
+__device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRing &r, int &it, int lg, int lane)
+{
+    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
+    const int n_tasks = *a.wl.n_groups * tiles * a.splits;
+    for (int task = blockIdx.x; task < n_tasks; task += gridDim.x, ++it) {
+        const GroupTask t = group_task(a, task);
+        const int ab = it & 1;
+        const int start = a.wl.g_start[t.g], count = a.wl.g_count[t.g];
+        const bool ok = dmbar_wait(&r.tfull[ab], ((uint32_t)it >> 1) & 1u, r.dead);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t acc = r.tmem + ab * 128 + ((uint32_t)(lg * kWarp) << 16);
+        const int row = t.row0 + lg * kWarp + lane;
+        if (NMAT == 2) {
+            for (int i = 0; i < count; ++i) {
+                const int tok = a.wl.pair_token[start + i];
+                const float inv = a.inv_rms[tok];  // W (inv * h) = inv * (W h)
+                const float g = inv * tmem_ld1(acc + tok), u = inv * tmem_ld1(acc + 64 + tok);
+                if (ok && row < a.rows)
+                    a.act[(size_t)(start + i) * a.rows + row] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
+            }
+        } else {
+            for (int i0 = 0; i0 < count; i0 += 8) {
+                float y[8];
+                tmem_ld8(acc + i0, y);
+                if (ok && row < a.rows) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (i0 + i < count) {
+                            const int slot = a.wl.pair_slot[start + i0 + i];
+                            a.part[((size_t)slot * a.splits + t.z) * a.rows + row] = y[i];
+                        }
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) dmbar_arrive(&r.tempty[ab]);
+        if (!ok) return;
+    }
+}
+
+// One projection as a kernel of its own (per-layer launches).
 template <int NMAT>
 __global__ void __launch_bounds__(kGroupThreads, 1)
 dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
                    const __grid_constant__ CUtensorMap map_x, GroupArgs a)
 {
-    constexpr int kGroupKBoxes = group_kboxes<NMAT>(), kGroupKStage = group_kstage<NMAT>();
     extern __shared__ uint8_t dsm_raw[];
     __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2];
     __shared__ uint32_t s_tmem;
     __shared__ int s_dead;
-    uint8_t *dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, warp = tid / kWarp, lane = tid % kWarp;
-    const int np = a.np;
-    const int NS = group_stages<NMAT>(np), STAGE = group_stage_bytes<NMAT>(np), act_bytes = group_act_bytes(np);
-    const int n_groups = *a.wl.n_groups;
-    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
-    const int n_tasks = n_groups * tiles * a.splits;
-
+    GroupRing r;
+    r.dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
+    r.full = full, r.empty = empty, r.tfull = tfull, r.tempty = tempty, r.dead = &s_dead;
+    r.NS = group_stages<NMAT>(a.np), r.slot = group_stage_bytes<NMAT>(a.np);
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) dmbar_init(&full[s], 1), dmbar_init(&empty[s], 1);
-        for (int b = 0; b < 2; ++b) dmbar_init(&tfull[b], 1), dmbar_init(&tempty[b], 4);
         s_dead = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        group_ring_init(r);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dsmem_u32(&s_tmem)),
@@ -157,122 +299,29 @@ dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_cons
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem = s_tmem;
+    r.tmem = s_tmem;
 
     if (warp == 0) {
-        // ---- TMA producer -----------------------------------------------------------------------
         if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0;
+            RingPos pos;
             int issued = 0;
-            for (int task = blockIdx.x; task < n_tasks && !s_dead; task += gridDim.x) {
-                const GroupTask t = group_task(a, task);
-                const int ge = a.wl.g_expert[t.g];
-                const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
-                const int xrow = NMAT == 2 ? 0 : a.wl.g_start[t.g];
-                for (int k = t.k0; k < t.k1; k += kGroupKStage) {
-                    if (!dmbar_wait(&empty[s], ph ^ 1u, &s_dead)) break;
-                    uint8_t *st = dsm + (size_t)s * STAGE;
-                    // boxes past the end of the reduction dimension are zero-filled and still count
-                    dmbar_expect_tx(&full[s], (uint32_t)(kGroupKBoxes * (NMAT * kGroupTileBytes + np * kDenseKStep * 2)));
-#pragma unroll
-                    for (int kb = 0; kb < kGroupKBoxes; ++kb) {
-                        uint8_t *sb = st + kb * (NMAT * kGroupTileBytes + act_bytes);
-                        tma_load_3d(sb, &map_w0, k + kb * kDenseKStep, t.row0, img, &full[s]);
-                        if (NMAT == 2)
-                            tma_load_3d(sb + kGroupTileBytes, &map_w1, k + kb * kDenseKStep, t.row0, img, &full[s]);
-                        tma_load_2d(sb + NMAT * kGroupTileBytes, &map_x, k + kb * kDenseKStep, xrow, &full[s]);
-                    }
-                    ++issued;
-                    if (++s == NS) s = 0, ph ^= 1u;
-                }
-            }
-            // every load that was issued has to land before the CTA may exit
-            for (int i = 0; i < min(issued, NS); ++i) {
-                if (s == 0) s = NS, ph ^= 1u;
-                --s;
-                dmbar_wait(&full[s], ph, &s_dead);
-            }
+            group_produce<NMAT>(&map_w0, &map_w1, &map_x, a, r, pos, issued);
+            group_drain(r, pos, issued);
         }
     } else if (warp == 1) {
-        // ---- MMA issue ----------------------------------------------------------------------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16(np);
-            int s = 0, it = 0;
-            uint32_t ph = 0;
-            for (int task = blockIdx.x; task < n_tasks && !s_dead; task += gridDim.x, ++it) {
-                const GroupTask t = group_task(a, task);
-                const int ab = it & 1;
-                if (!dmbar_wait(&tempty[ab], (((uint32_t)it >> 1) & 1u) ^ 1u, &s_dead)) break;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t acc = tmem + ab * 128;
-                bool first = true;
-                for (int k = t.k0; k < t.k1; k += kGroupKStage) {
-                    if (!dmbar_wait(&full[s], ph, &s_dead)) break;
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-                    for (int kb = 0; kb < kGroupKBoxes; ++kb) {
-                        const uint32_t st = dsmem_u32(dsm + (size_t)s * STAGE) + kb * (NMAT * kGroupTileBytes + act_bytes);
-#pragma unroll
-                        for (int j = 0; j < kDenseKStep / 16; ++j) {
-                            const uint64_t bd = umma_desc_sw128(st + NMAT * kGroupTileBytes, j);
-#pragma unroll
-                            for (int mat = 0; mat < NMAT; ++mat)
-                                umma_bf16(acc + mat * 64, umma_desc_sw128(st + mat * kGroupTileBytes, j), bd, idesc,
-                                          !first || kb > 0 || j > 0);
-                        }
-                    }
-                    first = false;
-                    umma_commit(&empty[s]);
-                    if (++s == NS) s = 0, ph ^= 1u;
-                }
-                umma_commit(&tfull[ab]);
-            }
+            RingPos pos;
+            int it = 0;
+            group_mma<NMAT>(a, r, pos, it);
         }
     } else {
-        // ---- epilogue: thread = one weight row (TMEM lane) -------------------------------------
-        const int lg = warp % 4;  // the TMEM lane quarter this warp may read
         int it = 0;
-        for (int task = blockIdx.x; task < n_tasks; task += gridDim.x, ++it) {
-            const GroupTask t = group_task(a, task);
-            const int ab = it & 1;
-            const int start = a.wl.g_start[t.g], count = a.wl.g_count[t.g];
-            const bool ok = dmbar_wait(&tfull[ab], ((uint32_t)it >> 1) & 1u, &s_dead);
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t acc = tmem + ab * 128 + ((uint32_t)(lg * kWarp) << 16);
-            const int row = t.row0 + lg * kWarp + lane;
-            if (NMAT == 2) {
-                for (int i = 0; i < count; ++i) {
-                    const int tok = a.wl.pair_token[start + i];
-                    const float inv = a.inv_rms[tok];  // W (inv * h) = inv * (W h)
-                    const float g = inv * tmem_ld1(acc + tok), u = inv * tmem_ld1(acc + 64 + tok);
-                    if (ok && row < a.rows)
-                        a.act[(size_t)(start + i) * a.rows + row] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
-                }
-            } else {
-                for (int i0 = 0; i0 < count; i0 += 8) {
-                    float y[8];
-                    tmem_ld8(acc + i0, y);
-                    if (ok && row < a.rows) {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if (i0 + i < count) {
-                                const int slot = a.wl.pair_slot[start + i0 + i];
-                                a.part[((size_t)slot * a.splits + t.z) * a.rows + row] = y[i];
-                            }
-                    }
-                }
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) dmbar_arrive(&tempty[ab]);
-            if (!ok) break;
-        }
+        group_epilogue<NMAT>(a, r, it, warp % 4, lane);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kGroupTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(r.tmem), "r"(kGroupTmemCols) : "memory");
     }
     if (tid == 0 && s_dead) *a.err = 1u;
 }

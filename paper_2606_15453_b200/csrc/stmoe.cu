@@ -17,6 +17,7 @@
 #include "ffn.cuh"
 #include "predictor.cuh"
 #include "router.cuh"
+#include "token_dense_kernel.cuh"
 #include "token_kernel.cuh"
 
 using namespace stmoe_dev;
@@ -315,6 +316,8 @@ struct stmoe {
     __nv_bfloat16 *d_xb = nullptr, *d_actb = nullptr;
     float *d_part_dense = nullptr;
     int dense_grid = 0;
+    bool dense_persistent = false;  // one cooperative kernel per decode step (token_dense_kernel.cuh)
+    int dense_dyn_bytes = 0;
 
     SlotCache cache;
     cudaStream_t copy_stream = nullptr;
@@ -530,6 +533,7 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
 // ---- tensor-core path (dense_group.cuh) ---------------------------------------------------
 constexpr int kDenseMinBatch = 4;
 constexpr int kDenseMaxSplits = 4;
+constexpr int kTokenDenseDynBytes = 220 * 1024;
 
 bool use_dense(const stmoe *s, int batch) { return s->dense && batch >= s->dense_min_batch; }
 
@@ -589,11 +593,28 @@ int dense_setup(stmoe *s)
     s->dense_grid = sm_count();
     s->dense_min_batch = kDenseMinBatch;
     s->dense = true;
+    if (s->persistent) {  // cooperative launches work and the per-layer buffers exist
+        void *k = s->rdt == STMOE_F32 ? (void *)decode_token_dense_kernel<0> : (void *)decode_token_dense_kernel<1>;
+        const int np = (B + 15) / 16 * 16;
+        const int slot = std::max(group_stage_bytes<1>(np), group_stage_bytes<2>(np));
+        const int need = (int)token_smem(B, c.top_k, c.n_shared) + 1024 + slot;  // at least one stage
+        int occ = 0;
+        if (need <= kTokenDenseDynBytes &&
+            cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokenDenseDynBytes) == cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kFfnThreads, kTokenDenseDynBytes) == cudaSuccess &&
+            occ >= 1) {
+            s->dense_persistent = true;
+            s->dense_dyn_bytes = kTokenDenseDynBytes;
+        }
+        (void)cudaGetLastError();
+    }
     return STMOE_OK;
 }
 
 // gate/up, down and the weighted sum of one layer step on the tensor-core kernels; the work
 // list (one entry per expert) and inv_rms come from the router kernel launched before
+int dense_down_splits(const stmoe *s, int batch, int *seg);
+
 // chained: h_in is the output of the previous layer's dense_ffn, whose bf16 copy is still in d_xb
 int dense_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, cudaStream_t st)
 {
@@ -619,10 +640,10 @@ int dense_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, c
                                                                                       s->map_x[np / 16 - 1], g);
     if (timed) CU_TRY(cudaEventRecord(e1, st));
     // down: split the reduction dimension until there are a few tasks per SM
-    const int entries = std::min(E, batch * c.top_k) + c.n_shared, tiles = (H + kDenseRows - 1) / kDenseRows;
-    int splits = std::max(1, std::min(kDenseMaxSplits, (4 * s->dense_grid + entries * tiles - 1) / (entries * tiles)));
-    int seg = ((I + splits - 1) / splits + group_kstage<1>() - 1) / group_kstage<1>() * group_kstage<1>();
-    splits = (I + seg - 1) / seg;  // no empty split
+    int seg = 0;
+    const int splits = dense_down_splits(s, batch, &seg);
+    const int tiles = (H + kDenseRows - 1) / kDenseRows;
+    (void)tiles;
     g.rows = H, g.kd = I, g.splits = splits, g.seg = seg;
     dense_group_kernel<1><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_down, s->map_down,
                                                                                       s->map_act[np / 16 - 1], g);
@@ -786,6 +807,54 @@ int token_persistent(stmoe *s, int batch, const float *h_in, float *h_out, int32
     void *args[] = {&a};
     CU_TRY(cudaLaunchCooperativeKernel(token_kernel(c.weight_dtype, s->rdt, a.mt), dim3(s->persistent_grid),
                                        dim3(kFfnThreads), args, token_smem(batch, c.top_k, c.n_shared), st));
+    s->launches += 1;
+    if (!s->built && s->host_t == c.profile_tokens - 1) {
+        const int rows = (c.n_layers - 1) * c.n_experts;
+        if (rows > 0) cct_build_kernel<<<(rows + 7) / 8, 256, 0, st>>>(s->pst, c.n_layers, c.n_experts, c.top_k);
+        s->launches += rows > 0;
+        s->built = true;
+        CU_TRY(cudaGetLastError());
+    }
+    s->host_t += 1;
+    return STMOE_OK;
+}
+
+int dense_down_splits(const stmoe *s, int batch, int *seg)
+{
+    const stmoe_config_t &c = s->cfg;
+    const int entries = std::min(c.n_experts, batch * c.top_k) + c.n_shared, tiles = (c.hidden + kDenseRows - 1) / kDenseRows;
+    int splits = std::max(1, std::min(kDenseMaxSplits, (4 * s->dense_grid + entries * tiles - 1) / (entries * tiles)));
+    *seg = ((c.inter + splits - 1) / splits + group_kstage<1>() - 1) / group_kstage<1>() * group_kstage<1>();
+    return (c.inter + *seg - 1) / *seg;  // no empty split
+}
+
+int token_dense(stmoe *s, int batch, const float *h_in, float *h_out, int32_t *routed_ids, float *routed_w,
+                int32_t *predicted_ids, int32_t *n_predicted, uint32_t *flags, cudaStream_t st)
+{
+    const stmoe_config_t &c = s->cfg;
+    TokenDenseArgs d{};
+    TokenArgs &a = d.t;
+    a.L = c.n_layers, a.B = batch, a.E = c.n_experts, a.K = c.top_k, a.n_shared = c.n_shared;
+    a.H = c.hidden, a.I = c.inter, a.S = 1, a.mt = kDenseMaxTokens;
+    a.renorm = (c.flags & STMOE_FLAG_RENORM_TOPK) ? 1 : 0;
+    a.eps = c.rms_eps, a.residual_scale = c.residual_scale;
+    a.h_in = h_in, a.h_out = h_out, a.hbuf = s->d_hbuf;
+    a.router = s->d_router;
+    a.rpart = s->d_rpart_all, a.sspart = s->d_sspart_all;
+    a.ids_all = s->d_ids, a.Bmax = c.max_batch;
+    a.ids_out = routed_ids, a.w_out = routed_w, a.flags_out = flags;
+    a.pred_ids = predicted_ids, a.n_pred = n_predicted, a.max_pred = s->max_pred;
+    a.pst = s->pst, a.P = c.profile_tokens, a.mode = c.predictor_mode;
+    a.barrier = s->d_barrier, a.err = s->d_err;
+    d.splits = dense_down_splits(s, batch, &d.seg);
+    d.img_shared_base = c.n_layers * c.n_experts;
+    d.dyn_bytes = s->dense_dyn_bytes;
+    d.xb = s->d_xb, d.actb = s->d_actb, d.part = s->d_part_dense;
+    const int np = (batch + 15) / 16 * 16;
+    CU_TRY(cudaMemsetAsync(s->d_barrier, 0, 4, st));
+    void *args[] = {&s->map_gate, &s->map_up, &s->map_down, &s->map_x[np / 16 - 1], &s->map_act[np / 16 - 1], &d};
+    void *k = s->rdt == STMOE_F32 ? (void *)decode_token_dense_kernel<0> : (void *)decode_token_dense_kernel<1>;
+    CU_TRY(cudaLaunchCooperativeKernel(k, dim3(s->dense_grid), dim3(kFfnThreads), args, (size_t)s->dense_dyn_bytes, st));
     s->launches += 1;
     if (!s->built && s->host_t == c.profile_tokens - 1) {
         const int rows = (c.n_layers - 1) * c.n_experts;
@@ -1078,6 +1147,8 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, i
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const stmoe_config_t &c = s->cfg;
     const bool build_due = !s->built && s->host_t == c.profile_tokens - 1;
+    if (s->dense_persistent && !s->time_kernels && use_dense(s, batch))
+        return token_dense(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
     if (s->persistent && !s->time_kernels && !use_dense(s, batch))
         return token_persistent(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
     if (offloaded(s) || s->time_kernels || s->graph_off || build_due)

@@ -1,0 +1,189 @@
+// One decode step of a resident bf16 stack with several sequences as a single persistent kernel
+// whose expert FFN runs on the tensor cores (the batched counterpart of token_kernel.cuh).
+//
+// One 512-thread CTA per SM, launched cooperatively, walks the layers:
+//   F   weighted sum + residual of the previous layer from its down-projection partial sums
+//       (layer 0: the input), written as fp32 (router, residual) and bf16 (gate/up operand)
+//                                                                          -> grid barrier
+//   R   split-K router GEMV tasks over all warps of the grid               -> grid barrier
+//   T   every CTA runs softmax / top-K / grouping (one work-list entry per expert) itself
+//   GU  gate/up tiles on tcgen05: warp 0 feeds TMA, warp 1 issues MMAs, warps 2-5 read the
+//       accumulators; the predictor (Algorithms 1-3) runs on one more warp of the last CTA
+//                                                                          -> grid barrier
+//   D   down-projection tiles the same way                                 -> grid barrier
+// The stage ring, its barriers and the tensor-memory columns are set up once and carried through
+// all phases and layers.  Data written with ordinary stores and then fetched by TMA from another
+// SM (the bf16 hidden state, the gated activations) is fenced for the async proxy on both sides
+// of the grid barrier in between.
+#pragma once
+#include "dense_group.cuh"
+#include "token_kernel.cuh"
+
+namespace stmoe_dev {
+
+struct TokenDenseArgs {
+    TokenArgs t;            // mt = 64; act/part/tile_done/blob unused
+    int splits, seg;        // down projection: splits of the reduction dimension, columns per split
+    int img_shared_base;    // image index of layer 0's first shared expert (= L * E)
+    int dyn_bytes;          // dynamic shared memory of the launch
+    __nv_bfloat16 *xb;      // [64][H]
+    __nv_bfloat16 *actb;    // [pairs + 64][I]
+    float *part;            // [pairs][splits][H]
+};
+
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+template <int RDT>
+__global__ void __launch_bounds__(kFfnThreads, 1)
+decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __grid_constant__ CUtensorMap map_up,
+                          const __grid_constant__ CUtensorMap map_down, const __grid_constant__ CUtensorMap map_x,
+                          const __grid_constant__ CUtensorMap map_act, TokenDenseArgs d)
+{
+    constexpr int NW = kFfnThreads / kWarp;
+    const TokenArgs &a = d.t;
+    extern __shared__ __align__(16) int dyn[];  // work list | ids | prev ids | gate weights | stage ring
+    __shared__ int s_scan[2 * (kMaxExperts + 1)];
+    __shared__ int s_score[kMaxExperts];
+    __shared__ float s_inv[kMaxBatch];
+    __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2];
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_dead;
+    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
+    const int L = a.L, B = a.B, E = a.E, K = a.K, H = a.H, I = a.I;
+    const int KS = K + a.n_shared, pairs = B * KS, np = (B + 15) / 16 * 16;
+    const int C = router_chunks<RDT>(H, B);
+
+    WorkList wl;
+    wl.n_groups = dyn, wl.g_expert = dyn + 4, wl.g_start = dyn + 4 + pairs, wl.g_count = dyn + 4 + 2 * pairs;
+    wl.pair_token = dyn + 4 + 3 * pairs, wl.pair_slot = dyn + 4 + 4 * pairs;
+    int *s_ids = dyn + 4 + 5 * pairs;
+    int *s_prev = s_ids + B * K;
+    float *s_w = reinterpret_cast<float *>(s_prev + B * K);
+    const int list_bytes = (int)sizeof(int) * (4 + 5 * pairs + 3 * B * K);
+
+    GroupRing r;
+    r.dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dyn) + list_bytes + 1023) & ~(uintptr_t)1023);
+    r.full = full, r.empty = empty, r.tfull = tfull, r.tempty = tempty, r.dead = &s_dead;
+    r.slot = max(group_stage_bytes<1>(np), group_stage_bytes<2>(np));
+    r.NS = min(kGroupMaxStages, (int)((reinterpret_cast<uint8_t *>(dyn) + d.dyn_bytes - r.dsm) / r.slot));
+    if (threadIdx.x == 0) {
+        s_dead = r.NS < 1;  // cannot happen with the host's sizing; never run a ring without stages
+        group_ring_init(r);
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dsmem_u32(&s_tmem)),
+                     "r"(kGroupTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    r.tmem = s_tmem;
+
+    unsigned target = 0;
+    const bool lead = blockIdx.x == 0;
+    const bool pred_cta = blockIdx.x == gridDim.x - 1;
+    RingPos ppos, mpos;              // producer / MMA thread
+    int issued = 0, mit = 0, eit = 0;  // loads issued (producer); tasks done (MMA thread, epilogue threads)
+    const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gthreads = gridDim.x * blockDim.x;
+
+    // arguments of the weighted sum that finishes layer lp
+    auto finish_args = [&](int lp) {
+        FfnArgs f{};
+        f.part = d.part, f.w = s_w;
+        f.h = lp == 0 ? a.h_in : a.hbuf + (size_t)lp * B * H;
+        f.H = H, f.B = B, f.K = K, f.n_shared = a.n_shared, f.residual_scale = a.residual_scale;
+        return f;
+    };
+
+    for (int l = 0; l < L && !s_dead; ++l) {
+        const float *h = l == 0 ? a.h_in : a.hbuf + (size_t)l * B * H;
+
+        // ---- F ---------------------------------------------------------------------------------
+        if (l == 0) {
+            for (int i = gtid; i < B * H; i += gthreads) d.xb[i] = __float2bfloat16_rn(h[i]);
+        } else {
+            const FfnArgs fp = finish_args(l - 1);
+            float *hl = a.hbuf + (size_t)l * B * H;
+            for (int i = gtid; i < B * H; i += gthreads) {
+                const float v = finish_value(fp, i / H, i % H, d.splits);
+                hl[i] = v;
+                d.xb[i] = __float2bfloat16_rn(v);
+            }
+        }
+        fence_async_proxy();
+        grid_barrier(a.barrier, a.err, target, &s_dead);
+
+        // ---- R ---------------------------------------------------------------------------------
+        RouterArgs ra;
+        ra.h = h, ra.W = a.router + (size_t)l * E * H * Fmt<RDT>::kBytes, ra.H = H, ra.eps = a.eps;
+        ra.part = a.rpart + (size_t)l * C * B * E, ra.ss_part = a.sspart + (size_t)l * C * B;
+        ra.arrivals = nullptr, ra.inv_rms = s_inv, ra.logits_out = nullptr;
+        TopkArgs &tk = ra.tk;
+        tk.logits = nullptr, tk.B = B, tk.E = E, tk.K = K, tk.n_shared = a.n_shared, tk.mt = a.mt, tk.renorm = a.renorm;
+        tk.ids = s_ids, tk.w = s_w;
+        tk.ids_out = (lead && a.ids_out) ? a.ids_out + (size_t)l * B * K : nullptr;
+        tk.w_out = (lead && a.w_out) ? a.w_out + (size_t)l * B * K : nullptr;
+        tk.flags_out = (lead && a.flags_out) ? a.flags_out + (size_t)l * B : nullptr;
+        tk.near_tie_counter = lead ? a.pst.stats + 4 : nullptr;
+        tk.wl = wl;
+        router_tasks<RDT, false>(ra, warp * gridDim.x + blockIdx.x, NW * gridDim.x, lane);
+        grid_barrier(a.barrier, a.err, target, &s_dead);
+
+        // ---- T ---------------------------------------------------------------------------------
+        router_finalize<RDT>(ra, s_ids, s_scan, NW);
+        __syncthreads();
+        if (lead)
+            for (int i = threadIdx.x; i < B * K; i += blockDim.x) a.ids_all[(size_t)l * a.Bmax * K + i] = s_ids[i];
+
+        // ---- GU (+ the predictor on one warp of the last CTA) -----------------------------------
+        GroupArgs g{};
+        g.wl = wl, g.E = E, g.img_routed0 = l * E, g.img_shared0 = d.img_shared_base + l * a.n_shared;
+        g.np = np, g.KS = KS, g.inv_rms = s_inv, g.act = d.actb, g.part = d.part, g.err = a.err;
+        g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + group_kstage<2>() - 1) / group_kstage<2>() * group_kstage<2>();
+        if (warp == 0) {
+            if (lane == 0) {
+                fence_async_proxy();
+                group_produce<2>(&map_gate, &map_up, &map_x, g, r, ppos, issued);
+            }
+        } else if (warp == 1) {
+            if (lane == 0) group_mma<2>(g, r, mpos, mit);
+        } else if (warp < 6) {
+            group_epilogue<2>(g, r, eit, warp % 4, lane);
+            fence_async_proxy();  // the gated activations are fetched by TMA in the next phase
+        } else if (pred_cta && warp == NW - 1) {
+            predictor_step_warp(a, l, s_ids, s_prev, s_score, lane);
+        }
+        grid_barrier(a.barrier, a.err, target, &s_dead);
+
+        // ---- D ---------------------------------------------------------------------------------
+        g.rows = H, g.kd = I, g.splits = d.splits, g.seg = d.seg;
+        if (warp == 0) {
+            if (lane == 0) {
+                fence_async_proxy();
+                group_produce<1>(&map_down, &map_down, &map_act, g, r, ppos, issued);
+            }
+        } else if (warp == 1) {
+            if (lane == 0) group_mma<1>(g, r, mpos, mit);
+        } else if (warp < 6) {
+            group_epilogue<1>(g, r, eit, warp % 4, lane);
+        }
+        for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
+        grid_barrier(a.barrier, a.err, target, &s_dead);
+    }
+    // the last layer's output
+    if (!s_dead) {
+        const FfnArgs fl = finish_args(L - 1);
+        for (int i = gtid; i < B * H; i += gthreads) a.h_out[i] = finish_value(fl, i / H, i % H, d.splits);
+    }
+    if (warp == 0 && lane == 0) group_drain(r, ppos, issued);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && s_dead) *a.err = 1u;
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(r.tmem), "r"(kGroupTmemCols) : "memory");
+    }
+}
+
+}  // namespace stmoe_dev
