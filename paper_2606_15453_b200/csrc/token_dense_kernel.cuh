@@ -8,7 +8,7 @@
 //   R   split-K router GEMV tasks over all warps of the grid               -> grid barrier
 //   T   every CTA runs softmax / top-K / grouping (one work-list entry per expert) itself
 //   GU  gate/up tiles on tcgen05: warp 0 feeds TMA, warp 1 issues MMAs, warps 2-5 read the
-//       accumulators; the predictor (Algorithms 1-3) runs on one more warp of the last CTA
+//       accumulators; the predictor (Algorithms 1-3) runs on the other ten warps of the last CTA
 //                                                                          -> grid barrier
 //   D   down-projection tiles the same way                                 -> grid barrier
 // The stage ring, its barriers and the tensor-memory columns are set up once and carried through
@@ -43,7 +43,6 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
     const TokenArgs &a = d.t;
     extern __shared__ __align__(16) int dyn[];  // work list | ids | prev ids | gate weights | stage ring
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
-    __shared__ int s_score[kMaxExperts];
     __shared__ float s_inv[kMaxBatch];
     __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2];
     __shared__ uint32_t s_tmem;
@@ -101,6 +100,7 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         const float *h = l == 0 ? a.h_in : a.hbuf + (size_t)l * B * H;
 
         // ---- F ---------------------------------------------------------------------------------
+        DBG_STAMP(l * 8 + 0);
         if (l == 0) {
             for (int i = gtid; i < B * H; i += gthreads) d.xb[i] = __float2bfloat16_rn(h[i]);
         } else {
@@ -114,6 +114,7 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         }
         fence_async_proxy();
         grid_barrier(a.barrier, a.err, target, &s_dead);
+        DBG_STAMP(l * 8 + 1);
 
         // ---- R ---------------------------------------------------------------------------------
         RouterArgs ra;
@@ -130,6 +131,7 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         tk.wl = wl;
         router_tasks<RDT, false>(ra, warp * gridDim.x + blockIdx.x, NW * gridDim.x, lane);
         grid_barrier(a.barrier, a.err, target, &s_dead);
+        DBG_STAMP(l * 8 + 2);
 
         // ---- T ---------------------------------------------------------------------------------
         router_finalize<RDT>(ra, s_ids, s_scan, NW);
@@ -138,6 +140,7 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
             for (int i = threadIdx.x; i < B * K; i += blockDim.x) a.ids_all[(size_t)l * a.Bmax * K + i] = s_ids[i];
 
         // ---- GU (+ the predictor on one warp of the last CTA) -----------------------------------
+        DBG_STAMP(l * 8 + 3);
         GroupArgs g{};
         g.wl = wl, g.E = E, g.img_routed0 = l * E, g.img_shared0 = d.img_shared_base + l * a.n_shared;
         g.np = np, g.KS = KS, g.inv_rms = s_inv, g.act = d.actb, g.part = d.part, g.err = a.err;
@@ -152,10 +155,11 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         } else if (warp < 6) {
             group_epilogue<2>(g, r, eit, warp % 4, lane);
             fence_async_proxy();  // the gated activations are fetched by TMA in the next phase
-        } else if (pred_cta && warp == NW - 1) {
-            predictor_step_warp(a, l, s_ids, s_prev, s_score, lane);
+        } else if (pred_cta) {  // the ten warps without a role in this phase
+            predictor_step_group(a, l, s_ids, s_prev, warp - 6, NW - 6, lane);
         }
-        grid_barrier(a.barrier, a.err, target, &s_dead);
+        grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 4);
+        DBG_STAMP(l * 8 + 5);
 
         // ---- D ---------------------------------------------------------------------------------
         g.rows = H, g.kd = I, g.splits = d.splits, g.seg = d.seg;
@@ -170,7 +174,8 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
             group_epilogue<1>(g, r, eit, warp % 4, lane);
         }
         for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
-        grid_barrier(a.barrier, a.err, target, &s_dead);
+        grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 6);
+        DBG_STAMP(l * 8 + 7);
     }
     // the last layer's output
     if (!s_dead) {

@@ -53,19 +53,25 @@ struct TokenArgs {
     unsigned *err;                  // [1]
 };
 
-// Algorithms 1-3 for one layer step on a single warp (same arithmetic and order as
-// predictor_step_kernel; rows are updated in place in global memory, which only this warp
-// touches during the launch).  cur/prev: routing of this and the previous layer [B][K].
-__device__ __forceinline__ void predictor_step_warp(const TokenArgs &a, int layer, const int *cur, const int *prev,
-                                                    int *s_score, int lane)
+// Algorithms 1-3 for one layer step on `nw` warps of one CTA (this is warp `wi` of them; all nw
+// call together), same arithmetic and order as predictor_step_kernel.  The tables live in global
+// memory, which only these warps touch during the launch.  Work is split so that no two warps
+// ever need the same data: table rows (Algorithm 3) by row index, with each warp walking the
+// batch in order, so a row sees its updates in the sequential order; predictions (Algorithm 2,
+// Eq. 1) and their scoring by sequence.  Scores are kept in registers (lane f % 32 holds expert
+// f in slot f / 32), so the warps need no shared memory.  cur/prev: routing of this and the
+// previous layer [B][K].
+__device__ __noinline__ void predictor_step_group(const TokenArgs &a, int layer, const int *cur, const int *prev,
+                                                  int wi, int nw, int lane)
 {
+    constexpr int SL = kMaxExperts / kWarp;  // score slots per lane
     const int E = a.E, K = a.K, L = a.L, B = a.B;
     const PredState &st = a.pst;
     const long long t = *st.t;
     const bool runtime = t >= a.P;
     const bool last_profiling = (!runtime) && t == a.P - 1 && layer == L - 1;
     if (runtime) {
-        for (int b = 0; b < B; ++b) {
+        for (int b = wi; b < B; b += nw) {
             const bool valid = st.pred_valid[b] != 0;
             int np = 0, nh = 0;
             if (valid) {
@@ -87,16 +93,16 @@ __device__ __forceinline__ void predictor_step_warp(const TokenArgs &a, int laye
         if (layer > 0) {
             uint8_t *gid = st.cct_id + (size_t)(layer - 1) * E * K;
             uint8_t *gcf = st.cct_conf + (size_t)(layer - 1) * E * K;
-            for (int b = 0; b < B; ++b)
-                for (int k = 0; k < K; ++k) {
-                    const int e = prev[b * K + k];
-                    update_row(gid + e * K, gcf + e * K, K, cur + b * K, lane);
-                    __syncwarp();
-                }
+            for (int i = 0; i < B * K; ++i) {
+                const int e = prev[i];
+                if (e % nw != wi) continue;  // warp-uniform
+                update_row(gid + e * K, gcf + e * K, K, cur + (i / K) * K, lane);
+                __syncwarp();
+            }
         }
     } else if (layer > 0) {
         uint32_t *Co = st.Co + (size_t)(layer - 1) * E * E;
-        for (int i = lane; i < B * K * K; i += kWarp) {
+        for (int i = wi * kWarp + lane; i < B * K * K; i += nw * kWarp) {
             const int b = i / (K * K), r = i % (K * K);
             atomicAdd(&Co[(size_t)prev[b * K + r / K] * E + cur[b * K + r % K]], 1u);
         }
@@ -109,29 +115,48 @@ __device__ __forceinline__ void predictor_step_warp(const TokenArgs &a, int laye
     const bool temporal = predict_now && (a.mode & 1);
     int32_t *pred_ids = a.pred_ids ? a.pred_ids + (size_t)layer * B * a.max_pred : nullptr;
     int32_t *n_pred = a.n_pred ? a.n_pred + (size_t)layer * B : nullptr;
-    for (int b = 0; b < B; ++b) {
-        for (int f = lane; f < kMaxExperts; f += kWarp) s_score[f] = 0;
-        __syncwarp();
+    const uint8_t *cid = st.cct_id + (size_t)layer * E * K;
+    const uint8_t *ccf = st.cct_conf + (size_t)layer * E * K;
+    for (int b = wi; b < B; b += nw) {
+        int sc[SL];
+#pragma unroll
+        for (int w = 0; w < SL; ++w) sc[w] = 0;
+        // lane j adds `add` to the score of expert `id` (add = 0: nothing), for all lanes in turn
+        auto scatter = [&](int id, int add, int n_lanes) {
+            for (int j = 0; j < n_lanes; ++j) {
+                const int idj = __shfl_sync(kFull, id, j), addj = __shfl_sync(kFull, add, j);
+                if (lane == (idj & 31)) {
+#pragma unroll
+                    for (int w = 0; w < SL; ++w)
+                        if (w == (idj >> 5)) sc[w] += addj;
+                }
+            }
+        };
         if (spatial) {
-            const uint8_t *cid = st.cct_id + (size_t)layer * E * K;
-            const uint8_t *ccf = st.cct_conf + (size_t)layer * E * K;
-            for (int k = 0; k < K; ++k) {
-                const int e = cur[b * K + k];
-                if (lane < K) s_score[cid[e * K + lane]] += ccf[e * K + lane];
-                __syncwarp();
+            // the K candidates of each of the K routed experts' rows, 32 (row, slot) pairs per trip
+            for (int i0 = 0; i0 < K * K; i0 += kWarp) {
+                const int i = i0 + lane;
+                int id = 0, add = 0;
+                if (i < K * K) {
+                    const int e = cur[b * K + i / K];
+                    id = cid[e * K + i % K], add = ccf[e * K + i % K];
+                }
+                scatter(id, add, min(kWarp, K * K - i0));
             }
         }
         if (temporal) {
+            int id = 0, add = 0;
             if (lane < K) {
                 const int hte = st.HT[((size_t)b * L + next) * K + lane];
-                if (hte >= 0) s_score[hte] += kThreshold;
+                if (hte >= 0) id = hte, add = kThreshold;
             }
-            __syncwarp();
+            scatter(id, add, K);
         }
         int count = 0;
-        for (int w = 0; w < kMaxExperts / kWarp; ++w) {
+#pragma unroll
+        for (int w = 0; w < SL; ++w) {
             const int f = w * kWarp + lane;
-            const bool in = f < E && s_score[f] >= kThreshold;
+            const bool in = f < E && sc[w] >= kThreshold;
             const unsigned msk = __ballot_sync(kFull, in);
             if (lane == 0) st.pred_mask[b * 8 + w] = msk;
             if (in) {
@@ -148,12 +173,13 @@ __device__ __forceinline__ void predictor_step_warp(const TokenArgs &a, int laye
         }
         __syncwarp();
     }
-    for (int i = lane; i < B * K; i += kWarp) {
+    for (int i = wi * kWarp + lane; i < B * K; i += nw * kWarp) {
         const int b = i / K, k = i % K;
         st.HT[((size_t)b * L + layer) * K + k] = (int16_t)cur[b * K + k];
     }
-    __syncwarp();
-    if (lane == 0 && layer == L - 1) *st.t = t + 1;
+    // every warp has read the step counter before one of them advances it
+    if (nw > 1) asm volatile("bar.sync 3, %0;" ::"r"(nw * kWarp) : "memory");
+    if (wi == 0 && lane == 0 && layer == L - 1) *st.t = t + 1;
 }
 
 // Bounded grid barrier on a monotonically increasing counter.
@@ -188,7 +214,6 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs 
     constexpr int NW = kFfnThreads / kWarp;
     extern __shared__ __align__(16) int dyn[];  // work list | ids | prev ids | gate weights
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
-    __shared__ int s_score[kMaxExperts];
     __shared__ float s_inv[kMaxBatch];
     __shared__ int s_next[3], s_dead;
     const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
@@ -245,7 +270,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs 
         fa.w = s_w, fa.h_out = h_next, fa.tile_done = a.tile_done + (size_t)l * tiles;
         fa.B = B, fa.K = K, fa.n_shared = a.n_shared, fa.residual_scale = a.residual_scale;
         gate_up_phase<DT, MTMAX>(fa, s_next, [&]() {
-            if (pred_cta && warp == NW - 1) predictor_step_warp(a, l, s_ids, s_prev, s_score, lane);
+            if (pred_cta && warp == NW - 1) predictor_step_group(a, l, s_ids, s_prev, 0, 1, lane);
         });
         grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 4);
         DBG_STAMP(l * 8 + 5);
