@@ -20,9 +20,19 @@ __device__ __forceinline__ void dbg_stamp(int idx)
         if (idx >= 16 && idx < 24) g_dbg_phases[4096 + blockIdx.x * 8 + (idx - 16)] = t;  // layer 2, every CTA
     }
 }
+__device__ __forceinline__ void dbg_stamp_lane0(int idx)
+{
+    if (threadIdx.x % 32 == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        g_dbg_phases[idx] = t;
+    }
+}
 #define DBG_STAMP(i) dbg_stamp(i)
+#define DBG_STAMP_WARP(i) dbg_stamp_lane0(i)
 #else
 #define DBG_STAMP(i)
+#define DBG_STAMP_WARP(i)
 #endif
 
 constexpr int kWarp = 32;

@@ -67,6 +67,53 @@ __device__ __forceinline__ void update_row(uint8_t *ids, uint8_t *conf, int K, c
     if (act) ids[lane] = (uint8_t)id, conf[lane] = (uint8_t)cf;
 }
 
+// Algorithm 3 for the rows of one sequence's previous-layer experts, several rows at a time: the
+// warp is cut into groups of G lanes (G = the power of two >= K) and each group updates one row
+// exactly as update_row does.  The rows of one sequence are distinct, so they do not depend on
+// one another.  take(k) says whether row prev[k] belongs to this warp.
+template <typename Take>
+__device__ __forceinline__ void update_rows_grouped(uint8_t *gid, uint8_t *gcf, int K, const int32_t *prev,
+                                                    const int32_t *F, int lane, Take take)
+{
+    int G = 1;
+    while (G < K) G <<= 1;
+    const int per = kWarp / G, sub = lane / G, sl = lane % G;
+    const unsigned gmask = G == kWarp ? kFull : ((1u << G) - 1u);
+    const unsigned mine = __ballot_sync(kFull, lane < K && take(prev[lane]));
+    const int nrows = __popc(mine);
+    const int myf = sl < K ? F[sl] : -2;  // group lane k also carries routed expert k (ascending)
+    for (int r0 = 0; r0 < nrows; r0 += per) {
+        const int r = r0 + sub;
+        const bool row_ok = r < nrows;
+        const int e = row_ok ? prev[__fns(mine, 0, r + 1)] : 0;
+        uint8_t *ids = gid + (size_t)e * K, *conf = gcf + (size_t)e * K;
+        const bool act = row_ok && sl < K;
+        int id = act ? ids[sl] : -1, cf = act ? conf[sl] : 0;
+        bool hit = false, held = false;
+        for (int k = 0; k < K; ++k) {
+            hit |= (id == __shfl_sync(kFull, myf, k, G));
+            held |= (myf == __shfl_sync(kFull, id, k, G));
+        }
+        const bool replace = act && !hit && cf == 0;
+        if (act) {
+            if (hit)
+                cf = min(cf + 1, kConfMax);
+            else if (cf > 0)
+                cf -= 1;
+        }
+        const unsigned rep = (__ballot_sync(kFull, replace) >> (sub * G)) & gmask;
+        const unsigned avail = (__ballot_sync(kFull, act && !held) >> (sub * G)) & gmask;
+        // routed experts the row does not hold, lowest id first; the n-th replacing slot (in slot
+        // order) takes the n-th of them
+        const int nth = __popc(rep & ((1u << sl) - 1u)) + 1;
+        const unsigned pos = replace ? __fns(avail, 0, nth) : 0u;
+        const int g = __shfl_sync(kFull, myf, pos & (unsigned)(G - 1), G);
+        if (replace && pos != 0xffffffffu) id = g, cf = kConfInit;
+        if (act) ids[sl] = (uint8_t)id, conf[sl] = (uint8_t)cf;
+        __syncwarp();
+    }
+}
+
 __global__ void __launch_bounds__(256) predictor_step_kernel(PredArgs a)
 {
     constexpr int NW = 8;

@@ -59,17 +59,34 @@ struct TokenArgs {
 // ever need the same data: table rows (Algorithm 3) by row index, with each warp walking the
 // batch in order, so a row sees its updates in the sequential order; predictions (Algorithm 2,
 // Eq. 1) and their scoring by sequence.  Scores are kept in registers (lane f % 32 holds expert
-// f in slot f / 32), so the warps need no shared memory.  cur/prev: routing of this and the
+// f), so the warps need no shared memory.  cur/prev: routing of this and the
 // previous layer [B][K].
-__device__ __noinline__ void predictor_step_group(const TokenArgs &a, int layer, const int *cur, const int *prev,
-                                                  int wi, int nw, int lane)
+__device__ __forceinline__ void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+
+__device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int layer, const int *cur, const int *prev,
+                                                     int wi, int nw, int lane)
 {
-    constexpr int SL = kMaxExperts / kWarp;  // score slots per lane
     const int E = a.E, K = a.K, L = a.L, B = a.B;
     const PredState &st = a.pst;
     const long long t = *st.t;
     const bool runtime = t >= a.P;
     const bool last_profiling = (!runtime) && t == a.P - 1 && layer == L - 1;
+    DBG_STAMP_WARP(2010);
+    if (runtime) {
+        // Every table row this step touches, pulled into L1 in one trip: the rows are then read
+        // one after the other (Algorithm 3 is sequential per row), each of which would otherwise
+        // be a trip to L2 of its own.  The tables are private to these warps' SM during the launch.
+        for (int i = wi * kWarp + lane; i < B * K; i += nw * kWarp) {
+            if (layer > 0) {
+                prefetch_l1(st.cct_id + ((size_t)(layer - 1) * E + prev[i]) * K);
+                prefetch_l1(st.cct_conf + ((size_t)(layer - 1) * E + prev[i]) * K);
+            }
+            if (layer < L - 1) {
+                prefetch_l1(st.cct_id + ((size_t)layer * E + cur[i]) * K);
+                prefetch_l1(st.cct_conf + ((size_t)layer * E + cur[i]) * K);
+            }
+        }
+    }
     if (runtime) {
         for (int b = wi; b < B; b += nw) {
             const bool valid = st.pred_valid[b] != 0;
@@ -90,15 +107,12 @@ __device__ __noinline__ void predictor_step_group(const TokenArgs &a, int layer,
                 atomicAdd(&st.stats[3], (unsigned long long)nh);
             }
         }
+        DBG_STAMP_WARP(2011);
         if (layer > 0) {
             uint8_t *gid = st.cct_id + (size_t)(layer - 1) * E * K;
             uint8_t *gcf = st.cct_conf + (size_t)(layer - 1) * E * K;
-            for (int i = 0; i < B * K; ++i) {
-                const int e = prev[i];
-                if (e % nw != wi) continue;  // warp-uniform
-                update_row(gid + e * K, gcf + e * K, K, cur + (i / K) * K, lane);
-                __syncwarp();
-            }
+            for (int b = 0; b < B; ++b)
+                update_rows_grouped(gid, gcf, K, prev + b * K, cur + b * K, lane, [&](int e) { return e % nw == wi; });
         }
     } else if (layer > 0) {
         uint32_t *Co = st.Co + (size_t)(layer - 1) * E * E;
@@ -108,6 +122,7 @@ __device__ __noinline__ void predictor_step_group(const TokenArgs &a, int layer,
         }
     }
     __syncwarp();
+    DBG_STAMP_WARP(2012);
 
     const bool predict_now = runtime || last_profiling;
     const int next = (layer + 1) % L;
@@ -118,17 +133,20 @@ __device__ __noinline__ void predictor_step_group(const TokenArgs &a, int layer,
     const uint8_t *cid = st.cct_id + (size_t)layer * E * K;
     const uint8_t *ccf = st.cct_conf + (size_t)layer * E * K;
     for (int b = wi; b < B; b += nw) {
-        int sc[SL];
-#pragma unroll
-        for (int w = 0; w < SL; ++w) sc[w] = 0;
+        // Scores of the eight experts lane, lane+32, ... packed one byte each into two registers
+        // (a score is at most 3K + 2 <= 98: K rows of confidence <= 3, plus the history bonus).
+        unsigned lo = 0u, hi = 0u;
         // lane j adds `add` to the score of expert `id` (add = 0: nothing), for all lanes in turn
         auto scatter = [&](int id, int add, int n_lanes) {
             for (int j = 0; j < n_lanes; ++j) {
                 const int idj = __shfl_sync(kFull, id, j), addj = __shfl_sync(kFull, add, j);
+                const int slot = idj >> 5;
+                const unsigned inc = (unsigned)addj << ((slot & 3) * 8);
                 if (lane == (idj & 31)) {
-#pragma unroll
-                    for (int w = 0; w < SL; ++w)
-                        if (w == (idj >> 5)) sc[w] += addj;
+                    if (slot < 4)
+                        lo += inc;
+                    else
+                        hi += inc;
                 }
             }
         };
@@ -154,9 +172,10 @@ __device__ __noinline__ void predictor_step_group(const TokenArgs &a, int layer,
         }
         int count = 0;
 #pragma unroll
-        for (int w = 0; w < SL; ++w) {
+        for (int w = 0; w < kMaxExperts / kWarp; ++w) {
             const int f = w * kWarp + lane;
-            const bool in = f < E && sc[w] >= kThreshold;
+            const int score = (int)(((w < 4 ? lo : hi) >> ((w & 3) * 8)) & 0xffu);
+            const bool in = f < E && score >= kThreshold;
             const unsigned msk = __ballot_sync(kFull, in);
             if (lane == 0) st.pred_mask[b * 8 + w] = msk;
             if (in) {
@@ -173,10 +192,12 @@ __device__ __noinline__ void predictor_step_group(const TokenArgs &a, int layer,
         }
         __syncwarp();
     }
+    DBG_STAMP_WARP(2013);
     for (int i = wi * kWarp + lane; i < B * K; i += nw * kWarp) {
         const int b = i / K, k = i % K;
         st.HT[((size_t)b * L + layer) * K + k] = (int16_t)cur[b * K + k];
     }
+    DBG_STAMP_WARP(2014);
     // every warp has read the step counter before one of them advances it
     if (nw > 1) asm volatile("bar.sync 3, %0;" ::"r"(nw * kWarp) : "memory");
     if (wi == 0 && lane == 0 && layer == L - 1) *st.t = t + 1;
