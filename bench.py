@@ -191,6 +191,8 @@ def main():
                     help="idle the compute stream this long after every layer: a stand-in for the attention "
                          "block the paper overlaps expert prefetch with (Section 4.3.4); 0 = pure MoE stack")
     ap.add_argument("--resident", action="store_true", help="keep every expert in HBM (cache_slots = 0)")
+    ap.add_argument("--no-dense", action="store_true",
+                    help="batched steps of resident bf16 stacks on the CUDA-core kernels instead of the tcgen05 ones")
     args = ap.parse_args()
 
     cfg = stacks.CONFIGS[args.workload]
@@ -216,7 +218,9 @@ def main():
 
     import paper_2606_15453_b200 as P
     P.build()
-    st = load_stack(cfg, batch, dev, prefetch_limit=args.prefetch_limit, mode=args.mode)  # a full replica per rank
+    import paper_2606_15453_b200 as P
+    st = load_stack(cfg, batch, dev, prefetch_limit=args.prefetch_limit, mode=args.mode,
+                    flags=P.FLAG_NO_DENSE if args.no_dense else 0)  # a full replica per rank
     L, K, H = cfg.n_layers, cfg.top_k, cfg.hidden
     n_tok = cfg.profile_tokens + args.warmup + args.steps
     x_host = stacks.token_inputs(cfg, batch, n_tok).pin_memory()
@@ -314,6 +318,9 @@ def main():
                                       "cache_hits", "cache_misses", "kernel_launches")}
     step_gbs = statistics.mean(step_bytes) / (ms / args.steps * 1e-3) / 1e9
     persistent = cfg.cache_slots == 0          # resident stacks: one kernel launch per decode step
+    # batched steps of resident bf16 stacks: expert FFN on tcgen05 tiles (the library's default threshold)
+    dense = persistent and cfg.dtype == "bf16" and batch >= 4 and not args.no_dense
+    top_kernel = ("decode_token_dense_kernel" if dense else "decode_token_kernel") if persistent else "gate_up_kernel"
     per_layer = NCU_TRAFFIC_BYTES_PER_LAYER.get(args.workload) if batch == 1 else None
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -322,6 +329,7 @@ def main():
         "config": {"workload": cfg.name, "batch": batch, "layers": L, "experts": cfg.n_experts,
                    "top_k": K, "hidden": H, "inter": cfg.inter, "parallelism": f"replicas x{world}",
                    "profile_tokens": cfg.profile_tokens, "l2": "inputs_larger_than_l2",
+                   "ffn_path": "tcgen05 tiles (TMA-fed, TMEM accumulators)" if dense else "weight-streaming GEMV on CUDA cores",
                    "resident_weight_gb": round(L * (cfg.n_experts + cfg.n_shared) * cfg.expert_bytes / 1e9, 1)},
         "clocks": clocks,
         "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT,
@@ -329,7 +337,7 @@ def main():
                 "d2h_bytes_per_step": batch * H * 4 + L * batch * K * 4},
         "gpu_launches": run["kernel_launches"],
         "roofline": {"bound": "hbm",
-                     "kernel": "decode_token_kernel" if persistent else "gate_up_kernel",
+                     "kernel": top_kernel,
                      "achieved": step_gbs if persistent else achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": (step_gbs if persistent else achieved or 0.0) / peak,
