@@ -191,6 +191,8 @@ def main():
                     help="idle the compute stream this long after every layer: a stand-in for the attention "
                          "block the paper overlaps expert prefetch with (Section 4.3.4); 0 = pure MoE stack")
     ap.add_argument("--resident", action="store_true", help="keep every expert in HBM (cache_slots = 0)")
+    ap.add_argument("--dense-min-batch", type=int, default=0,
+                    help="smallest batch that takes the tcgen05 path (0: the library's default, 2)")
     ap.add_argument("--no-dense", action="store_true",
                     help="batched steps of resident bf16 stacks on the CUDA-core kernels instead of the tcgen05 ones")
     args = ap.parse_args()
@@ -221,6 +223,8 @@ def main():
     import paper_2606_15453_b200 as P
     st = load_stack(cfg, batch, dev, prefetch_limit=args.prefetch_limit, mode=args.mode,
                     flags=P.FLAG_NO_DENSE if args.no_dense else 0)  # a full replica per rank
+    if args.dense_min_batch:
+        st.set_dense_min_batch(args.dense_min_batch)
     L, K, H = cfg.n_layers, cfg.top_k, cfg.hidden
     n_tok = cfg.profile_tokens + args.warmup + args.steps
     x_host = stacks.token_inputs(cfg, batch, n_tok).pin_memory()
@@ -319,7 +323,7 @@ def main():
     step_gbs = statistics.mean(step_bytes) / (ms / args.steps * 1e-3) / 1e9
     persistent = cfg.cache_slots == 0          # resident stacks: one kernel launch per decode step
     # batched steps of resident bf16 stacks: expert FFN on tcgen05 tiles (the library's default threshold)
-    dense = persistent and cfg.dtype == "bf16" and batch >= 4 and not args.no_dense
+    dense = persistent and cfg.dtype == "bf16" and batch >= (args.dense_min_batch or 2) and not args.no_dense
     top_kernel = ("decode_token_dense_kernel" if dense else "decode_token_kernel") if persistent else "gate_up_kernel"
     per_layer = NCU_TRAFFIC_BYTES_PER_LAYER.get(args.workload) if batch == 1 else None
     out = {

@@ -58,7 +58,7 @@ extern "C" {
                                       CUDA graph) instead of the single persistent kernel */
 
 #define STMOE_FLAG_NO_DENSE 4 /* never use the tensor-core FFN kernels: by default resident bf16 stacks run
-                                decode steps of at least stmoe_set_dense_min_batch() sequences (default 4)
+                                decode steps of at least stmoe_set_dense_min_batch() sequences (default 2)
                                 with one work-list entry per expert on tcgen05 tiles, rounding the
                                 normalised hidden state and the gated activations to bf16 */
 

@@ -531,7 +531,7 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
 }
 
 // ---- tensor-core path (dense_group.cuh) ---------------------------------------------------
-constexpr int kDenseMinBatch = 4;
+constexpr int kDenseMinBatch = 2;
 constexpr int kDenseMaxSplits = 4;
 constexpr int kTokenDenseDynBytes = 220 * 1024;
 
