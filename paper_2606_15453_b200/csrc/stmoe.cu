@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "dense_ffn.cuh"
+#include "dense8_group.cuh"
 #include "dense_group.cuh"
 #include "device_utils.cuh"
 #include "ffn.cuh"
@@ -316,6 +317,9 @@ struct stmoe {
     __nv_bfloat16 *d_xb = nullptr, *d_actb = nullptr;
     float *d_part_dense = nullptr;
     int dense_grid = 0;
+    bool dense8 = false;            // fp8 stacks: dense8_group.cuh (per-layer kernels only)
+    CUtensorMap map8_gate{}, map8_up{}, map8_down{}, map8_x[4]{}, map8_act[4]{};
+    __half *d_xb16 = nullptr, *d_act16 = nullptr;
     bool dense_persistent = false;  // one cooperative kernel per decode step (token_dense_kernel.cuh)
     int dense_dyn_bytes = 0;
 
@@ -535,7 +539,7 @@ constexpr int kDenseMinBatch = 2;
 constexpr int kDenseMaxSplits = 4;
 constexpr int kTokenDenseDynBytes = 220 * 1024;
 
-bool use_dense(const stmoe *s, int batch) { return s->dense && batch >= s->dense_min_batch; }
+bool use_dense(const stmoe *s, int batch) { return (s->dense || s->dense8) && batch >= s->dense_min_batch; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -544,11 +548,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 // bf16 tensor of `rank` dimensions (dims[0] innermost, strides in bytes for dims 1..), boxes of
 // 64 columns x box_rows rows (x 1 image), 128-byte swizzle, zero fill outside
 int encode_map(EncodeTiledFn fn, CUtensorMap *m, void *base, int rank, const cuuint64_t *dims,
-               const cuuint64_t *strides, int box_rows)
+               const cuuint64_t *strides, int box_rows, CUtensorMapDataType dt = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+               int box_cols = kDenseKStep)
 {
-    cuuint32_t box[3] = {(cuuint32_t)kDenseKStep, (cuuint32_t)box_rows, 1};
+    cuuint32_t box[3] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1};
     cuuint32_t es[3] = {1, 1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, dims, strides, box, es,
+    return fn(m, dt, (cuuint32_t)rank, base, dims, strides, box, es,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
                ? STMOE_OK
@@ -614,6 +619,97 @@ int dense_setup(stmoe *s)
 // gate/up, down and the weighted sum of one layer step on the tensor-core kernels; the work
 // list (one entry per expert) and inv_rms come from the router kernel launched before
 int dense_down_splits(const stmoe *s, int batch, int *seg);
+
+// fp8 stacks: tensor maps over the e4m3 images (128 x 128-byte boxes) and f16 activation buffers
+int dense8_setup(stmoe *s)
+{
+    const stmoe_config_t &c = s->cfg;
+    const int L = c.n_layers, E = c.n_experts, B = c.max_batch, H = c.hidden, I = c.inter;
+    int dev = 0, major = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (major != 10) return STMOE_OK;
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr) != cudaSuccess || !sym) {
+        (void)cudaGetLastError();
+        return STMOE_OK;
+    }
+    EncodeTiledFn enc = (EncodeTiledFn)sym;
+    const size_t pairs = (size_t)B * s->KS;
+    CU_TRY(cudaMalloc(&s->d_xb16, sizeof(__half) * (size_t)kDenseMaxTokens * H));
+    CU_TRY(cudaMemset(s->d_xb16, 0, sizeof(__half) * (size_t)kDenseMaxTokens * H));
+    CU_TRY(cudaMalloc(&s->d_act16, sizeof(__half) * (pairs + kDenseMaxTokens) * I));
+    CU_TRY(cudaMemset(s->d_act16, 0, sizeof(__half) * (pairs + kDenseMaxTokens) * I));
+    CU_TRY(cudaMalloc(&s->d_part_dense, sizeof(float) * pairs * kDenseMaxSplits * H));
+    const cuuint64_t n_img = (cuuint64_t)L * (E + c.n_shared);
+    const cuuint64_t gd[3] = {(cuuint64_t)H, (cuuint64_t)I, n_img}, gs[2] = {(cuuint64_t)H, s->img_bytes};
+    const cuuint64_t dd[3] = {(cuuint64_t)I, (cuuint64_t)H, n_img}, ds[2] = {(cuuint64_t)I, s->img_bytes};
+    const CUtensorMapDataType u8 = CU_TENSOR_MAP_DATA_TYPE_UINT8, f16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    ST_TRY(encode_map(enc, &s->map8_gate, s->d_resident, 3, gd, gs, kDenseRows, u8, kGroup8KStage));
+    ST_TRY(encode_map(enc, &s->map8_up, s->d_resident + (size_t)I * H, 3, gd, gs, kDenseRows, u8, kGroup8KStage));
+    ST_TRY(encode_map(enc, &s->map8_down, s->d_resident + 2 * (size_t)I * H, 3, dd, ds, kDenseRows, u8, kGroup8KStage));
+    for (int i = 0; i < 4; ++i) {
+        const cuuint64_t xd[2] = {(cuuint64_t)H, (cuuint64_t)kDenseMaxTokens}, xs[1] = {(cuuint64_t)H * 2};
+        const cuuint64_t ad[2] = {(cuuint64_t)I, (cuuint64_t)(pairs + kDenseMaxTokens)}, as[1] = {(cuuint64_t)I * 2};
+        ST_TRY(encode_map(enc, &s->map8_x[i], s->d_xb16, 2, xd, xs, 16 * (i + 1), f16));
+        ST_TRY(encode_map(enc, &s->map8_act[i], s->d_act16, 2, ad, as, 16 * (i + 1), f16));
+    }
+    CU_TRY(cudaFuncSetAttribute(dense8_group_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
+    CU_TRY(cudaFuncSetAttribute(dense8_group_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
+    s->dense_grid = sm_count();
+    s->dense_min_batch = kDenseMinBatch;
+    s->dense8 = true;
+    return STMOE_OK;
+}
+
+int dense8_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, cudaStream_t st)
+{
+    const stmoe_config_t &c = s->cfg;
+    const int E = c.n_experts, H = c.hidden, I = c.inter, np = (batch + 15) / 16 * 16;
+    cudaEvent_t e0 = nullptr, e1 = nullptr, e2 = nullptr;
+    const bool timed = s->time_kernels;
+    if (timed) {
+        ST_TRY(get_event(s, &e0));
+        ST_TRY(get_event(s, &e1));
+        ST_TRY(get_event(s, &e2));
+        CU_TRY(cudaEventRecord(e0, st));
+    }
+    if (!chained) {
+        dense8_cast_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fa.h, batch * H, s->d_xb16);
+        s->launches += 1;
+    }
+    Group8Args a8{};
+    GroupArgs &g = a8.g;
+    g.wl = fa.wl, g.E = E, g.img_routed0 = layer * E, g.img_shared0 = c.n_layers * E + layer * c.n_shared;
+    g.np = np, g.KS = s->KS, g.inv_rms = fa.inv_rms, g.part = s->d_part_dense, g.err = s->d_err;
+    a8.store = s->d_resident, a8.img_bytes = s->img_bytes, a8.act16 = s->d_act16;
+    g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kGroup8KStage - 1) / kGroup8KStage * kGroup8KStage;
+    a8.scale_off = 0;
+    dense8_group_kernel<2><<<s->dense_grid, kGroup8Threads, kGroupSmemBytes, st>>>(s->map8_gate, s->map8_up,
+                                                                                   s->map8_x[np / 16 - 1], a8);
+    if (timed) CU_TRY(cudaEventRecord(e1, st));
+    int seg = 0;
+    int splits = dense_down_splits(s, batch, &seg);
+    seg = (seg + kGroup8KStage - 1) / kGroup8KStage * kGroup8KStage;
+    splits = (I + seg - 1) / seg;
+    g.rows = H, g.kd = I, g.splits = splits, g.seg = seg;
+    a8.scale_off = 2 * I;
+    dense8_group_kernel<1><<<s->dense_grid, kGroup8Threads, kGroupSmemBytes, st>>>(s->map8_down, s->map8_down,
+                                                                                   s->map8_act[np / 16 - 1], a8);
+    FfnArgs fc = fa;
+    fc.part = s->d_part_dense;
+    dense8_combine_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fc, splits, s->d_xb16);
+    if (timed) {
+        CU_TRY(cudaEventRecord(e2, st));
+        s->spans.push_back(TimedSpan{e0, e1, 2});
+        s->spans.push_back(TimedSpan{e1, e2, 3});
+        s->timed_ffn += 1;
+    }
+    s->launches += 3;
+    CU_TRY(cudaGetLastError());
+    return STMOE_OK;
+}
 
 // chained: h_in is the output of the previous layer's dense_ffn, whose bf16 copy is still in d_xb
 int dense_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, cudaStream_t st)
@@ -747,7 +843,9 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
         fa.blob = s->d_blob_table + (size_t)layer * (E + c.n_shared);
     }
     s->launches += 1;
-    if (dense)
+    if (dense && s->dense8)
+        ST_TRY(dense8_ffn(s, layer, batch, chained, fa, st));
+    else if (dense)
         ST_TRY(dense_ffn(s, layer, batch, chained, fa, st));
     else
         ST_TRY(run_ffn(s, c.weight_dtype, mt, mt == 1 ? s->plan1 : s->plan4, fa, st));
@@ -911,7 +1009,7 @@ int stmoe_destroy(stmoe_t *s)
                    s->pst.Co, s->pst.cct_id, s->pst.cct_conf, s->pst.HT, s->pst.t, s->pst.pred_mask,
                    s->pst.pred_valid, s->pst.stats, s->d_rpart, s->d_sspart, s->d_arrivals, s->d_tile_done, s->d_hbuf, s->d_rpart_all, s->d_sspart_all,
                    s->d_act_all, s->d_part_all, s->d_tiles_all, s->d_barrier, s->d_err, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
-                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense};
+                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense, s->d_xb16, s->d_act16};
     if (s->d_shared && s->d_resident && s->d_shared > s->d_resident) dev[2] = nullptr;  // one allocation
     for (void *p : dev)
         if (p) cudaFree(p);
@@ -1067,6 +1165,10 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
         const int rc = dense_setup(s);
         if (rc != STMOE_OK) return fail(rc);
     }
+    if (c.cache_slots == 0 && c.weight_dtype == STMOE_FP8_E4M3 && !(c.flags & STMOE_FLAG_NO_DENSE) && B >= 2) {
+        const int rc = dense8_setup(s);
+        if (rc != STMOE_OK) return fail(rc);
+    }
     if (c.profile_tokens == 0 && L > 1) {
         const int rows = (L - 1) * E;
         cct_build_kernel<<<(rows + 7) / 8, 256>>>(s->pst, L, E, K);
@@ -1090,7 +1192,7 @@ int stmoe_set_kernel_timing(stmoe_t *s, int on)
 
 int stmoe_set_dense_min_batch(stmoe_t *s, int min_batch)
 {
-    if (!s || !s->dense || min_batch < 2 || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
+    if (!s || !(s->dense || s->dense8) || min_batch < 2 || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
     s->dense_min_batch = min_batch;
     return STMOE_OK;
 }

@@ -36,6 +36,49 @@ def test_dense_layer_steps_match_oracle(B, shape):
     pr.close()
 
 
+@pytest.mark.parametrize("B,shape", [
+    (4, dict(hidden=512, inter=384, n_experts=8, top_k=2, n_shared=0)),
+    (9, dict(hidden=272, inter=208, n_experts=16, top_k=3, n_shared=1)),     # ragged row and column tiles
+    (33, dict(hidden=1024, inter=768, n_experts=32, top_k=8, n_shared=0)),
+    (64, dict(hidden=256, inter=1536, n_experts=64, top_k=6, n_shared=2)),
+])
+def test_dense_fp8_layer_steps_match_oracle(B, shape):
+    """fp8 weights: e4m3 tiles widened to f16 in shared memory, f16 activations, row scales in the epilogue."""
+    cfg = stacks.CONFIGS["C4"].scaled(n_layers=3, profile_tokens=2, cache_slots=0, **shape)
+    pr = Pair(cfg, B)
+    x = stacks.token_inputs(cfg, B, 3).numpy()
+    skipped = 0
+    for t in range(3):
+        h = x[t]
+        for l in range(cfg.n_layers):
+            o = pr.oracle.layer_step(l, h)
+            g = pr.gpu_step(l, h)
+            skipped += check_layer(cfg, g, o, h, where=f"t={t} l={l}")
+            h = o["h_out"]
+    st = pr.stack.stats()
+    assert st["kernel_launches"] == 3 * cfg.n_layers * 6 + 1
+    assert skipped <= B
+    pr.close()
+
+
+def test_dense_fp8_decode_token_agrees_with_cuda_core_path():
+    cfg = stacks.CONFIGS["C4"].scaled(n_layers=3, profile_tokens=3, cache_slots=0, hidden=512, inter=384,
+                                      n_experts=16, top_k=4, n_shared=0)
+    B, T = 6, 5
+    graph = _run_tokens(cfg, B, T, 0, torch.cuda.Stream())
+    eager = _run_tokens(cfg, B, T, 0, torch.cuda.current_stream())
+    core = _run_tokens(cfg, B, T, P.FLAG_NO_DENSE, torch.cuda.Stream())
+    for a, b in zip(graph[0], eager[0]):
+        assert all(torch.equal(u, v) for u, v in zip(a, b))
+    assert graph[1] == eager[1]
+    assert graph[2]["kernel_launches"] > core[2]["kernel_launches"]
+    for t, (a, c) in enumerate(zip(graph[0], core[0])):
+        scale = c[0].abs().max().item()
+        assert (a[0] - c[0]).abs().max().item() <= 2e-2 * scale, t
+        if t == 0:
+            assert torch.equal(a[1][0], c[1][0])
+
+
 def _run_tokens(cfg, B, T, flags, stream, min_batch=None):
     pr = Pair(cfg, B, oracle=False, flags=flags)
     if min_batch is not None:
