@@ -192,7 +192,7 @@ def main():
                          "block the paper overlaps expert prefetch with (Section 4.3.4); 0 = pure MoE stack")
     ap.add_argument("--resident", action="store_true", help="keep every expert in HBM (cache_slots = 0)")
     ap.add_argument("--dense-min-batch", type=int, default=0,
-                    help="smallest batch that takes the tcgen05 path (0: the library's default, 2)")
+                    help="smallest batch that takes the tcgen05 path (0: the library's default, 2 for bf16, 4 for fp8)")
     ap.add_argument("--no-dense", action="store_true",
                     help="batched steps of resident bf16 stacks on the CUDA-core kernels instead of the tcgen05 ones")
     args = ap.parse_args()
@@ -323,8 +323,15 @@ def main():
     step_gbs = statistics.mean(step_bytes) / (ms / args.steps * 1e-3) / 1e9
     persistent = cfg.cache_slots == 0          # resident stacks: one kernel launch per decode step
     # batched steps of resident bf16 stacks: expert FFN on tcgen05 tiles (the library's default threshold)
-    dense = persistent and cfg.dtype == "bf16" and batch >= (args.dense_min_batch or 2) and not args.no_dense
-    top_kernel = ("decode_token_dense_kernel" if dense else "decode_token_kernel") if persistent else "gate_up_kernel"
+    dense = persistent and not args.no_dense and (
+        (cfg.dtype == "bf16" and batch >= (args.dense_min_batch or 2)) or
+        (cfg.dtype == "fp8" and batch >= (args.dense_min_batch or 4)))
+    top_kernel = "gate_up_kernel"
+    if persistent:
+        top_kernel = "decode_token_kernel"
+        if dense:   # fp8: per-layer tcgen05 kernels replayed as a graph; bf16: one persistent kernel
+            top_kernel = "decode_token_dense_kernel" if cfg.dtype == "bf16" else "dense8_group_kernel<2>"
+    whole_step = persistent and not (dense and cfg.dtype == "fp8")   # the top kernel is one launch per decode step
     per_layer = NCU_TRAFFIC_BYTES_PER_LAYER.get(args.workload) if batch == 1 else None
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -342,13 +349,13 @@ def main():
         "gpu_launches": run["kernel_launches"],
         "roofline": {"bound": "hbm",
                      "kernel": top_kernel,
-                     "achieved": step_gbs if persistent else achieved, "peak": peak,
+                     "achieved": step_gbs if whole_step else achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s",
-                     "frac": (step_gbs if persistent else achieved or 0.0) / peak,
-                     "frac_of_8000": (step_gbs if persistent else achieved or 0.0) / 8000.0,
-                     "traffic": per_layer * L if (persistent and per_layer) else None,
-                     "algorithmic_bytes_per_launch": statistics.mean(step_bytes) if persistent else gate_up_bytes,
-                     "us_per_launch": ms / args.steps * 1e3 if persistent else gu_ms * 1e3,
+                     "frac": (step_gbs if whole_step else achieved or 0.0) / peak,
+                     "frac_of_8000": (step_gbs if whole_step else achieved or 0.0) / 8000.0,
+                     "traffic": per_layer * L if (whole_step and per_layer) else None,
+                     "algorithmic_bytes_per_launch": statistics.mean(step_bytes) if whole_step else gate_up_bytes,
+                     "us_per_launch": ms / args.steps * 1e3 if whole_step else gu_ms * 1e3,
                      "per_layer_kernels": {
                          "note": "second pass over the same steps as per-layer kernels, events around each",
                          "gate_up": {"achieved": achieved, "us_per_launch": gu_ms * 1e3,

@@ -57,10 +57,11 @@ extern "C" {
 #define STMOE_FLAG_NO_PERSISTENT 2 /* resident stacks: decode steps as per-layer kernels (replayed as a
                                       CUDA graph) instead of the single persistent kernel */
 
-#define STMOE_FLAG_NO_DENSE 4 /* never use the tensor-core FFN kernels: by default resident bf16 stacks run
-                                decode steps of at least stmoe_set_dense_min_batch() sequences (default 2)
-                                with one work-list entry per expert on tcgen05 tiles, rounding the
-                                normalised hidden state and the gated activations to bf16 */
+#define STMOE_FLAG_NO_DENSE 4 /* never use the tensor-core FFN kernels: by default resident bf16 and fp8
+                                stacks run decode steps of at least stmoe_set_dense_min_batch() sequences
+                                (default 2 for bf16, 4 for fp8) with one work-list entry per expert on
+                                tcgen05 tiles, rounding the hidden state and the gated activations to
+                                bf16 (bf16 stacks) or f16 (fp8 stacks, whose weights are widened to f16) */
 
 /* per-sequence result flags of a layer step */
 #define STMOE_TOKEN_NEAR_TIE 1u /* K-th and (K+1)-th router logit closer than 1e-4 */

@@ -4,16 +4,17 @@
 // weight rows x one split, persistent CTA per SM, weights as the MMA's M operand).  tcgen05 has no
 // fp8 x 16-bit mode, and rounding the activations to fp8 would not fit the error bound, so the
 // weights are widened on the way: TMA lands the e4m3 tile (128 rows x 128 columns, 16 KB) in a
-// staging ring, six converter warps rewrite it as two f16 operand tiles (e4m3 -> f16 is exact) in
+// staging ring, eight converter warps rewrite it as two f16 operand tiles (e4m3 -> f16 is exact) in
 // the 128-byte swizzled layout, and the MMA runs in f16 x f16 -> fp32 against f16 activations.
 // The per-output-channel scales belong to the weight rows = accumulator lanes and are applied in
 // the epilogue.
 //   warp 0       TMA producer: weight tile(s) + two activation boxes per stage
-//   warp 1       MMA issue (8 K=16 steps per stage and matrix), tensor-memory owner
+//   warp 1       MMA issue (4 K=16 steps per 64-column half of a stage and matrix), tensor-memory owner
 //   warps 2-5    epilogue (two accumulator buffers)
-//   warps 6-11   converters
-// Rings: `NS` staging stages (fp8 weights + activation boxes) and one operand buffer; a stage is
-// released when its MMAs have completed.  Every wait is bounded.
+//   warps 6-13   converters
+// Rings: `NS` staging stages (fp8 weights + activation boxes) and two (gate/up) or four (down)
+// operand buffers of one 64-column half each, so the conversion of one half overlaps the MMAs of
+// another; a stage is released when its MMAs have completed.  Every wait is bounded.
 #pragma once
 #include <cuda_fp16.h>
 
@@ -21,11 +22,13 @@
 
 namespace stmoe_dev {
 
-constexpr int kGroup8Threads = 384;
-constexpr int kGroup8ConvWarps = 6;
+constexpr int kGroup8Threads = 448;
+constexpr int kGroup8ConvWarps = 8;
 constexpr int kGroup8KStage = 128;                                  // fp8 columns per stage
 constexpr int kGroup8StageW = kDenseRows * kGroup8KStage;           // 16 KB of e4m3 per matrix and stage
-constexpr int kGroup8OperandBytes = 2 * kGroupTileBytes;            // two f16 sub-tiles per matrix
+// operand buffers (one 64-column f16 half-tile per matrix each): the converters may run this many
+// halves ahead of the MMAs; the down projection's halves are short, so it gets more of them
+template <int NMAT> __host__ __device__ constexpr int group8_operand_buffers() { return NMAT == 2 ? 2 : 4; }
 
 struct Group8Args {
     GroupArgs g;                 // act/part as in GroupArgs (act unused), inv_rms, work list, sizes
@@ -41,7 +44,7 @@ template <int NMAT> __host__ __device__ constexpr int group8_stage_bytes(int np)
 }
 template <int NMAT> __host__ __device__ constexpr int group8_stages(int np)
 {
-    const int n = (kGroupSmemBytes - 1024 - NMAT * kGroup8OperandBytes) / group8_stage_bytes<NMAT>(np);
+    const int n = (kGroupSmemBytes - 1024 - group8_operand_buffers<NMAT>() * NMAT * kGroupTileBytes) / group8_stage_bytes<NMAT>(np);
     return n < kGroupMaxStages ? n : kGroupMaxStages;
 }
 __host__ __device__ constexpr uint32_t umma_idesc_f16(int n)
@@ -77,14 +80,15 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
 {
     const GroupArgs &a = a8.g;
     extern __shared__ uint8_t dsm_raw[];
-    __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2], ofull, oempty;
+    constexpr int NOB = group8_operand_buffers<NMAT>();
+    __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2], ofull[NOB], oempty[NOB];
     __shared__ uint32_t s_tmem;
     __shared__ int s_dead;
     const int tid = threadIdx.x, warp = tid / kWarp, lane = tid % kWarp;
     const int np = a.np, act_bytes = group_act_bytes(np);
     const int NS = group8_stages<NMAT>(np), STAGE = group8_stage_bytes<NMAT>(np);
     uint8_t *dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *opnd = dsm + (size_t)NS * STAGE;  // NMAT x 2 f16 sub-tiles
+    uint8_t *opnd = dsm + (size_t)NS * STAGE;  // NOB buffers x NMAT f16 half-tiles
     const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
     const int n_tasks = *a.wl.n_groups * tiles * a.splits;
     volatile int *dead = &s_dead;
@@ -92,7 +96,7 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) dmbar_init(&full[s], 1), dmbar_init(&empty[s], 1);
         for (int b = 0; b < 2; ++b) dmbar_init(&tfull[b], 1), dmbar_init(&tempty[b], 4);
-        dmbar_init(&ofull, kGroup8ConvWarps), dmbar_init(&oempty, 1);
+        for (int b = 0; b < NOB; ++b) dmbar_init(&ofull[b], kGroup8ConvWarps), dmbar_init(&oempty[b], 1);
         s_dead = NS < 1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -142,8 +146,7 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
         // ---- MMA issue ----------------------------------------------------------------------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_f16(np);
-            int s = 0, it = 0, stage_no = 0;
-            uint32_t ph = 0;
+            int s = 0, it = 0, half_no = 0;  // half_no counts 64-column halves; operand buffer = half_no % NOB
             for (int task = blockIdx.x; task < n_tasks && !*dead; task += gridDim.x, ++it) {
                 const GroupTask t = group_task(a, task);
                 const int ab = it & 1;
@@ -151,26 +154,29 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t acc = tmem + ab * 128;
                 bool first = true, ok = true;
-                for (int k = t.k0; k < t.k1; k += kGroup8KStage, ++stage_no) {
-                    ok = dmbar_wait(&ofull, (uint32_t)stage_no & 1u, dead);  // operands converted (implies the stage landed)
-                    if (!ok) break;
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                for (int k = t.k0; k < t.k1 && ok; k += kGroup8KStage) {
                     const uint32_t xs = dsmem_u32(dsm + (size_t)s * STAGE + NMAT * kGroup8StageW);
-                    const uint32_t ws = dsmem_u32(opnd);
 #pragma unroll
-                    for (int sub = 0; sub < 2; ++sub)
+                    for (int sub = 0; sub < 2; ++sub, ++half_no) {
+                        const int ob = half_no % NOB;
+                        ok = ok && dmbar_wait(&ofull[ob], (uint32_t)(half_no / NOB) & 1u, dead);  // converted (implies landed)
+                        if (!ok) break;
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint32_t ws = dsmem_u32(opnd) + ob * NMAT * kGroupTileBytes;
 #pragma unroll
                         for (int j = 0; j < kDenseKStep / 16; ++j) {
                             const uint64_t bd = umma_desc_sw128(xs + sub * act_bytes, j);
 #pragma unroll
                             for (int mat = 0; mat < NMAT; ++mat)
-                                umma_f16(acc + mat * 64, umma_desc_sw128(ws + (mat * 2 + sub) * kGroupTileBytes, j), bd,
-                                         idesc, !first || sub > 0 || j > 0);
+                                umma_f16(acc + mat * 64, umma_desc_sw128(ws + mat * kGroupTileBytes, j), bd, idesc,
+                                         !first || sub > 0 || j > 0);
                         }
+                        umma_commit(&oempty[ob]);  // this operand buffer may be rewritten
+                    }
+                    if (!ok) break;
                     first = false;
-                    umma_commit(&oempty);    // the operand buffer may be rewritten
-                    umma_commit(&empty[s]);  // the stage (fp8 tile already consumed, activation boxes now too)
-                    if (++s == NS) s = 0, ph ^= 1u;
+                    umma_commit(&empty[s]);  // the stage: fp8 tile consumed by the converters, activation boxes by these MMAs
+                    if (++s == NS) s = 0;
                 }
                 if (!ok) break;
                 umma_commit(&tfull[ab]);
@@ -223,30 +229,42 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
         }
     } else {
         // ---- converters: e4m3 staging tile -> two f16 operand tiles per matrix -------------------
-        const int ct = (warp - 6) * kWarp + lane;  // 0 .. 191
-        int s = 0, stage_no = 0;
+        // Thread = (row rb of 64, one of a half's four 16-byte fp8 chunks); it handles rows rb and
+        // rb + 64 of every matrix, so all of its shared-memory offsets are fixed up front.
+        const int ct = (warp - 6) * kWarp + lane;  // 0 .. 255
+        const int cl = ct & 3, rb = ct >> 2, r7 = rb & 7;
+        const int src_off[2] = {rb * 128 + ((cl ^ r7) << 4), rb * 128 + (((4 + cl) ^ r7) << 4)};
+        const int dst_lo = rb * 128 + (((cl * 2) ^ r7) << 4), dst_hi = rb * 128 + (((cl * 2 + 1) ^ r7) << 4);
+        int s = 0, half_no = 0;
         uint32_t ph = 0;
         bool ok = true;
         for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x) {
             const GroupTask t = group_task(a, task);
-            for (int k = t.k0; k < t.k1; k += kGroup8KStage, ++stage_no) {
-                ok = dmbar_wait(&full[s], ph, dead);                                      // the fp8 tile has landed
-                if (ok && stage_no > 0) ok = dmbar_wait(&oempty, (uint32_t)(stage_no - 1) & 1u, dead);  // previous MMAs done
-                if (!ok) break;
+            for (int k = t.k0; k < t.k1 && ok; k += kGroup8KStage) {
+                ok = dmbar_wait(&full[s], ph, dead);  // the fp8 tile has landed
                 const uint8_t *st = dsm + (size_t)s * STAGE;
-                for (int i = ct; i < NMAT * kDenseRows * 8; i += kGroup8ConvWarps * kWarp) {
-                    const int mat = i >> 10, r = (i >> 3) & 127, c = i & 7;
-                    const uint4 v = *reinterpret_cast<const uint4 *>(st + mat * kGroup8StageW + r * 128 + ((c ^ (r & 7)) << 4));
-                    uint4 lo, hi;
-                    e4m3x16_to_f16(v, lo, hi);
-                    uint8_t *dst = opnd + (mat * 2 + (c >> 2)) * kGroupTileBytes + r * 128;
-                    const int c2 = (c & 3) * 2;
-                    *reinterpret_cast<uint4 *>(dst + ((c2 ^ (r & 7)) << 4)) = lo;
-                    *reinterpret_cast<uint4 *>(dst + (((c2 + 1) ^ (r & 7)) << 4)) = hi;
+#pragma unroll
+                for (int sub = 0; sub < 2; ++sub, ++half_no) {
+                    if (!ok) break;
+                    const int ob = half_no % NOB, use = half_no / NOB;
+                    if (use > 0) ok = dmbar_wait(&oempty[ob], (uint32_t)(use - 1) & 1u, dead);  // its previous MMAs are done
+                    if (!ok) break;
+                    uint8_t *ow = opnd + ob * NMAT * kGroupTileBytes;
+#pragma unroll
+                    for (int mat = 0; mat < NMAT; ++mat)
+#pragma unroll
+                        for (int pass = 0; pass < 2; ++pass) {
+                            const uint4 v = *reinterpret_cast<const uint4 *>(st + mat * kGroup8StageW + pass * 64 * 128 + src_off[sub]);
+                            uint4 lo, hi;
+                            e4m3x16_to_f16(v, lo, hi);
+                            uint8_t *dst = ow + mat * kGroupTileBytes + pass * 64 * 128;
+                            *reinterpret_cast<uint4 *>(dst + dst_lo) = lo;
+                            *reinterpret_cast<uint4 *>(dst + dst_hi) = hi;
+                        }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) dmbar_arrive(&ofull[ob]);
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) dmbar_arrive(&ofull);
                 if (++s == NS) s = 0, ph ^= 1u;
             }
         }

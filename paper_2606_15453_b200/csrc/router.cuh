@@ -510,9 +510,9 @@ __device__ __forceinline__ void router_finalize(const RouterArgs &a, int *s_ids,
 }
 
 template <int DT>
-__global__ void __launch_bounds__(256) router_fused_kernel(RouterArgs a)
+__global__ void __launch_bounds__(512) router_fused_kernel(RouterArgs a)
 {
-    constexpr int NW = 8;
+    const int NW = blockDim.x / kWarp;  // 8 warps; 16 for larger batches (the last CTA routes one sequence per warp)
     __shared__ int s_ids[kMaxBatch * kMaxTopK];
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
     __shared__ int s_last;

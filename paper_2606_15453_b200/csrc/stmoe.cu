@@ -535,7 +535,8 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
 }
 
 // ---- tensor-core path (dense_group.cuh) ---------------------------------------------------
-constexpr int kDenseMinBatch = 2;
+constexpr int kDenseMinBatch = 2;   // bf16 stacks: measured ahead of the CUDA-core kernels from two sequences on
+constexpr int kDense8MinBatch = 4;  // fp8 stacks (conversion-bound kernels): from four
 constexpr int kDenseMaxSplits = 4;
 constexpr int kTokenDenseDynBytes = 220 * 1024;
 
@@ -658,7 +659,7 @@ int dense8_setup(stmoe *s)
     CU_TRY(cudaFuncSetAttribute(dense8_group_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
     CU_TRY(cudaFuncSetAttribute(dense8_group_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
     s->dense_grid = sm_count();
-    s->dense_min_batch = kDenseMinBatch;
+    s->dense_min_batch = kDense8MinBatch;
     s->dense8 = true;
     return STMOE_OK;
 }
@@ -810,17 +811,18 @@ int layer_step(stmoe *s, int layer, int batch, const float *h_in, float *h_out, 
     ta.wl = s->wlm.wl;
     {
         const int C = s->rdt == STMOE_F32 ? router_chunks<0>(H, batch) : router_chunks<1>(H, batch);
-        const int grid = std::min((E * C + 7) / 8, 2 * s->plan1.grid_gate_up);
+        const int threads = batch > 8 ? 512 : 256, nw = threads / kWarp;
+        const int grid = std::min((E * C + nw - 1) / nw, 2 * s->plan1.grid_gate_up);
         if (s->rdt == STMOE_F32) {
             if (layer > 0 && !offloaded(s))
-                launch_pdl(router_fused_kernel<0>, grid, 256, st, ra);
+                launch_pdl(router_fused_kernel<0>, grid, threads, st, ra);
             else
-                router_fused_kernel<0><<<grid, 256, 0, st>>>(ra);
+                router_fused_kernel<0><<<grid, threads, 0, st>>>(ra);
         } else {
             if (layer > 0 && !offloaded(s))
-                launch_pdl(router_fused_kernel<1>, grid, 256, st, ra);
+                launch_pdl(router_fused_kernel<1>, grid, threads, st, ra);
             else
-                router_fused_kernel<1><<<grid, 256, 0, st>>>(ra);
+                router_fused_kernel<1><<<grid, threads, 0, st>>>(ra);
         }
     }
     CU_TRY(cudaGetLastError());
