@@ -12,9 +12,9 @@
 //   warp 1       MMA issue (4 K=16 steps per 64-column half of a stage and matrix), tensor-memory owner
 //   warps 2-5    epilogue (two accumulator buffers)
 //   warps 6-13   converters
-// Rings: `NS` staging stages (fp8 weights + activation boxes) and two (gate/up) or four (down)
-// operand buffers of one 64-column half each, so the conversion of one half overlaps the MMAs of
-// another; a stage is released when its MMAs have completed.  Every wait is bounded.
+// Rings: `NS` staging stages (fp8 weights + activation boxes) and two operand buffers, so the
+// conversion of one unit overlaps the MMAs of the other; a stage is released when its MMAs have
+// completed.  Every wait is bounded.
 #pragma once
 #include <cuda_fp16.h>
 
@@ -26,9 +26,11 @@ constexpr int kGroup8Threads = 448;
 constexpr int kGroup8ConvWarps = 8;
 constexpr int kGroup8KStage = 128;                                  // fp8 columns per stage
 constexpr int kGroup8StageW = kDenseRows * kGroup8KStage;           // 16 KB of e4m3 per matrix and stage
-// operand buffers (one 64-column f16 half-tile per matrix each): the converters may run this many
-// halves ahead of the MMAs; the down projection's halves are short, so it gets more of them
-template <int NMAT> __host__ __device__ constexpr int group8_operand_buffers() { return NMAT == 2 ? 2 : 4; }
+// Two operand buffers, so that the conversion of one unit overlaps the MMAs of the other.  A unit
+// is one 64-column half of a stage for gate/up (two matrices) and the whole stage for the down
+// projection (one matrix: fewer, longer hand-offs), 32 KB of f16 either way.
+template <int NMAT> __host__ __device__ constexpr int group8_unit_halves() { return NMAT == 2 ? 1 : 2; }
+template <int NMAT> __host__ __device__ constexpr int group8_operand_buffers() { return 2; }
 
 struct Group8Args {
     GroupArgs g;                 // act/part as in GroupArgs (act unused), inv_rms, work list, sizes
@@ -44,7 +46,8 @@ template <int NMAT> __host__ __device__ constexpr int group8_stage_bytes(int np)
 }
 template <int NMAT> __host__ __device__ constexpr int group8_stages(int np)
 {
-    const int n = (kGroupSmemBytes - 1024 - group8_operand_buffers<NMAT>() * NMAT * kGroupTileBytes) / group8_stage_bytes<NMAT>(np);
+    const int n = (kGroupSmemBytes - 1024 - group8_operand_buffers<NMAT>() * group8_unit_halves<NMAT>() * NMAT * kGroupTileBytes) /
+                  group8_stage_bytes<NMAT>(np);
     return n < kGroupMaxStages ? n : kGroupMaxStages;
 }
 __host__ __device__ constexpr uint32_t umma_idesc_f16(int n)
@@ -80,7 +83,7 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
 {
     const GroupArgs &a = a8.g;
     extern __shared__ uint8_t dsm_raw[];
-    constexpr int NOB = group8_operand_buffers<NMAT>();
+    constexpr int NOB = group8_operand_buffers<NMAT>(), UH = group8_unit_halves<NMAT>(), UNIT = UH * NMAT * kGroupTileBytes;
     __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2], ofull[NOB], oempty[NOB];
     __shared__ uint32_t s_tmem;
     __shared__ int s_dead;
@@ -88,7 +91,7 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
     const int np = a.np, act_bytes = group_act_bytes(np);
     const int NS = group8_stages<NMAT>(np), STAGE = group8_stage_bytes<NMAT>(np);
     uint8_t *dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *opnd = dsm + (size_t)NS * STAGE;  // NOB buffers x NMAT f16 half-tiles
+    uint8_t *opnd = dsm + (size_t)NS * STAGE;  // NOB buffers x (NMAT x UH) f16 half-tiles
     const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
     const int n_tasks = *a.wl.n_groups * tiles * a.splits;
     volatile int *dead = &s_dead;
@@ -146,7 +149,7 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
         // ---- MMA issue ----------------------------------------------------------------------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_f16(np);
-            int s = 0, it = 0, half_no = 0;  // half_no counts 64-column halves; operand buffer = half_no % NOB
+            int s = 0, it = 0, half_no = 0;  // half_no counts units; operand buffer = half_no % NOB
             for (int task = blockIdx.x; task < n_tasks && !*dead; task += gridDim.x, ++it) {
                 const GroupTask t = group_task(a, task);
                 const int ab = it & 1;
@@ -157,19 +160,23 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
                 for (int k = t.k0; k < t.k1 && ok; k += kGroup8KStage) {
                     const uint32_t xs = dsmem_u32(dsm + (size_t)s * STAGE + NMAT * kGroup8StageW);
 #pragma unroll
-                    for (int sub = 0; sub < 2; ++sub, ++half_no) {
+                    for (int unit = 0; unit < 2 / UH; ++unit, ++half_no) {
                         const int ob = half_no % NOB;
                         ok = ok && dmbar_wait(&ofull[ob], (uint32_t)(half_no / NOB) & 1u, dead);  // converted (implies landed)
                         if (!ok) break;
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        const uint32_t ws = dsmem_u32(opnd) + ob * NMAT * kGroupTileBytes;
+                        const uint32_t ws = dsmem_u32(opnd) + ob * UNIT;
 #pragma unroll
-                        for (int j = 0; j < kDenseKStep / 16; ++j) {
-                            const uint64_t bd = umma_desc_sw128(xs + sub * act_bytes, j);
+                        for (int h = 0; h < UH; ++h) {
+                            const int sub = unit * UH + h;
 #pragma unroll
-                            for (int mat = 0; mat < NMAT; ++mat)
-                                umma_f16(acc + mat * 64, umma_desc_sw128(ws + mat * kGroupTileBytes, j), bd, idesc,
-                                         !first || sub > 0 || j > 0);
+                            for (int j = 0; j < kDenseKStep / 16; ++j) {
+                                const uint64_t bd = umma_desc_sw128(xs + sub * act_bytes, j);
+#pragma unroll
+                                for (int mat = 0; mat < NMAT; ++mat)
+                                    umma_f16(acc + mat * 64, umma_desc_sw128(ws + (mat * UH + h) * kGroupTileBytes, j), bd,
+                                             idesc, !first || sub > 0 || j > 0);
+                            }
                         }
                         umma_commit(&oempty[ob]);  // this operand buffer may be rewritten
                     }
@@ -244,23 +251,26 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
                 ok = dmbar_wait(&full[s], ph, dead);  // the fp8 tile has landed
                 const uint8_t *st = dsm + (size_t)s * STAGE;
 #pragma unroll
-                for (int sub = 0; sub < 2; ++sub, ++half_no) {
+                for (int unit = 0; unit < 2 / UH; ++unit, ++half_no) {
                     if (!ok) break;
                     const int ob = half_no % NOB, use = half_no / NOB;
                     if (use > 0) ok = dmbar_wait(&oempty[ob], (uint32_t)(use - 1) & 1u, dead);  // its previous MMAs are done
                     if (!ok) break;
-                    uint8_t *ow = opnd + ob * NMAT * kGroupTileBytes;
+                    uint8_t *ow = opnd + ob * UNIT;
 #pragma unroll
-                    for (int mat = 0; mat < NMAT; ++mat)
+                    for (int h = 0; h < UH; ++h)
 #pragma unroll
-                        for (int pass = 0; pass < 2; ++pass) {
-                            const uint4 v = *reinterpret_cast<const uint4 *>(st + mat * kGroup8StageW + pass * 64 * 128 + src_off[sub]);
-                            uint4 lo, hi;
-                            e4m3x16_to_f16(v, lo, hi);
-                            uint8_t *dst = ow + mat * kGroupTileBytes + pass * 64 * 128;
-                            *reinterpret_cast<uint4 *>(dst + dst_lo) = lo;
-                            *reinterpret_cast<uint4 *>(dst + dst_hi) = hi;
-                        }
+                        for (int mat = 0; mat < NMAT; ++mat)
+#pragma unroll
+                            for (int pass = 0; pass < 2; ++pass) {
+                                const uint4 v = *reinterpret_cast<const uint4 *>(st + mat * kGroup8StageW + pass * 64 * 128 +
+                                                                                 src_off[unit * UH + h]);
+                                uint4 lo, hi;
+                                e4m3x16_to_f16(v, lo, hi);
+                                uint8_t *dst = ow + (mat * UH + h) * kGroupTileBytes + pass * 64 * 128;
+                                *reinterpret_cast<uint4 *>(dst + dst_lo) = lo;
+                                *reinterpret_cast<uint4 *>(dst + dst_hi) = hi;
+                            }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) dmbar_arrive(&ofull[ob]);
