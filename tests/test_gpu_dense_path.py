@@ -126,6 +126,23 @@ def test_dense_decode_token_agrees_with_cuda_core_path(B):
             assert torch.equal(a[1][0], c[1][0])      # layer 0 routing sees identical inputs
 
 
+def test_dense_paths_agree_at_maximum_batch_and_k():
+    """64 sequences x top-32: the work list takes 65 KB of the persistent kernel's shared memory and
+    leaves a single stage for the ring."""
+    cfg = stacks.CONFIGS["C2"].scaled(n_layers=2, profile_tokens=2, hidden=144, inter=96, n_experts=40, top_k=32,
+                                      n_shared=0)
+    one = _run_tokens(cfg, 64, 4, 0, torch.cuda.Stream())
+    graph = _run_tokens(cfg, 64, 4, P.FLAG_NO_PERSISTENT, torch.cuda.Stream())
+    core = _run_tokens(cfg, 64, 4, P.FLAG_NO_DENSE, torch.cuda.Stream())
+    for a, b in zip(one[0], graph[0]):
+        assert all(torch.equal(u, v) for u, v in zip(a, b))
+    assert one[1] == graph[1]
+    assert one[2]["kernel_launches"] < graph[2]["kernel_launches"]
+    for a, c in zip(one[0][:1], core[0][:1]):
+        assert torch.equal(a[1][0], c[1][0])
+        assert (a[0] - c[0]).abs().max().item() <= 2e-2 * c[0].abs().max().item()
+
+
 def test_dense_path_off_for_small_batches_and_fp32():
     cfg = stacks.CONFIGS["C0"].scaled(n_layers=2)
     pr = Pair(cfg, 8, oracle=False)        # fp32 weights: no tensor-core path

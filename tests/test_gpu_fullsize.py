@@ -1,7 +1,8 @@
 """Full-size parity: the benchmark workload (Mixtral-shaped bf16 stack, 32 layers, 90 GB of
 resident experts, batch 1) through the same entry point and launch configuration bench.py
 times (stmoe_decode_token -> persistent decode-step kernel), against the CPU oracle running
-its own residual stream for whole decode steps."""
+its own residual stream for whole decode steps; and the DeepSeek-V2-Lite-shaped stack at batch 8
+through the persistent tensor-core kernel."""
 import numpy as np
 import pytest
 import torch
@@ -54,4 +55,52 @@ def test_c1_full_size_decode_steps_match_oracle():
             checked_outputs += 1
     assert pr.stack.export_state() == replay.export()
     assert checked_outputs == 1
+    pr.close()
+
+
+def test_c2_full_size_batch8_tensor_core_step_matches_oracle():
+    """C2 at full size (26 layers, 64 + 2 experts, 29.7 GB) with eight sequences: the launch
+    bench.py times for `--workload C2 --batch 8` (decode_token_dense_kernel)."""
+    free = torch.cuda.mem_get_info()[0]
+    cfg = stacks.CONFIGS["C2"].scaled(profile_tokens=1)
+    need = cfg.n_layers * (cfg.n_experts + cfg.n_shared) * cfg.expert_bytes + (8 << 30)
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of free HBM, {free >> 30} GiB available")
+    B, T = 8, 3
+    pr = Pair(cfg, B)
+    L, K = cfg.n_layers, cfg.top_k
+    x = stacks.token_inputs(cfg, B, T)
+    ids = torch.empty(L, B, K, dtype=torch.int32, device=DEV)
+    w = torch.empty(L, B, K, dtype=torch.float32, device=DEV)
+    pred = torch.empty(L, B, pr.stack.max_pred, dtype=torch.int32, device=DEV)
+    npred = torch.empty(L, B, dtype=torch.int32, device=DEV)
+    flags = torch.empty(L, B, dtype=torch.int32, device=DEV)
+    ho = torch.empty(B, cfg.hidden, device=DEV)
+    replay = O.Predictor(L, cfg.n_experts, K, B, cfg.profile_tokens, "st")
+    checked = 0
+    for t in range(T):
+        pr.stack.decode_token(x[t].to(DEV), ho, ids, w, pred, npred, flags)
+        torch.cuda.synchronize()
+        g_ids, g_pred, g_np = ids.cpu().numpy(), pred.cpu().numpy(), npred.cpu().numpy()
+        for l in range(L):   # the predictor is bit-exact on the GPU's own routing, always
+            rp = replay.step(l, g_ids[l])
+            assert g_np[l].tolist() == rp["n_pred"].tolist() and (g_pred[l] == rp["pred_ids"]).all(), (t, l)
+        if t > 0:
+            continue
+        h_ref, per = pr.oracle.decode_token(x[t].numpy())
+        o_ids = np.stack([r["ids"] for r in per])
+        got = ho.cpu().numpy()
+        for b in range(B):
+            # a sequence is comparable while its routing agrees with the oracle's in every layer
+            if (o_ids[:, b] != g_ids[:, b]).any():
+                assert sum(int(r["ties"][b]) for r in per) + int(flags[:, b].sum()) > 0, \
+                    f"sequence {b}: routing diverged from the oracle without a near tie"
+                continue
+            assert rel_err(got[b], h_ref[b]) <= TOL["bf16"], b
+            assert rel_err(got[b] - x[t][b].numpy(), h_ref[b] - x[t][b].numpy()) <= 2e-2, b
+            checked += 1
+    assert pr.stack.export_state() == replay.export()
+    assert checked >= B // 2
+    st = pr.stack.stats()
+    assert st["kernel_launches"] <= T + 1      # one persistent launch per step (+ the table build)
     pr.close()
