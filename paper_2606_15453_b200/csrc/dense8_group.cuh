@@ -3,18 +3,20 @@
 // Same task structure as dense_group.cuh (one work-list entry per expert, a task = entry x 128
 // weight rows x one split, persistent CTA per SM, weights as the MMA's M operand).  tcgen05 has no
 // fp8 x 16-bit mode, and rounding the activations to fp8 would not fit the error bound, so the
-// weights are widened on the way: TMA lands the e4m3 tile (128 rows x 128 columns, 16 KB) in a
-// staging ring, eight converter warps rewrite it as two f16 operand tiles (e4m3 -> f16 is exact) in
-// the 128-byte swizzled layout, and the MMA runs in f16 x f16 -> fp32 against f16 activations.
-// The per-output-channel scales belong to the weight rows = accumulator lanes and are applied in
-// the epilogue.
-//   warp 0       TMA producer: weight tile(s) + two activation boxes per stage
-//   warp 1       MMA issue (4 K=16 steps per 64-column half of a stage and matrix), tensor-memory owner
+// weights are widened on the way: TMA lands e4m3 boxes (128 rows x 128 columns, 16 KB) in a
+// staging ring, eight converter warps turn each row into f16 pairs (e4m3 -> f16 is exact) and write
+// them straight into tensor memory (tcgen05.st; a thread owns the row = TMEM lane of its warp's
+// lane quarter), and the MMA runs f16 x f16 -> fp32 with its A operand from tensor memory and the
+// f16 activations from shared memory.  A weight byte thus crosses shared memory twice (TMA write,
+// converter read).  The per-output-channel scales belong to the weight rows = accumulator lanes and
+// are applied in the epilogue.
+//   warp 0       TMA producer: two weight boxes (gate and up of the same columns, or two
+//                consecutive column boxes of the down matrix) + the activation boxes of a stage
+//   warp 1       MMA issue (8 K=16 steps per box), tensor-memory owner
 //   warps 2-5    epilogue (two accumulator buffers)
-//   warps 6-13   converters
-// Rings: `NS` staging stages (fp8 weights + activation boxes) and two operand buffers, so the
-// conversion of one unit overlaps the MMAs of the other; a stage is released when its MMAs have
-// completed.  Every wait is bounded.
+//   warps 6-13   converters, two per lane quarter: one weight box each
+// Tensor memory: columns [0,256) two accumulator buffers, [256,512) two A buffers of 2 x 64 columns
+// (a box = 128 reduction columns, two f16 per 32-bit column).  Every wait is bounded.
 #pragma once
 #include <cuda_fp16.h>
 
@@ -23,14 +25,10 @@
 namespace stmoe_dev {
 
 constexpr int kGroup8Threads = 448;
-constexpr int kGroup8ConvWarps = 8;
-constexpr int kGroup8KStage = 128;                                  // fp8 columns per stage
-constexpr int kGroup8StageW = kDenseRows * kGroup8KStage;           // 16 KB of e4m3 per matrix and stage
-// Two operand buffers, so that the conversion of one unit overlaps the MMAs of the other.  A unit
-// is one 64-column half of a stage for gate/up (two matrices) and the whole stage for the down
-// projection (one matrix: fewer, longer hand-offs), 32 KB of f16 either way.
-template <int NMAT> __host__ __device__ constexpr int group8_unit_halves() { return NMAT == 2 ? 1 : 2; }
-template <int NMAT> __host__ __device__ constexpr int group8_operand_buffers() { return 2; }
+constexpr int kGroup8BoxCols = 128;                                 // fp8 columns of a weight box
+constexpr int kGroup8BoxBytes = kDenseRows * kGroup8BoxCols;        // 16 KB of e4m3
+// reduction columns per stage: gate/up share one box position, the down projection takes two
+template <int NMAT> __host__ __device__ constexpr int group8_kstage() { return NMAT == 2 ? kGroup8BoxCols : 2 * kGroup8BoxCols; }
 
 struct Group8Args {
     GroupArgs g;                 // act/part as in GroupArgs (act unused), inv_rms, work list, sizes
@@ -40,25 +38,20 @@ struct Group8Args {
     int scale_off;               // element offset of this projection's scales in the image's scale vector
 };
 
+// two weight boxes + one 64-column f16 activation box per 64 reduction columns
 template <int NMAT> __host__ __device__ constexpr int group8_stage_bytes(int np)
 {
-    return NMAT * kGroup8StageW + 2 * group_act_bytes(np);
+    return 2 * kGroup8BoxBytes + (group8_kstage<NMAT>() / kDenseKStep) * group_act_bytes(np);
 }
 template <int NMAT> __host__ __device__ constexpr int group8_stages(int np)
 {
-    const int n = (kGroupSmemBytes - 1024 - group8_operand_buffers<NMAT>() * group8_unit_halves<NMAT>() * NMAT * kGroupTileBytes) /
-                  group8_stage_bytes<NMAT>(np);
+    const int n = (kGroupSmemBytes - 1024) / group8_stage_bytes<NMAT>(np);
     return n < kGroupMaxStages ? n : kGroupMaxStages;
 }
 __host__ __device__ constexpr uint32_t umma_idesc_f16(int n)
 {
     return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kDenseRows >> 4) << 24);  // f16 x f16 -> f32
 }
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t a, uint64_t b, uint32_t idesc, bool accumulate)
-{
-    umma_bf16(tmem_d, a, b, idesc, accumulate);  // same instruction; the operand types are in idesc
-}
-
 // 16 e4m3 values -> 16 f16 values (two 16-byte chunks)
 __device__ __forceinline__ void e4m3x16_to_f16(const uint4 &v, uint4 &lo, uint4 &hi)
 {
@@ -76,22 +69,42 @@ __device__ __forceinline__ void e4m3x16_to_f16(const uint4 &v, uint4 &lo, uint4 
     hi = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
+__device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t b, uint32_t idesc, bool accumulate)
+{
+    asm volatile(
+        "{.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;}"
+        :
+        : "r"(tmem_d), "r"(tmem_a), "l"(b), "r"(idesc), "r"((uint32_t)accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+                 :
+                 : "r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+                   "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+                 : "memory");
+}
+
+// NMAT = 2: gate and up projections with the SiLU epilogue; NMAT = 1: down projection.
 template <int NMAT>
 __global__ void __launch_bounds__(kGroup8Threads, 1)
 dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
-                    const __grid_constant__ CUtensorMap map_x, Group8Args a8)
+                     const __grid_constant__ CUtensorMap map_x, Group8Args a8)
 {
+    constexpr int ACOLS = 128;                           // tensor-memory columns of one A buffer (two boxes)
+    constexpr int KSTAGE = group8_kstage<NMAT>(), XBOXES = KSTAGE / kDenseKStep;
     const GroupArgs &a = a8.g;
     extern __shared__ uint8_t dsm_raw[];
-    constexpr int NOB = group8_operand_buffers<NMAT>(), UH = group8_unit_halves<NMAT>(), UNIT = UH * NMAT * kGroupTileBytes;
-    __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2], ofull[NOB], oempty[NOB];
+    __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2], afull[2], aempty[2];
     __shared__ uint32_t s_tmem;
     __shared__ int s_dead;
     const int tid = threadIdx.x, warp = tid / kWarp, lane = tid % kWarp;
     const int np = a.np, act_bytes = group_act_bytes(np);
     const int NS = group8_stages<NMAT>(np), STAGE = group8_stage_bytes<NMAT>(np);
     uint8_t *dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *opnd = dsm + (size_t)NS * STAGE;  // NOB buffers x (NMAT x UH) f16 half-tiles
     const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
     const int n_tasks = *a.wl.n_groups * tiles * a.splits;
     volatile int *dead = &s_dead;
@@ -99,13 +112,12 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) dmbar_init(&full[s], 1), dmbar_init(&empty[s], 1);
         for (int b = 0; b < 2; ++b) dmbar_init(&tfull[b], 1), dmbar_init(&tempty[b], 4);
-        for (int b = 0; b < NOB; ++b) dmbar_init(&ofull[b], kGroup8ConvWarps), dmbar_init(&oempty[b], 1);
+        for (int b = 0; b < 2; ++b) dmbar_init(&afull[b], 8), dmbar_init(&aempty[b], 1);
         s_dead = NS < 1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dsmem_u32(&s_tmem)),
-                     "r"(kGroupTmemCols)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dsmem_u32(&s_tmem)), "r"(512)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -125,15 +137,20 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
                 const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
                 const int xrow = NMAT == 2 ? 0 : a.wl.g_start[t.g];
                 bool ok = true;
-                for (int k = t.k0; k < t.k1 && ok; k += kGroup8KStage) {
+                for (int k = t.k0; k < t.k1 && ok; k += KSTAGE) {
                     ok = dmbar_wait(&empty[s], ph ^ 1u, dead);
                     if (!ok) break;
                     uint8_t *st = dsm + (size_t)s * STAGE;
-                    dmbar_expect_tx(&full[s], (uint32_t)(NMAT * kGroup8StageW + 2 * np * kDenseKStep * 2));
+                    // boxes past the end of the reduction dimension are zero-filled and still count
+                    dmbar_expect_tx(&full[s], (uint32_t)(2 * kGroup8BoxBytes + XBOXES * np * kDenseKStep * 2));
                     tma_load_3d(st, &map_w0, k, t.row0, img, &full[s]);
-                    if (NMAT == 2) tma_load_3d(st + kGroup8StageW, &map_w1, k, t.row0, img, &full[s]);
-                    tma_load_2d(st + NMAT * kGroup8StageW, &map_x, k, xrow, &full[s]);
-                    tma_load_2d(st + NMAT * kGroup8StageW + act_bytes, &map_x, k + kDenseKStep, xrow, &full[s]);
+                    if (NMAT == 2)
+                        tma_load_3d(st + kGroup8BoxBytes, &map_w1, k, t.row0, img, &full[s]);
+                    else
+                        tma_load_3d(st + kGroup8BoxBytes, &map_w0, k + kGroup8BoxCols, t.row0, img, &full[s]);
+#pragma unroll
+                    for (int x = 0; x < XBOXES; ++x)
+                        tma_load_2d(st + 2 * kGroup8BoxBytes + x * act_bytes, &map_x, k + x * kDenseKStep, xrow, &full[s]);
                     ++issued;
                     if (++s == NS) s = 0, ph ^= 1u;
                 }
@@ -146,10 +163,10 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
             }
         }
     } else if (warp == 1) {
-        // ---- MMA issue ----------------------------------------------------------------------------
+        // ---- MMA issue: A from tensor memory, B (activations) from shared memory -------------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_f16(np);
-            int s = 0, it = 0, half_no = 0;  // half_no counts units; operand buffer = half_no % NOB
+            int s = 0, it = 0, stage_no = 0;
             for (int task = blockIdx.x; task < n_tasks && !*dead; task += gridDim.x, ++it) {
                 const GroupTask t = group_task(a, task);
                 const int ab = it & 1;
@@ -157,32 +174,27 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t acc = tmem + ab * 128;
                 bool first = true, ok = true;
-                for (int k = t.k0; k < t.k1 && ok; k += kGroup8KStage) {
-                    const uint32_t xs = dsmem_u32(dsm + (size_t)s * STAGE + NMAT * kGroup8StageW);
-#pragma unroll
-                    for (int unit = 0; unit < 2 / UH; ++unit, ++half_no) {
-                        const int ob = half_no % NOB;
-                        ok = ok && dmbar_wait(&ofull[ob], (uint32_t)(half_no / NOB) & 1u, dead);  // converted (implies landed)
-                        if (!ok) break;
-                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        const uint32_t ws = dsmem_u32(opnd) + ob * UNIT;
-#pragma unroll
-                        for (int h = 0; h < UH; ++h) {
-                            const int sub = unit * UH + h;
-#pragma unroll
-                            for (int j = 0; j < kDenseKStep / 16; ++j) {
-                                const uint64_t bd = umma_desc_sw128(xs + sub * act_bytes, j);
-#pragma unroll
-                                for (int mat = 0; mat < NMAT; ++mat)
-                                    umma_f16(acc + mat * 64, umma_desc_sw128(ws + (mat * UH + h) * kGroupTileBytes, j), bd,
-                                             idesc, !first || sub > 0 || j > 0);
-                            }
-                        }
-                        umma_commit(&oempty[ob]);  // this operand buffer may be rewritten
-                    }
+                for (int k = t.k0; k < t.k1; k += KSTAGE, ++stage_no) {
+                    const int buf = stage_no & 1;
+                    ok = dmbar_wait(&afull[buf], ((uint32_t)stage_no >> 1) & 1u, dead);  // converted (implies landed)
                     if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t xs = dsmem_u32(dsm + (size_t)s * STAGE + 2 * kGroup8BoxBytes);
+                    const uint32_t abuf = tmem + 256 + buf * ACOLS;
+#pragma unroll
+                    for (int bx = 0; bx < 2; ++bx)
+#pragma unroll
+                        for (int j = 0; j < kGroup8BoxCols / 16; ++j) {
+                            // gate/up: both boxes multiply the same activation columns into their own
+                            // accumulators; down: the second box continues the reduction
+                            const int xb = (NMAT == 2 ? 0 : bx * 2) + (j >> 2);
+                            const uint64_t bd = umma_desc_sw128(xs + xb * act_bytes, j & 3);
+                            umma_f16_ts(acc + (NMAT == 2 ? bx * 64 : 0), abuf + bx * 64 + j * 8, bd, idesc,
+                                        !first || j > 0 || (NMAT == 1 && bx > 0));
+                        }
                     first = false;
-                    umma_commit(&empty[s]);  // the stage: fp8 tile consumed by the converters, activation boxes by these MMAs
+                    umma_commit(&aempty[buf]);  // this A buffer may be rewritten
+                    umma_commit(&empty[s]);     // and the stage reloaded
                     if (++s == NS) s = 0;
                 }
                 if (!ok) break;
@@ -200,7 +212,6 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
             const int ge = a.wl.g_expert[t.g];
             const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
             const int row = t.row0 + lg * kWarp + lane;
-            // bf16 scales behind the three matrices: [gate I | up I | down H]
             const uint16_t *sc = reinterpret_cast<const uint16_t *>(a8.store + (size_t)img * a8.img_bytes +
                                                                     3 * (size_t)a.rows * a.kd) + a8.scale_off;
             const int srow = min(row, a.rows - 1);
@@ -235,46 +246,41 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
             if (!ok) break;
         }
     } else {
-        // ---- converters: e4m3 staging tile -> two f16 operand tiles per matrix -------------------
-        // Thread = (row rb of 64, one of a half's four 16-byte fp8 chunks); it handles rows rb and
-        // rb + 64 of every matrix, so all of its shared-memory offsets are fixed up front.
-        const int ct = (warp - 6) * kWarp + lane;  // 0 .. 255
-        const int cl = ct & 3, rb = ct >> 2, r7 = rb & 7;
-        const int src_off[2] = {rb * 128 + ((cl ^ r7) << 4), rb * 128 + (((4 + cl) ^ r7) << 4)};
-        const int dst_lo = rb * 128 + (((cl * 2) ^ r7) << 4), dst_hi = rb * 128 + (((cl * 2 + 1) ^ r7) << 4);
-        int s = 0, half_no = 0;
+        // ---- converters: thread = one weight row; its e4m3 columns -> f16 pairs -> tensor memory ----
+        // Two warps share a lane quarter: one weight box of the stage each.
+        const int cw = warp - 6, lq = warp % 4, bx = cw >> 2;
+        const int r = lq * kWarp + lane, r7 = r & 7;
+        const uint32_t lane_base = tmem + 256 + ((uint32_t)(lq * kWarp) << 16) + bx * 64;
+        int s = 0, stage_no = 0;
         uint32_t ph = 0;
         bool ok = true;
         for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x) {
             const GroupTask t = group_task(a, task);
-            for (int k = t.k0; k < t.k1 && ok; k += kGroup8KStage) {
+            for (int k = t.k0; k < t.k1 && ok; k += KSTAGE, ++stage_no) {
+                const int buf = stage_no & 1, use = stage_no >> 1;
                 ok = dmbar_wait(&full[s], ph, dead);  // the fp8 tile has landed
-                const uint8_t *st = dsm + (size_t)s * STAGE;
+                if (ok && use > 0) ok = dmbar_wait(&aempty[buf], (uint32_t)(use - 1) & 1u, dead);  // its previous MMAs are done
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint8_t *row_ptr = dsm + (size_t)s * STAGE + bx * kGroup8BoxBytes + r * 128;
 #pragma unroll
-                for (int unit = 0; unit < 2 / UH; ++unit, ++half_no) {
-                    if (!ok) break;
-                    const int ob = half_no % NOB, use = half_no / NOB;
-                    if (use > 0) ok = dmbar_wait(&oempty[ob], (uint32_t)(use - 1) & 1u, dead);  // its previous MMAs are done
-                    if (!ok) break;
-                    uint8_t *ow = opnd + ob * UNIT;
+                for (int c0 = 0; c0 < 8; c0 += 2) {
+                    uint32_t v[16];
 #pragma unroll
-                    for (int h = 0; h < UH; ++h)
-#pragma unroll
-                        for (int mat = 0; mat < NMAT; ++mat)
-#pragma unroll
-                            for (int pass = 0; pass < 2; ++pass) {
-                                const uint4 v = *reinterpret_cast<const uint4 *>(st + mat * kGroup8StageW + pass * 64 * 128 +
-                                                                                 src_off[unit * UH + h]);
-                                uint4 lo, hi;
-                                e4m3x16_to_f16(v, lo, hi);
-                                uint8_t *dst = ow + (mat * UH + h) * kGroupTileBytes + pass * 64 * 128;
-                                *reinterpret_cast<uint4 *>(dst + dst_lo) = lo;
-                                *reinterpret_cast<uint4 *>(dst + dst_hi) = hi;
-                            }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) dmbar_arrive(&ofull[ob]);
+                    for (int h = 0; h < 2; ++h) {
+                        const int c = c0 + h;
+                        const uint4 raw = *reinterpret_cast<const uint4 *>(row_ptr + ((c ^ r7) << 4));
+                        uint4 lo, hi;
+                        e4m3x16_to_f16(raw, lo, hi);
+                        v[8 * h] = lo.x, v[8 * h + 1] = lo.y, v[8 * h + 2] = lo.z, v[8 * h + 3] = lo.w;
+                        v[8 * h + 4] = hi.x, v[8 * h + 5] = hi.y, v[8 * h + 6] = hi.z, v[8 * h + 7] = hi.w;
+                    }
+                    tmem_st16(lane_base + buf * ACOLS + c0 * 8, v);
                 }
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) dmbar_arrive(&afull[buf]);
                 if (++s == NS) s = 0, ph ^= 1u;
             }
         }
@@ -282,7 +288,7 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kGroupTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
     }
     if (tid == 0 && s_dead) *a.err = 1u;
 }

@@ -647,9 +647,9 @@ int dense8_setup(stmoe *s)
     const cuuint64_t gd[3] = {(cuuint64_t)H, (cuuint64_t)I, n_img}, gs[2] = {(cuuint64_t)H, s->img_bytes};
     const cuuint64_t dd[3] = {(cuuint64_t)I, (cuuint64_t)H, n_img}, ds[2] = {(cuuint64_t)I, s->img_bytes};
     const CUtensorMapDataType u8 = CU_TENSOR_MAP_DATA_TYPE_UINT8, f16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
-    ST_TRY(encode_map(enc, &s->map8_gate, s->d_resident, 3, gd, gs, kDenseRows, u8, kGroup8KStage));
-    ST_TRY(encode_map(enc, &s->map8_up, s->d_resident + (size_t)I * H, 3, gd, gs, kDenseRows, u8, kGroup8KStage));
-    ST_TRY(encode_map(enc, &s->map8_down, s->d_resident + 2 * (size_t)I * H, 3, dd, ds, kDenseRows, u8, kGroup8KStage));
+    ST_TRY(encode_map(enc, &s->map8_gate, s->d_resident, 3, gd, gs, kDenseRows, u8, kGroup8BoxCols));
+    ST_TRY(encode_map(enc, &s->map8_up, s->d_resident + (size_t)I * H, 3, gd, gs, kDenseRows, u8, kGroup8BoxCols));
+    ST_TRY(encode_map(enc, &s->map8_down, s->d_resident + 2 * (size_t)I * H, 3, dd, ds, kDenseRows, u8, kGroup8BoxCols));
     for (int i = 0; i < 4; ++i) {
         const cuuint64_t xd[2] = {(cuuint64_t)H, (cuuint64_t)kDenseMaxTokens}, xs[1] = {(cuuint64_t)H * 2};
         const cuuint64_t ad[2] = {(cuuint64_t)I, (cuuint64_t)(pairs + kDenseMaxTokens)}, as[1] = {(cuuint64_t)I * 2};
@@ -685,14 +685,14 @@ int dense8_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, 
     g.wl = fa.wl, g.E = E, g.img_routed0 = layer * E, g.img_shared0 = c.n_layers * E + layer * c.n_shared;
     g.np = np, g.KS = s->KS, g.inv_rms = fa.inv_rms, g.part = s->d_part_dense, g.err = s->d_err;
     a8.store = s->d_resident, a8.img_bytes = s->img_bytes, a8.act16 = s->d_act16;
-    g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kGroup8KStage - 1) / kGroup8KStage * kGroup8KStage;
+    g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + group8_kstage<2>() - 1) / group8_kstage<2>() * group8_kstage<2>();
     a8.scale_off = 0;
     dense8_group_kernel<2><<<s->dense_grid, kGroup8Threads, kGroupSmemBytes, st>>>(s->map8_gate, s->map8_up,
                                                                                    s->map8_x[np / 16 - 1], a8);
     if (timed) CU_TRY(cudaEventRecord(e1, st));
     int seg = 0;
     int splits = dense_down_splits(s, batch, &seg);
-    seg = (seg + kGroup8KStage - 1) / kGroup8KStage * kGroup8KStage;
+    seg = (seg + group8_kstage<1>() - 1) / group8_kstage<1>() * group8_kstage<1>();
     splits = (I + seg - 1) / seg;
     g.rows = H, g.kd = I, g.splits = splits, g.seg = seg;
     a8.scale_off = 2 * I;
