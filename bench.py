@@ -192,7 +192,7 @@ def main():
                          "block the paper overlaps expert prefetch with (Section 4.3.4); 0 = pure MoE stack")
     ap.add_argument("--resident", action="store_true", help="keep every expert in HBM (cache_slots = 0)")
     ap.add_argument("--dense-min-batch", type=int, default=0,
-                    help="smallest batch that takes the tcgen05 path (0: the library's default, 2 for bf16, 4 for fp8)")
+                    help="smallest batch that takes the tcgen05 path (0: the library's default, 2 for bf16, 3 for fp8)")
     ap.add_argument("--no-dense", action="store_true",
                     help="batched steps of resident bf16 stacks on the CUDA-core kernels instead of the tcgen05 ones")
     args = ap.parse_args()
@@ -223,7 +223,7 @@ def main():
     import paper_2606_15453_b200 as P
     st = load_stack(cfg, batch, dev, prefetch_limit=args.prefetch_limit, mode=args.mode,
                     flags=P.FLAG_NO_DENSE if args.no_dense else 0)  # a full replica per rank
-    if args.dense_min_batch:
+    if args.dense_min_batch and not args.no_dense:
         st.set_dense_min_batch(args.dense_min_batch)
     L, K, H = cfg.n_layers, cfg.top_k, cfg.hidden
     n_tok = cfg.profile_tokens + args.warmup + args.steps
@@ -325,7 +325,7 @@ def main():
     # batched steps of resident bf16 stacks: expert FFN on tcgen05 tiles (the library's default threshold)
     dense = persistent and not args.no_dense and (
         (cfg.dtype == "bf16" and batch >= (args.dense_min_batch or 2)) or
-        (cfg.dtype == "fp8" and batch >= (args.dense_min_batch or 4)))
+        (cfg.dtype == "fp8" and batch >= (args.dense_min_batch or 3)))
     top_kernel = "gate_up_kernel"
     if persistent:
         top_kernel = "decode_token_kernel"

@@ -536,7 +536,7 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
 
 // ---- tensor-core path (dense_group.cuh) ---------------------------------------------------
 constexpr int kDenseMinBatch = 2;   // bf16 stacks: measured ahead of the CUDA-core kernels from two sequences on
-constexpr int kDense8MinBatch = 4;  // fp8 stacks (conversion-bound kernels): from four
+constexpr int kDense8MinBatch = 3;  // fp8 stacks (the conversion costs issue slots): level at two, ahead from three
 constexpr int kDenseMaxSplits = 4;
 constexpr int kTokenDenseDynBytes = 220 * 1024;
 
