@@ -474,8 +474,15 @@ __device__ __forceinline__ void finalize_tokens(const RouterArgs &a, int *s_ids,
         for (int v = 0; v < VPL; ++v) {
             const int j = v * kWarp + lane;
             float s = 0.f;
-            if (j < E)
-                for (int c = 0; c < C; ++c) s += __ldcg(a.part + ((size_t)c * B + b) * E + j);
+            for (int c0 = 0; c0 < C; c0 += 8) {  // eight chunk partials per trip to L2, summed in chunk order
+                float t[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    t[i] = (c0 + i < C && j < E) ? __ldcg(a.part + ((size_t)(c0 + i) * B + b) * E + j) : 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (c0 + i < C) s += t[i];
+            }
             z[v] = j < E ? s * inv : -INFINITY;
             if (j < E && a.logits_out) a.logits_out[(size_t)b * E + j] = z[v];
         }
