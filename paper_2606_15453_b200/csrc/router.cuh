@@ -469,21 +469,30 @@ __device__ __forceinline__ void finalize_tokens(const RouterArgs &a, int *s_ids,
         ss = warp_sum(ss);
         const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
         if (lane == 0) a.inv_rms[b] = inv;
+        // partial logits of this lane's experts: eight chunks of every expert per trip to L2,
+        // summed in chunk order
         float z[VPL];
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) z[v] = 0.f;
+        for (int c0 = 0; c0 < C; c0 += 8) {
+            float t[VPL][8];
+#pragma unroll
+            for (int v = 0; v < VPL; ++v)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int j = v * kWarp + lane;
+                    t[v][i] = (c0 + i < C && j < E) ? __ldcg(a.part + ((size_t)(c0 + i) * B + b) * E + j) : 0.f;
+                }
+#pragma unroll
+            for (int v = 0; v < VPL; ++v)
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (c0 + i < C) z[v] += t[v][i];
+        }
 #pragma unroll
         for (int v = 0; v < VPL; ++v) {
             const int j = v * kWarp + lane;
-            float s = 0.f;
-            for (int c0 = 0; c0 < C; c0 += 8) {  // eight chunk partials per trip to L2, summed in chunk order
-                float t[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    t[i] = (c0 + i < C && j < E) ? __ldcg(a.part + ((size_t)(c0 + i) * B + b) * E + j) : 0.f;
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (c0 + i < C) s += t[i];
-            }
-            z[v] = j < E ? s * inv : -INFINITY;
+            z[v] = j < E ? z[v] * inv : -INFINITY;
             if (j < E && a.logits_out) a.logits_out[(size_t)b * E + j] = z[v];
         }
         route_token<VPL>(z, nullptr, s_ids + b * a.tk.K, a.tk, b, lane);

@@ -700,7 +700,7 @@ int dense8_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, 
                                                                                    s->map8_act[np / 16 - 1], a8);
     FfnArgs fc = fa;
     fc.part = s->d_part_dense;
-    dense8_combine_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fc, splits, s->d_xb16);
+    dense8_combine_kernel<<<std::min(8 * s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fc, splits, s->d_xb16);
     if (timed) {
         CU_TRY(cudaEventRecord(e2, st));
         s->spans.push_back(TimedSpan{e0, e1, 2});
@@ -746,7 +746,7 @@ int dense_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, c
                                                                                       s->map_act[np / 16 - 1], g);
     FfnArgs fc = fa;
     fc.part = s->d_part_dense;
-    dense_combine_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fc, splits, s->d_xb);
+    dense_combine_kernel<<<std::min(8 * s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fc, splits, s->d_xb);
     if (timed) {
         CU_TRY(cudaEventRecord(e2, st));
         s->spans.push_back(TimedSpan{e0, e1, 2});
