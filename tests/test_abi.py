@@ -45,3 +45,25 @@ def test_product_does_not_import_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in src.lower() or f == "__init__.py" and False, f
+
+
+def test_binding_constants_match_the_header():
+    text = open(os.path.join(ROOT, "include", "stmoe.h")).read()
+    defs = {m.group(1): int(m.group(2), 0) for m in re.finditer(r"#define\s+(STMOE_[A-Z0-9_]+)\s+\(?(-?\d+)u?\)?", text)}
+    assert defs["STMOE_FLAG_RENORM_TOPK"] == P.FLAG_RENORM_TOPK
+    assert defs["STMOE_FLAG_NO_PERSISTENT"] == P.FLAG_NO_PERSISTENT
+    assert defs["STMOE_FLAG_NO_DENSE"] == P.FLAG_NO_DENSE
+    assert len({defs[k] for k in defs if k.startswith("STMOE_FLAG_")}) == 3      # distinct bits
+    for name, code in P.DTYPE.items():
+        assert defs[{"f32": "STMOE_F32", "bf16": "STMOE_BF16", "fp8": "STMOE_FP8_E4M3"}[name]] == code
+    for name, code in P.MODE.items():
+        assert defs["STMOE_PRED_" + name.upper()] == code
+
+
+def test_dense_entry_points_reject_bad_arguments_without_device_work():
+    lib = P.lib()
+    lib.stmoe_expert_ffn_dense_scratch_bytes.restype = ctypes.c_size_t
+    assert lib.stmoe_expert_ffn_dense_scratch_bytes(0, 128, 128) == 0        # no tokens
+    assert lib.stmoe_expert_ffn_dense_scratch_bytes(65, 128, 128) == 0       # more than 64 tokens
+    assert lib.stmoe_expert_ffn_dense_scratch_bytes(5, 128, 256) >= 16 * (128 + 256) * 2
+    assert lib.stmoe_set_dense_min_batch(None, 4) == -1
