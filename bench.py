@@ -329,9 +329,11 @@ def main():
     top_kernel = "gate_up_kernel"
     if persistent:
         top_kernel = "decode_token_kernel"
-        if dense:   # fp8: per-layer tcgen05 kernels replayed as a graph; bf16: one persistent kernel
-            top_kernel = "decode_token_dense_kernel" if cfg.dtype == "bf16" else "dense8_group_kernel<2>"
-    whole_step = persistent and not (dense and cfg.dtype == "fp8")   # the top kernel is one launch per decode step
+        if dense:   # bf16 and fp8: one persistent kernel with the tcgen05 phases
+            top_kernel = "decode_token_dense_kernel"
+            if cfg.dtype == "fp8" and batch > 4:   # larger fp8 batches: per-layer tcgen05 kernels replayed as a graph
+                top_kernel = "dense8_group_kernel<2>"
+    whole_step = top_kernel.startswith("decode_token")   # the top kernel is one launch per decode step
     per_layer = NCU_TRAFFIC_BYTES_PER_LAYER.get(args.workload) if batch == 1 else None
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

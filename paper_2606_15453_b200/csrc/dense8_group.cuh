@@ -88,33 +88,220 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]
                  : "memory");
 }
 
+// The stage ring of dense_group.cuh plus the hand-off barriers of the two A buffers in tensor memory.
+struct Group8Ring {
+    GroupRing r;  // r.tmem: base of 512 columns
+    uint64_t *afull, *aempty;
+};
+struct Group8Pos {  // per role: ring position and the number of stages handled so far
+    int s = 0;
+    uint32_t ph = 0;
+    int stage_no = 0;
+};
+constexpr int kGroup8ACols = 128;  // tensor-memory columns of one A buffer (two boxes)
+
+__device__ __forceinline__ void group8_ring_init(const Group8Ring &q)
+{
+    for (int b = 0; b < 2; ++b) dmbar_init(&q.afull[b], 8), dmbar_init(&q.aempty[b], 1);
+    group_ring_init(q.r);
+}
+
+// One thread: the TMA loads of this CTA's tasks.  NMAT = 2: gate and up; NMAT = 1: down.
+template <int NMAT>
+__device__ __forceinline__ void group8_produce(const CUtensorMap *map_w0, const CUtensorMap *map_w1,
+                                               const CUtensorMap *map_x, const GroupArgs &a, const Group8Ring &q,
+                                               Group8Pos &pos, int &issued)
+{
+    constexpr int KSTAGE = group8_kstage<NMAT>(), XBOXES = KSTAGE / kDenseKStep;
+    const GroupRing &r = q.r;
+    const int np = a.np, act_bytes = group_act_bytes(np);
+    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
+    const int n_tasks = *a.wl.n_groups * tiles * a.splits;
+    for (int task = blockIdx.x; task < n_tasks && !*r.dead; task += gridDim.x) {
+        const GroupTask t = group_task(a, task);
+        const int ge = a.wl.g_expert[t.g];
+        const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
+        const int xrow = NMAT == 2 ? 0 : a.wl.g_start[t.g];
+        for (int k = t.k0; k < t.k1; k += KSTAGE) {
+            if (!dmbar_wait(&r.empty[pos.s], pos.ph ^ 1u, r.dead)) return;
+            uint8_t *st = r.dsm + (size_t)pos.s * r.slot;
+            // boxes past the end of the reduction dimension are zero-filled and still count
+            dmbar_expect_tx(&r.full[pos.s], (uint32_t)(2 * kGroup8BoxBytes + XBOXES * np * kDenseKStep * 2));
+            tma_load_3d(st, map_w0, k, t.row0, img, &r.full[pos.s]);
+            if (NMAT == 2)
+                tma_load_3d(st + kGroup8BoxBytes, map_w1, k, t.row0, img, &r.full[pos.s]);
+            else
+                tma_load_3d(st + kGroup8BoxBytes, map_w0, k + kGroup8BoxCols, t.row0, img, &r.full[pos.s]);
+#pragma unroll
+            for (int x = 0; x < XBOXES; ++x)
+                tma_load_2d(st + 2 * kGroup8BoxBytes + x * act_bytes, map_x, k + x * kDenseKStep, xrow, &r.full[pos.s]);
+            ++issued;
+            if (++pos.s == r.NS) pos.s = 0, pos.ph ^= 1u;
+        }
+    }
+}
+
+// One thread: MMAs with A from tensor memory, B (activations) from shared memory.  `it` counts
+// the CTA's tasks across calls (accumulator buffer = it & 1).
+template <int NMAT>
+__device__ __forceinline__ void group8_mma(const GroupArgs &a, const Group8Ring &q, Group8Pos &pos, int &it)
+{
+    constexpr int KSTAGE = group8_kstage<NMAT>();
+    const GroupRing &r = q.r;
+    const int np = a.np, act_bytes = group_act_bytes(np);
+    const uint32_t idesc = umma_idesc_f16(np);
+    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
+    const int n_tasks = *a.wl.n_groups * tiles * a.splits;
+    for (int task = blockIdx.x; task < n_tasks && !*r.dead; task += gridDim.x, ++it) {
+        const GroupTask t = group_task(a, task);
+        const int ab = it & 1;
+        if (!dmbar_wait(&r.tempty[ab], (((uint32_t)it >> 1) & 1u) ^ 1u, r.dead)) return;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t acc = r.tmem + ab * 128;
+        bool first = true;
+        for (int k = t.k0; k < t.k1; k += KSTAGE, ++pos.stage_no) {
+            const int buf = pos.stage_no & 1;
+            if (!dmbar_wait(&q.afull[buf], ((uint32_t)pos.stage_no >> 1) & 1u, r.dead)) return;  // converted (implies landed)
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t xs = dsmem_u32(r.dsm + (size_t)pos.s * r.slot + 2 * kGroup8BoxBytes);
+            const uint32_t abuf = r.tmem + 256 + buf * kGroup8ACols;
+#pragma unroll
+            for (int bx = 0; bx < 2; ++bx)
+#pragma unroll
+                for (int j = 0; j < kGroup8BoxCols / 16; ++j) {
+                    // gate/up: both boxes multiply the same activation columns into their own
+                    // accumulators; down: the second box continues the reduction
+                    const int xb = (NMAT == 2 ? 0 : bx * 2) + (j >> 2);
+                    const uint64_t bd = umma_desc_sw128(xs + xb * act_bytes, j & 3);
+                    umma_f16_ts(acc + (NMAT == 2 ? bx * 64 : 0), abuf + bx * 64 + j * 8, bd, idesc,
+                                !first || j > 0 || (NMAT == 1 && bx > 0));
+                }
+            first = false;
+            umma_commit(&q.aempty[buf]);      // this A buffer may be rewritten
+            umma_commit(&r.empty[pos.s]);     // and the stage reloaded
+            if (++pos.s == r.NS) pos.s = 0;
+        }
+        umma_commit(&r.tfull[ab]);
+    }
+}
+
+// Four warps (lg = warp index % 4): thread = one weight row (TMEM lane); applies the row scales.
+template <int NMAT>
+__device__ __forceinline__ void group8_epilogue(const Group8Args &a8, const Group8Ring &q, int &it, int lg, int lane)
+{
+    const GroupArgs &a = a8.g;
+    const GroupRing &r = q.r;
+    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
+    const int n_tasks = *a.wl.n_groups * tiles * a.splits;
+    for (int task = blockIdx.x; task < n_tasks; task += gridDim.x, ++it) {
+        const GroupTask t = group_task(a, task);
+        const int ab = it & 1;
+        const int start = a.wl.g_start[t.g], count = a.wl.g_count[t.g];
+        const int ge = a.wl.g_expert[t.g];
+        const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
+        const int row = t.row0 + lg * kWarp + lane;
+        // bf16 scales behind the three matrices: [gate I | up I | down H]
+        const uint16_t *sc = reinterpret_cast<const uint16_t *>(a8.store + (size_t)img * a8.img_bytes +
+                                                                3 * (size_t)a.rows * a.kd) + a8.scale_off;
+        const int srow = min(row, a.rows - 1);
+        const float s0 = bf16_to_f32(sc[srow]), s1 = NMAT == 2 ? bf16_to_f32(sc[a.rows + srow]) : 0.f;
+        const bool ok = dmbar_wait(&r.tfull[ab], ((uint32_t)it >> 1) & 1u, r.dead);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t acc = r.tmem + ab * 128 + ((uint32_t)(lg * kWarp) << 16);
+        if (NMAT == 2) {
+            for (int i = 0; i < count; ++i) {
+                const int tok = a.wl.pair_token[start + i];
+                const float inv = a.inv_rms[tok];  // W (inv * h) = inv * (W h)
+                const float g = inv * s0 * tmem_ld1(acc + tok), u = inv * s1 * tmem_ld1(acc + 64 + tok);
+                if (ok && row < a.rows) a8.act16[(size_t)(start + i) * a.rows + row] = __float2half_rn(g / (1.f + expf(-g)) * u);
+            }
+        } else {
+            for (int i0 = 0; i0 < count; i0 += 8) {
+                float y[8];
+                tmem_ld8(acc + i0, y);
+                if (ok && row < a.rows) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (i0 + i < count) {
+                            const int slot = a.wl.pair_slot[start + i0 + i];
+                            a.part[((size_t)slot * a.splits + t.z) * a.rows + row] = s0 * y[i];
+                        }
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) dmbar_arrive(&r.tempty[ab]);
+        if (!ok) return;
+    }
+}
+
+// Eight warps, two per lane quarter lq (cw = 0..7: the warp's number among the converters; the
+// warp must sit in lane quarter lq = its warp index % 4): thread = one weight row; the e4m3
+// columns of its box become f16 pairs in tensor memory.
+template <int NMAT>
+__device__ __forceinline__ void group8_convert(const GroupArgs &a, const Group8Ring &q, Group8Pos &pos, int cw, int lq,
+                                               int lane)
+{
+    constexpr int KSTAGE = group8_kstage<NMAT>();
+    const GroupRing &r = q.r;
+    const int bx = cw >> 2;
+    const int row = lq * kWarp + lane, r7 = row & 7;
+    const uint32_t lane_base = r.tmem + 256 + ((uint32_t)(lq * kWarp) << 16) + bx * 64;
+    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
+    const int n_tasks = *a.wl.n_groups * tiles * a.splits;
+    for (int task = blockIdx.x; task < n_tasks; task += gridDim.x) {
+        const GroupTask t = group_task(a, task);
+        for (int k = t.k0; k < t.k1; k += KSTAGE, ++pos.stage_no) {
+            const int buf = pos.stage_no & 1, use = pos.stage_no >> 1;
+            if (!dmbar_wait(&r.full[pos.s], pos.ph, r.dead)) return;                                         // the boxes have landed
+            if (use > 0 && !dmbar_wait(&q.aempty[buf], (uint32_t)(use - 1) & 1u, r.dead)) return;  // its previous MMAs are done
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint8_t *row_ptr = r.dsm + (size_t)pos.s * r.slot + bx * kGroup8BoxBytes + row * 128;
+#pragma unroll
+            for (int c0 = 0; c0 < 8; c0 += 2) {
+                uint32_t v[16];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint4 raw = *reinterpret_cast<const uint4 *>(row_ptr + (((c0 + h) ^ r7) << 4));
+                    uint4 lo, hi;
+                    e4m3x16_to_f16(raw, lo, hi);
+                    v[8 * h] = lo.x, v[8 * h + 1] = lo.y, v[8 * h + 2] = lo.z, v[8 * h + 3] = lo.w;
+                    v[8 * h + 4] = hi.x, v[8 * h + 5] = hi.y, v[8 * h + 6] = hi.z, v[8 * h + 7] = hi.w;
+                }
+                tmem_st16(lane_base + buf * kGroup8ACols + c0 * 8, v);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) dmbar_arrive(&q.afull[buf]);
+            if (++pos.s == r.NS) pos.s = 0, pos.ph ^= 1u;
+        }
+    }
+}
+
+// One projection as a kernel of its own (per-layer launches).
 // NMAT = 2: gate and up projections with the SiLU epilogue; NMAT = 1: down projection.
 template <int NMAT>
 __global__ void __launch_bounds__(kGroup8Threads, 1)
 dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
-                     const __grid_constant__ CUtensorMap map_x, Group8Args a8)
+                    const __grid_constant__ CUtensorMap map_x, Group8Args a8)
 {
-    constexpr int ACOLS = 128;                           // tensor-memory columns of one A buffer (two boxes)
-    constexpr int KSTAGE = group8_kstage<NMAT>(), XBOXES = KSTAGE / kDenseKStep;
     const GroupArgs &a = a8.g;
     extern __shared__ uint8_t dsm_raw[];
     __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2], afull[2], aempty[2];
     __shared__ uint32_t s_tmem;
     __shared__ int s_dead;
     const int tid = threadIdx.x, warp = tid / kWarp, lane = tid % kWarp;
-    const int np = a.np, act_bytes = group_act_bytes(np);
-    const int NS = group8_stages<NMAT>(np), STAGE = group8_stage_bytes<NMAT>(np);
-    uint8_t *dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
-    const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
-    const int n_tasks = *a.wl.n_groups * tiles * a.splits;
-    volatile int *dead = &s_dead;
-
+    Group8Ring q;
+    GroupRing &r = q.r;
+    r.dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
+    r.full = full, r.empty = empty, r.tfull = tfull, r.tempty = tempty, r.dead = &s_dead;
+    q.afull = afull, q.aempty = aempty;
+    r.NS = group8_stages<NMAT>(a.np), r.slot = group8_stage_bytes<NMAT>(a.np);
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) dmbar_init(&full[s], 1), dmbar_init(&empty[s], 1);
-        for (int b = 0; b < 2; ++b) dmbar_init(&tfull[b], 1), dmbar_init(&tempty[b], 4);
-        for (int b = 0; b < 2; ++b) dmbar_init(&afull[b], 8), dmbar_init(&aempty[b], 1);
-        s_dead = NS < 1;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s_dead = r.NS < 1;
+        group8_ring_init(q);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dsmem_u32(&s_tmem)), "r"(512)
@@ -124,171 +311,34 @@ dense8_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_con
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem = s_tmem;
+    r.tmem = s_tmem;
 
     if (warp == 0) {
-        // ---- TMA producer -----------------------------------------------------------------------
         if (lane == 0) {
-            int s = 0, issued = 0;
-            uint32_t ph = 0;
-            for (int task = blockIdx.x; task < n_tasks && !*dead; task += gridDim.x) {
-                const GroupTask t = group_task(a, task);
-                const int ge = a.wl.g_expert[t.g];
-                const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
-                const int xrow = NMAT == 2 ? 0 : a.wl.g_start[t.g];
-                bool ok = true;
-                for (int k = t.k0; k < t.k1 && ok; k += KSTAGE) {
-                    ok = dmbar_wait(&empty[s], ph ^ 1u, dead);
-                    if (!ok) break;
-                    uint8_t *st = dsm + (size_t)s * STAGE;
-                    // boxes past the end of the reduction dimension are zero-filled and still count
-                    dmbar_expect_tx(&full[s], (uint32_t)(2 * kGroup8BoxBytes + XBOXES * np * kDenseKStep * 2));
-                    tma_load_3d(st, &map_w0, k, t.row0, img, &full[s]);
-                    if (NMAT == 2)
-                        tma_load_3d(st + kGroup8BoxBytes, &map_w1, k, t.row0, img, &full[s]);
-                    else
-                        tma_load_3d(st + kGroup8BoxBytes, &map_w0, k + kGroup8BoxCols, t.row0, img, &full[s]);
-#pragma unroll
-                    for (int x = 0; x < XBOXES; ++x)
-                        tma_load_2d(st + 2 * kGroup8BoxBytes + x * act_bytes, &map_x, k + x * kDenseKStep, xrow, &full[s]);
-                    ++issued;
-                    if (++s == NS) s = 0, ph ^= 1u;
-                }
-                if (!ok) break;
-            }
-            for (int i = 0; i < min(issued, NS); ++i) {  // every load that was issued has to land
-                if (s == 0) s = NS, ph ^= 1u;
-                --s;
-                dmbar_wait(&full[s], ph, dead);
-            }
+            Group8Pos pos;
+            int issued = 0;
+            group8_produce<NMAT>(&map_w0, &map_w1, &map_x, a, q, pos, issued);
+            RingPos rp;
+            rp.s = pos.s, rp.ph = pos.ph;
+            group_drain(r, rp, issued);
         }
     } else if (warp == 1) {
-        // ---- MMA issue: A from tensor memory, B (activations) from shared memory -------------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_f16(np);
-            int s = 0, it = 0, stage_no = 0;
-            for (int task = blockIdx.x; task < n_tasks && !*dead; task += gridDim.x, ++it) {
-                const GroupTask t = group_task(a, task);
-                const int ab = it & 1;
-                if (!dmbar_wait(&tempty[ab], (((uint32_t)it >> 1) & 1u) ^ 1u, dead)) break;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t acc = tmem + ab * 128;
-                bool first = true, ok = true;
-                for (int k = t.k0; k < t.k1; k += KSTAGE, ++stage_no) {
-                    const int buf = stage_no & 1;
-                    ok = dmbar_wait(&afull[buf], ((uint32_t)stage_no >> 1) & 1u, dead);  // converted (implies landed)
-                    if (!ok) break;
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t xs = dsmem_u32(dsm + (size_t)s * STAGE + 2 * kGroup8BoxBytes);
-                    const uint32_t abuf = tmem + 256 + buf * ACOLS;
-#pragma unroll
-                    for (int bx = 0; bx < 2; ++bx)
-#pragma unroll
-                        for (int j = 0; j < kGroup8BoxCols / 16; ++j) {
-                            // gate/up: both boxes multiply the same activation columns into their own
-                            // accumulators; down: the second box continues the reduction
-                            const int xb = (NMAT == 2 ? 0 : bx * 2) + (j >> 2);
-                            const uint64_t bd = umma_desc_sw128(xs + xb * act_bytes, j & 3);
-                            umma_f16_ts(acc + (NMAT == 2 ? bx * 64 : 0), abuf + bx * 64 + j * 8, bd, idesc,
-                                        !first || j > 0 || (NMAT == 1 && bx > 0));
-                        }
-                    first = false;
-                    umma_commit(&aempty[buf]);  // this A buffer may be rewritten
-                    umma_commit(&empty[s]);     // and the stage reloaded
-                    if (++s == NS) s = 0;
-                }
-                if (!ok) break;
-                umma_commit(&tfull[ab]);
-            }
+            Group8Pos pos;
+            int it = 0;
+            group8_mma<NMAT>(a, q, pos, it);
         }
     } else if (warp < 6) {
-        // ---- epilogue: thread = one weight row (TMEM lane) -------------------------------------
-        const int lg = warp % 4;
         int it = 0;
-        for (int task = blockIdx.x; task < n_tasks; task += gridDim.x, ++it) {
-            const GroupTask t = group_task(a, task);
-            const int ab = it & 1;
-            const int start = a.wl.g_start[t.g], count = a.wl.g_count[t.g];
-            const int ge = a.wl.g_expert[t.g];
-            const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
-            const int row = t.row0 + lg * kWarp + lane;
-            const uint16_t *sc = reinterpret_cast<const uint16_t *>(a8.store + (size_t)img * a8.img_bytes +
-                                                                    3 * (size_t)a.rows * a.kd) + a8.scale_off;
-            const int srow = min(row, a.rows - 1);
-            const float s0 = bf16_to_f32(sc[srow]), s1 = NMAT == 2 ? bf16_to_f32(sc[a.rows + srow]) : 0.f;
-            const bool ok = dmbar_wait(&tfull[ab], ((uint32_t)it >> 1) & 1u, dead);
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t acc = tmem + ab * 128 + ((uint32_t)(lg * kWarp) << 16);
-            if (NMAT == 2) {
-                for (int i = 0; i < count; ++i) {
-                    const int tok = a.wl.pair_token[start + i];
-                    const float inv = a.inv_rms[tok];
-                    const float g = inv * s0 * tmem_ld1(acc + tok), u = inv * s1 * tmem_ld1(acc + 64 + tok);
-                    if (ok && row < a.rows) a8.act16[(size_t)(start + i) * a.rows + row] = __float2half_rn(g / (1.f + expf(-g)) * u);
-                }
-            } else {
-                for (int i0 = 0; i0 < count; i0 += 8) {
-                    float y[8];
-                    tmem_ld8(acc + i0, y);
-                    if (ok && row < a.rows) {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if (i0 + i < count) {
-                                const int slot = a.wl.pair_slot[start + i0 + i];
-                                a.part[((size_t)slot * a.splits + t.z) * a.rows + row] = s0 * y[i];
-                            }
-                    }
-                }
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) dmbar_arrive(&tempty[ab]);
-            if (!ok) break;
-        }
+        group8_epilogue<NMAT>(a8, q, it, warp % 4, lane);
     } else {
-        // ---- converters: thread = one weight row; its e4m3 columns -> f16 pairs -> tensor memory ----
-        // Two warps share a lane quarter: one weight box of the stage each.
-        const int cw = warp - 6, lq = warp % 4, bx = cw >> 2;
-        const int r = lq * kWarp + lane, r7 = r & 7;
-        const uint32_t lane_base = tmem + 256 + ((uint32_t)(lq * kWarp) << 16) + bx * 64;
-        int s = 0, stage_no = 0;
-        uint32_t ph = 0;
-        bool ok = true;
-        for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x) {
-            const GroupTask t = group_task(a, task);
-            for (int k = t.k0; k < t.k1 && ok; k += KSTAGE, ++stage_no) {
-                const int buf = stage_no & 1, use = stage_no >> 1;
-                ok = dmbar_wait(&full[s], ph, dead);  // the fp8 tile has landed
-                if (ok && use > 0) ok = dmbar_wait(&aempty[buf], (uint32_t)(use - 1) & 1u, dead);  // its previous MMAs are done
-                if (!ok) break;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint8_t *row_ptr = dsm + (size_t)s * STAGE + bx * kGroup8BoxBytes + r * 128;
-#pragma unroll
-                for (int c0 = 0; c0 < 8; c0 += 2) {
-                    uint32_t v[16];
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int c = c0 + h;
-                        const uint4 raw = *reinterpret_cast<const uint4 *>(row_ptr + ((c ^ r7) << 4));
-                        uint4 lo, hi;
-                        e4m3x16_to_f16(raw, lo, hi);
-                        v[8 * h] = lo.x, v[8 * h + 1] = lo.y, v[8 * h + 2] = lo.z, v[8 * h + 3] = lo.w;
-                        v[8 * h + 4] = hi.x, v[8 * h + 5] = hi.y, v[8 * h + 6] = hi.z, v[8 * h + 7] = hi.w;
-                    }
-                    tmem_st16(lane_base + buf * ACOLS + c0 * 8, v);
-                }
-                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) dmbar_arrive(&afull[buf]);
-                if (++s == NS) s = 0, ph ^= 1u;
-            }
-        }
+        Group8Pos pos;
+        group8_convert<NMAT>(a, q, pos, warp - 6, warp % 4, lane);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(r.tmem), "r"(512) : "memory");
     }
     if (tid == 0 && s_dead) *a.err = 1u;
 }

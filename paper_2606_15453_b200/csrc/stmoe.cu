@@ -536,6 +536,7 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
 
 // ---- tensor-core path (dense_group.cuh) ---------------------------------------------------
 constexpr int kDenseMinBatch = 2;   // bf16 stacks: measured ahead of the CUDA-core kernels from two sequences on
+constexpr int kDense8PersistentMaxBatch = 4;
 constexpr int kDense8MinBatch = 3;  // fp8 stacks (the conversion costs issue slots): level at two, ahead from three
 constexpr int kDenseMaxSplits = 4;
 constexpr int kTokenDenseDynBytes = 220 * 1024;
@@ -560,6 +561,8 @@ int encode_map(EncodeTiledFn fn, CUtensorMap *m, void *base, int rank, const cuu
                ? STMOE_OK
                : STMOE_ERR_CUDA;
 }
+
+void *token_dense_kernel(int rdt, bool w8);
 
 int dense_setup(stmoe *s)
 {
@@ -600,7 +603,7 @@ int dense_setup(stmoe *s)
     s->dense_min_batch = kDenseMinBatch;
     s->dense = true;
     if (s->persistent) {  // cooperative launches work and the per-layer buffers exist
-        void *k = s->rdt == STMOE_F32 ? (void *)decode_token_dense_kernel<0> : (void *)decode_token_dense_kernel<1>;
+        void *k = token_dense_kernel(s->rdt, false);
         const int np = (B + 15) / 16 * 16;
         const int slot = std::max(group_stage_bytes<1>(np), group_stage_bytes<2>(np));
         const int need = (int)token_smem(B, c.top_k, c.n_shared) + 1024 + slot;  // at least one stage
@@ -661,6 +664,21 @@ int dense8_setup(stmoe *s)
     s->dense_grid = sm_count();
     s->dense_min_batch = kDense8MinBatch;
     s->dense8 = true;
+    if (s->persistent) {  // cooperative launches work and the per-layer buffers exist
+        void *k = token_dense_kernel(s->rdt, true);
+        const int np = (B + 15) / 16 * 16;
+        const int slot = std::max(group8_stage_bytes<1>(np), group8_stage_bytes<2>(np));
+        const int need = (int)token_smem(B, c.top_k, c.n_shared) + 1024 + slot;  // at least one stage
+        int occ = 0;
+        if (need <= kTokenDenseDynBytes &&
+            cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokenDenseDynBytes) == cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kFfnThreads, kTokenDenseDynBytes) == cudaSuccess &&
+            occ >= 1) {
+            s->dense_persistent = true;
+            s->dense_dyn_bytes = kTokenDenseDynBytes;
+        }
+        (void)cudaGetLastError();
+    }
     return STMOE_OK;
 }
 
@@ -919,6 +937,12 @@ int token_persistent(stmoe *s, int batch, const float *h_in, float *h_out, int32
     return STMOE_OK;
 }
 
+void *token_dense_kernel(int rdt, bool w8)
+{
+    if (w8) return rdt == STMOE_F32 ? (void *)decode_token_dense_kernel<0, 2> : (void *)decode_token_dense_kernel<1, 2>;
+    return rdt == STMOE_F32 ? (void *)decode_token_dense_kernel<0, 1> : (void *)decode_token_dense_kernel<1, 1>;
+}
+
 int dense_down_splits(const stmoe *s, int batch, int *seg)
 {
     const stmoe_config_t &c = s->cfg;
@@ -949,11 +973,19 @@ int token_dense(stmoe *s, int batch, const float *h_in, float *h_out, int32_t *r
     d.splits = dense_down_splits(s, batch, &d.seg);
     d.img_shared_base = c.n_layers * c.n_experts;
     d.dyn_bytes = s->dense_dyn_bytes;
-    d.xb = s->d_xb, d.actb = s->d_actb, d.part = s->d_part_dense;
+    const bool w8 = s->dense8;
+    d.xb = w8 ? (void *)s->d_xb16 : (void *)s->d_xb, d.actb = w8 ? (void *)s->d_act16 : (void *)s->d_actb;
+    d.part = s->d_part_dense, d.store = s->d_resident, d.img_bytes = s->img_bytes;
+    if (w8) {  // the fp8 down projection walks two boxes per stage
+        d.seg = (d.seg + group8_kstage<1>() - 1) / group8_kstage<1>() * group8_kstage<1>();
+        d.splits = (c.inter + d.seg - 1) / d.seg;
+    }
     const int np = (batch + 15) / 16 * 16;
     CU_TRY(cudaMemsetAsync(s->d_barrier, 0, 4, st));
-    void *args[] = {&s->map_gate, &s->map_up, &s->map_down, &s->map_x[np / 16 - 1], &s->map_act[np / 16 - 1], &d};
-    void *k = s->rdt == STMOE_F32 ? (void *)decode_token_dense_kernel<0> : (void *)decode_token_dense_kernel<1>;
+    void *args_bf16[] = {&s->map_gate, &s->map_up, &s->map_down, &s->map_x[np / 16 - 1], &s->map_act[np / 16 - 1], &d};
+    void *args_fp8[] = {&s->map8_gate, &s->map8_up, &s->map8_down, &s->map8_x[np / 16 - 1], &s->map8_act[np / 16 - 1], &d};
+    void **args = w8 ? args_fp8 : args_bf16;
+    void *k = token_dense_kernel(s->rdt, w8);
     CU_TRY(cudaLaunchCooperativeKernel(k, dim3(s->dense_grid), dim3(kFfnThreads), args, (size_t)s->dense_dyn_bytes, st));
     s->launches += 1;
     if (!s->built && s->host_t == c.profile_tokens - 1) {
@@ -1251,7 +1283,9 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, i
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const stmoe_config_t &c = s->cfg;
     const bool build_due = !s->built && s->host_t == c.profile_tokens - 1;
-    if (s->dense_persistent && !s->time_kernels && use_dense(s, batch))
+    // fp8: the persistent kernel is ahead only for small batches (measured on the C4 shape: +6 % at 3
+    // sequences, +2 % at 4, -6 % at 8 and 32, where its ring has a stage less and the predictor two warps)
+    if (s->dense_persistent && !s->time_kernels && use_dense(s, batch) && (!s->dense8 || batch <= kDense8PersistentMaxBatch))
         return token_dense(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
     if (s->persistent && !s->time_kernels && !use_dense(s, batch))
         return token_persistent(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);

@@ -16,6 +16,9 @@
 // SM (the bf16 hidden state, the gated activations) is fenced for the async proxy on both sides
 // of the grid barrier in between.
 #pragma once
+#include <type_traits>
+
+#include "dense8_group.cuh"
 #include "dense_group.cuh"
 #include "token_kernel.cuh"
 
@@ -26,14 +29,18 @@ struct TokenDenseArgs {
     int splits, seg;        // down projection: splits of the reduction dimension, columns per split
     int img_shared_base;    // image index of layer 0's first shared expert (= L * E)
     int dyn_bytes;          // dynamic shared memory of the launch
-    __nv_bfloat16 *xb;      // [64][H]
-    __nv_bfloat16 *actb;    // [pairs + 64][I]
+    void *xb;               // [64][H] bf16 (bf16 weights) or f16 (fp8 weights)
+    void *actb;             // [pairs + 64][I], same type
     float *part;            // [pairs][splits][H]
+    const uint8_t *store;   // fp8: first expert image (for the row scales) and the image pitch
+    unsigned long long img_bytes;
 };
 
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-template <int RDT>
+// RDT: router weight type; WDT: expert weight type, 1 = bf16 (dense_group.cuh), 2 = fp8 e4m3
+// (dense8_group.cuh: warps 6-13 convert, the predictor gets warps 14-15).
+template <int RDT, int WDT>
 __global__ void __launch_bounds__(kFfnThreads, 1)
 decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __grid_constant__ CUtensorMap map_up,
                           const __grid_constant__ CUtensorMap map_down, const __grid_constant__ CUtensorMap map_x,
@@ -44,7 +51,9 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
     extern __shared__ __align__(16) int dyn[];  // work list | ids | prev ids | gate weights | stage ring
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
     __shared__ float s_inv[kMaxBatch];
-    __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2];
+    using XT = typename std::conditional<WDT == 1, __nv_bfloat16, __half>::type;  // activation operand type
+    constexpr int kTmemCols = WDT == 1 ? kGroupTmemCols : 512;
+    __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2], afull[2], aempty[2];
     __shared__ uint32_t s_tmem;
     __shared__ int s_dead;
     const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
@@ -60,18 +69,21 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
     float *s_w = reinterpret_cast<float *>(s_prev + B * K);
     const int list_bytes = (int)sizeof(int) * (4 + 5 * pairs + 3 * B * K);
 
-    GroupRing r;
+    Group8Ring q;
+    GroupRing &r = q.r;
     r.dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dyn) + list_bytes + 1023) & ~(uintptr_t)1023);
     r.full = full, r.empty = empty, r.tfull = tfull, r.tempty = tempty, r.dead = &s_dead;
-    r.slot = max(group_stage_bytes<1>(np), group_stage_bytes<2>(np));
+    q.afull = afull, q.aempty = aempty;
+    r.slot = WDT == 1 ? max(group_stage_bytes<1>(np), group_stage_bytes<2>(np))
+                      : max(group8_stage_bytes<1>(np), group8_stage_bytes<2>(np));
     r.NS = min(kGroupMaxStages, (int)((reinterpret_cast<uint8_t *>(dyn) + d.dyn_bytes - r.dsm) / r.slot));
     if (threadIdx.x == 0) {
         s_dead = r.NS < 1;  // cannot happen with the host's sizing; never run a ring without stages
-        group_ring_init(r);
+        group8_ring_init(q);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dsmem_u32(&s_tmem)),
-                     "r"(kGroupTmemCols)
+                     "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -83,8 +95,16 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
     unsigned target = 0;
     const bool lead = blockIdx.x == 0;
     const bool pred_cta = blockIdx.x == gridDim.x - 1;
-    RingPos ppos, mpos;              // producer / MMA thread
+    RingPos ppos, mpos;              // producer / MMA thread (bf16 weights)
+    Group8Pos ppos8, mpos8, cpos8;   // producer / MMA thread / converter warps (fp8 weights)
     int issued = 0, mit = 0, eit = 0;  // loads issued (producer); tasks done (MMA thread, epilogue threads)
+    XT *xb = static_cast<XT *>(d.xb), *actb = static_cast<XT *>(d.actb);
+    auto to_xt = [](float v) {
+        if constexpr (WDT == 1)
+            return __float2bfloat16_rn(v);
+        else
+            return __float2half_rn(v);
+    };
     const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gthreads = gridDim.x * blockDim.x;
 
     // arguments of the weighted sum that finishes layer lp
@@ -102,14 +122,14 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         // ---- F ---------------------------------------------------------------------------------
         DBG_STAMP(l * 8 + 0);
         if (l == 0) {
-            for (int i = gtid; i < B * H; i += gthreads) d.xb[i] = __float2bfloat16_rn(h[i]);
+            for (int i = gtid; i < B * H; i += gthreads) xb[i] = to_xt(h[i]);
         } else {
             const FfnArgs fp = finish_args(l - 1);
             float *hl = a.hbuf + (size_t)l * B * H;
             for (int i = gtid; i < B * H; i += gthreads) {
                 const float v = finish_value(fp, i / H, i % H, d.splits);
                 hl[i] = v;
-                d.xb[i] = __float2bfloat16_rn(v);
+                xb[i] = to_xt(v);
             }
         }
         fence_async_proxy();
@@ -141,37 +161,73 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
 
         // ---- GU (+ the predictor on one warp of the last CTA) -----------------------------------
         DBG_STAMP(l * 8 + 3);
-        GroupArgs g{};
+        Group8Args g8{};
+        GroupArgs &g = g8.g;
         g.wl = wl, g.E = E, g.img_routed0 = l * E, g.img_shared0 = d.img_shared_base + l * a.n_shared;
-        g.np = np, g.KS = KS, g.inv_rms = s_inv, g.act = d.actb, g.part = d.part, g.err = a.err;
-        g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + group_kstage<2>() - 1) / group_kstage<2>() * group_kstage<2>();
+        g.np = np, g.KS = KS, g.inv_rms = s_inv, g.part = d.part, g.err = a.err;
+        g8.store = d.store, g8.img_bytes = d.img_bytes;
+        if constexpr (WDT == 1)
+            g.act = actb;
+        else
+            g8.act16 = actb;
+        constexpr int kGuStage = WDT == 1 ? group_kstage<2>() : group8_kstage<2>();
+        g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kGuStage - 1) / kGuStage * kGuStage;
+        g8.scale_off = 0;
         if (warp == 0) {
             if (lane == 0) {
                 fence_async_proxy();
-                group_produce<2>(&map_gate, &map_up, &map_x, g, r, ppos, issued);
+                if constexpr (WDT == 1)
+                    group_produce<2>(&map_gate, &map_up, &map_x, g, r, ppos, issued);
+                else
+                    group8_produce<2>(&map_gate, &map_up, &map_x, g, q, ppos8, issued);
             }
         } else if (warp == 1) {
-            if (lane == 0) group_mma<2>(g, r, mpos, mit);
+            if (lane == 0) {
+                if constexpr (WDT == 1)
+                    group_mma<2>(g, r, mpos, mit);
+                else
+                    group8_mma<2>(g, q, mpos8, mit);
+            }
         } else if (warp < 6) {
-            group_epilogue<2>(g, r, eit, warp % 4, lane);
+            if constexpr (WDT == 1)
+                group_epilogue<2>(g, r, eit, warp % 4, lane);
+            else
+                group8_epilogue<2>(g8, q, eit, warp % 4, lane);
             fence_async_proxy();  // the gated activations are fetched by TMA in the next phase
-        } else if (pred_cta) {  // the ten warps without a role in this phase
-            predictor_step_group(a, l, s_ids, s_prev, warp - 6, NW - 6, lane);
+        } else if (WDT == 2 && warp < 14) {
+            group8_convert<2>(g, q, cpos8, warp - 6, warp % 4, lane);
+        } else if (pred_cta) {  // the warps without a role in this phase: ten (bf16) or two (fp8)
+            constexpr int kFirst = WDT == 1 ? 6 : 14;
+            predictor_step_group(a, l, s_ids, s_prev, warp - kFirst, NW - kFirst, lane);
         }
         grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 4);
         DBG_STAMP(l * 8 + 5);
 
         // ---- D ---------------------------------------------------------------------------------
         g.rows = H, g.kd = I, g.splits = d.splits, g.seg = d.seg;
+        g8.scale_off = 2 * I;
         if (warp == 0) {
             if (lane == 0) {
                 fence_async_proxy();
-                group_produce<1>(&map_down, &map_down, &map_act, g, r, ppos, issued);
+                if constexpr (WDT == 1)
+                    group_produce<1>(&map_down, &map_down, &map_act, g, r, ppos, issued);
+                else
+                    group8_produce<1>(&map_down, &map_down, &map_act, g, q, ppos8, issued);
             }
         } else if (warp == 1) {
-            if (lane == 0) group_mma<1>(g, r, mpos, mit);
+            if (lane == 0) {
+                if constexpr (WDT == 1)
+                    group_mma<1>(g, r, mpos, mit);
+                else
+                    group8_mma<1>(g, q, mpos8, mit);
+            }
         } else if (warp < 6) {
-            group_epilogue<1>(g, r, eit, warp % 4, lane);
+            if constexpr (WDT == 1)
+                group_epilogue<1>(g, r, eit, warp % 4, lane);
+            else
+                group8_epilogue<1>(g8, q, eit, warp % 4, lane);
+        } else if (WDT == 2 && warp < 14) {
+            group8_convert<1>(g, q, cpos8, warp - 6, warp % 4, lane);
         }
         for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
         grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 6);
@@ -182,12 +238,15 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         const FfnArgs fl = finish_args(L - 1);
         for (int i = gtid; i < B * H; i += gthreads) a.h_out[i] = finish_value(fl, i / H, i % H, d.splits);
     }
-    if (warp == 0 && lane == 0) group_drain(r, ppos, issued);
+    if (warp == 0 && lane == 0) {
+        if (WDT == 2) ppos.s = ppos8.s, ppos.ph = ppos8.ph;
+        group_drain(r, ppos, issued);
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (threadIdx.x == 0 && s_dead) *a.err = 1u;
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(r.tmem), "r"(kGroupTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(r.tmem), "r"(kTmemCols) : "memory");
     }
 }
 
