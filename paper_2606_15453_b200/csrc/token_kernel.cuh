@@ -211,8 +211,10 @@ __device__ __forceinline__ void grid_barrier(unsigned *counter, unsigned *err, u
     __syncthreads();
     if (dbg_idx >= 0) DBG_STAMP(dbg_idx);
     if (threadIdx.x == 0 && !*s_dead) {
-        __threadfence();
-        atomicAdd(counter, 1u);
+        // Release at GPU scope: the CTA barrier above orders every thread's writes before this
+        // thread's arrival (cumulativity), so no separate fence is needed; the acquiring load below
+        // and the CTA barrier after it do the same on the way out.
+        asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(counter), "r"(1u) : "memory");
         int spins = 0;
         for (;;) {
             unsigned seen;
@@ -224,7 +226,6 @@ __device__ __forceinline__ void grid_barrier(unsigned *counter, unsigned *err, u
                 break;
             }
         }
-        __threadfence();
     }
     __syncthreads();
 }
