@@ -218,17 +218,23 @@ __device__ __forceinline__ float finish_value(const FfnArgs &a, int b, int c, in
 __device__ __forceinline__ void finish_rows(const FfnArgs &a, int r0, int nrows, int want_per_row, int S, int lane)
 {
     const int H = a.H;
-    __threadfence();
+    // The warp's lanes have stored their partial sums; the warp barrier orders those stores before
+    // lane 0's counter update, whose release makes them visible to whoever reads the count, and whose
+    // acquire (handed to the other lanes by the shuffle) orders the finisher's loads after every
+    // earlier contributor's release: one acquire-release atomic instead of two full fences.
     __syncwarp();
     for (int rr = r0; rr < r0 + nrows;) {
         const int tile = rr / kTileRows;
         const int n = min(r0 + nrows, (tile + 1) * kTileRows) - rr;
         const int tile_rows = min(kTileRows, H - tile * kTileRows);
         unsigned prev = 0;
-        if (lane == 0) prev = atomicAdd(a.tile_done + tile, (unsigned)n);
+        if (lane == 0)
+            asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], %2;"
+                         : "=r"(prev)
+                         : "l"(a.tile_done + tile), "r"((unsigned)n)
+                         : "memory");
         prev = __shfl_sync(kFull, prev, 0);
         if (prev + n == (unsigned)(want_per_row * tile_rows)) {
-            __threadfence();
             if (lane == 0) a.tile_done[tile] = 0u;
             const int c = tile * kTileRows + lane;
             if (lane < tile_rows)
