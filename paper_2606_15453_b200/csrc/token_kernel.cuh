@@ -215,17 +215,21 @@ __device__ __forceinline__ void grid_barrier(unsigned *counter, unsigned *err, u
         // thread's arrival (cumulativity), so no separate fence is needed; the acquiring load below
         // and the CTA barrier after it do the same on the way out.
         asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(counter), "r"(1u) : "memory");
+        // poll with relaxed loads (the error word only now and then), acquire once on the way out
         int spins = 0;
         for (;;) {
             unsigned seen;
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+            asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
             if (seen >= target) break;
-            if (++spins > kBarrierSpinLimit || *((volatile unsigned *)err)) {
+            if (++spins > kBarrierSpinLimit || ((spins & 255) == 0 && *((volatile unsigned *)err))) {
                 *err = 1u;
                 *s_dead = 1;
                 break;
             }
         }
+        unsigned seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+        (void)seen;
     }
     __syncthreads();
 }
