@@ -227,9 +227,7 @@ __device__ __forceinline__ void grid_barrier(unsigned *counter, unsigned *err, u
                 break;
             }
         }
-        unsigned seen;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
-        (void)seen;
+        asm volatile("{.reg .u32 t;\n\tld.acquire.gpu.global.u32 t, [%0];}" ::"l"(counter) : "memory");
     }
     __syncthreads();
 }
