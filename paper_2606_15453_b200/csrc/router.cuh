@@ -535,12 +535,16 @@ __global__ void __launch_bounds__(512) router_fused_kernel(RouterArgs a)
     const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
     router_tasks<DT, true>(a, blockIdx.x * NW + warp, gridDim.x * NW, lane);
     pdl_wait();  // warps without a task: nothing below may run ahead of the previous kernel either
-    __threadfence();
+    // arrival: the CTA barrier orders the warps' partial stores before thread 0's acquire-release
+    // atomic, which publishes them and, for the CTA that arrives last, brings in everyone else's
     __syncthreads();
-    if (threadIdx.x == 0) s_last = (atomicAdd(a.arrivals, 1u) == gridDim.x - 1);
+    if (threadIdx.x == 0) {
+        unsigned prev;
+        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(prev) : "l"(a.arrivals) : "memory");
+        s_last = prev == gridDim.x - 1;
+    }
     __syncthreads();
     if (!s_last) return;
-    __threadfence();
     if (threadIdx.x == 0) *a.arrivals = 0u;
     router_finalize<DT>(a, s_ids, s_scan, NW);
 }
