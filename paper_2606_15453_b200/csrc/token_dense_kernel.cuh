@@ -1,14 +1,15 @@
-// One decode step of a resident bf16 stack with several sequences as a single persistent kernel
-// whose expert FFN runs on the tensor cores (the batched counterpart of token_kernel.cuh).
+// One decode step of a resident bf16 or fp8 stack with several sequences as a single persistent
+// kernel whose expert FFN runs on the tensor cores (the batched counterpart of token_kernel.cuh).
 //
 // One 512-thread CTA per SM, launched cooperatively, walks the layers:
 //   F   weighted sum + residual of the previous layer from its down-projection partial sums
-//       (layer 0: the input), written as fp32 (router, residual) and bf16 (gate/up operand)
+//       (layer 0: the input), written as fp32 (router, residual) and bf16 / f16 (gate/up operand)
 //                                                                          -> grid barrier
 //   R   split-K router GEMV tasks over all warps of the grid               -> grid barrier
 //   T   every CTA runs softmax / top-K / grouping (one work-list entry per expert) itself
 //   GU  gate/up tiles on tcgen05: warp 0 feeds TMA, warp 1 issues MMAs, warps 2-5 read the
-//       accumulators; the predictor (Algorithms 1-3) runs on the other ten warps of the last CTA
+//       accumulators (fp8 weights: warps 6-13 widen them into tensor memory); the predictor
+//       (Algorithms 1-3) runs on the remaining warps of the last CTA
 //                                                                          -> grid barrier
 //   D   down-projection tiles the same way                                 -> grid barrier
 // The stage ring, its barriers and the tensor-memory columns are set up once and carried through
