@@ -186,6 +186,8 @@ def main():
     ap.add_argument("--cpu-sample-layers", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefetch-limit", type=int, default=0, help="offloaded stacks: copies per layer step")
+    ap.add_argument("--prefetch-min-score", type=int, default=0,
+                    help="offloaded stacks: prefetch only predictions with at least this score")
     ap.add_argument("--mode", default="st", choices=["off", "temporal", "spatial", "st"])
     ap.add_argument("--inter-layer-gap-us", type=float, default=0.0,
                     help="idle the compute stream this long after every layer: a stand-in for the attention "
@@ -223,6 +225,8 @@ def main():
     import paper_2606_15453_b200 as P
     st = load_stack(cfg, batch, dev, prefetch_limit=args.prefetch_limit, mode=args.mode,
                     flags=P.FLAG_NO_DENSE if args.no_dense else 0)  # a full replica per rank
+    if args.prefetch_min_score:
+        st.set_prefetch_min_score(args.prefetch_min_score)
     if args.dense_min_batch and not args.no_dense:
         st.set_dense_min_batch(args.dense_min_batch)
     L, K, H = cfg.n_layers, cfg.top_k, cfg.hidden
@@ -383,7 +387,8 @@ def main():
                   "exposed_ms": s1["exposed_ms"] - s0["exposed_ms"],
                   "hidden_frac": 1.0 - (s1["exposed_ms"] - s0["exposed_ms"])
                   / max(s1["transfer_ms"] - s0["transfer_ms"], 1e-9),
-                  "prefetch_limit": args.prefetch_limit, "mode": args.mode,
+                  "prefetch_limit": args.prefetch_limit, "prefetch_min_score": args.prefetch_min_score,
+                  "mode": args.mode,
                   "inter_layer_gap_us": args.inter_layer_gap_us},
     }
     if world == 1 and not args.no_cpu_baseline:

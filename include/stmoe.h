@@ -165,6 +165,13 @@ int stmoe_max_predicted(const stmoe_t *s); /* min(E, K*K+K) */
  * Off by default. */
 int stmoe_set_kernel_timing(stmoe_t *s, int on);
 
+/* Offloaded stacks: prefetch only queue entries whose score (Eq. 1, summed over the batch's
+ * sequences) is at least min_score; entries below it are ignored as if they had not been
+ * predicted (they are neither copied nor protected from eviction).  0 (default) prefetches the
+ * whole predicted set, the paper's policy; higher values trade recall for fewer wasted copies.
+ * Between decode steps; routing, outputs and predictor tables are unaffected. */
+int stmoe_set_prefetch_min_score(stmoe_t *s, int min_score);
+
 /* Smallest batch that takes the tensor-core FFN path (see STMOE_FLAG_NO_DENSE); between decode
  * steps.  min_batch < 2 or a stack without that path: STMOE_ERR_BAD_ARG. */
 int stmoe_set_dense_min_batch(stmoe_t *s, int min_batch);

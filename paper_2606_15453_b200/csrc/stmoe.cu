@@ -323,6 +323,7 @@ struct stmoe {
     bool dense_persistent = false;  // one cooperative kernel per decode step (token_dense_kernel.cuh)
     int dense_dyn_bytes = 0;
 
+    int prefetch_min_score = 0;  // queue entries below this summed score are not prefetched
     SlotCache cache;
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_route = nullptr;
@@ -502,7 +503,8 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
     }
 
     // prefetch the queued experts of the next layer (priority order)
-    const int nq = s->h_queue[0];
+    int nq = s->h_queue[0];
+    while (nq > 0 && s->h_queue[1 + E + nq - 1] < s->prefetch_min_score) --nq;  // the queue is in score order
     for (int i = 0; i < nq; ++i) {
         const int32_t sl = ch.slot_of[(size_t)next * E + s->h_queue[1 + i]];
         if (sl >= 0) ch.protect(sl);
@@ -1221,6 +1223,13 @@ int stmoe_set_kernel_timing(stmoe_t *s, int on)
 {
     if (!s) return STMOE_ERR_BAD_ARG;
     s->time_kernels = on != 0;
+    return STMOE_OK;
+}
+
+int stmoe_set_prefetch_min_score(stmoe_t *s, int min_score)
+{
+    if (!s || min_score < 0 || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
+    s->prefetch_min_score = min_score;
     return STMOE_OK;
 }
 

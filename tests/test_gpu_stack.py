@@ -13,9 +13,11 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def _teacher_forced(cfg, B, tokens, mode="st", prefetch_limit=0, flags=0):
+def _teacher_forced(cfg, B, tokens, mode="st", prefetch_limit=0, flags=0, min_score=0):
     """Feed both sides the oracle's hidden state at every (token, layer)."""
     pr = Pair(cfg, B, mode=mode, prefetch_limit=prefetch_limit, flags=flags)
+    if min_score:
+        pr.stack.set_prefetch_min_score(min_score)
     x = stacks.token_inputs(cfg, B, tokens).numpy()
     replay = O.Predictor(cfg.n_layers, cfg.n_experts, cfg.top_k, B, cfg.profile_tokens, mode)
     cache = O.CacheModel(cfg.cache_slots, cfg.n_layers, cfg.n_experts) if cfg.cache_slots else None
@@ -31,7 +33,8 @@ def _teacher_forced(cfg, B, tokens, mode="st", prefetch_limit=0, flags=0):
             assert g["n_pred"].tolist() == rp["n_pred"].tolist(), (t, l)
             assert (g["pred_ids"] == rp["pred_ids"]).all(), (t, l)
             if cache is not None:
-                cache.step(l, np.unique(g["ids"]), (l + 1) % cfg.n_layers, rp["queue_ids"],
+                cache.step(l, np.unique(g["ids"]), (l + 1) % cfg.n_layers,
+                           rp["queue_ids"][rp["queue_score"] >= min_score],
                            prefetch_limit)
             h = o["h_out"]
     assert pr.stack.export_state() == replay.export()
@@ -164,6 +167,16 @@ def test_decode_token_paths_agree(B, shape):
         for k in ("runtime_steps", "routed", "predicted", "hits", "decode_steps", "near_ties"):
             assert st[k] == ref_stats[k], k
     assert ref_stats["kernel_launches"] < results[1][2]["kernel_launches"]
+
+
+def test_prefetch_min_score_policy_matches_filtered_oracle_queue():
+    """Prefetching only predictions with a score of at least m = the cache model driven by the
+    oracle's queue cut at that score; fewer copies are issued than with the whole predicted set."""
+    cfg = stacks.CONFIGS["C0"].scaled(cache_slots=12, profile_tokens=6)
+    _, all_ = _teacher_forced(cfg, 2, 20)
+    _, cut = _teacher_forced(cfg, 2, 20, min_score=5)
+    assert 0 < cut["prefetch_issued"] < all_["prefetch_issued"]
+    assert cut["hits"] == all_["hits"] and cut["predicted"] == all_["predicted"]   # the predictor itself is untouched
 
 
 def test_argument_and_state_errors():
