@@ -292,3 +292,67 @@ def test_replacement_takes_lowest_missing_id_and_never_duplicates():
     O.update(E, K, [3], [1, 2], ids, conf)
     assert ids[3].tolist() == [1, 2, 7] and conf[3].tolist() == [1, 1, 0]
     assert ids[0].tolist() == [1, 2, 7]                      # other rows untouched
+
+
+GOLDEN_B2 = os.path.join(os.path.dirname(__file__), "golden", "cct_batch2_example.txt")
+
+
+def test_worked_example_batch_of_two_pins_queue_scores():
+    """Hand-worked two-sequence steps: the prefetch queue carries the sum of the sequences'
+    Eq. 1 scores (not their maximum, not one sequence's), ordered by (score descending, id
+    ascending); the shared table is updated sequence 0 first."""
+    recs = []
+    with open(GOLDEN_B2) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                key, val = line.split(":", 1)
+                recs.append((key.strip(), val.strip()))
+
+    def queue(val):
+        pairs = [p.split(":") for p in val.split()]
+        return [int(a) for a, _ in pairs], [int(b) for _, b in pairs]
+
+    def token(val):
+        seqs = [[list(map(int, side.split())) for side in s.split("->")] for s in val.split("|")]
+        return [s[0] for s in seqs], [s[1] for s in seqs]          # layer-0 routing, layer-1 routing
+
+    E, K = 4, 2
+    p = O.Predictor(L=2, E=E, K=K, B=2, P=2, mode="st")
+    it = iter(recs)
+    out1 = None
+    for _ in range(2):                                             # profiling
+        key, val = next(it)
+        assert key == "token"
+        r0, r1 = token(val)
+        out0 = p.step(0, r0)
+        assert out0["queue_ids"].size == 0 and (out0["n_pred"] == 0).all()
+        out1 = p.step(1, r1)
+    tb = p.tables()
+    assert tb["built"] == 1 and tb["t"] == 2
+    assert tb["cct_id"][0].tolist() == _rows(next(it)[1])
+    assert tb["cct_conf"][0].tolist() == _rows(next(it)[1])
+    key, val = next(it)
+    assert key == "queue_next"
+    ids, sc = queue(val)
+    assert out1["queue_ids"].tolist() == ids and out1["queue_score"].tolist() == sc
+
+    for key, val in it:
+        assert key == "token"
+        r0, r1 = token(val)
+        tb = p.tables()
+        want = [[int(v) for v in next(it)[1].split()] for _ in range(2)]
+        for b in range(2):                                         # Algorithm 2 + Eq. 1 per sequence
+            score, _, mask = O.predict(E, K, r0[b], tb["cct_id"][0].copy(), tb["cct_conf"][0].copy(),
+                                       tb["HT"][b, 1].copy())
+            assert score.tolist() == want[b]
+        out0 = p.step(0, r0)
+        ids, sc = queue(next(it)[1])
+        assert out0["queue_ids"].tolist() == ids and out0["queue_score"].tolist() == sc
+        for b in range(2):
+            n = out0["n_pred"][b]
+            assert out0["pred_ids"][b, :n].tolist() == [f for f in range(E) if want[b][f] >= 2]
+        out1 = p.step(1, r1)
+        assert p.tables()["cct_conf"][0].tolist() == _rows(next(it)[1])
+        ids, sc = queue(next(it)[1])
+        assert out1["queue_ids"].tolist() == ids and out1["queue_score"].tolist() == sc
