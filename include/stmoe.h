@@ -144,7 +144,11 @@ int stmoe_load_experts(stmoe_t *s, int layer, int first_expert, int count, const
  * Resident stacks: the call only enqueues work on cuda_stream.  Stacks with cache_slots > 0:
  * the call waits on the host (bounded, STMOE_ERR_TIMEOUT) for this layer's routing, issues
  * demand and prefetch copies on the library's copy stream and fences them with events.
- * Prediction never changes routing or output (Section 4.3.4). */
+ * Prediction never changes routing or output (Section 4.3.4).
+ * A step that returns an error other than STMOE_ERR_BAD_ARG / STMOE_ERR_STATE may already have
+ * applied Algorithm 3 and the history overwrite for this layer; the stack is then marked failed
+ * and every further step returns STMOE_ERR_STATE until stmoe_import_state restores a consistent
+ * image (retrying the layer would apply the update twice). */
 int stmoe_decode_step(stmoe_t *s, int layer, int batch, const float *h_in, float *h_out,
                       int32_t *routed_ids, float *routed_w, int32_t *predicted_ids,
                       int32_t *n_predicted, uint32_t *flags, void *cuda_stream);
@@ -230,7 +234,10 @@ int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t *ids, cons
  *   - Returns STMOE_ERR_TOO_LARGE when stmoe_moe_ffn_scratch_bytes(batch, top_k, hidden, inter)
  *     exceeds 8 MiB (for example batch 64, top_k 8, hidden 4096, inter 14336).
  *   - The first call on each device looks up the area's device address (with that device
- *     current); make that first call before starting any stream capture.
+ *     current); make that first call before starting any stream capture, and from one host
+ *     thread (later calls may come from any thread).
+ *   - Arguments out of range are STMOE_ERR_BAD_ARG, as in stmoe_moe_ffn; only a well-formed
+ *     problem that does not fit is STMOE_ERR_TOO_LARGE.
  *   - All calls on a device share the one area, which keeps whatever the last call left; the
  *     call clears the counters that must start at zero itself.  Two calls whose kernels can
  *     overlap on the GPU (different streams, no ordering between them) race on it: order

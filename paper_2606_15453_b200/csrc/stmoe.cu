@@ -274,6 +274,7 @@ struct stmoe {
     int next_layer = 0;
     int64_t host_t = 0;
     bool built = false;
+    bool failed = false;  // a layer step broke off after the predictor had run: tables and counters are ahead of next_layer
 
     uint8_t *d_router = nullptr;    // [L][E][H]
     uint8_t *d_resident = nullptr;  // [L][E] images (resident stacks)
@@ -1237,6 +1238,10 @@ int stmoe_set_dense_min_batch(stmoe_t *s, int min_batch)
 {
     if (!s || !(s->dense || s->dense8) || min_batch < 2 || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
     s->dense_min_batch = min_batch;
+    // a captured decode step holds the kernels of the path chosen at capture time: drop it so
+    // the next step is captured again with the new threshold
+    if (s->graph_exec) cudaGraphExecDestroy(s->graph_exec), s->graph_exec = nullptr;
+    memset(s->graph_key, 0, sizeof(s->graph_key));
     return STMOE_OK;
 }
 
@@ -1275,11 +1280,12 @@ int stmoe_decode_step(stmoe_t *s, int layer, int batch, const float *h_in, float
 {
     if (!s || !h_in || !h_out || batch < 1 || batch > s->cfg.max_batch || layer < 0 || layer >= s->cfg.n_layers)
         return STMOE_ERR_BAD_ARG;
-    if (layer != s->next_layer) return STMOE_ERR_STATE;
+    if (s->failed || layer != s->next_layer) return STMOE_ERR_STATE;
     int rc = layer_step(s, layer, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted,
                         flags, (cudaStream_t)cuda_stream);
     if (rc == STMOE_OK) rc = join_side(s, (cudaStream_t)cuda_stream);
     if (rc == STMOE_OK) s->next_layer = (layer + 1) % s->cfg.n_layers;
+    else s->failed = true;  // Algorithm 3 and the history overwrite of this step may already have run
     return rc;
 }
 
@@ -1288,7 +1294,7 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, i
                        void *cuda_stream)
 {
     if (!s || !h_in || !h_out || batch < 1 || batch > s->cfg.max_batch) return STMOE_ERR_BAD_ARG;
-    if (s->next_layer != 0) return STMOE_ERR_STATE;
+    if (s->failed || s->next_layer != 0) return STMOE_ERR_STATE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const stmoe_config_t &c = s->cfg;
     const bool build_due = !s->built && s->host_t == c.profile_tokens - 1;
@@ -1298,8 +1304,11 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, i
         return token_dense(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
     if (s->persistent && !s->time_kernels && !use_dense(s, batch))
         return token_persistent(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
-    if (offloaded(s) || s->time_kernels || s->graph_off || build_due)
-        return token_eager(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
+    if (offloaded(s) || s->time_kernels || s->graph_off || build_due) {
+        const int rc = token_eager(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
+        if (rc != STMOE_OK) s->failed = true;
+        return rc;
+    }
 
     const void *key[9] = {(const void *)(intptr_t)batch, h_in, h_out, routed_ids, routed_w, predicted_ids,
                           n_predicted, flags, st};
@@ -1408,7 +1417,7 @@ int stmoe_import_state(stmoe_t *s, const void *buf, size_t bytes)
     if (!s || !buf) return STMOE_ERR_BAD_ARG;
     const stmoe_config_t &c = s->cfg;
     if (bytes != state_bytes(c)) return STMOE_ERR_BAD_ARG;
-    if (s->next_layer != 0) return STMOE_ERR_STATE;
+    if (s->next_layer != 0 && !s->failed) return STMOE_ERR_STATE;
     const uint8_t *o = (const uint8_t *)buf;
     int32_t hdr[8];
     memcpy(hdr, o, 32), o += 32;
@@ -1432,6 +1441,7 @@ int stmoe_import_state(stmoe_t *s, const void *buf, size_t bytes)
     CU_TRY(cudaMemset(s->pst.pred_valid, 0, (size_t)c.max_batch * 4));
     s->host_t = t;
     s->built = hdr[7] != 0;
+    s->failed = false, s->next_layer = 0;  // the image is a state between decode steps
     return STMOE_OK;
 }
 
@@ -1467,7 +1477,7 @@ int stmoe_predictor_step(stmoe_t *s, int layer, int batch, const int32_t *routed
 {
     if (!s || !routed_ids || batch < 1 || batch > s->cfg.max_batch || layer < 0 || layer >= s->cfg.n_layers)
         return STMOE_ERR_BAD_ARG;
-    if (layer != s->next_layer) return STMOE_ERR_STATE;
+    if (s->failed || layer != s->next_layer) return STMOE_ERR_STATE;
     const stmoe_config_t &c = s->cfg;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     int32_t *ids = s->d_ids + (size_t)layer * c.max_batch * c.top_k;
@@ -1487,7 +1497,7 @@ size_t stmoe_expert_image_bytes(int hidden, int inter, int weight_dtype)
 static size_t ffn_scratch_layout(int B, int K, int H, int I, int E, int S, size_t *o_tab, size_t *o_act, size_t *o_part,
                                  size_t *o_tiles)
 {
-    size_t o = round_up(sizeof(int) * (size_t)(4 + 5 * B * K), 256);
+    size_t o = round_up(sizeof(int) * (4 + 5 * (size_t)B * K), 256);
     *o_tab = o, o += round_up(sizeof(void *) * (size_t)E, 256);
     *o_act = o, o += round_up(sizeof(float) * (size_t)B * K * I, 256);
     *o_part = o, o += round_up(sizeof(float) * (size_t)B * K * S * H, 256);
@@ -1564,8 +1574,13 @@ extern "C" int stmoe_moe_ffn(const float *h, const float *inv_rms, const int32_t
     fa.H = hidden, fa.I = inter, fa.E = n_experts, fa.S = S;
     fa.w = w, fa.h_out = h_out, fa.tile_done = (unsigned *)(sc + o_tiles);
     fa.B = batch, fa.K = top_k, fa.n_shared = 0, fa.residual_scale = residual_scale;
-    static FfnPlan plans[3][2];
-    FfnPlan &plan = plans[weight_dtype][mt == 1 ? 0 : 1];
+    // launch shapes per device ordinal (the SM count differs between devices); filled on first use,
+    // and a repeated fill by a racing host thread writes the same values
+    static FfnPlan plans[64][3][2];
+    int dev = 0;
+    CU_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return STMOE_ERR_BAD_ARG;
+    FfnPlan &plan = plans[dev][weight_dtype][mt == 1 ? 0 : 1];
     if (plan.grid_down == 0) plan = make_plan(weight_dtype, mt);
     return run_ffn(nullptr, weight_dtype, mt, plan, fa, st);
 }
@@ -1584,7 +1599,12 @@ extern "C" int stmoe_moe_ffn_static(const float *h, const float *inv_rms, const 
                                     const void *experts, int weight_dtype, int batch, int n_experts, int top_k,
                                     int hidden, int inter, float residual_scale, float *h_out, void *cuda_stream)
 {
-    if (batch < 1 || top_k < 1 || hidden < 16 || inter < 16) return STMOE_ERR_BAD_ARG;
+    // the same argument checks as stmoe_moe_ffn, before the capacity check, so that a malformed
+    // call reads as a bad argument and the size below is computed from values in range
+    if (!h || !ids || !w || !experts || !h_out || batch < 1 || batch > kMaxBatch || n_experts < 1 ||
+        n_experts > kMaxExperts || top_k < 1 || top_k > kMaxTopK || top_k > n_experts || hidden < 16 ||
+        hidden % 16 || inter < 16 || inter % 16 || weight_dtype < STMOE_F32 || weight_dtype > STMOE_FP8_E4M3)
+        return STMOE_ERR_BAD_ARG;
     if (stmoe_moe_ffn_scratch_bytes(batch, top_k, hidden, inter) > (size_t)STMOE_STATIC_SCRATCH_BYTES)
         return STMOE_ERR_TOO_LARGE;
     int dev = -1;

@@ -11,7 +11,6 @@ import torch
 
 import paper_2606_15453_b200 as P
 from datagen import rng, stacks
-from helpers import TOL, rel_err
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -44,9 +43,42 @@ def test_static_scratch_matches_caller_scratch_on_two_calls_in_a_row():
         P.moe_ffn_static(h, inv, ids, w, img, dt, E, H, I, 0.1, got)
         torch.cuda.synchronize()
         assert torch.isfinite(got).all()
-        assert rel_err(got.cpu().numpy(), want.cpu().numpy()) <= TOL[dt]
-        moe_w, moe_g = (want - h).cpu().numpy() / 0.1, (got - h).cpu().numpy() / 0.1
-        assert rel_err(moe_g, moe_w) <= 1e-3
+        # the two entry points run the same kernels on the same inputs in the same fixed summation
+        # order, so the results must agree bit for bit; a tolerance would hide a slip in the layout
+        # of the built-in area that disturbs a single partial sum
+        assert torch.equal(got, want)
+
+
+def test_static_entry_point_allocates_no_device_memory():
+    """What the entry point is for: after its first call on the device (module load, address
+    look-up) further calls, at several problem sizes, leave the device's free memory and the
+    caching allocator's reservations exactly as they were."""
+    E, K, H, I, dt = 6, 2, 512, 1408, "bf16"
+    problems = [_problem(7 + i, B, E, K, H, I, dt) for i, B in enumerate((1, 4, 9, 2))]
+    outs = [torch.empty(B, H, device=DEV) for B in (1, 4, 9, 2)]
+    img, h, inv, ids, w = problems[0]
+    P.moe_ffn_static(h, inv, ids, w, img, dt, E, H, I, 0.1, outs[0])      # first call: set-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    reserved0, mallocs0 = torch.cuda.memory_reserved(), torch.cuda.memory_stats()["allocation.all.allocated"]
+    for _ in range(3):
+        for (img, h, inv, ids, w), out in zip(problems, outs):
+            P.moe_ffn_static(h, inv, ids, w, img, dt, E, H, I, 0.1, out)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    # nothing went through torch's caching allocator either (no segment reserved, no block handed out)
+    assert torch.cuda.memory_reserved() == reserved0
+    assert torch.cuda.memory_stats()["allocation.all.allocated"] == mallocs0
+
+
+def test_static_entry_point_reports_malformed_calls_as_bad_arguments():
+    h = torch.zeros(1, 520, device=DEV)
+    ids = torch.zeros(1, 2, dtype=torch.int32, device=DEV)
+    w = torch.zeros(1, 2, device=DEV)
+    img = torch.zeros(16, dtype=torch.uint8, device=DEV)
+    with pytest.raises(P.StmoeError, match="bad argument"):            # hidden not a multiple of 16
+        P.moe_ffn_static(h, None, ids, w, img, "bf16", 4, 520, 64, 0.1, torch.empty_like(h))
 
 
 def test_static_scratch_rejects_problems_beyond_its_capacity():
