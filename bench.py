@@ -195,6 +195,12 @@ def main():
     ap.add_argument("--resident", action="store_true", help="keep every expert in HBM (cache_slots = 0)")
     ap.add_argument("--dense-min-batch", type=int, default=0,
                     help="smallest batch that takes the tcgen05 path (0: the library's default, 2 for bf16, 3 for fp8)")
+    ap.add_argument("--stage-known-kb", type=int, default=-1,
+                    help="single-sequence resident steps: L2 staging of known weights, KiB per expert and SM "
+                         "(-1: the library's default, 0: off)")
+    ap.add_argument("--stage-pred-mb", type=float, default=-1.0,
+                    help="single-sequence resident steps: MB per layer of predicted experts' rows staged into L2 "
+                         "ahead of the router (-1: the library's default)")
     ap.add_argument("--no-dense", action="store_true",
                     help="batched steps of resident bf16 stacks on the CUDA-core kernels instead of the tcgen05 ones")
     args = ap.parse_args()
@@ -229,6 +235,9 @@ def main():
         st.set_prefetch_min_score(args.prefetch_min_score)
     if args.dense_min_batch and not args.no_dense:
         st.set_dense_min_batch(args.dense_min_batch)
+    if args.stage_known_kb >= 0 or args.stage_pred_mb >= 0:
+        st.set_onchip_staging(max(args.stage_known_kb, 0) << 10,
+                              int(max(args.stage_pred_mb, 0.0) * 1e6))
     L, K, H = cfg.n_layers, cfg.top_k, cfg.hidden
     n_tok = cfg.profile_tokens + args.warmup + args.steps
     x_host = stacks.token_inputs(cfg, batch, n_tok).pin_memory()

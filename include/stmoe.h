@@ -176,6 +176,21 @@ int stmoe_set_kernel_timing(stmoe_t *s, int on);
  * Between decode steps; routing, outputs and predictor tables are unaffected. */
 int stmoe_set_prefetch_min_score(stmoe_t *s, int min_score);
 
+/* On-chip staging in the single-sequence persistent decode step of resident stacks: the paper's
+ * idea of fetching experts before they are needed (Sections 4.1, 4.3.4), one memory level down.
+ * Weight rows are hinted into L2 while HBM would otherwise idle at a grid barrier; results never
+ * depend on it (bit-identical on or off).
+ *   known_bytes      weights whose addresses are already known: the down projection of the routed
+ *                    experts (known since the top-K) ahead of the barrier in front of it, at most
+ *                    known_bytes per expert and SM, and the next layer's shared experts ahead of
+ *                    its router.  0 = off (default: measured neutral to slower, the phases
+ *                    it overlaps with are not idle enough).
+ *   predicted_bytes  per layer, summed over the GPU: leading gate/up rows of the experts in
+ *                    Algorithm 2's prefetch set for the next layer, hinted ahead of that layer's
+ *                    router and top-K.  0 = off (default).
+ * Between decode steps. */
+int stmoe_set_onchip_staging(stmoe_t *s, int64_t known_bytes, int64_t predicted_bytes);
+
 /* Smallest batch that takes the tensor-core FFN path (see STMOE_FLAG_NO_DENSE); between decode
  * steps.  min_batch < 2 or a stack without that path: STMOE_ERR_BAD_ARG. */
 int stmoe_set_dense_min_batch(stmoe_t *s, int min_batch);

@@ -66,6 +66,7 @@ def lib():
         L.stmoe_set_kernel_timing.argtypes = [vp, i32]
         L.stmoe_set_dense_min_batch.argtypes = [vp, i32]
         L.stmoe_set_prefetch_min_score.argtypes = [vp, i32]
+        L.stmoe_set_onchip_staging.argtypes = [vp, i64, i64]
         L.stmoe_stats.argtypes = [vp, C.POINTER(Stats)]
         L.stmoe_export_state.argtypes = [vp, vp, C.POINTER(sz)]
         L.stmoe_import_state.argtypes = [vp, vp, sz]
@@ -176,6 +177,10 @@ class Stack:
 
     def set_prefetch_min_score(self, min_score: int) -> None:
         _check(lib().stmoe_set_prefetch_min_score(self._h, int(min_score)), "stmoe_set_prefetch_min_score")
+
+    def set_onchip_staging(self, known_bytes: int, predicted_bytes: int) -> None:
+        _check(lib().stmoe_set_onchip_staging(self._h, int(known_bytes), int(predicted_bytes)),
+               "stmoe_set_onchip_staging")
 
     def set_dense_min_batch(self, min_batch: int) -> None:
         _check(lib().stmoe_set_dense_min_batch(self._h, int(min_batch)), "stmoe_set_dense_min_batch")

@@ -460,6 +460,193 @@ __device__ __forceinline__ void down_phase(const FfnArgs &a, int *s_next)
     }
 }
 
+// ---- single-sequence schedule (persistent decode-step kernel, batch 1) ------------------------
+// With one sequence the work of a layer is static once the K routed ids are known: K routed
+// entries followed by the shared ones, one token each.  Two things differ from the general
+// phases above.
+//
+// Row-slice partition.  CTA c owns rows [c*RPE/G, (c+1)*RPE/G) of EVERY entry (RPE rows per
+// entry, G CTAs) instead of one contiguous range of the concatenated rows, so each CTA streams
+// the same share of every expert: when part of the weights already sits in L2 (see below) all
+// CTAs gain alike and none runs ahead of the others into the next grid barrier.
+//
+// On-chip staging.  Weights whose address is known before the phase that reads them are asked
+// into L2 (prefetch hints, no data returns to the SM) while HBM would otherwise idle at a phase
+// boundary: a warp that runs out of gate/up rows stages this CTA's rows of the down projection
+// (known since the top-K) before it waits at the grid barrier; a warp that runs out of
+// down-projection rows stages the next layer's shared experts (routing-independent) and a
+// bounded prefix of the experts predicted for the next layer (Algorithm 2's prefetch set, one
+// memory level below the paper's expert buffer: Section 4.3.4) before the barrier, the router
+// GEMV and the top-K of that layer.  Results do not depend on whether a line was staged.
+struct SliceTickets {
+    int lo, len;     // first row of the slice, rows of the slice (per entry)
+    int pitch;       // tickets per entry: len rounded up to whole claims, so no claim spans two entries
+    int total;       // entries * pitch
+    int base, rot, n;
+    __device__ void init(int rpe, int n_entries, int claim_rows)
+    {
+        n = n_entries;
+#ifdef STMOE_SINGLE_CONTIG
+        const int all = rpe * n_entries;
+        base = (int)((long long)all * blockIdx.x / gridDim.x);
+        total = (int)((long long)all * (blockIdx.x + 1) / gridDim.x) - base;
+        lo = 0, len = rpe, pitch = rpe, rot = 0;
+#else
+        base = 0;
+        lo = (int)((long long)rpe * blockIdx.x / gridDim.x);
+        len = (int)((long long)rpe * (blockIdx.x + 1) / gridDim.x) - lo;
+        // whole claims per entry: a claim that spanned two entries would run the row block twice,
+        // each time with some rows masked (measured: down phase 36 -> 48 us on the Mixtral shape)
+        pitch = (len + claim_rows - 1) / claim_rows * claim_rows;
+        rot = 0;
+        total = n_entries * pitch;
+#endif
+    }
+    // ticket v -> entry g and row offset o inside the slice (o >= len: padding, no row)
+    __device__ __forceinline__ void decode(int v, int &g, int &o) const
+    {
+        const int q = (base + v) / pitch;
+        o = (base + v) - q * pitch;
+        g = q + rot;
+        if (g >= n) g -= n;
+    }
+    __device__ int claim(int *s_tk, int R, int lane) const
+    {
+        int u = 0;
+        if (lane == 0) u = atomicAdd(s_tk, R);
+        return __shfl_sync(kFull, u, 0);
+    }
+};
+
+// Where the images of one layer's experts live (resident stacks: one allocation, routed images
+// [L][E] followed by the shared ones [L][n_shared]) and who is routed (shared memory).
+struct SingleCtx {
+    const uint8_t *routed0;  // image of (layer, expert 0)
+    const uint8_t *shared0;  // image of (layer, shared 0)
+    size_t img_bytes;
+    const int *s_ids;        // [K] routed ids, ascending
+    const float *s_inv;      // [1]
+    int K;
+    __device__ __forceinline__ const uint8_t *image(int g) const
+    {
+        return g < K ? routed0 + (size_t)s_ids[g] * img_bytes : shared0 + (size_t)(g - K) * img_bytes;
+    }
+    __device__ __forceinline__ void load(Entry<1> &en, int g) const
+    {
+        if (g == en.g) return;
+        en.g = g, en.cnt = 1, en.img = image(g);
+        en.tok[0] = 0, en.slot[0] = g, en.inv[0] = s_inv[0];
+    }
+};
+
+#ifndef STMOE_STAGE_PIECE
+#define STMOE_STAGE_PIECE 4096
+#endif
+// Hint [p, p+bytes) into L2, spread over `nw` warps of which this is number `w`: pieces of 4 KB,
+// one 128-byte line per lane.
+__device__ __forceinline__ void stage_range(const uint8_t *p, long long bytes, int w, int nw, int lane)
+{
+    for (long long o = (long long)w * STMOE_STAGE_PIECE; o < bytes; o += (long long)nw * STMOE_STAGE_PIECE) {
+        const int n = (int)min((long long)STMOE_STAGE_PIECE, bytes - o);
+#pragma unroll
+        for (int q = 0; q < STMOE_STAGE_PIECE / (kWarp * 128); ++q)
+            if ((q * kWarp + lane) * 128 < n) prefetch_l2(p + o + (q * kWarp + lane) * 128);
+    }
+}
+
+// This CTA's slice of the down projection of entries [g0, g1), at most cap bytes per entry.
+template <int DT>
+__device__ __forceinline__ void stage_down_slices(const FfnArgs &a, const SingleCtx &cx, const SliceTickets &td,
+                                                  int g0, int g1, long long cap, int w, int nw, int lane)
+{
+    constexpr int BYTES = Fmt<DT>::kBytes, EPL = Fmt<DT>::kEpl;
+    const int H = a.H, I = a.I, S = a.S;
+    const size_t row_bytes = (size_t)I * BYTES;
+    const int seg = ((I + S - 1) / S + kWarp * EPL - 1) / (kWarp * EPL) * (kWarp * EPL);
+    for (int g = g0; g < g1; ++g) {
+        const uint8_t *down = cx.image(g) + image_down(H, I, BYTES);
+        if (S == 1) {
+            stage_range(down + (size_t)td.lo * row_bytes, min(cap, (long long)td.len * (long long)row_bytes), w, nw, lane);
+        } else {  // rows cut into segments: one piece per (segment, row) of the slice
+            long long done = 0;
+            for (int u = td.lo + w; u < td.lo + td.len && done < cap; u += nw) {
+                const int sgm = u / H, r = u % H;
+                const int nb = min(seg, I - sgm * seg) * BYTES;
+                stage_range(down + (size_t)r * row_bytes + (size_t)sgm * seg * BYTES, nb, 0, 1, lane);
+                done += (long long)nb * nw;
+            }
+        }
+    }
+}
+
+// This CTA's slice of the gate and up matrices of the expert whose image is img: rows
+// [tg.lo, tg.lo + rows) of each.
+template <int DT>
+__device__ __forceinline__ void stage_gate_up_slice(const FfnArgs &a, const uint8_t *img, const SliceTickets &tg,
+                                                    int rows, int w, int nw, int lane)
+{
+    constexpr int BYTES = Fmt<DT>::kBytes;
+    const size_t row_bytes = (size_t)a.H * BYTES;
+    const long long n = (long long)min(rows, tg.len) * (long long)row_bytes;
+    stage_range(img + image_gate(a.H, a.I, BYTES) + (size_t)tg.lo * row_bytes, n, w, nw, lane);
+    stage_range(img + image_up(a.H, a.I, BYTES) + (size_t)tg.lo * row_bytes, n, w, nw, lane);
+}
+
+// Gate/up rows of this CTA's slices.  side(): once per warp before it starts claiming.
+// done(): once per warp when no rows are left (staging of what comes next).
+template <int DT, typename Side, typename Done>
+__device__ __forceinline__ void gate_up_single(const FfnArgs &a, const SingleCtx &cx, const SliceTickets &tk, int *s_tk,
+                                               Side side, Done done)
+{
+    using TS = TileShape<DT>;
+    constexpr int RC = TS::RG1;
+    const int lane = threadIdx.x % kWarp;
+    side();
+    Entry<1> en;
+    for (int v0 = tk.claim(s_tk, RC, lane); v0 < tk.total; v0 = tk.claim(s_tk, RC, lane)) {
+        const int vend = min(v0 + RC, tk.total);
+        for (int v = v0; v < vend;) {
+            int g, o;
+            tk.decode(v, g, o);
+            if (o >= tk.len) break;  // padding at the end of an entry's tickets
+            const int nrows = min(vend - v, tk.len - o);
+            v += nrows;
+            cx.load(en, g);
+            gate_up_block<DT, TS::RG1, 1, TS::UG1>(a, en, tk.lo + o, nrows, lane);
+        }
+    }
+    done();
+}
+
+// Down-projection rows of this CTA's slices with the fused weighted sum (n_entries entries
+// contribute to every output row).
+template <int DT, typename Done>
+__device__ __forceinline__ void down_single(const FfnArgs &a, const SingleCtx &cx, const SliceTickets &tk, int *s_tk,
+                                            int n_entries, Done done)
+{
+    using TS = TileShape<DT>;
+    constexpr int EPL = Fmt<DT>::kEpl, RC = TS::RD1;
+    const int lane = threadIdx.x % kWarp;
+    const int H = a.H, I = a.I, S = a.S;
+    const int seg = ((I + S - 1) / S + kWarp * EPL - 1) / (kWarp * EPL) * (kWarp * EPL);
+    Entry<1> en;
+    for (int v0 = tk.claim(s_tk, RC, lane); v0 < tk.total; v0 = tk.claim(s_tk, RC, lane)) {
+        const int vend = min(v0 + RC, tk.total);
+        for (int v = v0; v < vend;) {
+            int g, o;
+            tk.decode(v, g, o);
+            if (o >= tk.len) break;  // padding at the end of an entry's tickets
+            const int u = tk.lo + o, sgm = u / H, r0 = u % H;
+            const int nrows = min(min(vend - v, tk.len - o), H - r0);
+            v += nrows;
+            cx.load(en, g);
+            down_block<DT, TS::RD1, 1, TS::UD1>(a, en, sgm, seg, r0, nrows, lane);
+            finish_rows(a, r0, nrows, n_entries * S, S, lane);
+        }
+    }
+    done();
+}
+
 template <int DT, int MTMAX>
 __global__ void __launch_bounds__(kFfnThreads, 1) down_kernel(FfnArgs a)
 {

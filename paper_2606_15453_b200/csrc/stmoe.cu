@@ -324,6 +324,9 @@ struct stmoe {
     bool dense_persistent = false;  // one cooperative kernel per decode step (token_dense_kernel.cuh)
     int dense_dyn_bytes = 0;
 
+    // on-chip staging of the single-sequence persistent kernel (see ffn.cuh)
+    long long stage_down_bytes = 0, stage_pred_bytes = 0;
+    int stage_shared = 0;
     int prefetch_min_score = 0;  // queue entries below this summed score are not prefetched
     SlotCache cache;
     cudaStream_t copy_stream = nullptr;
@@ -924,6 +927,8 @@ int token_persistent(stmoe *s, int batch, const float *h_in, float *h_out, int32
     a.pred_ids = predicted_ids, a.n_pred = n_predicted, a.max_pred = s->max_pred;
     a.pst = s->pst, a.P = c.profile_tokens, a.mode = c.predictor_mode;
     a.barrier = s->d_barrier, a.err = s->d_err;
+    a.store = s->d_resident, a.img_bytes = s->img_bytes;
+    a.stage_down_bytes = s->stage_down_bytes, a.stage_pred_bytes = s->stage_pred_bytes, a.stage_shared = s->stage_shared;
     CU_TRY(cudaMemsetAsync(s->d_barrier, 0, 4, st));
     void *args[] = {&a};
     CU_TRY(cudaLaunchCooperativeKernel(token_kernel(c.weight_dtype, s->rdt, a.mt), dim3(s->persistent_grid),
@@ -1231,6 +1236,15 @@ int stmoe_set_prefetch_min_score(stmoe_t *s, int min_score)
 {
     if (!s || min_score < 0 || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
     s->prefetch_min_score = min_score;
+    return STMOE_OK;
+}
+
+int stmoe_set_onchip_staging(stmoe_t *s, int64_t known_bytes, int64_t predicted_bytes)
+{
+    if (!s || known_bytes < 0 || predicted_bytes < 0 || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
+    s->stage_shared = known_bytes > 0;
+    s->stage_down_bytes = known_bytes;
+    s->stage_pred_bytes = predicted_bytes;
     return STMOE_OK;
 }
 

@@ -51,6 +51,12 @@ struct TokenArgs {
     int P, mode;
     unsigned *barrier;              // [1] zero at launch
     unsigned *err;                  // [1]
+    // single-sequence schedule: resident images by address arithmetic, on-chip staging budgets
+    const uint8_t *store;           // routed images [L][E], then shared images [L][n_shared]
+    size_t img_bytes;
+    long long stage_down_bytes;     // per entry and CTA: down-projection bytes staged ahead of the GU->D barrier
+    long long stage_pred_bytes;     // per layer, whole GPU: gate/up bytes of predicted experts staged ahead (0: off)
+    int stage_shared;               // stage the next layer's shared experts ahead of its router
 };
 
 // Algorithms 1-3 for one layer step on `nw` warps of one CTA (this is warp `wi` of them; all nw
@@ -232,6 +238,127 @@ __device__ __forceinline__ void grid_barrier(unsigned *counter, unsigned *err, u
     __syncthreads();
 }
 
+// Next layer's routing-independent and predicted weights, asked into L2 by a warp that has run
+// out of rows in the current layer (or, for layer 0, at the start of the launch): this CTA's
+// slices of the shared experts' three matrices, then of the first rows of the gate and up
+// matrices of the experts in the prefetch set of Algorithm 2 for that layer (lowest ids first
+// when the budget does not cover them all).  The set was written by the predictor warp at least
+// one grid barrier ago and is not overwritten before the next layer's top-K, which needs the
+// barrier this warp has yet to arrive at.
+template <int DT>
+__device__ __forceinline__ void stage_layer_ahead(const TokenArgs &a, int layer, const FfnArgs &fa,
+                                                  const SliceTickets &tg, const SliceTickets &td, int w, int nw,
+                                                  int lane)
+{
+    constexpr int BYTES = Fmt<DT>::kBytes;
+    const uint8_t *routed0 = a.store + (size_t)layer * a.E * a.img_bytes;
+    const uint8_t *shared0 = a.store + ((size_t)a.L * a.E + (size_t)layer * a.n_shared) * a.img_bytes;
+    if (a.stage_shared) {
+        SingleCtx cx{routed0, shared0, a.img_bytes, nullptr, nullptr, 0};  // K = 0: entry g is shared expert g
+        for (int i = 0; i < a.n_shared; ++i) stage_gate_up_slice<DT>(fa, cx.image(i), tg, tg.len, w, nw, lane);
+        stage_down_slices<DT>(fa, cx, td, 0, a.n_shared, a.stage_down_bytes, w, nw, lane);
+    }
+    if (a.stage_pred_bytes > 0 && __ldcg(a.pst.pred_valid) != 0u) {
+        unsigned msk = lane < kMaxExperts / kWarp ? __ldcg(a.pst.pred_mask + lane) : 0u;
+        const int n_pred = __reduce_add_sync(kFull, __popc(msk));
+        if (n_pred > 0) {
+            const long long per_row = 2ll * a.H * BYTES * gridDim.x;  // one gate + one up row in every CTA
+            const int rows_all = (int)(a.stage_pred_bytes / per_row);  // rows the budget buys per CTA
+            const int n_take = min(n_pred, max(rows_all, 1));
+            const int rows = max(rows_all / n_take, 1);
+            int taken = 0;
+            for (int wd = 0; wd < kMaxExperts / kWarp && taken < n_take; ++wd) {
+                unsigned m = __shfl_sync(kFull, msk, wd);
+                while (m && taken < n_take) {
+                    const int f = wd * kWarp + __ffs(m) - 1;
+                    m &= m - 1;
+                    stage_gate_up_slice<DT>(fa, routed0 + (size_t)f * a.img_bytes, tg, rows, w, nw, lane);
+                    ++taken;
+                }
+            }
+        }
+    }
+}
+
+// One decode step for a single sequence (see "single-sequence schedule" in ffn.cuh).
+template <int DT, int RDT>
+__device__ __forceinline__ void decode_token_single(const TokenArgs &a, int *dyn, int *s_scan, float *s_inv, int *s_next,
+                                                    int *s_dead)
+{
+    constexpr int NW = kFfnThreads / kWarp;
+    const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
+    const int L = a.L, E = a.E, K = a.K, H = a.H, I = a.I, S = a.S;
+    const int KS = K + a.n_shared;
+    const int C = router_chunks<RDT>(H, 1), tiles = (H + kTileRows - 1) / kTileRows;
+    int *s_ids = dyn + 4 + 5 * KS;
+    int *s_prev = s_ids + K;
+    float *s_w = reinterpret_cast<float *>(s_prev + K);
+    unsigned target = 0;
+    const bool lead = blockIdx.x == 0;
+    const bool pred_cta = blockIdx.x == gridDim.x - 1;
+    SliceTickets tg, td;
+    tg.init(I, KS, TileShape<DT>::RG1);
+    td.init(S * H, KS, TileShape<DT>::RD1);
+    FfnArgs fa;
+    fa.inv_rms = s_inv, fa.H = H, fa.I = I, fa.E = E, fa.S = S, fa.w = s_w;
+    fa.B = 1, fa.K = K, fa.n_shared = a.n_shared, fa.residual_scale = a.residual_scale;
+    stage_layer_ahead<DT>(a, 0, fa, tg, td, warp, NW, lane);
+
+    for (int l = 0; l < L; ++l) {
+        const float *h = l == 0 ? a.h_in : a.hbuf + (size_t)l * H;
+        float *h_next = l == L - 1 ? a.h_out : a.hbuf + (size_t)(l + 1) * H;
+        if (threadIdx.x == 0) s_next[0] = 0, s_next[1] = 0;  // row tickets of the two phases (read after barriers)
+
+        // ---- R: split-K router GEMV -------------------------------------------------------
+        RouterArgs ra;
+        ra.h = h, ra.W = a.router + (size_t)l * E * H * Fmt<RDT>::kBytes, ra.H = H, ra.eps = a.eps;
+        ra.part = a.rpart + (size_t)l * C * E, ra.ss_part = a.sspart + (size_t)l * C;
+        ra.arrivals = nullptr, ra.inv_rms = s_inv, ra.logits_out = nullptr;
+        TopkArgs &tk = ra.tk;
+        tk.logits = nullptr, tk.B = 1, tk.E = E, tk.K = K, tk.n_shared = a.n_shared, tk.mt = 1, tk.renorm = a.renorm;
+        tk.ids = s_ids, tk.w = s_w;
+        tk.ids_out = (lead && a.ids_out) ? a.ids_out + (size_t)l * K : nullptr;
+        tk.w_out = (lead && a.w_out) ? a.w_out + (size_t)l * K : nullptr;
+        tk.flags_out = (lead && a.flags_out) ? a.flags_out + l : nullptr;
+        tk.near_tie_counter = lead ? a.pst.stats + 4 : nullptr;
+        tk.wl.n_groups = nullptr;  // no work list: the entries are the K routed ids, then the shared experts
+        DBG_STAMP(l * 8 + 0);
+        router_tasks<RDT, false>(ra, warp * gridDim.x + blockIdx.x, NW * gridDim.x, lane);  // over the SMs first
+        grid_barrier(a.barrier, a.err, target, s_dead, l * 8 + 1);
+        DBG_STAMP(l * 8 + 2);
+
+        // ---- T: softmax / top-K, redundantly per CTA --------------------------------------
+        router_finalize<RDT>(ra, s_ids, s_scan, NW);
+        __syncthreads();
+        if (lead && threadIdx.x < K) a.ids_all[(size_t)l * a.Bmax * K + threadIdx.x] = s_ids[threadIdx.x];
+        DBG_STAMP(l * 8 + 3);
+
+        // ---- GU (+ the predictor on one warp of the last CTA) -----------------------------
+        SingleCtx cx;
+        cx.routed0 = a.store + (size_t)l * E * a.img_bytes;
+        cx.shared0 = a.store + ((size_t)L * E + (size_t)l * a.n_shared) * a.img_bytes;
+        cx.img_bytes = a.img_bytes, cx.s_ids = s_ids, cx.s_inv = s_inv, cx.K = K;
+        fa.h = h, fa.act = a.act + (size_t)l * KS * I, fa.part = a.part + (size_t)l * KS * S * H;
+        fa.h_out = h_next, fa.tile_done = a.tile_done + (size_t)l * tiles;
+        gate_up_single<DT>(
+            fa, cx, tg, s_next,
+            [&]() {
+                if (pred_cta && warp == NW - 1) predictor_step_group(a, l, s_ids, s_prev, 0, 1, lane);
+            },
+            [&]() { stage_down_slices<DT>(fa, cx, td, 0, K, a.stage_down_bytes, warp, NW, lane); });
+        grid_barrier(a.barrier, a.err, target, s_dead, l * 8 + 4);
+        DBG_STAMP(l * 8 + 5);
+
+        // ---- D ---------------------------------------------------------------------------
+        down_single<DT>(fa, cx, td, s_next + 1, KS, [&]() {
+            if (l + 1 < L) stage_layer_ahead<DT>(a, l + 1, fa, tg, td, warp, NW, lane);
+        });
+        if (threadIdx.x < K) s_prev[threadIdx.x] = s_ids[threadIdx.x];
+        grid_barrier(a.barrier, a.err, target, s_dead, l * 8 + 6);
+        DBG_STAMP(l * 8 + 7);
+    }
+}
+
 template <int DT, int RDT, int MTMAX>
 __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs a)
 {
@@ -256,6 +383,9 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs 
     const bool lead = blockIdx.x == 0;
     const bool pred_cta = blockIdx.x == gridDim.x - 1;
 
+    if constexpr (MTMAX == 1) {
+        decode_token_single<DT, RDT>(a, dyn, s_scan, s_inv, s_next, &s_dead);
+    } else
     for (int l = 0; l < L; ++l) {
         const float *h = l == 0 ? a.h_in : a.hbuf + (size_t)l * B * H;
         float *h_next = l == L - 1 ? a.h_out : a.hbuf + (size_t)(l + 1) * B * H;

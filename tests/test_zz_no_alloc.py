@@ -82,7 +82,7 @@ def test_static_entry_point_reports_malformed_calls_as_bad_arguments():
 
 
 def test_static_scratch_rejects_problems_beyond_its_capacity():
-    E, K, H, I = 4, 8, 4096, 14336
+    E, K, H, I = 8, 8, 4096, 14336
     B = 64
     assert P.moe_ffn_scratch_bytes(B, K, H, I) > (8 << 20)
     h = torch.zeros(B, H, device=DEV)
