@@ -63,6 +63,13 @@ extern "C" {
                                 tcgen05 tiles, rounding the hidden state and the gated activations to
                                 bf16 (bf16 stacks) or f16 (fp8 stacks, whose weights are widened to f16) */
 
+#define STMOE_FLAG_NO_FUSED 8 /* resident stacks, one sequence: by default stmoe_decode_token runs a kernel
+                                that streams each expert's gate, up and (from a transposed copy made at
+                                load time: one third more weight memory) down rows together, one
+                                streaming phase and two grid barriers per layer; its sums are exact in
+                                fixed point, so results are reproducible but differ in the last bits
+                                from the three-phase kernels.  This flag keeps the three-phase kernel. */
+
 /* per-sequence result flags of a layer step */
 #define STMOE_TOKEN_NEAR_TIE 1u /* K-th and (K+1)-th router logit closer than 1e-4 */
 

@@ -19,6 +19,7 @@ MODE = {"off": 0, "temporal": 1, "spatial": 2, "st": 3}
 FLAG_RENORM_TOPK = 1
 FLAG_NO_PERSISTENT = 2
 FLAG_NO_DENSE = 4
+FLAG_NO_FUSED = 8
 
 
 class StmoeError(RuntimeError):

@@ -19,6 +19,7 @@
 #include "predictor.cuh"
 #include "router.cuh"
 #include "token_dense_kernel.cuh"
+#include "token_fused_kernel.cuh"
 #include "token_kernel.cuh"
 
 using namespace stmoe_dev;
@@ -310,6 +311,14 @@ struct stmoe {
     int persistent_grid = 0;
     float *d_hbuf = nullptr, *d_rpart_all = nullptr, *d_sspart_all = nullptr, *d_act_all = nullptr, *d_part_all = nullptr;
     unsigned *d_tiles_all = nullptr, *d_barrier = nullptr;
+
+    // single-sequence decode step with one streaming phase per layer (token_fused_kernel.cuh)
+    bool fused = false;
+    uint8_t *d_down_t = nullptr;            // transposed down projections, one per image
+    size_t down_t_bytes = 0;
+    float *d_zpart = nullptr;
+    unsigned long long *d_acc = nullptr;
+    int poll_limit = kBarrierSpinLimit;
 
     // tensor-core path for batched steps of resident bf16 stacks (dense_group.cuh)
     bool dense = false;
@@ -945,6 +954,50 @@ int token_persistent(stmoe *s, int batch, const float *h_in, float *h_out, int32
     return STMOE_OK;
 }
 
+void *token_fused_kernel(int dt)
+{
+    if (dt == STMOE_F32) return (void *)decode_token_fused_kernel<0, 0>;
+    if (dt == STMOE_BF16) return (void *)decode_token_fused_kernel<1, 1>;
+    return (void *)decode_token_fused_kernel<2, 1>;
+}
+
+int token_fused(stmoe *s, const float *h_in, float *h_out, int32_t *routed_ids, float *routed_w,
+                int32_t *predicted_ids, int32_t *n_predicted, uint32_t *flags, cudaStream_t st)
+{
+    const stmoe_config_t &c = s->cfg;
+    FusedArgs f{};
+    TokenArgs &a = f.t;
+    a.L = c.n_layers, a.B = 1, a.E = c.n_experts, a.K = c.top_k, a.n_shared = c.n_shared;
+    a.H = c.hidden, a.I = c.inter, a.S = 1, a.mt = 1;
+    a.renorm = (c.flags & STMOE_FLAG_RENORM_TOPK) ? 1 : 0;
+    a.eps = c.rms_eps, a.residual_scale = c.residual_scale;
+    a.h_in = h_in, a.h_out = h_out;
+    a.router = s->d_router;
+    a.ids_all = s->d_ids, a.Bmax = c.max_batch;
+    a.ids_out = routed_ids, a.w_out = routed_w, a.flags_out = flags;
+    a.pred_ids = predicted_ids, a.n_pred = n_predicted, a.max_pred = s->max_pred;
+    a.pst = s->pst, a.P = c.profile_tokens, a.mode = c.predictor_mode;
+    a.barrier = s->d_barrier, a.err = s->d_err;
+    a.store = s->d_resident, a.img_bytes = s->img_bytes;
+    f.down_t = s->d_down_t, f.down_t_bytes = s->down_t_bytes;
+    f.zpart = s->d_zpart, f.acc = s->d_acc, f.poll_limit = s->poll_limit;
+    CU_TRY(cudaMemsetAsync(s->d_barrier, 0, 4, st));
+    CU_TRY(cudaMemsetAsync(s->d_acc, 0, 8 * (size_t)c.n_layers * c.hidden, st));
+    void *args[] = {&f};
+    CU_TRY(cudaLaunchCooperativeKernel(token_fused_kernel(c.weight_dtype), dim3(s->persistent_grid), dim3(kFfnThreads),
+                                       args, kFusedRingBytes, st));
+    s->launches += 1;
+    if (!s->built && s->host_t == c.profile_tokens - 1) {
+        const int rows = (c.n_layers - 1) * c.n_experts;
+        if (rows > 0) cct_build_kernel<<<(rows + 7) / 8, 256, 0, st>>>(s->pst, c.n_layers, c.n_experts, c.top_k);
+        s->launches += rows > 0;
+        s->built = true;
+        CU_TRY(cudaGetLastError());
+    }
+    s->host_t += 1;
+    return STMOE_OK;
+}
+
 void *token_dense_kernel(int rdt, bool w8)
 {
     if (w8) return rdt == STMOE_F32 ? (void *)decode_token_dense_kernel<0, 2> : (void *)decode_token_dense_kernel<1, 2>;
@@ -1051,7 +1104,8 @@ int stmoe_destroy(stmoe_t *s)
                    s->pst.Co, s->pst.cct_id, s->pst.cct_conf, s->pst.HT, s->pst.t, s->pst.pred_mask,
                    s->pst.pred_valid, s->pst.stats, s->d_rpart, s->d_sspart, s->d_arrivals, s->d_tile_done, s->d_hbuf, s->d_rpart_all, s->d_sspart_all,
                    s->d_act_all, s->d_part_all, s->d_tiles_all, s->d_barrier, s->d_err, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
-                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense, s->d_xb16, s->d_act16};
+                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense, s->d_xb16, s->d_act16,
+                   s->d_down_t, s->d_zpart, s->d_acc};
     if (s->d_shared && s->d_resident && s->d_shared > s->d_resident) dev[2] = nullptr;  // one allocation
     for (void *p : dev)
         if (p) cudaFree(p);
@@ -1203,6 +1257,28 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
             s->persistent_grid = sm_count();
         }
     }
+    if (s->persistent && !(c.flags & STMOE_FLAG_NO_FUSED) &&
+        fused_shape_ok(H, 16 / dtype_bytes(c.weight_dtype))) {
+        // a second, transposed copy of every down projection; if it does not fit the stack stays
+        // on the three-phase kernel
+        const size_t n_img = (size_t)L * (E + c.n_shared);
+        s->down_t_bytes = (size_t)H * I * dtype_bytes(c.weight_dtype);
+        int occ = 0;
+        void *k = token_fused_kernel(c.weight_dtype);
+        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedRingBytes) == cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kFfnThreads, kFusedRingBytes) == cudaSuccess && occ >= 1 &&
+            cudaMalloc(&s->d_down_t, n_img * s->down_t_bytes) == cudaSuccess &&
+            cudaMalloc(&s->d_zpart, sizeof(float) * (size_t)L * E) == cudaSuccess &&
+            cudaMalloc(&s->d_acc, 8 * (size_t)L * H) == cudaSuccess) {
+            s->fused = true;
+        } else {
+            (void)cudaGetLastError();
+            if (s->d_down_t) cudaFree(s->d_down_t);
+            if (s->d_zpart) cudaFree(s->d_zpart);
+            if (s->d_acc) cudaFree(s->d_acc);
+            s->d_down_t = nullptr, s->d_zpart = nullptr, s->d_acc = nullptr;
+        }
+    }
     if (c.cache_slots == 0 && c.weight_dtype == STMOE_BF16 && !(c.flags & STMOE_FLAG_NO_DENSE) && B >= 2) {
         const int rc = dense_setup(s);
         if (rc != STMOE_OK) return fail(rc);
@@ -1284,7 +1360,19 @@ int stmoe_load_experts(stmoe_t *s, int layer, int first_expert, int count, const
         CU_TRY(cudaMemcpy(img + image_down(c.hidden, c.inter, wb), (const uint8_t *)down + i * mat, mat, cudaMemcpyDefault));
         if (scales)
             CU_TRY(cudaMemcpy(img + image_scales(c.hidden, c.inter, wb), (const uint8_t *)scales + i * sc, sc, cudaMemcpyDefault));
+        if (s->fused) {  // W_d [H][I] -> [I][H] for the row-triple kernel
+            const size_t idx = is_shared ? (size_t)c.n_layers * c.n_experts + (size_t)layer * c.n_shared + first_expert + i
+                                         : (size_t)layer * c.n_experts + first_expert + i;
+            const uint8_t *in = img + image_down(c.hidden, c.inter, wb);
+            uint8_t *out = s->d_down_t + idx * s->down_t_bytes;
+            const dim3 grid((c.inter + 31) / 32, (c.hidden + 31) / 32), block(32, 8);
+            if (wb == 4) transpose_kernel<uint32_t><<<grid, block>>>((const uint32_t *)in, (uint32_t *)out, c.hidden, c.inter);
+            else if (wb == 2) transpose_kernel<uint16_t><<<grid, block>>>((const uint16_t *)in, (uint16_t *)out, c.hidden, c.inter);
+            else transpose_kernel<uint8_t><<<grid, block>>>(in, out, c.hidden, c.inter);
+            CU_TRY(cudaGetLastError());
+        }
     }
+    if (s->fused) CU_TRY(cudaDeviceSynchronize());
     return STMOE_OK;
 }
 
@@ -1316,6 +1404,8 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, i
     // sequences, +2 % at 4, -6 % at 8 and 32, where its ring has a stage less and the predictor two warps)
     if (s->dense_persistent && !s->time_kernels && use_dense(s, batch) && (!s->dense8 || batch <= kDense8PersistentMaxBatch))
         return token_dense(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
+    if (s->fused && batch == 1 && !s->time_kernels)
+        return token_fused(s, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
     if (s->persistent && !s->time_kernels && !use_dense(s, batch))
         return token_persistent(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
     if (offloaded(s) || s->time_kernels || s->graph_off || build_due) {

@@ -97,3 +97,48 @@ def replay_predictor(cfg, batch, mode, trace_ids):
     """Drive the oracle predictor with a routed-id trace [(layer, ids[B][K]) ...]."""
     p = O.Predictor(cfg.n_layers, cfg.n_experts, cfg.top_k, batch, cfg.profile_tokens, mode)
     return p, [p.step(layer, ids) for layer, ids in trace_ids]
+
+
+def decode_tokens_vs_oracle(cfg, B, T, min_checked, flags=0):
+    """Whole decode steps through stmoe_decode_token (the persistent kernels) against the oracle
+    running its own residual stream; a sequence is compared while its routing agrees in every
+    layer (a disagreement needs a flagged near tie).  The predictor is replayed on the GPU's
+    routing, bit-exact.  Returns the stack's statistics."""
+    pr = Pair(cfg, B, flags=flags)
+    L, K = cfg.n_layers, cfg.top_k
+    x = stacks.token_inputs(cfg, B, T)
+    ids = torch.empty(L, B, K, dtype=torch.int32, device=pr.dev)
+    w = torch.empty(L, B, K, dtype=torch.float32, device=pr.dev)
+    pred = torch.empty(L, B, pr.stack.max_pred, dtype=torch.int32, device=pr.dev)
+    npred = torch.empty(L, B, dtype=torch.int32, device=pr.dev)
+    flags = torch.empty(L, B, dtype=torch.int32, device=pr.dev)   # (the stack's flags were consumed above)
+    ho = torch.empty(B, cfg.hidden, device=pr.dev)
+    replay = O.Predictor(L, cfg.n_experts, K, B, cfg.profile_tokens, "st")
+    checked = 0
+    for t in range(T):
+        pr.stack.decode_token(x[t].to(pr.dev), ho, ids, w, pred, npred, flags)
+        torch.cuda.synchronize()
+        g_ids, g_w = ids.cpu().numpy(), w.cpu().numpy()
+        for l in range(L):
+            rp = replay.step(l, g_ids[l])
+            assert npred[l].cpu().tolist() == rp["n_pred"].tolist(), (t, l)
+            assert (pred[l].cpu().numpy() == rp["pred_ids"]).all(), (t, l)
+        h_ref, per = pr.oracle.decode_token(x[t].numpy())
+        o_ids = np.stack([r["ids"] for r in per])
+        o_w = np.stack([r["w"] for r in per])
+        got = ho.cpu().numpy()
+        for b in range(B):
+            if (o_ids[:, b] != g_ids[:, b]).any():
+                assert sum(int(r["ties"][b]) for r in per) + int(flags[:, b].sum()) > 0, \
+                    f"t={t} sequence {b}: routing diverged from the oracle without a near tie"
+                continue
+            assert np.abs(g_w[0, b] - o_w[0, b]).max() < 2e-5          # layer 0 sees identical inputs
+            assert rel_err(got[b], h_ref[b]) <= TOL[cfg.dtype], (t, b)
+            xin = x[t][b].numpy()
+            assert rel_err(got[b] - xin, h_ref[b] - xin) <= TOL[cfg.dtype], (t, b)
+            checked += 1
+    assert pr.stack.export_state() == replay.export()
+    assert checked >= min_checked
+    st = pr.stack.stats()            # raises if a bounded wait inside a kernel ran out
+    pr.close()
+    return st

@@ -53,7 +53,8 @@ def test_binding_constants_match_the_header():
     assert defs["STMOE_FLAG_RENORM_TOPK"] == P.FLAG_RENORM_TOPK
     assert defs["STMOE_FLAG_NO_PERSISTENT"] == P.FLAG_NO_PERSISTENT
     assert defs["STMOE_FLAG_NO_DENSE"] == P.FLAG_NO_DENSE
-    assert len({defs[k] for k in defs if k.startswith("STMOE_FLAG_")}) == 3      # distinct bits
+    assert defs["STMOE_FLAG_NO_FUSED"] == P.FLAG_NO_FUSED
+    assert len({defs[k] for k in defs if k.startswith("STMOE_FLAG_")}) == 4      # distinct bits
     for name, code in P.DTYPE.items():
         assert defs[{"f32": "STMOE_F32", "bf16": "STMOE_BF16", "fp8": "STMOE_FP8_E4M3"}[name]] == code
     for name, code in P.MODE.items():

@@ -131,8 +131,8 @@ def test_tiny_cache_thrashes_but_stays_correct():
     (64, dict(hidden=144, inter=96, n_experts=40, top_k=32, n_shared=0)),      # maximum batch and K
 ])
 def test_decode_token_paths_agree(B, shape):
-    """decode_token has three execution paths for a resident stack: the persistent one-kernel
-    step (default), per-layer kernels replayed as a CUDA graph (capturable stream), and per-layer
+    """decode_token has three execution paths for a resident stack that share their arithmetic:
+    the persistent three-phase kernel, per-layer kernels replayed as a CUDA graph (capturable stream), and per-layer
     kernels launched one by one (default stream).  Outputs, routing, predictions, tables and
     counters must be identical, bit for bit."""
     cfg = stacks.CONFIGS["C2"].scaled(n_layers=3, profile_tokens=3, **shape)
@@ -141,7 +141,7 @@ def test_decode_token_paths_agree(B, shape):
     results = []
     for path in ("persistent", "graph", "eager"):
         pr = Pair(cfg, B, oracle=False,
-                  flags=P.FLAG_NO_DENSE | (0 if path == "persistent" else P.FLAG_NO_PERSISTENT))
+                  flags=P.FLAG_NO_DENSE | P.FLAG_NO_FUSED | (0 if path == "persistent" else P.FLAG_NO_PERSISTENT))
         L, K = cfg.n_layers, cfg.top_k
         ids = torch.empty(L, B, K, dtype=torch.int32, device=DEV)
         w = torch.empty(L, B, K, dtype=torch.float32, device=DEV)

@@ -13,7 +13,7 @@ DEV = "cuda:0"
 
 
 def _run(cfg, T, flags=0, staging=None):
-    pr = Pair(cfg, 1, oracle=False, flags=flags)
+    pr = Pair(cfg, 1, oracle=False, flags=flags | P.FLAG_NO_FUSED)    # the three-phase kernel family
     if staging is not None:
         pr.stack.set_onchip_staging(*staging)
     L, K = cfg.n_layers, cfg.top_k
