@@ -954,11 +954,13 @@ int token_persistent(stmoe *s, int batch, const float *h_in, float *h_out, int32
     return STMOE_OK;
 }
 
-void *token_fused_kernel(int dt)
+void *token_fused_kernel(const stmoe_config_t &c)
 {
-    if (dt == STMOE_F32) return (void *)decode_token_fused_kernel<0, 0>;
-    if (dt == STMOE_BF16) return (void *)decode_token_fused_kernel<1, 1>;
-    return (void *)decode_token_fused_kernel<2, 1>;
+    const int dt = c.weight_dtype;
+    const int ch = fused_chunks(c.hidden, 16 / dtype_bytes(dt), c.inter, c.top_k, sm_count());
+    if (dt == STMOE_F32) return ch == 2 ? (void *)decode_token_fused_kernel<0, 0, 2> : (void *)decode_token_fused_kernel<0, 0, 1>;
+    if (dt == STMOE_BF16) return ch == 2 ? (void *)decode_token_fused_kernel<1, 1, 2> : (void *)decode_token_fused_kernel<1, 1, 1>;
+    return (void *)decode_token_fused_kernel<2, 1, 1>;
 }
 
 int token_fused(stmoe *s, const float *h_in, float *h_out, int32_t *routed_ids, float *routed_w,
@@ -984,8 +986,8 @@ int token_fused(stmoe *s, const float *h_in, float *h_out, int32_t *routed_ids, 
     CU_TRY(cudaMemsetAsync(s->d_barrier, 0, 4, st));
     CU_TRY(cudaMemsetAsync(s->d_acc, 0, 8 * (size_t)c.n_layers * c.hidden, st));
     void *args[] = {&f};
-    CU_TRY(cudaLaunchCooperativeKernel(token_fused_kernel(c.weight_dtype), dim3(s->persistent_grid), dim3(kFfnThreads),
-                                       args, kFusedRingBytes, st));
+    CU_TRY(cudaLaunchCooperativeKernel(token_fused_kernel(c), dim3(s->persistent_grid), dim3(kFfnThreads),
+                                       args, (size_t)fused_smem_bytes(c.hidden), st));
     s->launches += 1;
     if (!s->built && s->host_t == c.profile_tokens - 1) {
         const int rows = (c.n_layers - 1) * c.n_experts;
@@ -1264,9 +1266,9 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
         const size_t n_img = (size_t)L * (E + c.n_shared);
         s->down_t_bytes = (size_t)H * I * dtype_bytes(c.weight_dtype);
         int occ = 0;
-        void *k = token_fused_kernel(c.weight_dtype);
-        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedRingBytes) == cudaSuccess &&
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kFfnThreads, kFusedRingBytes) == cudaSuccess && occ >= 1 &&
+        void *k = token_fused_kernel(c);
+        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, fused_smem_bytes(H)) == cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kFfnThreads, fused_smem_bytes(H)) == cudaSuccess && occ >= 1 &&
             cudaMalloc(&s->d_down_t, n_img * s->down_t_bytes) == cudaSuccess &&
             cudaMalloc(&s->d_zpart, sizeof(float) * (size_t)L * E) == cudaSuccess &&
             cudaMalloc(&s->d_acc, 8 * (size_t)L * H) == cudaSuccess) {

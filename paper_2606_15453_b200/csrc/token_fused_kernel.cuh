@@ -53,18 +53,36 @@ struct FusedArgs {
 };
 
 constexpr int kFusedRows = 2;          // rows per block
-constexpr int kFusedStages = 4;        // ring stages per unit (blocks in flight)
+constexpr int kFusedStages = 4;        // ring stages per unit (blocks in flight) with one chunk per thread
 // ring bytes: units * stages * 3 matrices * rows * (H * element bytes) = 512 threads * 16 B * 24
 constexpr int kFusedRingBytes = kFfnThreads * 16 * 3 * kFusedRows * kFusedStages;
+// dynamic shared memory: the ring, then H floats in which the CTA's units add up their outputs
+__host__ __device__ inline int fused_smem_bytes(int H) { return kFusedRingBytes + H * 4; }
 constexpr int kFusedMaxUnits = 8;      // units per CTA (TPR >= 64)
 constexpr float kFixScale = 1099511627776.0f;            // 2^40
-constexpr double kFixInv = 9.094947017729282379150390625e-13;  // 2^-40
+constexpr float kFixInv = 9.094947017729282379150390625e-13f;  // 2^-40 (exact in fp32)
 
-// Which shapes the kernel covers: a unit must be 2..16 whole warps.
+// Which shapes the kernel covers: a unit must be 2..16 whole warps (with one chunk per thread).
 __host__ __device__ inline bool fused_shape_ok(int H, int epl)
 {
     const int tpr = H / epl;
-    return H % epl == 0 && (tpr == 64 || tpr == 128 || tpr == 256 || tpr == 512);
+    return H % epl == 0 && H <= 4096 && (tpr == 64 || tpr == 128 || tpr == 256 || tpr == 512);
+}
+// Chunks per thread: two where the unit then still has two whole warps, the registers allow it
+// (not the 16-column fp8 layout) and every unit still gets at least six row blocks of the routed
+// experts per layer: two chunks halve the per-block bookkeeping per byte but double the number
+// of units, and with few blocks per unit the one-block difference between units shows at the
+// layer's closing barrier (measured: Qwen3-30B shape, 5.2 blocks per unit, 25.8 us per layer with
+// two chunks against 24.0 with one; DeepSeek-V2-Lite shape, 7.2 blocks, 30.7 against 32.2).
+#ifndef STMOE_FUSED_MAX_CHUNKS
+#define STMOE_FUSED_MAX_CHUNKS 2
+#endif
+__host__ __device__ inline int fused_chunks(int H, int epl, int I, int K, int n_ctas)
+{
+    if (STMOE_FUSED_MAX_CHUNKS < 2 || epl >= 16 || H / epl < 128) return 1;
+    const long long units = (long long)(n_ctas - 1) * (kFfnThreads / (H / (epl * 2)));
+    const long long blocks = (long long)K * ((I + kFusedRows - 1) / kFusedRows);
+    return blocks >= 6 * units ? 2 : 1;
 }
 
 struct UnitCtx {
@@ -136,17 +154,24 @@ __device__ __forceinline__ void unit_sum4(UnitCtx &u, float (&v)[4])
     for (int i = 0; i < 4; ++i) v[i] = __shfl_sync(kFull, t, i);
 }
 
-// Grid barrier whose participants are the units (one arrival each).
-__device__ __forceinline__ void units_arrive(const UnitCtx &u, unsigned *counter)
+// Grid barrier with one arrival and one poller per CTA (the units of a CTA meet at a CTA barrier
+// first: with several hundred units on the GPU, per-unit arrivals and pollers on one counter cost
+// several microseconds per barrier).
+// The CTA barrier of the threads that take part in the layer loop: all 512 of a streaming CTA, the
+// first 256 of the service CTA (its last warp runs the predictor on its own, the rest idle).
+struct CtaBar {
+    int id, width;
+    __device__ __forceinline__ void sync() const { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(width) : "memory"); }
+};
+__device__ __forceinline__ void cta_arrive(const CtaBar &cb, unsigned *counter)
 {
-    unit_sync(u);  // orders every thread's writes before the leader's release
-    if (u.t == 0) asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(counter), "r"(1u) : "memory");
+    cb.sync();  // orders every thread's writes before the release below
+    if (threadIdx.x == 0) asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(counter), "r"(1u) : "memory");
 }
-
-__device__ __forceinline__ void units_wait(const UnitCtx &u, unsigned *counter, unsigned *err, unsigned target,
-                                           volatile int *s_dead, int poll_limit)
+__device__ __forceinline__ void cta_wait(const CtaBar &cb, unsigned *counter, unsigned *err, unsigned target,
+                                         volatile int *s_dead, int poll_limit)
 {
-    if (u.t == 0 && !*s_dead) {
+    if (threadIdx.x == 0 && !*s_dead) {
         int spins = 0;
         for (;;) {
             unsigned seen;
@@ -160,382 +185,520 @@ __device__ __forceinline__ void units_wait(const UnitCtx &u, unsigned *counter, 
         }
         asm volatile("{.reg .u32 t;\n\tld.acquire.gpu.global.u32 t, [%0];}" ::"l"(counter) : "memory");
     }
-    unit_sync(u);
+    cb.sync();
 }
 
-// Registers of one block in flight: kFusedRows rows of the three matrices (16 bytes each).
-struct FusedBlock {
-    uint4 g[kFusedRows], u[kFusedRows], d[kFusedRows];
+// The row blocks a unit streams in one layer.  The blocks of a list of entries form one index
+// space (bpe = ceil(I / R) blocks per entry); a unit owns a contiguous range of the shared
+// experts' space and one of the routed experts' space, each equal to within one block for all
+// units.  Block q of the unit's layer sequence: q < nq_s is global block first_s + q of the shared
+// experts, the others are global block first_r + q - nq_s of the routed ones; global block g is
+// rows [bi*R, bi*R + nrows) of entry g / bpe, bi = g % bpe.
+struct FusedPlan {
+    int rows, bpe, first_s, nq_s, first_r, nq_r;
+    __device__ __forceinline__ int nq() const { return nq_s + nq_r; }
+    __device__ __forceinline__ int nrows(int bi) const { return min(kFusedRows, rows - bi * kFusedRows); }
 };
 
-// The row blocks a unit streams for a list of entries.  The blocks of all entries form one index
-// space (bpe = ceil(I / R) blocks per entry); a unit owns a contiguous range of it, equal to
-// within one block for all units.  Block q of the unit is global block first + q: rows
-// [bi*R, bi*R + nrows) of entry (first + q) / bpe, bi = (first + q) % bpe.
-template <int DT> struct FusedStream {
-    static constexpr int EPL = Fmt<DT>::kEpl, BYTES = Fmt<DT>::kBytes, R = kFusedRows;
-    const FusedArgs &fa;
-    int layer, rows, bpe, first;   // rows per entry (I), blocks per entry, this unit's first global block
-    bool shared;            // entries are the shared experts (weight 1), else the routed ones
-    const int *s_ids;
-    const float *s_w;
-    size_t col_off;         // byte offset of this thread's columns in a row
-
-    __device__ __forceinline__ size_t image_index(int entry) const
+// Walks the blocks of a unit's layer sequence without a division: next rows of the entry, next
+// entry, next segment (shared -> routed).
+struct FusedCursor {
+    bool sh;
+    int entry, bi;
+    __device__ __forceinline__ void start(const FusedPlan &pl, bool shared_seg)
     {
-        const TokenArgs &a = fa.t;
-        return shared ? (size_t)a.L * a.E + (size_t)layer * a.n_shared + entry : (size_t)layer * a.E + s_ids[entry];
+        sh = shared_seg;
+        const int g = shared_seg ? pl.first_s : pl.first_r;
+        entry = g / pl.bpe, bi = g - entry * pl.bpe;
     }
-    // the unit's first thread: bulk copies of block q into ring stage `stage`
-    __device__ __forceinline__ void issue(int q, uint8_t *stage, uint64_t *full) const
+    __device__ __forceinline__ void next(const FusedPlan &pl)
     {
-        const TokenArgs &a = fa.t;
-        const int entry = (first + q) / bpe, bi = (first + q) % bpe;
-        const int i0 = bi * R, nrows = min(R, rows - i0);
-        const size_t idx = image_index(entry), row_bytes = (size_t)a.H * BYTES;
-        const uint8_t *img = a.store + idx * a.img_bytes;
-        const uint8_t *src[3] = {img + image_gate(a.H, a.I, BYTES) + (size_t)i0 * row_bytes,
-                                 img + image_up(a.H, a.I, BYTES) + (size_t)i0 * row_bytes,
-                                 fa.down_t + idx * fa.down_t_bytes + (size_t)i0 * row_bytes};
-        const uint32_t bytes = (uint32_t)(nrows * row_bytes);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the stage was last read through the generic proxy
-        dmbar_expect_tx(full, 3 * bytes);
-#pragma unroll
-        for (int m = 0; m < 3; ++m)
-            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         :
-                         : "r"(dsmem_u32(stage + (size_t)m * R * row_bytes)), "l"(src[m]), "r"(bytes), "r"(dsmem_u32(full))
-                         : "memory");
-    }
-    // every thread: its 16 bytes of each row of block q from the stage
-    __device__ __forceinline__ void fetch(int q, const uint8_t *stage, FusedBlock &b) const
-    {
-        const TokenArgs &a = fa.t;
-        const int nrows = min(R, rows - ((first + q) % bpe) * R);
-        const size_t row_bytes = (size_t)a.H * BYTES;
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            if (r < nrows) {
-                b.g[r] = *reinterpret_cast<const uint4 *>(stage + (size_t)r * row_bytes + col_off);
-                b.u[r] = *reinterpret_cast<const uint4 *>(stage + (size_t)(R + r) * row_bytes + col_off);
-                b.d[r] = *reinterpret_cast<const uint4 *>(stage + (size_t)(2 * R + r) * row_bytes + col_off);
-            } else {
-                b.g[r] = b.u[r] = b.d[r] = make_uint4(0u, 0u, 0u, 0u);
-            }
-        }
+        if (++bi == pl.bpe) bi = 0, ++entry;
     }
 };
 
-template <int DT, int RDT>
+__device__ __forceinline__ size_t fused_image_index(const TokenArgs &a, int layer, bool shared, int entry, const int *s_ids)
+{
+    return shared ? (size_t)a.L * a.E + (size_t)layer * a.n_shared + entry : (size_t)layer * a.E + s_ids[entry];
+}
+
+// The unit's first thread: bulk copies of one block (rows [i0, i0+nrows) of the three matrices of
+// image idx) into a ring stage.
+template <int DT>
+__device__ __forceinline__ void fused_issue(const FusedArgs &fa, size_t idx, int i0, int nrows, uint8_t *stage, uint64_t *full)
+{
+    constexpr int BYTES = Fmt<DT>::kBytes, R = kFusedRows;
+    const TokenArgs &a = fa.t;
+    const size_t row_bytes = (size_t)a.H * BYTES;
+    const uint8_t *img = a.store + idx * a.img_bytes;
+    const uint8_t *src[3] = {img + image_gate(a.H, a.I, BYTES) + (size_t)i0 * row_bytes,
+                             img + image_up(a.H, a.I, BYTES) + (size_t)i0 * row_bytes,
+                             fa.down_t + idx * fa.down_t_bytes + (size_t)i0 * row_bytes};
+    const uint32_t bytes = (uint32_t)(nrows * row_bytes);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the stage was last read through the generic proxy
+    dmbar_expect_tx(full, 3 * bytes);
+#pragma unroll
+    for (int m = 0; m < 3; ++m)
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     :
+                     : "r"(dsmem_u32(stage + (size_t)m * R * row_bytes)), "l"(src[m]), "r"(bytes), "r"(dsmem_u32(full))
+                     : "memory");
+}
+
+// Bounded wait for a stage's copies: the hardware suspends the thread inside try_wait (up to the
+// hint, in nanoseconds), so a waiting unit issues few instructions beside a working one.
+__device__ __forceinline__ bool fused_wait(uint64_t *bar, uint32_t parity, volatile int *dead)
+{
+    for (int spins = 0; spins < (1 << 18); ++spins) {
+        uint32_t ok;
+        asm volatile(
+            "{.reg .pred p;\n\t"
+#ifdef STMOE_FUSED_WAIT_HINT
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+#else
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+#endif
+            "selp.u32 %0, 1, 0, p;}"
+            : "=r"(ok)
+            : "r"(dsmem_u32(bar)), "r"(parity), "r"(2000u)
+            : "memory");
+        if (ok) return true;
+        if ((spins & 15) == 15 && *dead) return false;
+    }
+    *dead = 1;
+    return false;
+}
+
+// CH: 16-byte chunks of a row a thread owns (chunk j = columns [(t + j*TPR)*EPL, +EPL)).  Two
+// chunks halve the per-block bookkeeping (waits, reductions, barriers) per byte, which is what
+// bounds the kernel once the copies keep HBM busy; they need twice the registers for the
+// thread's columns of h and of the output, which the 16-column fp8 layout does not have.
+template <int DT, int RDT, int CH>
 __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(FusedArgs fa)
 {
     constexpr int EPL = Fmt<DT>::kEpl, BYTES = Fmt<DT>::kBytes, R = kFusedRows;
-    constexpr int EPLR = Fmt<RDT>::kEpl, NRL = EPL / EPLR;  // router loads per thread and row
+    // The ring is 192 KB per CTA whatever the unit size: a CTA of two-chunk threads has twice the
+    // units, each with half the stages (the bytes in flight per SM are the same).
+    constexpr int NS = kFusedStages / CH;
+    constexpr int EPLR = Fmt<RDT>::kEpl, NRL = EPL / EPLR;  // router loads per chunk and row
     static_assert(R == 2, "unit_sum4 reduces the two dot products of two rows");
     const TokenArgs &a = fa.t;
     const int L = a.L, E = a.E, K = a.K, H = a.H, I = a.I;
     __shared__ __align__(16) float s_red[kFusedMaxUnits][2 * 64];
-    __shared__ uint32_t s_key[kFusedMaxUnits][kMaxExperts];
-    __shared__ uint8_t s_sel[kFusedMaxUnits][kMaxExperts];
-    __shared__ int s_ids[kFusedMaxUnits][kMaxTopK];
-    __shared__ float s_w[kFusedMaxUnits][kMaxTopK];
-    __shared__ float s_pick[kFusedMaxUnits][2];
+    __shared__ uint32_t s_key[kMaxExperts];
+    __shared__ float s_tk[3][8];   // top-K: per-warp maxima, sums, selected sums
+    __shared__ int s_cnt[8];       // top-K: selected experts per warp
+    __shared__ int s_ids[kMaxTopK];
+    __shared__ float s_w[kMaxTopK];
+    __shared__ float s_pick[2];
     __shared__ int s_prev[kMaxTopK];
-    __shared__ int s_dead;
+    __shared__ int s_dead, s_ready;  // s_ready: layers whose routing the service CTA has recorded
     __shared__ __align__(8) uint64_t s_full[kFusedMaxUnits][kFusedStages];
-    extern __shared__ __align__(128) uint8_t ring[];  // [unit][stage][gate rows | up rows | down^T rows]
+    extern __shared__ __align__(128) uint8_t ring[];  // [unit][stage][gate rows | up rows | down^T rows], then H floats
 
     UnitCtx u;
-    u.tpr = H / EPL;
+    u.tpr = H / (EPL * CH);
     u.grp = threadIdx.x / u.tpr, u.t = threadIdx.x % u.tpr;
     u.wig = u.t / kWarp, u.nwg = u.tpr / kWarp, u.lane = threadIdx.x % kWarp;
     u.bar_id = 1 + u.grp;
     u.red = s_red[u.grp], u.par = 0;
     const int ng = kFfnThreads / u.tpr;
-    const int unit = blockIdx.x * ng + u.grp, n_units = gridDim.x * ng;
     const bool service = blockIdx.x == gridDim.x - 1;
     const int n_stream = (gridDim.x - 1) * ng;
+    // The service CTA's last warp runs the predictor on its own, layer after layer, from the
+    // routing its first 256 threads record (whole units when a unit has at most 256 threads); the
+    // threads between idle.  The predictor then never holds up a grid barrier.
+    const bool async_pred = service && u.tpr <= 256;
+    const CtaBar cb{async_pred ? 13 : 0, async_pred ? 256 : kFfnThreads};
+    const int unit = blockIdx.x * ng + u.grp;
+    const int n_units = async_pred ? n_stream + 256 / u.tpr : gridDim.x * ng;  // who router rows are dealt to
     if (threadIdx.x == 0) {
-        s_dead = 0;
+        s_dead = 0, s_ready = 0;
         for (int i = 0; i < kFusedMaxUnits * kFusedStages; ++i) dmbar_init(&s_full[0][0] + i, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     unsigned target = 0;
-    const size_t stage_bytes = (size_t)3 * R * H * BYTES;
-    uint8_t *my_ring = ring + (size_t)u.grp * kFusedStages * stage_bytes;
+    const size_t row_bytes = (size_t)H * BYTES, stage_bytes = 3 * R * row_bytes;
+    uint8_t *my_ring = ring + (size_t)u.grp * NS * stage_bytes;
+    float *ysum = reinterpret_cast<float *>(ring + kFusedRingBytes);
     uint64_t *my_full = s_full[u.grp];
-    unsigned blocks_done = 0;  // blocks this unit has consumed so far: ring position and phase
 
     // this thread's columns of the hidden state, carried in registers through all layers
-    const int c0 = u.t * EPL;
-    float h[EPL], y[EPL];
+    int c0[CH];
+    float h[CH][EPL], y[CH][EPL];
 #pragma unroll
-    for (int e = 0; e < EPL; e += 4) {
-        const float4 v = ld_f4(a.h_in + c0 + e);
-        h[e] = v.x, h[e + 1] = v.y, h[e + 2] = v.z, h[e + 3] = v.w;
+    for (int j = 0; j < CH; ++j) {
+        c0[j] = (u.t + j * u.tpr) * EPL;
+#pragma unroll
+        for (int e = 0; e < EPL; e += 4) {
+            const float4 v = ld_f4(a.h_in + c0[j] + e);
+            h[j][e] = v.x, h[j][e + 1] = v.y, h[j][e + 2] = v.z, h[j][e + 3] = v.w;
+        }
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) y[j][e] = 0.f;
     }
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) y[e] = 0.f;
 
-    FusedStream<DT> fs{fa};
-    fs.rows = I, fs.bpe = (I + R - 1) / R;
-    fs.col_off = (size_t)c0 * BYTES;
-    fs.s_ids = s_ids[u.grp], fs.s_w = s_w[u.grp];
+    // The service CTA keeps the predictor's tables (CCT of every layer pair, history table, the
+    // predicted set, the step counter) in its unused ring for the whole launch and writes them back
+    // at the end: with the other SMs streaming at full rate a dependent access to global memory
+    // costs two to three microseconds, and Algorithms 2 and 3 are chains of such accesses (measured:
+    // 17-38 us per layer from global memory, which made this CTA the last to arrive at every barrier).
+    TokenArgs ap = a;
+    const size_t cct_bytes = (size_t)(L > 1 ? L - 1 : 0) * E * K, ht_bytes = (size_t)L * K * 2;
+    const size_t cct_pad = (cct_bytes + 15) / 16 * 16, ht_pad = (ht_bytes + 15) / 16 * 16;
+    const bool tables_staged = service && 2 * cct_pad + ht_pad + 64 <= (size_t)kFusedRingBytes;
+    auto copy_bytes = [&](uint8_t *dst, const uint8_t *src, size_t n) {
+        for (size_t i = threadIdx.x; i < n; i += kFfnThreads) dst[i] = src[i];
+    };
+    if (tables_staged) {
+        uint8_t *sm = ring;
+        copy_bytes(sm, a.pst.cct_id, cct_bytes);
+        copy_bytes(sm + cct_pad, a.pst.cct_conf, cct_bytes);
+        copy_bytes(sm + 2 * cct_pad, reinterpret_cast<const uint8_t *>(a.pst.HT), ht_bytes);
+        copy_bytes(sm + 2 * cct_pad + ht_pad, reinterpret_cast<const uint8_t *>(a.pst.pred_mask), 32);
+        copy_bytes(sm + 2 * cct_pad + ht_pad + 32, reinterpret_cast<const uint8_t *>(a.pst.pred_valid), 4);
+        copy_bytes(sm + 2 * cct_pad + ht_pad + 48, reinterpret_cast<const uint8_t *>(a.pst.t), 8);
+        ap.pst.cct_id = sm, ap.pst.cct_conf = sm + cct_pad;
+        ap.pst.HT = reinterpret_cast<int16_t *>(sm + 2 * cct_pad);
+        ap.pst.pred_mask = reinterpret_cast<uint32_t *>(sm + 2 * cct_pad + ht_pad);
+        ap.pst.pred_valid = reinterpret_cast<uint32_t *>(sm + 2 * cct_pad + ht_pad + 32);
+        ap.pst.t = reinterpret_cast<long long *>(sm + 2 * cct_pad + ht_pad + 48);
+    }
+    int *s_hist = reinterpret_cast<int *>(ring + (tables_staged ? 2 * cct_pad + ht_pad + 64 : 0));  // [L][K], service CTA
+    __syncthreads();
+    if (async_pred && threadIdx.x >= kFfnThreads - kWarp) {
+        for (int l = 0; l < L; ++l) {
+            int spins = 0;
+            while (*(volatile int *)&s_ready <= l && !*(volatile int *)&s_dead) {
+                if (++spins > (1 << 24)) {
+                    s_dead = 1;
+                    break;
+                }
+                __nanosleep(64);
+            }
+            if (*(volatile int *)&s_ready <= l) break;  // gave up: the error word is set at the end
+            __syncwarp();
+            predictor_step_group(ap, l, s_hist + (size_t)l * K, s_hist + (size_t)(l > 0 ? l - 1 : 0) * K, 0, 1, u.lane);
+        }
+    }
+    const bool in_loop = !(async_pred && threadIdx.x >= 256);
 
-    for (int l = 0; l < L; ++l) {
-        fs.layer = l;
+    FusedPlan pl;
+    pl.rows = I, pl.bpe = (I + R - 1) / R;
+    {
+        const long long all_s = (long long)a.n_shared * pl.bpe, all_r = (long long)K * pl.bpe;
+        pl.first_s = service ? 0 : (int)(all_s * unit / n_stream);
+        pl.nq_s = service ? 0 : (int)(all_s * (unit + 1) / n_stream) - pl.first_s;
+        pl.first_r = service ? 0 : (int)(all_r * unit / n_stream);
+        pl.nq_r = service ? 0 : (int)(all_r * (unit + 1) / n_stream) - pl.first_r;
+    }
+    const int nq = pl.nq();
+    // Ring position: `done` = blocks the unit has consumed since the start of the launch (stage =
+    // count % NS, phase = count / NS).  The copies run up to NS blocks ahead and do not stop at a
+    // layer's end: the next layer's shared experts are known, its routed experts only after its
+    // top-K.  What is issued next is the first thread's business alone.
+    unsigned done = 0, issued = 0;
+    int iss_layer = 0, iss_seq = 0;
+    FusedCursor iss;
+    iss.start(pl, pl.nq_s > 0);
+
+    for (int l = 0; in_loop && l < L; ++l) {
         // ---- RMSNorm factor (every unit, same bits) -------------------------------------------
         float ss = 0.f;
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) ss = fmaf(h[e], h[e], ss);
+        for (int j = 0; j < CH; ++j)
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) ss = fmaf(h[j][e], h[j][e], ss);
         ss = unit_sum(u, ss);
         const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
 
         // ---- router rows dealt over the units ------------------------------------------------
         DBG_STAMP(l * 8 + 0);
-        for (int j = unit; j < E; j += n_units) {
-            const uint8_t *row = a.router + ((size_t)l * E + j) * H * Fmt<RDT>::kBytes + (size_t)c0 * Fmt<RDT>::kBytes;
+        for (int jr = unit; jr < E; jr += n_units) {
+            const uint8_t *row = a.router + ((size_t)l * E + jr) * H * Fmt<RDT>::kBytes;
             float p = 0.f;
 #pragma unroll
-            for (int q = 0; q < NRL; ++q) {
-                float wf[EPLR];
-                Fmt<RDT>::unpack(ld_stream16(row + q * 16), wf);
+            for (int j = 0; j < CH; ++j)
 #pragma unroll
-                for (int e = 0; e < EPLR; ++e) p = fmaf(wf[e], h[q * EPLR + e], p);
-            }
+                for (int q = 0; q < NRL; ++q) {
+                    float wf[EPLR];
+                    Fmt<RDT>::unpack(ld_stream16(row + (size_t)c0[j] * Fmt<RDT>::kBytes + q * 16), wf);
+#pragma unroll
+                    for (int e = 0; e < EPLR; ++e) p = fmaf(wf[e], h[j][q * EPLR + e], p);
+                }
             p = unit_sum(u, p);
-            if (u.t == 0) fa.zpart[(size_t)l * E + j] = p;
+            if (u.t == 0) fa.zpart[(size_t)l * E + jr] = p;
         }
-        target += n_units;
-        units_arrive(u, a.barrier);
+        target += gridDim.x;
+        cta_arrive(cb, a.barrier);
         DBG_STAMP(l * 8 + 1);
 
-        // One pass over a list of entries: loads run one block ahead of the arithmetic.
-        auto stream = [&](bool shared_entries, int n_entries) {
-            fs.shared = shared_entries;
-            const long long all = (long long)n_entries * fs.bpe;
-            fs.first = (int)(all * unit / n_stream);
-            const int nq = (int)(all * (unit + 1) / n_stream) - fs.first;
-            if (nq == 0) return;
-            float ye[DT == 2 ? EPL : 1];  // fp8: per-expert sums before the output-channel scales
-            if (DT == 2) {
+        // ---- softmax / top-K once the logits have arrived: the CTA's first 256 threads, thread j
+        // owns expert j (rank counting: no dependent rounds); the other threads wait at the CTA
+        // barrier.  Every unit calls this once per layer, at the block where it first needs routing.
+        bool routed_known = false;
+        auto route = [&]() {
+            cta_wait(cb, a.barrier, a.err, target, &s_dead, fa.poll_limit);
+            DBG_STAMP(l * 8 + 2);
+            if (threadIdx.x < 256) {
+                auto sync256 = []() { asm volatile("bar.sync 14, 256;" ::: "memory"); };
+                const int j = threadIdx.x, wj = j / kWarp;
+                const float z = j < E ? __ldcg(fa.zpart + (size_t)l * E + j) * inv : -INFINITY;
+                const uint32_t key = j < E ? float_key(z) : 0u;
+                s_key[j] = key;
+                const float wm = warp_max(z);
+                if (u.lane == 0) s_tk[0][wj] = wm;
+                sync256();
+                float zmax = s_tk[0][0];
 #pragma unroll
-                for (int e = 0; e < EPL; ++e) ye[e] = 0.f;
-            }
-            auto compute = [&](int q, const FusedBlock &b) {
-                const int entry = (fs.first + q) / fs.bpe, bi = (fs.first + q) % fs.bpe;
-                const int i0 = bi * R;
-                float v[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    float wg[EPL], wu[EPL];
-                    Fmt<DT>::unpack(b.g[r], wg);
-                    Fmt<DT>::unpack(b.u[r], wu);
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e) {
-                        v[2 * r] = fmaf(wg[e], h[e], v[2 * r]);
-                        v[2 * r + 1] = fmaf(wu[e], h[e], v[2 * r + 1]);
-                    }
-                }
-                unit_sum4(u, v);
-                const float wgt = shared_entries ? 1.f : fs.s_w[entry];
-                const uint16_t *sc = nullptr;
-                if (DT == 2)
-                    sc = reinterpret_cast<const uint16_t *>(a.store + fs.image_index(entry) * a.img_bytes +
-                                                            image_scales(H, I, BYTES));
-                // odd lanes evaluate row 1, even lanes row 0; one exchange gives every lane both
-                const int r_mine = u.lane & 1;
-                float gv = (r_mine ? v[2] : v[0]) * inv, uv = (r_mine ? v[3] : v[1]) * inv;
-                if (DT == 2 && i0 + r_mine < I) {
-                    gv *= bf16_to_f32(sc[i0 + r_mine]);
-                    uv *= bf16_to_f32(sc[I + i0 + r_mine]);
-                }
-                const float act_mine = gv / (1.f + expf(-gv)) * uv;  // rows past the end: zero weights, act = 0
-                const float act_other = __shfl_xor_sync(kFull, act_mine, 1);
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const float act = (r == r_mine) ? act_mine : act_other;
-                    float wd[EPL];
-                    Fmt<DT>::unpack(b.d[r], wd);
-                    if (DT == 2) {
-#pragma unroll
-                        for (int e = 0; e < EPL; ++e) ye[e] = fmaf(act, wd[e], ye[e]);
-                    } else {
-                        const float aw = act * wgt;
-#pragma unroll
-                        for (int e = 0; e < EPL; ++e) y[e] = fmaf(aw, wd[e], y[e]);
-                    }
-                }
-                if (DT == 2 && (bi == fs.bpe - 1 || q == nq - 1)) {  // done with this expert: output-channel scales, gate weight
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e) {
-                        y[e] = fmaf(wgt * bf16_to_f32(sc[2 * I + c0 + e]), ye[e], y[e]);
-                        ye[e] = 0.f;
-                    }
-                }
-            };
-            constexpr int D = kFusedStages - 1;  // blocks the copies run ahead
-            if (u.t == 0)
-                for (int d = 0; d < D && d < nq; ++d) {
-                    const unsigned pos = blocks_done + d;
-                    fs.issue(d, my_ring + (pos % kFusedStages) * stage_bytes, my_full + pos % kFusedStages);
-                }
-            for (int q = 0; q < nq; ++q) {
-                const unsigned pos = blocks_done + q;
-                if (u.t == 0 && q + D < nq) {  // into the stage of block q-1, which the unit has left behind
-                    const unsigned pn = pos + D;
-                    fs.issue(q + D, my_ring + (pn % kFusedStages) * stage_bytes, my_full + pn % kFusedStages);
-                }
-                dmbar_wait(my_full + pos % kFusedStages, (pos / kFusedStages) & 1u, &s_dead);
-                FusedBlock b;
-                fs.fetch(q, my_ring + (pos % kFusedStages) * stage_bytes, b);
-                compute(q, b);
-            }
-            blocks_done += nq;
-        };
-
-        // ---- shared experts: independent of the routing, streamed while the logits travel -----
-        if (!service) stream(true, a.n_shared);
-        units_wait(u, a.barrier, a.err, target, &s_dead, fa.poll_limit);
-        DBG_STAMP(l * 8 + 2);
-
-        // ---- softmax / top-K, by every unit for itself ----------------------------------------
-        {
-            constexpr int VPT = kMaxExperts / 64;  // experts a thread owns at the smallest unit
-            float z[VPT], ex[VPT];
-            uint32_t key[VPT];
-            float zmax = -INFINITY;
-#pragma unroll
-            for (int q = 0; q < VPT; ++q) {
-                const int j = u.t + q * u.tpr;
-                z[q] = j < E ? __ldcg(fa.zpart + (size_t)l * E + j) * inv : -INFINITY;
-                key[q] = j < E ? float_key(z[q]) : 0u;
-                if (j < kMaxExperts) s_key[u.grp][j] = key[q];
-                zmax = fmaxf(zmax, z[q]);
-            }
-            zmax = unit_max(u, zmax);
-            float sum = 0.f;
-#pragma unroll
-            for (int q = 0; q < VPT; ++q) {
-                ex[q] = (u.t + q * u.tpr) < E ? expf(z[q] - zmax) : 0.f;
-                sum += ex[q];
-            }
-            sum = unit_sum(u, sum);
-            bool sel[VPT];
-            float selsum = 0.f;
-#pragma unroll
-            for (int q = 0; q < VPT; ++q) {
-                const int j = u.t + q * u.tpr;
-                sel[q] = false;
-                if (j < E) {
-                    int rank = 0;
+                for (int w = 1; w < 8; ++w) zmax = fmaxf(zmax, s_tk[0][w]);
+                const float ex = j < E ? expf(z - zmax) : 0.f;
+                const float ws = warp_sum(ex);
+                if (u.lane == 0) s_tk[1][wj] = ws;
+                int rank = 0;
+                if (j < E)
                     for (int i = 0; i < E; ++i) {
-                        const uint32_t k = s_key[u.grp][i];
-                        rank += (k > key[q]) || (k == key[q] && i < j);
+                        const uint32_t k = s_key[i];
+                        rank += (k > key) || (k == key && i < j);
                     }
-                    sel[q] = rank < K;
-                    if (rank == K - 1) s_pick[u.grp][0] = z[q];
-                    if (rank == K) s_pick[u.grp][1] = z[q];
-                    s_sel[u.grp][j] = sel[q];
-                    if (sel[q]) selsum += ex[q];
-                }
-            }
-            selsum = unit_sum(u, selsum);  // its barrier also publishes s_sel and s_pick
+                const bool sel = j < E && rank < K;
+                if (j < E && rank == K - 1) s_pick[0] = z;
+                if (j < E && rank == K) s_pick[1] = z;
+                const unsigned msk = __ballot_sync(kFull, sel);
+                const float wsel = warp_sum(sel ? ex : 0.f);
+                if (u.lane == 0) s_cnt[wj] = __popc(msk), s_tk[2][wj] = wsel;
+                sync256();
+                float sum = 0.f, selsum = 0.f;
+                int pos = __popc(msk & ((1u << u.lane) - 1u));
 #pragma unroll
-            for (int q = 0; q < VPT; ++q) {
-                const int j = u.t + q * u.tpr;
-                if (j < E && sel[q]) {
-                    int pos = 0;
-                    for (int i = 0; i < j; ++i) pos += s_sel[u.grp][i];
-                    s_ids[u.grp][pos] = j;
-                    s_w[u.grp][pos] = ex[q] / (a.renorm ? selsum : sum);
+                for (int w = 0; w < 8; ++w) {
+                    sum += s_tk[1][w], selsum += s_tk[2][w];
+                    if (w < wj) pos += s_cnt[w];
                 }
+                if (sel) s_ids[pos] = j, s_w[pos] = ex / (a.renorm ? selsum : sum);
             }
-            unit_sync(u);
-            if (service && u.grp == 0) {  // the step's outputs
-                if (u.t < K) {
-                    const int id = s_ids[0][u.t];
-                    a.ids_all[(size_t)l * a.Bmax * K + u.t] = id;
-                    if (a.ids_out) a.ids_out[(size_t)l * K + u.t] = id;
-                    if (a.w_out) a.w_out[(size_t)l * K + u.t] = s_w[0][u.t];
+            cb.sync();
+            if (service) {  // the step's outputs
+                if (threadIdx.x < K) {
+                    const int id = s_ids[threadIdx.x];
+                    if (async_pred) s_hist[(size_t)l * K + threadIdx.x] = id;
+                    a.ids_all[(size_t)l * a.Bmax * K + threadIdx.x] = id;
+                    if (a.ids_out) a.ids_out[(size_t)l * K + threadIdx.x] = id;
+                    if (a.w_out) a.w_out[(size_t)l * K + threadIdx.x] = s_w[threadIdx.x];
                 }
-                if (u.t == 0) {
-                    const float gap = K < E ? s_pick[0][0] - s_pick[0][1] : INFINITY;
+                if (threadIdx.x == 0) {
+                    const float gap = K < E ? s_pick[0] - s_pick[1] : INFINITY;
                     const uint32_t f = gap < 1e-4f ? 1u : 0u;
                     if (a.flags_out) a.flags_out[l] = f;
                     if (f) atomicAdd(a.pst.stats + 4, 1ull);
                 }
+                if (async_pred && threadIdx.x < kWarp) {  // K <= 32: the ids were written by this warp
+                    __syncwarp();
+                    if (threadIdx.x == 0) {
+                        __threadfence_block();
+                        *(volatile int *)&s_ready = l + 1;
+                    }
+                }
             }
-        }
-        DBG_STAMP(l * 8 + 3);
+            routed_known = true;
+            DBG_STAMP(l * 8 + 3);
+        };
 
-        // ---- routed experts (streaming units); predictor (first warp of the service CTA) ------
+        // Keep the ring full (the unit's first thread only).
+        auto top_up = [&]() {
+            while (nq > 0 && issued - done < (unsigned)NS && iss_layer < L) {
+                // a routed block of a later layer, or of this one before its top-K: not known yet
+                if (!iss.sh && (iss_layer != l || !routed_known)) break;
+                const unsigned st = issued % NS;
+                fused_issue<DT>(fa, fused_image_index(a, iss_layer, iss.sh, iss.entry, s_ids), iss.bi * R,
+                                pl.nrows(iss.bi), my_ring + st * stage_bytes, my_full + st);
+                ++issued, ++iss_seq;
+                iss.next(pl);
+                if (iss_seq == pl.nq_s && pl.nq_r > 0) iss.start(pl, false);
+                if (iss_seq == nq) iss_seq = 0, ++iss_layer, iss.start(pl, pl.nq_s > 0);
+            }
+        };
+
+        // ---- the layer's row blocks: shared experts first (they need no routing) ---------------
+        float ye[DT == 2 ? EPL : 1];  // fp8 (CH = 1): per-expert sums before the output-channel scales
+        if (DT == 2) {
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) ye[e] = 0.f;
+        }
+        FusedCursor cu;
+        cu.start(pl, pl.nq_s > 0);
+        for (int q = 0; q < nq; ++q) {
+            // the block the first thread would issue now is a routed one: time for the top-K
+            if (!routed_known && q + NS - 1 >= pl.nq_s) route();
+            if (u.t == 0) top_up();
+            const unsigned st = done % NS;
+            fused_wait(my_full + st, (done / NS) & 1u, &s_dead);
+            if (q == pl.nq_s && q > 0) cu.start(pl, false);
+            const int i0 = cu.bi * R, nrows = pl.nrows(cu.bi);
+            const uint8_t *stage = my_ring + st * stage_bytes;
+            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            uint4 wd[R][CH];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int j = 0; j < CH; ++j) {
+                    const size_t off = (size_t)r * row_bytes + (size_t)c0[j] * BYTES;
+                    uint4 wg4 = make_uint4(0u, 0u, 0u, 0u), wu4 = wg4;
+                    wd[r][j] = wg4;
+                    if (r < nrows) {
+                        wg4 = *reinterpret_cast<const uint4 *>(stage + off);
+                        wu4 = *reinterpret_cast<const uint4 *>(stage + R * row_bytes + off);
+                        wd[r][j] = *reinterpret_cast<const uint4 *>(stage + 2 * R * row_bytes + off);
+                    }
+                    float wg[EPL], wu[EPL];
+                    Fmt<DT>::unpack(wg4, wg);
+                    Fmt<DT>::unpack(wu4, wu);
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) {
+                        v[2 * r] = fmaf(wg[e], h[j][e], v[2 * r]);
+                        v[2 * r + 1] = fmaf(wu[e], h[j][e], v[2 * r + 1]);
+                    }
+                }
+            unit_sum4(u, v);  // past its barrier every thread has read the stage: it may be refilled
+            ++done;
+            const float wgt = cu.sh ? 1.f : s_w[cu.entry];
+            const uint16_t *sc = nullptr;
+            if (DT == 2)
+                sc = reinterpret_cast<const uint16_t *>(a.store + fused_image_index(a, l, cu.sh, cu.entry, s_ids) * a.img_bytes +
+                                                        image_scales(H, I, BYTES));
+            // odd lanes evaluate row 1, even lanes row 0; one exchange gives every lane both
+            const int r_mine = u.lane & 1;
+            float gv = (r_mine ? v[2] : v[0]) * inv, uv = (r_mine ? v[3] : v[1]) * inv;
+            if (DT == 2 && i0 + r_mine < I) {
+                gv *= bf16_to_f32(sc[i0 + r_mine]);
+                uv *= bf16_to_f32(sc[I + i0 + r_mine]);
+            }
+            const float act_mine = gv / (1.f + expf(-gv)) * uv;  // rows past the end: zero weights, act = 0
+            const float act_other = __shfl_xor_sync(kFull, act_mine, 1);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float act = (r == r_mine) ? act_mine : act_other;
+                if (DT != 2) act *= wgt;
+#pragma unroll
+                for (int j = 0; j < CH; ++j) {
+                    float wf[EPL];
+                    Fmt<DT>::unpack(wd[r][j], wf);
+                    if (DT == 2) {
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) ye[e] = fmaf(act, wf[e], ye[e]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) y[j][e] = fmaf(act, wf[e], y[j][e]);
+                    }
+                }
+            }
+            if (DT == 2 && (cu.bi == pl.bpe - 1 || q == pl.nq_s - 1 || q == nq - 1)) {  // done with this expert
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) {
+                    y[0][e] = fmaf(wgt * bf16_to_f32(sc[2 * I + c0[0] + e]), ye[e], y[0][e]);
+                    ye[e] = 0.f;
+                }
+            }
+            cu.next(pl);
+        }
+        if (!routed_known) route();  // units without a routed block (the service CTA among them)
+        DBG_STAMP(l * 8 + 4);
+
         if (!service) {
-            stream(false, K);
-            DBG_STAMP(l * 8 + 4);
-            // the CTA's units add up in shared memory (unit order), then one exact atomic per column
-            float *ysum = reinterpret_cast<float *>(ring);  // every copy into the ring has been consumed
-            __syncthreads();
+            // the CTA's units add up in shared memory, unit by unit, then one exact atomic per column
+            for (int g = 0; g < ng; ++g) {
+                if (u.grp == g) {
 #pragma unroll
-            for (int e = 0; e < EPL; e += 4)
-                *reinterpret_cast<float4 *>(ysum + (size_t)u.grp * H + c0 + e) = make_float4(y[e], y[e + 1], y[e + 2], y[e + 3]);
+                    for (int j = 0; j < CH; ++j)
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) y[e] = 0.f;
-            __syncthreads();
+                        for (int e = 0; e < EPL; e += 4) {
+                            float4 *p = reinterpret_cast<float4 *>(ysum + c0[j] + e);
+                            float4 sv = make_float4(y[j][e], y[j][e + 1], y[j][e + 2], y[j][e + 3]);
+                            if (g > 0) {
+                                const float4 o = *p;
+                                sv.x += o.x, sv.y += o.y, sv.z += o.z, sv.w += o.w;
+                            }
+                            *p = sv;
+                        }
+                }
+                cb.sync();
+            }
+#pragma unroll
+            for (int j = 0; j < CH; ++j)
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) y[j][e] = 0.f;
             for (int c = threadIdx.x; c < H; c += kFfnThreads) {
-                float v = 0.f;
-                for (int g = 0; g < ng; ++g) v += ysum[(size_t)g * H + c];
-                const long long fx = __float2ll_rn(v * kFixScale);
+                const long long fx = __float2ll_rn(ysum[c] * kFixScale);
                 asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(fa.acc + (size_t)l * H + c), "l"(fx) : "memory");
             }
-            __syncthreads();  // the ring is written again only after everyone has read the sums
-        } else if (threadIdx.x < kWarp) {
-            predictor_step_group(a, l, s_ids[0], s_prev, 0, 1, u.lane);
-            if (u.lane < K) s_prev[u.lane] = s_ids[0][u.lane];
+        } else if (!async_pred && threadIdx.x < kWarp) {
+            // (units of 512 threads: no warp to spare, the predictor runs here, between the barriers)
+            // one warp: spreading Algorithms 2 and 3 of a single sequence over eight warps measured
+            // two to three times slower (the rows of one sequence are too few to split)
+            predictor_step_group(ap, l, s_ids, s_prev, 0, 1, u.lane);
+            if (u.lane < K) s_prev[u.lane] = s_ids[u.lane];
             __syncwarp();
         }
         DBG_STAMP(l * 8 + 5);
 
         // ---- h' = h + r * y, from the exact sums ----------------------------------------------
-        target += n_units;
-        units_arrive(u, a.barrier);
+        target += gridDim.x;
+        cta_arrive(cb, a.barrier);  // (its CTA barrier also orders the reads of ysum before the next layer's writes)
         DBG_STAMP(l * 8 + 6);
-        units_wait(u, a.barrier, a.err, target, &s_dead, fa.poll_limit);
-        {
-            const unsigned long long *acc = fa.acc + (size_t)l * H + c0;
+        // the next layer's shared experts start to arrive while the barrier completes (top_up stops at
+        // that layer's routed blocks: iss_layer is past l by now)
+        if (u.t == 0) top_up();
+        cta_wait(cb, a.barrier, a.err, target, &s_dead, fa.poll_limit);
+#pragma unroll
+        for (int j = 0; j < CH; ++j) {
+            const unsigned long long *acc = fa.acc + (size_t)l * H + c0[j];
 #pragma unroll
             for (int e = 0; e < EPL; e += 2) {
                 const ulonglong2 v = __ldcg(reinterpret_cast<const ulonglong2 *>(acc + e));
-                h[e] = fmaf(a.residual_scale, (float)((double)(long long)v.x * kFixInv), h[e]);
-                h[e + 1] = fmaf(a.residual_scale, (float)((double)(long long)v.y * kFixInv), h[e + 1]);
+                // one rounding (64-bit integer -> fp32), then an exact power of two: no fp64 arithmetic,
+                // which this GPU executes at a small fraction of the fp32 rate
+                h[j][e] = fmaf(a.residual_scale, __ll2float_rn((long long)v.x) * kFixInv, h[j][e]);
+                h[j][e + 1] = fmaf(a.residual_scale, __ll2float_rn((long long)v.y) * kFixInv, h[j][e + 1]);
             }
         }
         DBG_STAMP(l * 8 + 7);
     }
+    __syncthreads();  // the service CTA's predictor warp and its other threads meet again here
+    if (tables_staged) {
+        const uint8_t *sm = ring;
+        copy_bytes(a.pst.cct_id, sm, cct_bytes);
+        copy_bytes(a.pst.cct_conf, sm + cct_pad, cct_bytes);
+        copy_bytes(reinterpret_cast<uint8_t *>(a.pst.HT), sm + 2 * cct_pad, ht_bytes);
+        copy_bytes(reinterpret_cast<uint8_t *>(a.pst.pred_mask), sm + 2 * cct_pad + ht_pad, 32);
+        copy_bytes(reinterpret_cast<uint8_t *>(a.pst.pred_valid), sm + 2 * cct_pad + ht_pad + 32, 4);
+        copy_bytes(reinterpret_cast<uint8_t *>(a.pst.t), sm + 2 * cct_pad + ht_pad + 48, 8);
+    }
     if (s_dead) {  // a bounded wait ran out: report it, and do not leave while a copy may still land
         if (threadIdx.x == 0) *a.err = 1u;
         if (u.t == 0)
-            for (unsigned k = 0; k < (unsigned)kFusedStages && k < blocks_done; ++k) {
-                const unsigned pos = blocks_done - 1 - k;
+            for (unsigned k = 0; k < (unsigned)NS && k < issued; ++k) {
+                const unsigned pos = issued - 1 - k;
                 for (int spins = 0; spins < (1 << 20); ++spins) {
-                    uint32_t done;
+                    uint32_t ok;
                     asm volatile(
                         "{.reg .pred p;\n\t"
                         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
                         "selp.u32 %0, 1, 0, p;}"
-                        : "=r"(done)
-                        : "r"(dsmem_u32(my_full + pos % kFusedStages)), "r"((pos / kFusedStages) & 1u)
+                        : "=r"(ok)
+                        : "r"(dsmem_u32(my_full + pos % NS)), "r"((pos / NS) & 1u)
                         : "memory");
-                    if (done) break;
+                    if (ok) break;
                 }
             }
         __syncthreads();
     }
     if (unit == 0) {
 #pragma unroll
-        for (int e = 0; e < EPL; e += 4)
-            *reinterpret_cast<float4 *>(a.h_out + c0 + e) = make_float4(h[e], h[e + 1], h[e + 2], h[e + 3]);
+        for (int j = 0; j < CH; ++j)
+#pragma unroll
+            for (int e = 0; e < EPL; e += 4)
+                *reinterpret_cast<float4 *>(a.h_out + c0[j] + e) = make_float4(h[j][e], h[j][e + 1], h[j][e + 2], h[j][e + 3]);
     }
 }
 

@@ -70,7 +70,7 @@ struct TokenArgs {
 __device__ __forceinline__ void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
 
 __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int layer, const int *cur, const int *prev,
-                                                     int wi, int nw, int lane)
+                                                     int wi, int nw, int lane, int bar_id = 3)
 {
     const int E = a.E, K = a.K, L = a.L, B = a.B;
     const PredState &st = a.pst;
@@ -78,7 +78,7 @@ __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int lay
     const bool runtime = t >= a.P;
     const bool last_profiling = (!runtime) && t == a.P - 1 && layer == L - 1;
     DBG_STAMP_WARP(2010);
-    if (runtime) {
+    if (runtime && __isGlobal(st.cct_id)) {  // (a caller may keep the tables in shared memory: nothing to pull)
         // Every table row this step touches, pulled into L1 in one trip: the rows are then read
         // one after the other (Algorithm 3 is sequential per row), each of which would otherwise
         // be a trip to L2 of its own.  The tables are private to these warps' SM during the launch.
@@ -205,7 +205,7 @@ __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int lay
     }
     DBG_STAMP_WARP(2014);
     // every warp has read the step counter before one of them advances it
-    if (nw > 1) asm volatile("bar.sync 3, %0;" ::"r"(nw * kWarp) : "memory");
+    if (nw > 1) asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(nw * kWarp) : "memory");
     if (wi == 0 && lane == 0 && layer == L - 1) *st.t = t + 1;
 }
 
