@@ -69,6 +69,8 @@ def lib():
         L.orc_pred_export.argtypes = [vp, vp]
         L.orc_cache_create.restype = vp
         L.orc_cache_create.argtypes = [i64, i32, i32]
+        L.orc_cache_create2.restype = vp
+        L.orc_cache_create2.argtypes = [i64, i32, i32, i32, i32, i32]
         L.orc_cache_destroy.argtypes = [vp]
         L.orc_cache_step.restype = C.c_int
         L.orc_cache_step.argtypes = [vp, i32, vp, i32, i32, vp, i32, i32, vp, vp, vp]
@@ -265,11 +267,16 @@ def parse_state(blob: bytes) -> dict:
 
 
 class CacheModel:
-    """Integer model of verification, miss loading and prefetch (LRU slots)."""
+    """Integer model of verification, miss loading and prefetch.  window: bits of use history per
+    key that rank the victims before recency (0: none); by_turn: among equally used keys evict
+    the one whose layer's next turn is furthest; floor: most uses in its window a prefetch
+    victim may have (-1: no such test).  window 0 without by_turn is plain LRU."""
 
-    def __init__(self, slots: int, L: int, E: int):
+    def __init__(self, slots: int, L: int, E: int, window: int = 0, floor: int = -1, by_turn: bool = False):
         self.S, self.L, self.E = slots, L, E
-        self._h = lib().orc_cache_create(slots, L, E)
+        self._h = lib().orc_cache_create2(slots, L, E, window, floor, int(by_turn))
+        if not self._h:
+            raise ValueError("bad cache policy")
 
     def __del__(self):
         if getattr(self, "_h", None):

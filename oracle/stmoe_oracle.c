@@ -520,35 +520,54 @@ size_t orc_pred_export(const orc_pred_t *p, void *buf)
 
 /* The paper stages predicted experts in an on-chip buffer and fetches a
  * mispredicted expert at once (Section 4.3.4); it names no replacement
- * policy.  Model used here: S slots, least-recently-used replacement on a
- * clock that ticks once per layer step, lowest slot index on equal stamps
- * (empty slots carry stamp -1, so they are taken first).
+ * policy.  Model used here: S slots.
+ *   use history  every (layer, expert) key carries W bits: bit i = the key was
+ *            routed at its layer's turn i decode steps ago (bit 0 = this
+ *            step).  At the start of a layer's step the histories of that
+ *            layer's keys shift by one; routed keys then set bit 0.
+ *   victim   among the slots not protected in this step: an empty slot first,
+ *            else the key with the fewest uses in its window; then (by_turn)
+ *            the key whose layer's next turn is furthest away: a decode step
+ *            walks the layers in a fixed cycle, so a key of layer m waits
+ *            (m - layer) mod L layer steps, L for the layer in progress; then
+ *            the least recently used (a clock that ticks once per layer step);
+ *            then the lowest slot index.  W = 0 without by_turn is plain LRU.
+ *            (Once a decode step touches more keys than there are slots, LRU
+ *            evicts every key just before its next turn and the hit rate is
+ *            zero; use counts keep the popular keys and the turn order keeps a
+ *            stable subset among equally popular ones.)
  *   verify   each routed expert (ascending id): resident -> hit, else a
  *            demand load into a victim that no routed expert of this step
  *            occupies;
  *   prefetch each queued expert of the next layer, in queue order: skipped
  *            if resident, else loaded into a victim that holds neither a
  *            routed expert of this step nor any queued expert; dropped when
- *            no such slot exists or `limit` copies were issued this step.
+ *            no such slot exists, when `limit` copies were issued this step,
+ *            or when the victim's key has more than `floor` uses in its
+ *            window (floor < 0: no such test): a speculative copy may then
+ *            only take slots whose content has not been of use lately.
  * A prefetched expert that is evicted before its first use counts as wasted. */
 typedef struct {
     int64_t S, clock;
-    int32_t L, E;
+    int32_t L, E, W, floor, by_turn, cur_layer;
     int32_t *slot_of;   /* [L*E] slot or -1 */
     int32_t *tag;       /* [S]   layer*E+expert or -1 */
     int64_t *stamp;     /* [S] */
+    uint32_t *hist;     /* [L*E] use history, W <= 32 bits */
     uint8_t *pf_unused; /* [S] brought by prefetch, not used yet */
     uint8_t *guard;     /* [S] scratch: protected during the current pass */
     int64_t hits, misses, pf_issued, pf_useful, pf_wasted, pf_dropped, pf_resident;
 } orc_cache_t;
 
-orc_cache_t *orc_cache_create(int64_t S, int L, int E)
+orc_cache_t *orc_cache_create2(int64_t S, int L, int E, int W, int floor, int by_turn)
 {
+    if (W < 0 || W > 32) return NULL;
     orc_cache_t *c = (orc_cache_t *)calloc(1, sizeof(*c));
-    c->S = S, c->L = L, c->E = E;
+    c->S = S, c->L = L, c->E = E, c->W = W, c->floor = floor, c->by_turn = by_turn;
     c->slot_of = (int32_t *)malloc(sizeof(int32_t) * (size_t)L * E);
     c->tag = (int32_t *)malloc(sizeof(int32_t) * (size_t)S);
     c->stamp = (int64_t *)malloc(sizeof(int64_t) * (size_t)S);
+    c->hist = (uint32_t *)calloc((size_t)L * E, sizeof(uint32_t));
     c->pf_unused = (uint8_t *)calloc((size_t)S, 1);
     c->guard = (uint8_t *)calloc((size_t)S, 1);
     for (int i = 0; i < L * E; ++i) c->slot_of[i] = -1;
@@ -556,17 +575,41 @@ orc_cache_t *orc_cache_create(int64_t S, int L, int E)
     return c;
 }
 
+orc_cache_t *orc_cache_create(int64_t S, int L, int E) { return orc_cache_create2(S, L, E, 0, -1, 0); }
+
 void orc_cache_destroy(orc_cache_t *c)
 {
     if (!c) return;
-    free(c->slot_of), free(c->tag), free(c->stamp), free(c->pf_unused), free(c->guard), free(c);
+    free(c->slot_of), free(c->tag), free(c->stamp), free(c->hist), free(c->pf_unused), free(c->guard), free(c);
+}
+
+static int cache_uses(const orc_cache_t *c, int64_t s)
+{
+    if (c->tag[s] < 0) return -1; /* empty: before everything */
+    int n = 0;
+    for (uint32_t h = c->hist[c->tag[s]]; h; h >>= 1) n += (int)(h & 1u);
+    return n;
+}
+
+/* layer steps until the turn of the layer that the slot's key belongs to */
+static int cache_wait(const orc_cache_t *c, int64_t s)
+{
+    if (!c->by_turn || c->tag[s] < 0) return 0;
+    int d = (c->tag[s] / c->E - c->cur_layer) % c->L;
+    if (d < 0) d += c->L;
+    return d == 0 ? c->L : d;
 }
 
 static int64_t cache_victim(const orc_cache_t *c)
 {
     int64_t best = -1;
-    for (int64_t s = 0; s < c->S; ++s)
-        if (!c->guard[s] && (best < 0 || c->stamp[s] < c->stamp[best])) best = s;
+    int best_uses = 0, best_wait = 0;
+    for (int64_t s = 0; s < c->S; ++s) {
+        if (c->guard[s]) continue;
+        int u = cache_uses(c, s), w = cache_wait(c, s);
+        if (best < 0 || u < best_uses || (u == best_uses && (w > best_wait || (w == best_wait && c->stamp[s] < c->stamp[best]))))
+            best = s, best_uses = u, best_wait = w;
+    }
     return best;
 }
 
@@ -589,6 +632,9 @@ int orc_cache_step(orc_cache_t *c, int layer, const int32_t *U, int nU, int next
                    const int32_t *Q, int nQ, int limit, int32_t *u_slot, uint8_t *u_loaded,
                    int32_t *q_slot)
 {
+    const uint32_t mask = c->W >= 32 ? 0xffffffffu : ((1u << c->W) - 1u);
+    c->cur_layer = layer;
+    for (int e = 0; e < c->E; ++e) c->hist[layer * c->E + e] = (c->hist[layer * c->E + e] << 1) & mask;
     memset(c->guard, 0, (size_t)c->S);
     for (int i = 0; i < nU; ++i) {
         int32_t s = c->slot_of[layer * c->E + U[i]];
@@ -597,6 +643,7 @@ int orc_cache_step(orc_cache_t *c, int layer, const int32_t *U, int nU, int next
     for (int i = 0; i < nU; ++i) {
         int32_t key = layer * c->E + U[i];
         int64_t s = c->slot_of[key];
+        if (c->W > 0) c->hist[key] |= 1u;
         if (s >= 0) {
             c->hits += 1;
             if (c->pf_unused[s]) c->pf_useful += 1, c->pf_unused[s] = 0;
@@ -625,6 +672,7 @@ int orc_cache_step(orc_cache_t *c, int layer, const int32_t *U, int nU, int next
             continue;
         }
         int64_t s = (limit > 0 && issued >= limit) ? -1 : cache_victim(c);
+        if (s >= 0 && c->floor >= 0 && cache_uses(c, s) > c->floor) s = -1;
         if (s < 0) {
             c->pf_dropped += 1;
             continue;
