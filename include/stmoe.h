@@ -117,6 +117,7 @@ typedef struct {
     double gate_up_ms;        /* summed device time of the timed gate/up kernels          */
     double down_ms;           /* summed device time of the timed down kernels             */
     double router_ms;         /* summed device time of the timed router kernels           */
+    int64_t recovered_faults; /* slot-table inconsistencies found at verification and repaired by a demand load */
 } stmoe_stats_t;
 
 /* Create a stack for the current CUDA device.  Allocates weight storage (HBM
@@ -182,6 +183,57 @@ int stmoe_set_kernel_timing(stmoe_t *s, int on);
  * whole predicted set, the paper's policy; higher values trade recall for fewer wasted copies.
  * Between decode steps; routing, outputs and predictor tables are unaffected. */
 int stmoe_set_prefetch_min_score(stmoe_t *s, int min_score);
+
+/* Replacement policy of the HBM slot cache (the paper stages predicted experts and fetches
+ * misses at once, Section 4.3.4, and names no replacement policy).  Victims are taken in this
+ * order among the slots not needed by the step in progress: empty slots; the expert with the
+ * fewest uses in its history window (history_window bits per expert: routed at its layer's turn i
+ * decode steps ago; 0: not counted); with by_turn, the expert whose layer's next turn in the
+ * cyclic layer walk is furthest away; the least recently used; the lowest slot.  0, 0 is plain
+ * LRU.  prefetch_floor >= 0: a prefetch only takes a slot whose expert has at most that many uses
+ * in its window (0: only slots without recent use), otherwise the prediction is dropped; -1: no
+ * such test (every predicted expert is prefetched, the paper's behaviour).
+ * Default: LRU when a decode step cannot touch more experts than there are slots
+ * (n_layers * min(n_experts, max_batch * top_k) <= cache_slots), else a 16-step window with
+ * by_turn (LRU has hit rate zero on a cyclic walk that is larger than the cache); floor -1.
+ * Only before the first decode step of an offloaded stack. */
+int stmoe_set_cache_policy(stmoe_t *s, int history_window, int by_turn, int prefetch_floor);
+
+/* Bandwidth sensitivity (the paper's off-chip bandwidth axis): expert copies host -> HBM are issued
+ * in chunks of chunk_bytes with gap_us of idle time on the copy stream after each, which lowers
+ * the effective link speed to chunk_bytes / (chunk_bytes / link + gap_us).  0, 0: whole images at
+ * full speed (default).  Offloaded stacks, between decode steps. */
+int stmoe_set_copy_throttle(stmoe_t *s, int64_t chunk_bytes, int gap_us);
+
+/* Host-side fault injection for tests (nothing here faults or hangs the GPU).  Offloaded stacks,
+ * between decode steps:
+ *   DROP_PREFETCH n   the next n prefetch requests are lost (counted as dropped); the experts
+ *                     are demand-loaded if routed
+ *   FAIL_COPY n       the n-th next expert copy reports failure: the layer step returns
+ *                     STMOE_ERR_CUDA and the stack is failed until stmoe_import_state
+ *   DELAY_COPY_US us  the next expert copy is preceded by us microseconds (<= 10000) of idle
+ *                     time on the copy stream; the consuming kernels wait on the slot's event
+ *   CORRUPT_TAG slot  the slot's tag is overwritten: verification finds the mismatch, reloads
+ *                     the expert and counts it in recovered_faults
+ *   HOST_WAIT_MS ms   limit of the host's wait for a layer's routing (default 20000); when it
+ *                     runs out the step returns STMOE_ERR_TIMEOUT
+ * Any stack: POLL_LIMIT n = polls after which a grid-barrier wait of the single-sequence
+ * persistent kernel gives up (default 2^22). */
+#define STMOE_HOOK_DROP_PREFETCH 1
+#define STMOE_HOOK_FAIL_COPY 2
+#define STMOE_HOOK_DELAY_COPY_US 3
+#define STMOE_HOOK_CORRUPT_TAG 4
+#define STMOE_HOOK_HOST_WAIT_MS 5
+#define STMOE_HOOK_POLL_LIMIT 6
+int stmoe_test_hook(stmoe_t *s, int what, int64_t value);
+
+/* Runs the bounded waits of the persistent kernels on barriers that nobody completes, with a poll
+ * limit of a few thousand: which = 0 the grid barrier of the three-phase kernel, 1 the grid barrier
+ * of the single-sequence kernel, 2 an mbarrier wait of the tensor-core kernels, 3 the mbarrier wait
+ * of the single-sequence kernel's copy ring.  Each wait gives up, the stack's error word is set
+ * and stmoe_stats returns STMOE_ERR_TIMEOUT from then on (destroy the stack afterwards); the
+ * kernel itself ends normally.  Asynchronous on cuda_stream. */
+int stmoe_selftest_bounded_wait(stmoe_t *s, int which, int poll_limit, void *cuda_stream);
 
 /* On-chip staging in the single-sequence persistent decode step of resident stacks: the paper's
  * idea of fetching experts before they are needed (Sections 4.1, 4.3.4), one memory level down.

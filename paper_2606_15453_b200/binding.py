@@ -20,6 +20,7 @@ FLAG_RENORM_TOPK = 1
 FLAG_NO_PERSISTENT = 2
 FLAG_NO_DENSE = 4
 FLAG_NO_FUSED = 8
+HOOK_DROP_PREFETCH, HOOK_FAIL_COPY, HOOK_DELAY_COPY_US, HOOK_CORRUPT_TAG, HOOK_HOST_WAIT_MS, HOOK_POLL_LIMIT = 1, 2, 3, 4, 5, 6
 
 
 class StmoeError(RuntimeError):
@@ -41,7 +42,7 @@ class Stats(C.Structure):
         "prefetch_resident", "h2d_bytes_demand", "h2d_bytes_prefetch")] + \
         [("transfer_ms", C.c_double), ("exposed_ms", C.c_double), ("kernel_launches", C.c_int64),
          ("timed_ffn_launches", C.c_int64), ("gate_up_ms", C.c_double), ("down_ms", C.c_double),
-         ("router_ms", C.c_double)]
+         ("router_ms", C.c_double), ("recovered_faults", C.c_int64)]
 
 
 _lib = None
@@ -68,6 +69,10 @@ def lib():
         L.stmoe_set_dense_min_batch.argtypes = [vp, i32]
         L.stmoe_set_prefetch_min_score.argtypes = [vp, i32]
         L.stmoe_set_onchip_staging.argtypes = [vp, i64, i64]
+        L.stmoe_set_cache_policy.argtypes = [vp, i32, i32, i32]
+        L.stmoe_set_copy_throttle.argtypes = [vp, i64, i32]
+        L.stmoe_test_hook.argtypes = [vp, i32, i64]
+        L.stmoe_selftest_bounded_wait.argtypes = [vp, i32, i32, vp]
         L.stmoe_stats.argtypes = [vp, C.POINTER(Stats)]
         L.stmoe_export_state.argtypes = [vp, vp, C.POINTER(sz)]
         L.stmoe_import_state.argtypes = [vp, vp, sz]
@@ -182,6 +187,20 @@ class Stack:
     def set_onchip_staging(self, known_bytes: int, predicted_bytes: int) -> None:
         _check(lib().stmoe_set_onchip_staging(self._h, int(known_bytes), int(predicted_bytes)),
                "stmoe_set_onchip_staging")
+
+    def set_cache_policy(self, history_window: int, by_turn: bool, prefetch_floor: int = -1) -> None:
+        _check(lib().stmoe_set_cache_policy(self._h, int(history_window), int(by_turn), int(prefetch_floor)),
+               "stmoe_set_cache_policy")
+
+    def set_copy_throttle(self, chunk_bytes: int, gap_us: int) -> None:
+        _check(lib().stmoe_set_copy_throttle(self._h, int(chunk_bytes), int(gap_us)), "stmoe_set_copy_throttle")
+
+    def test_hook(self, what: int, value: int) -> None:
+        _check(lib().stmoe_test_hook(self._h, int(what), int(value)), "stmoe_test_hook")
+
+    def selftest_bounded_wait(self, which: int, poll_limit: int = 4096, stream=None) -> None:
+        _check(lib().stmoe_selftest_bounded_wait(self._h, int(which), int(poll_limit), _stream(stream)),
+               "stmoe_selftest_bounded_wait")
 
     def set_dense_min_batch(self, min_batch: int) -> None:
         _check(lib().stmoe_set_dense_min_batch(self._h, int(min_batch)), "stmoe_set_dense_min_batch")

@@ -41,9 +41,10 @@ __device__ __forceinline__ void dmbar_arrive(uint64_t *bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(dsmem_u32(bar)) : "memory");
 }
 // bounded wait on a phase parity; false when the limit ran out or another thread gave up
-__device__ __forceinline__ bool dmbar_wait(uint64_t *bar, uint32_t parity, volatile int *dead)
+__device__ __forceinline__ bool dmbar_wait(uint64_t *bar, uint32_t parity, volatile int *dead,
+                                           int spin_limit = kDenseSpinLimit)
 {
-    for (int spins = 0; spins < kDenseSpinLimit; ++spins) {
+    for (int spins = 0; spins < spin_limit; ++spins) {
         uint32_t done;
         asm volatile(
             "{.reg .pred p;\n\t"

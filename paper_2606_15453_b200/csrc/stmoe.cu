@@ -8,6 +8,7 @@
 #include <deque>
 #include <new>
 #include <set>
+#include <tuple>
 #include <utility>
 #include <vector>
 
@@ -201,29 +202,49 @@ struct WorkListMem {
 };
 
 // ---- host-side slot cache (verification, miss loading, prefetch; Sections 4.1, 4.3.4) ---
-// LRU on a clock that ticks once per layer step, lowest slot on equal stamps, empty slots
-// (stamp -1) first.  Kept in an ordered set so a victim is found without scanning all slots.
+// Victim order among the slots not protected in the current step: empty slots first, then the key
+// with the fewest uses in its history window (W bits per key: routed at its layer's turn i decode
+// steps ago), then (by_turn) the key whose layer's next turn is furthest away in the cyclic layer
+// walk, then the least recently used on a clock that ticks once per layer step, then the lowest
+// slot.  W = 0 without by_turn is plain LRU.  One ordered set per layer (uses, stamp, slot) makes a
+// victim a walk over the layers' first unprotected entries; only the keys of the layer in progress
+// change their use counts when its history shifts.
 struct SlotCache {
     int64_t S = 0, clock = 0;
-    int E = 0;
+    int E = 0, L = 0, W = 0, floor = -1, cur_layer = 0;
+    bool by_turn = false;
     std::vector<int32_t> slot_of, tag;
     std::vector<int64_t> stamp;
+    std::vector<uint32_t> hist;
     std::vector<uint8_t> pf_unused, guard;
-    std::set<std::pair<int64_t, int32_t>> order;  // (stamp, slot)
+    typedef std::tuple<int, int64_t, int32_t> Key;  // (uses, stamp, slot)
+    std::vector<std::set<Key>> by_layer;
+    std::set<int32_t> empty;
     std::vector<int32_t> guarded;
     int64_t hits = 0, misses = 0, pf_issued = 0, pf_useful = 0, pf_wasted = 0, pf_dropped = 0,
-            pf_resident = 0;
+            pf_resident = 0, tag_mismatches = 0;
 
-    void init(int64_t slots, int L, int experts)
+    void init(int64_t slots, int layers, int experts)
     {
-        S = slots, E = experts;
+        S = slots, E = experts, L = layers, clock = 0;
         slot_of.assign((size_t)L * E, -1);
         tag.assign((size_t)S, -1);
         stamp.assign((size_t)S, -1);
+        hist.assign((size_t)L * E, 0u);
         pf_unused.assign((size_t)S, 0);
         guard.assign((size_t)S, 0);
-        for (int32_t s = 0; s < S; ++s) order.insert({-1, s});
+        by_layer.assign((size_t)L, std::set<Key>());
+        empty.clear();
+        guarded.clear();
+        for (int32_t s = 0; s < S; ++s) empty.insert(s);
     }
+    static int popcount(uint32_t v)
+    {
+        int n = 0;
+        for (; v; v &= v - 1) ++n;
+        return n;
+    }
+    Key key_of(int32_t s) const { return Key(popcount(hist[tag[s]]), stamp[s], s); }
     void protect(int32_t s)
     {
         if (!guard[s]) guard[s] = 1, guarded.push_back(s);
@@ -233,27 +254,71 @@ struct SlotCache {
         for (int32_t s : guarded) guard[s] = 0;
         guarded.clear();
     }
-    void touch(int32_t s)
+    // a new turn of `layer`: its keys' histories shift by one
+    void begin_step(int layer)
     {
-        order.erase({stamp[s], s});
-        stamp[s] = clock;
-        order.insert({stamp[s], s});
+        cur_layer = layer;
+        const uint32_t mask = W >= 32 ? 0xffffffffu : ((1u << W) - 1u);
+        for (int e = 0; e < E; ++e) {
+            const int32_t key = layer * E + e;
+            const uint32_t h = (hist[key] << 1) & mask;
+            if (h == hist[key]) continue;
+            const int32_t s = slot_of[key];
+            if (s >= 0) by_layer[layer].erase(key_of(s));
+            hist[key] = h;
+            if (s >= 0) by_layer[layer].insert(key_of(s));
+        }
     }
+    // the routed key in slot s is used now
+    void use(int32_t s)
+    {
+        const int layer = tag[s] / E;
+        by_layer[layer].erase(key_of(s));
+        if (W > 0) hist[tag[s]] |= 1u;
+        stamp[s] = clock;
+        by_layer[layer].insert(key_of(s));
+    }
+    int uses_of(int32_t s) const { return tag[s] < 0 ? -1 : popcount(hist[tag[s]]); }
     int32_t victim() const
     {
-        for (const auto &it : order)
-            if (!guard[it.second]) return it.second;
-        return -1;
+        if (!empty.empty()) return *empty.begin();
+        bool have = false;
+        Key best;
+        int best_wait = 0;
+        for (int m = 0; m < L; ++m) {
+            auto it = by_layer[m].begin();
+            while (it != by_layer[m].end() && guard[std::get<2>(*it)]) ++it;
+            if (it == by_layer[m].end()) continue;
+            int wait = 0;
+            if (by_turn) {
+                wait = (m - cur_layer) % L;
+                if (wait < 0) wait += L;
+                if (wait == 0) wait = L;
+            }
+            const Key &k = *it;
+            const bool better = !have || std::get<0>(k) < std::get<0>(best) ||
+                                (std::get<0>(k) == std::get<0>(best) &&
+                                 (wait > best_wait ||
+                                  (wait == best_wait && (std::get<1>(k) < std::get<1>(best) ||
+                                                         (std::get<1>(k) == std::get<1>(best) && std::get<2>(k) < std::get<2>(best))))));
+            if (better) best = k, best_wait = wait, have = true;
+        }
+        return have ? std::get<2>(best) : -1;
     }
     void place(int32_t s, int32_t key, bool by_prefetch)
     {
         if (tag[s] >= 0) {
+            by_layer[tag[s] / E].erase(key_of(s));
             slot_of[tag[s]] = -1;
             if (pf_unused[s]) ++pf_wasted;
+        } else {
+            empty.erase(s);
         }
         tag[s] = key, slot_of[key] = s;
+        if (!by_prefetch && W > 0) hist[key] |= 1u;
         pf_unused[s] = by_prefetch;
-        touch(s);
+        stamp[s] = clock;
+        by_layer[key / E].insert(key_of(s));
     }
 };
 
@@ -337,6 +402,9 @@ struct stmoe {
     long long stage_down_bytes = 0, stage_pred_bytes = 0;
     int stage_shared = 0;
     int prefetch_min_score = 0;  // queue entries below this summed score are not prefetched
+    int host_wait_ms = kWaitTimeoutMs;     // limit of the host's wait for a layer's routing
+    int throttle_chunk = 0, throttle_gap_us = 0;  // expert copies in chunks with idle gaps (0: whole images)
+    int hook_drop_prefetch = 0, hook_fail_copy = 0, hook_delay_us = 0;  // host-side fault injection (tests)
     SlotCache cache;
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_route = nullptr;
@@ -421,6 +489,41 @@ int launch_predictor(stmoe *s, int layer, int batch, const int32_t *cur, const i
     return STMOE_OK;
 }
 
+// Bounded idle time on a stream (copy throttle, injected delays): spins on the global timer.
+__global__ void delay_kernel(long long ns)
+{
+    unsigned long long t0, t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+    for (int i = 0; i < (1 << 22); ++i) {
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        if ((long long)(t - t0) >= ns) break;
+        __nanosleep(200);
+    }
+}
+
+// One expert image host -> slot on the copy stream, whole or in throttled chunks.
+int copy_image(stmoe *s, int32_t slot, const uint8_t *src)
+{
+    if (s->hook_fail_copy > 0 && --s->hook_fail_copy == 0) return STMOE_ERR_CUDA;  // injected failure
+    if (s->hook_delay_us > 0) {
+        delay_kernel<<<1, 1, 0, s->copy_stream>>>(std::min<long long>(s->hook_delay_us, 10000) * 1000ll);
+        s->hook_delay_us = 0;
+    }
+    uint8_t *dst = s->d_slots + (size_t)slot * s->img_bytes;
+    if (s->throttle_chunk <= 0) {
+        CU_TRY(cudaMemcpyAsync(dst, src, s->img_bytes, cudaMemcpyHostToDevice, s->copy_stream));
+    } else {
+        for (size_t o = 0; o < s->img_bytes; o += (size_t)s->throttle_chunk) {
+            const size_t n = std::min(s->img_bytes - o, (size_t)s->throttle_chunk);
+            CU_TRY(cudaMemcpyAsync(dst + o, src + o, n, cudaMemcpyHostToDevice, s->copy_stream));
+            if (s->throttle_gap_us > 0) delay_kernel<<<1, 1, 0, s->copy_stream>>>((long long)s->throttle_gap_us * 1000ll);
+        }
+    }
+    CU_TRY(cudaEventRecord(s->slot_ready[slot], s->copy_stream));
+    s->slot_pending[slot] = 1;
+    return STMOE_OK;
+}
+
 // Verification, miss loading and prefetch for one layer step of an offloaded stack.
 int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
 {
@@ -442,8 +545,7 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
             (void)cudaGetLastError();
             return STMOE_ERR_CUDA;
         }
-        if (std::chrono::steady_clock::now() - t0 > std::chrono::milliseconds(kWaitTimeoutMs))
-            return STMOE_ERR_TIMEOUT;
+        if (std::chrono::steady_clock::now() - t0 > std::chrono::milliseconds(s->host_wait_ms)) return STMOE_ERR_TIMEOUT;
     }
     harvest_spans(s, false);
 
@@ -451,27 +553,29 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
     for (int i = 0; i < batch * K; ++i) routed[s->h_ids[i]] = 1;
 
     // verify: hits and demand loads (ascending expert id)
+    ch.begin_step(layer);
     ch.unprotect_all();
-    for (int e = 0; e < E; ++e)
-        if (routed[e] && ch.slot_of[(size_t)layer * E + e] >= 0) ch.protect(ch.slot_of[(size_t)layer * E + e]);
+    for (int e = 0; e < E; ++e) {
+        if (!routed[e]) continue;
+        const int32_t key = layer * E + e, sl = ch.slot_of[key];
+        if (sl >= 0 && ch.tag[sl] != key) {  // the slot does not hold what the table says: forget the entry, load again
+            ch.slot_of[key] = -1;
+            ++ch.tag_mismatches;
+        } else if (sl >= 0) {
+            ch.protect(sl);
+        }
+    }
     std::vector<cudaEvent_t> wait_on;
     bool any_copy = false;
     cudaEvent_t span_a = nullptr, span_b = nullptr;
-    auto begin_copies = [&]() -> int {
-        if (any_copy) return STMOE_OK;
-        ST_TRY(get_event(s, &span_a));
-        ST_TRY(get_event(s, &span_b));
-        CU_TRY(cudaEventRecord(span_a, s->copy_stream));
-        any_copy = true;
-        return STMOE_OK;
-    };
     auto copy_into = [&](int32_t slot, int lyr, int e) -> int {
-        ST_TRY(begin_copies());
-        CU_TRY(cudaMemcpyAsync(s->d_slots + (size_t)slot * s->img_bytes, image_ptr(s, lyr, e, false),
-                               s->img_bytes, cudaMemcpyHostToDevice, s->copy_stream));
-        CU_TRY(cudaEventRecord(s->slot_ready[slot], s->copy_stream));
-        s->slot_pending[slot] = 1;
-        return STMOE_OK;
+        if (!any_copy) {
+            ST_TRY(get_event(s, &span_a));
+            ST_TRY(get_event(s, &span_b));
+            CU_TRY(cudaEventRecord(span_a, s->copy_stream));
+            any_copy = true;
+        }
+        return copy_image(s, slot, image_ptr(s, lyr, e, false));
     };
     for (int e = 0; e < E; ++e) {
         if (!routed[e]) continue;
@@ -480,7 +584,7 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
         if (slot >= 0) {
             ++ch.hits;
             if (ch.pf_unused[slot]) ++ch.pf_useful, ch.pf_unused[slot] = 0;
-            ch.touch(slot);
+            ch.use(slot);
         } else {
             slot = ch.victim();
             if (slot < 0) return STMOE_ERR_STATE;
@@ -530,7 +634,9 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
             ++ch.pf_resident;
             continue;
         }
-        const int32_t slot = (c.prefetch_limit > 0 && issued >= c.prefetch_limit) ? -1 : ch.victim();
+        int32_t slot = (c.prefetch_limit > 0 && issued >= c.prefetch_limit) ? -1 : ch.victim();
+        if (slot >= 0 && ch.floor >= 0 && ch.uses_of(slot) > ch.floor) slot = -1;  // only slots without recent use
+        if (slot >= 0 && s->hook_drop_prefetch > 0) --s->hook_drop_prefetch, slot = -1;  // injected: a lost request
         if (slot < 0) {
             ++ch.pf_dropped;
             continue;
@@ -1178,6 +1284,9 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
         CR_TRY(cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking));
         CR_TRY(cudaEventCreateWithFlags(&s->ev_route, cudaEventDisableTiming));
         s->cache.init(c.cache_slots, L, E);
+        // A decode step that can touch more (layer, expert) keys than there are slots walks the
+        // cache in a cycle: use counts and the turn order decide there; otherwise plain LRU.
+        if ((int64_t)L * std::min(E, B * K) > c.cache_slots) s->cache.W = 16, s->cache.by_turn = true;
         s->slot_ready.resize((size_t)c.cache_slots);
         s->slot_pending.assign((size_t)c.cache_slots, 0);
         for (auto &e : s->slot_ready) CR_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
@@ -1315,6 +1424,60 @@ int stmoe_set_prefetch_min_score(stmoe_t *s, int min_score)
     if (!s || min_score < 0 || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
     s->prefetch_min_score = min_score;
     return STMOE_OK;
+}
+
+int stmoe_selftest_bounded_wait(stmoe_t *s, int which, int poll_limit, void *cuda_stream)
+{
+    if (!s || which < 0 || which > 3 || poll_limit < 1 || poll_limit > (1 << 16)) return STMOE_ERR_BAD_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (!s->d_barrier) CU_TRY(cudaMalloc(&s->d_barrier, 16));
+    CU_TRY(cudaMemsetAsync(s->d_barrier, 0, 4, st));
+    bounded_wait_selftest_kernel<<<2, 64, 0, st>>>(s->d_barrier, s->d_err, which, poll_limit);
+    CU_TRY(cudaGetLastError());
+    return STMOE_OK;
+}
+
+int stmoe_set_cache_policy(stmoe_t *s, int history_window, int by_turn, int prefetch_floor)
+{
+    if (!s || !offloaded(s) || history_window < 0 || history_window > 32 || prefetch_floor < -1 || s->next_layer != 0 ||
+        s->cache.clock != 0)
+        return STMOE_ERR_BAD_ARG;
+    s->cache.W = history_window, s->cache.by_turn = by_turn != 0, s->cache.floor = prefetch_floor;
+    return STMOE_OK;
+}
+
+int stmoe_set_copy_throttle(stmoe_t *s, int64_t chunk_bytes, int gap_us)
+{
+    if (!s || !offloaded(s) || chunk_bytes < 0 || chunk_bytes > (1ll << 30) || gap_us < 0 || gap_us > 10000 ||
+        s->next_layer != 0)
+        return STMOE_ERR_BAD_ARG;
+    s->throttle_chunk = (int)chunk_bytes, s->throttle_gap_us = gap_us;
+    return STMOE_OK;
+}
+
+int stmoe_test_hook(stmoe_t *s, int what, int64_t value)
+{
+    if (!s || value < 0 || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
+    if (what != STMOE_HOOK_POLL_LIMIT && !offloaded(s)) return STMOE_ERR_BAD_ARG;
+    switch (what) {
+    case STMOE_HOOK_DROP_PREFETCH: s->hook_drop_prefetch = (int)value; return STMOE_OK;
+    case STMOE_HOOK_FAIL_COPY: s->hook_fail_copy = (int)value; return STMOE_OK;
+    case STMOE_HOOK_DELAY_COPY_US: s->hook_delay_us = (int)std::min<int64_t>(value, 10000); return STMOE_OK;
+    case STMOE_HOOK_CORRUPT_TAG:
+        if (value >= s->cfg.cache_slots || s->cache.tag[(size_t)value] < 0) return STMOE_ERR_BAD_ARG;
+        // the slot now claims another expert of the same layer (the table entry of the true key stays)
+        {
+            SlotCache &ch = s->cache;
+            const int32_t sl = (int32_t)value, key = ch.tag[sl], layer = key / ch.E;
+            ch.by_layer[layer].erase(ch.key_of(sl));
+            ch.tag[sl] = layer * ch.E + (key % ch.E + 1) % ch.E;
+            ch.by_layer[layer].insert(ch.key_of(sl));
+        }
+        return STMOE_OK;
+    case STMOE_HOOK_HOST_WAIT_MS: s->host_wait_ms = (int)std::min<int64_t>(value, kWaitTimeoutMs); return STMOE_OK;
+    case STMOE_HOOK_POLL_LIMIT: s->poll_limit = (int)std::min<int64_t>(std::max<int64_t>(value, 1), kBarrierSpinLimit); return STMOE_OK;
+    default: return STMOE_ERR_BAD_ARG;
+    }
 }
 
 int stmoe_set_onchip_staging(stmoe_t *s, int64_t known_bytes, int64_t predicted_bytes)
@@ -1481,6 +1644,7 @@ int stmoe_stats(stmoe_t *s, stmoe_stats_t *out)
     out->prefetch_issued = ch.pf_issued, out->prefetch_useful = ch.pf_useful;
     out->prefetch_wasted = ch.pf_wasted, out->prefetch_dropped = ch.pf_dropped;
     out->prefetch_resident = ch.pf_resident;
+    out->recovered_faults = ch.tag_mismatches;
     out->h2d_bytes_demand = s->bytes_demand, out->h2d_bytes_prefetch = s->bytes_prefetch;
     out->transfer_ms = s->transfer_ms, out->exposed_ms = s->exposed_ms;
     out->kernel_launches = s->launches, out->timed_ffn_launches = s->timed_ffn;
@@ -1547,6 +1711,13 @@ int stmoe_import_state(stmoe_t *s, const void *buf, size_t bytes)
     CU_TRY(cudaMemset(s->pst.pred_valid, 0, (size_t)c.max_batch * 4));
     s->host_t = t;
     s->built = hdr[7] != 0;
+    if (s->failed && offloaded(s)) {  // the slot table may be mid-step: start from an empty cache, same policy
+        const int W = s->cache.W, floor = s->cache.floor;
+        const bool by_turn = s->cache.by_turn;
+        s->cache.init(c.cache_slots, c.n_layers, c.n_experts);
+        s->cache.W = W, s->cache.floor = floor, s->cache.by_turn = by_turn;
+        std::fill(s->slot_pending.begin(), s->slot_pending.end(), 0);
+    }
     s->failed = false, s->next_layer = 0;  // the image is a state between decode steps
     return STMOE_OK;
 }

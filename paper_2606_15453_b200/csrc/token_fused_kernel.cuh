@@ -247,9 +247,9 @@ __device__ __forceinline__ void fused_issue(const FusedArgs &fa, size_t idx, int
 
 // Bounded wait for a stage's copies: the hardware suspends the thread inside try_wait (up to the
 // hint, in nanoseconds), so a waiting unit issues few instructions beside a working one.
-__device__ __forceinline__ bool fused_wait(uint64_t *bar, uint32_t parity, volatile int *dead)
+__device__ __forceinline__ bool fused_wait(uint64_t *bar, uint32_t parity, volatile int *dead, int spin_limit = 1 << 22)
 {
-    for (int spins = 0; spins < (1 << 18); ++spins) {
+    for (int spins = 0; spins < spin_limit; ++spins) {
         uint32_t ok;
         asm volatile(
             "{.reg .pred p;\n\t"
@@ -699,6 +699,34 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
 #pragma unroll
             for (int e = 0; e < EPL; e += 4)
                 *reinterpret_cast<float4 *>(a.h_out + c0[j] + e) = make_float4(h[j][e], h[j][e + 1], h[j][e + 2], h[j][e + 3]);
+    }
+}
+
+// The bounded waits of the persistent kernels, run on barriers that nobody completes: two CTAs of
+// 64 threads call the same helpers the kernels use, with a small poll limit; every wait gives up,
+// raises the error word and returns.  which: 0 grid_barrier (token_kernel.cuh), 1 cta_wait
+// (this file), 2 dmbar_wait (tensor-core kernels), 3 fused_wait (this file's copy ring).
+__global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(unsigned *counter, unsigned *err, int which, int limit)
+{
+    __shared__ int s_dead;
+    __shared__ __align__(8) uint64_t s_bar;
+    if (threadIdx.x == 0) {
+        s_dead = 0;
+        dmbar_init(&s_bar, 1);  // one arrival expected, none comes
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (which == 0) {
+        unsigned target = 1;  // one more arrival than there are CTAs
+        grid_barrier(counter, err, target, &s_dead, -1, limit);
+    } else if (which == 1) {
+        const CtaBar cb{0, 64};
+        cta_arrive(cb, counter);
+        cta_wait(cb, counter, err, gridDim.x + 1, &s_dead, limit);
+    } else if (which == 2) {
+        if (!dmbar_wait(&s_bar, 0u, &s_dead, limit) && threadIdx.x == 0) *err = 1u;
+    } else {
+        if (!fused_wait(&s_bar, 0u, &s_dead, limit) && threadIdx.x == 0) *err = 1u;
     }
 }
 

@@ -211,7 +211,7 @@ __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int lay
 
 // Bounded grid barrier on a monotonically increasing counter.
 __device__ __forceinline__ void grid_barrier(unsigned *counter, unsigned *err, unsigned &target, volatile int *s_dead,
-                                             int dbg_idx = -1)
+                                             int dbg_idx = -1, int spin_limit = kBarrierSpinLimit)
 {
     target += gridDim.x;
     __syncthreads();
@@ -227,7 +227,7 @@ __device__ __forceinline__ void grid_barrier(unsigned *counter, unsigned *err, u
             unsigned seen;
             asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
             if (seen >= target) break;
-            if (++spins > kBarrierSpinLimit || ((spins & 255) == 0 && *((volatile unsigned *)err))) {
+            if (++spins > spin_limit || ((spins & 255) == 0 && *((volatile unsigned *)err))) {
                 *err = 1u;
                 *s_dead = 1;
                 break;

@@ -10,6 +10,13 @@ from oracle.stack import OracleStack
 TOL = {"f32": 1e-4, "bf16": 2e-2, "fp8": 5e-2}   # max|err| / ||ref||_inf
 
 
+def cache_policy(cfg, batch):
+    """The slot-cache policy the library picks by default: plain LRU unless a decode step can touch
+    more (layer, expert) keys than there are slots, then a 16-step use window and the turn order."""
+    cyclic = cfg.n_layers * min(cfg.n_experts, batch * cfg.top_k) > cfg.cache_slots
+    return dict(window=16 if cyclic else 0, by_turn=cyclic)
+
+
 def rel_err(got, ref):
     got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
     return float(np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-30))

@@ -10,7 +10,7 @@ import torch
 import oracle as O
 import paper_2606_15453_b200 as P
 from datagen import stacks
-from helpers import Pair, check_layer, decode_tokens_vs_oracle as _decode_token_vs_oracle
+from helpers import Pair, cache_policy, check_layer, decode_tokens_vs_oracle as _decode_token_vs_oracle
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -70,7 +70,9 @@ def test_slot_manager_at_c3_depth_and_slot_count(B):
     npred = torch.empty(L, B, dtype=torch.int32, device=DEV)
     ho = torch.empty(B, cfg.hidden, device=DEV)
     replay = O.Predictor(L, cfg.n_experts, K, B, cfg.profile_tokens, "st")
-    cache = O.CacheModel(cfg.cache_slots, L, cfg.n_experts)
+    policy = cache_policy(cfg, B)
+    assert policy["by_turn"] == (B == 16)       # batch 16 touches 48 x 128 keys per step, more than 1536 slots
+    cache = O.CacheModel(cfg.cache_slots, L, cfg.n_experts, **policy)
     for t in range(T):
         pr.stack.decode_token(x[t], ho, ids, None, pred, npred)
         torch.cuda.synchronize()

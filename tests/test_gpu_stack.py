@@ -7,7 +7,7 @@ import torch
 import oracle as O
 import paper_2606_15453_b200 as P
 from datagen import stacks
-from helpers import Pair, check_layer
+from helpers import Pair, cache_policy, check_layer
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -20,7 +20,7 @@ def _teacher_forced(cfg, B, tokens, mode="st", prefetch_limit=0, flags=0, min_sc
         pr.stack.set_prefetch_min_score(min_score)
     x = stacks.token_inputs(cfg, B, tokens).numpy()
     replay = O.Predictor(cfg.n_layers, cfg.n_experts, cfg.top_k, B, cfg.profile_tokens, mode)
-    cache = O.CacheModel(cfg.cache_slots, cfg.n_layers, cfg.n_experts) if cfg.cache_slots else None
+    cache = O.CacheModel(cfg.cache_slots, cfg.n_layers, cfg.n_experts, **cache_policy(cfg, B)) if cfg.cache_slots else None
     skipped = 0
     for t in range(tokens):
         h = x[t]
