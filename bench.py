@@ -31,11 +31,6 @@ sys.path.insert(0, ROOT)
 from datagen import stacks  # noqa: E402
 
 METRIC, UNIT = "decode_tokens_per_s", "tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_token_kernel launch, from the ncu
-# capture summarised in profiles/decode_token_kernel_c1_2layers_ncu_full.md.  The capture ran a
-# 2-layer stack of the same shape (1409.598 MB read + 4.767 MB written); traffic grows in
-# proportion to the layer count, so the full launch is that figure x layers / 2.
-NCU_TRAFFIC_BYTES_PER_LAYER = {"C1": (1409598000 + 4766976) / 2}
 
 
 def measured_peaks():
@@ -99,6 +94,8 @@ def load_stack(cfg, batch, dev, **kw):
                 w = stacks.expert_weights(cfg, l, e, shared, device=dev)
                 sc = torch.cat([w["gate_scale"], w["up_scale"], w["down_scale"]]) \
                     if cfg.dtype == "fp8" else None
+                # load_experts copies at once, outside torch's streams: the generator must be done
+                torch.cuda.current_stream().synchronize()
                 st.load_experts(l, e, w["gate"], w["up"], w["down"], sc, shared)
         del w
     return st
@@ -146,6 +143,13 @@ def cpu_oracle_sample(cfg, batch, layers, tokens, dev):
     return spent, O.get_threads()
 
 
+def workload_config(cfg, batch, world):
+    """The workload both arms (this library, the CPU oracle) are timed on: identical keys and values."""
+    return {"workload": cfg.name, "batch": batch, "layers": cfg.n_layers, "experts": cfg.n_experts,
+            "top_k": cfg.top_k, "hidden": cfg.hidden, "inter": cfg.inter, "profile_tokens": cfg.profile_tokens,
+            "parallelism": f"replicas x{world}", "l2": "inputs_larger_than_l2"}
+
+
 def run_reference(args, cfg, batch):
     """--impl reference: the oracle on the host cores, each step a bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
@@ -164,13 +168,168 @@ def run_reference(args, cfg, batch):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_token * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype,
         "data": "synthetic",
-        "config": {"workload": cfg.name, "batch": batch, "layers": cfg.n_layers,
-                   "experts": cfg.n_experts, "top_k": cfg.top_k, "hidden": cfg.hidden,
-                   "inter": cfg.inter},
+        "config": workload_config(cfg, batch, args.gpus),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def profile_value(name):
+    """A figure recorded in an ncu summary under profiles/ ("<name>: <number>" on a line of its
+    own), or None: the DRAM traffic in the roofline object comes from there, not from a literal here."""
+    import glob
+    import re
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.md"))):
+        m = re.search(r"^" + re.escape(name) + r":\s*([0-9.eE+]+)\s*$", open(path).read(), flags=re.M)
+        if m:
+            return float(m.group(1)), os.path.basename(path)
+    return None, None
+
+
+def top_kernel_name(cfg, batch, args):
+    """The kernel that dominates a decode step of this workload (one launch per step for resident stacks)."""
+    if cfg.cache_slots:
+        return "gate_up_kernel"
+    dense = not args.no_dense and ((cfg.dtype == "bf16" and batch >= (args.dense_min_batch or 2)) or
+                                   (cfg.dtype == "fp8" and batch >= (args.dense_min_batch or 3)))
+    if dense:
+        return "dense8_group_kernel<2>" if cfg.dtype == "fp8" and batch > 4 else "decode_token_dense_kernel"
+    epl = {"f32": 4, "bf16": 8, "fp8": 16}[cfg.dtype]
+    fused = batch == 1 and not args.no_fused and cfg.hidden % epl == 0 and cfg.hidden <= 4096 and \
+        cfg.hidden // epl in (64, 128, 256, 512)
+    return "decode_token_fused_kernel" if fused else "decode_token_kernel"
+
+
+def measure(cfg, batch, st, args, dev, world, stream, with_e2e):
+    """Profiling steps, warm-up, K timed decode steps on resident inputs, an untimed pass that records
+    the routing (for the algorithmic bytes), optionally the end-to-end pass.  Returns a dict."""
+    import torch.distributed as dist
+    L, K, H = cfg.n_layers, cfg.top_k, cfg.hidden
+    steps, warmup = args.steps, args.warmup
+    n_tok = cfg.profile_tokens + warmup + steps
+    x_host = stacks.token_inputs(cfg, batch, n_tok).pin_memory()
+    x_dev = x_host.to(dev)
+    h_out = torch.empty(batch, H, device=dev)
+    ids = torch.empty(L, batch, K, dtype=torch.int32, device=dev)
+    pred = torch.empty(L, batch, st.max_pred, dtype=torch.int32, device=dev)
+    npred = torch.empty(L, batch, dtype=torch.int32, device=dev)
+    h_in = torch.empty(batch, H, device=dev)
+    local = dev.index or 0
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    gap_cycles = int(args.inter_layer_gap_us * 1965)      # torch.cuda._sleep spins on the SM clock
+
+    def decode(h_src):
+        h_in.copy_(h_src)
+        if gap_cycles <= 0:
+            st.decode_token(h_in, h_out, ids, None, pred, npred)
+            return
+        for l in range(L):                                # per-layer entry point + attention stand-in
+            st.decode_step(l, h_in if l == 0 else h_out, h_out, ids[l], None, pred[l], npred[l])
+            torch.cuda._sleep(gap_cycles)
+
+    t = 0
+    for _ in range(cfg.profile_tokens + warmup):          # the profiling phase of Algorithm 1, then warm-up
+        decode(x_dev[t])
+        t += 1
+    s0 = st.stats()
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for i in range(steps):
+        decode(x_dev[t + i])
+    ev1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    s1 = st.stats()
+
+    # the routing of the same steps (it depends on the inputs only), for the algorithmic bytes
+    ids_seen = []
+    for i in range(steps):
+        decode(x_dev[t + i])
+        ids_seen.append(ids.cpu().numpy().copy())
+    e2e_ms = None
+    if with_e2e:
+        out_host = torch.empty(batch, H).pin_memory()
+        ids_host = torch.empty(L, batch, K, dtype=torch.int32).pin_memory()
+        barrier()
+        w0 = time.perf_counter()
+        for i in range(steps):
+            h_in.copy_(x_host[t + i], non_blocking=True)
+            st.decode_token(h_in, h_out, ids, None, pred, npred)
+            out_host.copy_(h_out, non_blocking=True)
+            ids_host.copy_(ids, non_blocking=True)
+            torch.cuda.synchronize()
+        e2e_ms = (time.perf_counter() - w0) * 1e3
+        barrier()
+    times = torch.tensor([ms, e2e_ms or 0.0], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = (float(v) for v in times.cpu())
+    step_bytes = [algorithmic_bytes(cfg, a) for a in ids_seen]
+    return dict(ms=ms, e2e_ms=e2e_ms, clocks=clocks, s0=s0, s1=s1, step_bytes=step_bytes, steps=steps)
+
+
+def summarise(cfg, batch, m, args, world, peak):
+    """The fields shared by the headline line and the secondary records."""
+    tokens = m["steps"] * batch * world
+    value = tokens / (m["ms"] * 1e-3)
+    step_gbs = statistics.mean(m["step_bytes"]) / (m["ms"] / m["steps"] * 1e-3) / 1e9
+    s0, s1 = m["s0"], m["s1"]
+    run = {k: s1[k] - s0[k] for k in ("runtime_steps", "routed", "predicted", "hits", "near_ties", "cache_hits",
+                                      "cache_misses", "kernel_launches", "prefetch_issued", "prefetch_useful",
+                                      "prefetch_wasted", "transfer_ms", "exposed_ms")}
+    out = {"workload": cfg.name, "batch": batch, "value": value, "unit": UNIT, "ms_per_step": m["ms"] / m["steps"],
+           "algorithmic_bytes_per_step": statistics.mean(m["step_bytes"]), "achieved_gbs": step_gbs,
+           "frac": step_gbs / peak, "frac_of_8000": step_gbs / 8000.0, "kernel": top_kernel_name(cfg, batch, args),
+           "clocks": m["clocks"], "gpu_launches": run["kernel_launches"],
+           "predictor": {"recall": run["hits"] / max(run["routed"], 1), "precision": run["hits"] / max(run["predicted"], 1),
+                         "mean_predicted": run["predicted"] / max(run["runtime_steps"], 1), "near_ties": run["near_ties"]}}
+    if cfg.cache_slots:
+        h2d = (s1["h2d_bytes_demand"] + s1["h2d_bytes_prefetch"] - s0["h2d_bytes_demand"] - s0["h2d_bytes_prefetch"])
+        transfer, exposed = run["transfer_ms"], run["exposed_ms"]
+        out["cache"] = {
+            "slots": cfg.cache_slots, "hits": run["cache_hits"], "misses": run["cache_misses"],
+            "hit_rate": run["cache_hits"] / max(run["cache_hits"] + run["cache_misses"], 1),
+            "prefetch_issued": run["prefetch_issued"], "prefetch_useful": run["prefetch_useful"],
+            "prefetch_wasted": run["prefetch_wasted"], "h2d_gb": h2d / 1e9, "transfer_ms": transfer, "exposed_ms": exposed,
+            "hidden_frac": 1.0 - exposed / max(transfer, 1e-9),
+            # no more of the transfer time can be hidden than the compute stream is busy: the rest of
+            # the step it waits for copies whatever the predictor does (the link is the bound)
+            "hidden_bound": min(1.0, max(m["ms"] - exposed, 0.0) / max(transfer, 1e-9)),
+            "prefetch_limit": args.prefetch_limit, "prefetch_min_score": args.prefetch_min_score,
+            "prefetch_floor": args.prefetch_floor, "mode": args.mode, "inter_layer_gap_us": args.inter_layer_gap_us,
+            "copy_throttle": [args.throttle_chunk_kb, args.throttle_gap_us]}
+    return out
+
+
+def make_stack(cfg, batch, dev, args):
+    import paper_2606_15453_b200 as P
+    flags = (P.FLAG_NO_DENSE if args.no_dense else 0) | (P.FLAG_NO_FUSED if args.no_fused else 0)
+    st = load_stack(cfg, batch, dev, prefetch_limit=args.prefetch_limit, mode=args.mode, flags=flags)
+    if args.prefetch_min_score:
+        st.set_prefetch_min_score(args.prefetch_min_score)
+    if args.dense_min_batch and not args.no_dense:
+        st.set_dense_min_batch(args.dense_min_batch)
+    if args.stage_known_kb >= 0 or args.stage_pred_mb >= 0:
+        st.set_onchip_staging(max(args.stage_known_kb, 0) << 10, int(max(args.stage_pred_mb, 0.0) * 1e6))
+    if cfg.cache_slots:
+        if args.cache_policy != "default" or args.prefetch_floor >= 0:
+            window, by_turn = {"default": (16, True) if cfg.n_layers * min(cfg.n_experts, batch * cfg.top_k) > cfg.cache_slots
+                               else (0, False), "lru": (0, False), "counts": (16, False), "turn": (16, True)}[args.cache_policy]
+            st.set_cache_policy(window, by_turn, args.prefetch_floor)
+        if args.throttle_chunk_kb:
+            st.set_copy_throttle(args.throttle_chunk_kb << 10, args.throttle_gap_us)
+    return st
 
 
 def main():
@@ -185,9 +344,17 @@ def main():
     ap.add_argument("--ref-layers", type=int, default=2)
     ap.add_argument("--cpu-sample-layers", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true",
+                    help="skip the short runs of the other resident configurations that the default run appends")
     ap.add_argument("--prefetch-limit", type=int, default=0, help="offloaded stacks: copies per layer step")
     ap.add_argument("--prefetch-min-score", type=int, default=0,
                     help="offloaded stacks: prefetch only predictions with at least this score")
+    ap.add_argument("--prefetch-floor", type=int, default=-1,
+                    help="offloaded stacks: a prefetch only takes a slot whose expert has at most this many uses in "
+                         "its history window (-1: no such test)")
+    ap.add_argument("--cache-policy", default="default", choices=["default", "lru", "counts", "turn"])
+    ap.add_argument("--throttle-chunk-kb", type=int, default=0, help="offloaded stacks: expert copies in chunks of this size ...")
+    ap.add_argument("--throttle-gap-us", type=int, default=0, help="... with this much idle time after each (link-speed sweep)")
     ap.add_argument("--mode", default="st", choices=["off", "temporal", "spatial", "st"])
     ap.add_argument("--inter-layer-gap-us", type=float, default=0.0,
                     help="idle the compute stream this long after every layer: a stand-in for the attention "
@@ -196,13 +363,15 @@ def main():
     ap.add_argument("--dense-min-batch", type=int, default=0,
                     help="smallest batch that takes the tcgen05 path (0: the library's default, 2 for bf16, 3 for fp8)")
     ap.add_argument("--stage-known-kb", type=int, default=-1,
-                    help="single-sequence resident steps: L2 staging of known weights, KiB per expert and SM "
+                    help="three-phase single-sequence kernel: L2 staging of known weights, KiB per expert and SM "
                          "(-1: the library's default, 0: off)")
     ap.add_argument("--stage-pred-mb", type=float, default=-1.0,
-                    help="single-sequence resident steps: MB per layer of predicted experts' rows staged into L2 "
+                    help="three-phase single-sequence kernel: MB per layer of predicted experts' rows staged into L2 "
                          "ahead of the router (-1: the library's default)")
     ap.add_argument("--no-dense", action="store_true",
                     help="batched steps of resident bf16 stacks on the CUDA-core kernels instead of the tcgen05 ones")
+    ap.add_argument("--no-fused", action="store_true",
+                    help="single-sequence resident steps on the three-phase kernel instead of the one-phase one")
     args = ap.parse_args()
 
     cfg = stacks.CONFIGS[args.workload]
@@ -228,181 +397,76 @@ def main():
 
     import paper_2606_15453_b200 as P
     P.build()
-    import paper_2606_15453_b200 as P
-    st = load_stack(cfg, batch, dev, prefetch_limit=args.prefetch_limit, mode=args.mode,
-                    flags=P.FLAG_NO_DENSE if args.no_dense else 0)  # a full replica per rank
-    if args.prefetch_min_score:
-        st.set_prefetch_min_score(args.prefetch_min_score)
-    if args.dense_min_batch and not args.no_dense:
-        st.set_dense_min_batch(args.dense_min_batch)
-    if args.stage_known_kb >= 0 or args.stage_pred_mb >= 0:
-        st.set_onchip_staging(max(args.stage_known_kb, 0) << 10,
-                              int(max(args.stage_pred_mb, 0.0) * 1e6))
-    L, K, H = cfg.n_layers, cfg.top_k, cfg.hidden
-    n_tok = cfg.profile_tokens + args.warmup + args.steps
-    x_host = stacks.token_inputs(cfg, batch, n_tok).pin_memory()
-    x_dev = x_host.to(dev)
-    h_out = torch.empty(batch, H, device=dev)
-    ids = torch.empty(L, batch, K, dtype=torch.int32, device=dev)
-    pred = torch.empty(L, batch, st.max_pred, dtype=torch.int32, device=dev)
-    npred = torch.empty(L, batch, dtype=torch.int32, device=dev)
+    default_run = (args.workload == "C1" and batch == 1 and not args.layers and not args.resident
+                   and not args.no_secondary and world == 1)
+    # the default run also times C1 at batch 4 on the same 90 GB stack (a full replica per rank)
+    st = make_stack(cfg, 4 if default_run else batch, dev, args)
     stream = torch.cuda.Stream()            # a capturable stream: decode steps replay as a CUDA graph
     torch.cuda.set_stream(stream)
-    h_in = torch.empty(batch, H, device=dev)
-
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    gap_cycles = int(args.inter_layer_gap_us * 1965)      # torch.cuda._sleep spins on the SM clock
-
-    def decode(h_src):
-        h_in.copy_(h_src)
-        if gap_cycles <= 0:
-            st.decode_token(h_in, h_out, ids, None, pred, npred)
-            return
-        for l in range(L):                                # per-layer entry point + attention stand-in
-            st.decode_step(l, h_in if l == 0 else h_out, h_out, ids[l], None, pred[l], npred[l])
-            torch.cuda._sleep(gap_cycles)
-
-    # set-up: the profiling phase of Algorithm 1, then warm-up
-    t = 0
-    for _ in range(cfg.profile_tokens + args.warmup):
-        decode(x_dev[t])
-        t += 1
-    s0 = st.stats()
-
-    # ---- timed region: K decode steps, inputs resident in HBM --------------------------------
-    sampler = ClockSampler(local)
-    barrier()
-    sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ids_seen = []
-    ev0.record(stream)
-    for i in range(args.steps):
-        decode(x_dev[t + i])
-    ev1.record(stream)
-    barrier()
-    clocks = sampler.stop()
-    ms = ev0.elapsed_time(ev1)
-    s1 = st.stats()
-
-    # ---- same steps again with the FFN kernels bracketed by events (roofline of the top kernel)
-    st.set_kernel_timing(True)
-    for i in range(args.steps):
-        h_in.copy_(x_dev[t + i])
-        st.decode_token(h_in, h_out, ids, None, pred, npred)
-        ids_seen.append(ids.cpu().numpy().copy())
-    st.set_kernel_timing(False)
-    s2 = st.stats()
-
-    # ---- end to end: pinned host input copied in, results copied out, every step -------------
-    out_host = torch.empty(batch, H).pin_memory()
-    ids_host = torch.empty(L, batch, K, dtype=torch.int32).pin_memory()
-    barrier()
-    w0 = time.perf_counter()
-    for i in range(args.steps):
-        h_in.copy_(x_host[t + i], non_blocking=True)
-        st.decode_token(h_in, h_out, ids, None, pred, npred)
-        out_host.copy_(h_out, non_blocking=True)
-        ids_host.copy_(ids, non_blocking=True)
-        torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - w0
-    barrier()
-
-    times = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = (float(v) for v in times.cpu())
+    L, K, H = cfg.n_layers, cfg.top_k, cfg.hidden
+    m = measure(cfg, batch, st, args, dev, world, stream, with_e2e=True)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    tokens = args.steps * batch * world
-    value = tokens / (ms * 1e-3)
     peak, peak_kind = measured_peaks()
-    step_bytes = [algorithmic_bytes(cfg, a) for a in ids_seen]
-    n_ffn = s2["timed_ffn_launches"]
-    gate_up_bytes = sum(sum((len(np.unique(a[l])) + cfg.n_shared) for l in range(L)) for a in ids_seen) \
-        * (2 * cfg.expert_bytes // 3) / max(n_ffn, 1)
-    gu_ms = s2["gate_up_ms"] / max(n_ffn, 1)
-    dn_ms = s2["down_ms"] / max(n_ffn, 1)
-    achieved = gate_up_bytes / (gu_ms * 1e-3) / 1e9 if gu_ms > 0 else None
-    run = {k: s1[k] - s0[k] for k in ("runtime_steps", "routed", "predicted", "hits", "near_ties",
-                                      "cache_hits", "cache_misses", "kernel_launches")}
-    step_gbs = statistics.mean(step_bytes) / (ms / args.steps * 1e-3) / 1e9
+    head = summarise(cfg, batch, m, args, world, peak)
+    tokens = args.steps * batch * world
     persistent = cfg.cache_slots == 0          # resident stacks: one kernel launch per decode step
-    # batched steps of resident bf16 stacks: expert FFN on tcgen05 tiles (the library's default threshold)
-    dense = persistent and not args.no_dense and (
-        (cfg.dtype == "bf16" and batch >= (args.dense_min_batch or 2)) or
-        (cfg.dtype == "fp8" and batch >= (args.dense_min_batch or 3)))
-    top_kernel = "gate_up_kernel"
-    if persistent:
-        top_kernel = "decode_token_kernel"
-        if dense:   # bf16 and fp8: one persistent kernel with the tcgen05 phases
-            top_kernel = "decode_token_dense_kernel"
-            if cfg.dtype == "fp8" and batch > 4:   # larger fp8 batches: per-layer tcgen05 kernels replayed as a graph
-                top_kernel = "dense8_group_kernel<2>"
-    whole_step = top_kernel.startswith("decode_token")   # the top kernel is one launch per decode step
-    per_layer = NCU_TRAFFIC_BYTES_PER_LAYER.get(args.workload) if batch == 1 else None
+    whole_step = head["kernel"].startswith("decode_token")
+    traffic, traffic_src = (None, None)
+    if whole_step and batch == 1 and args.workload == "C1" and not args.no_fused:
+        per_layer, traffic_src = profile_value("dram_bytes_per_layer_c1_batch1_" + head["kernel"])
+        traffic = per_layer * L if per_layer else None
     out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": cfg.name, "batch": batch, "layers": L, "experts": cfg.n_experts,
-                   "top_k": K, "hidden": H, "inter": cfg.inter, "parallelism": f"replicas x{world}",
-                   "profile_tokens": cfg.profile_tokens, "l2": "inputs_larger_than_l2",
-                   "ffn_path": "tcgen05 tiles (TMA-fed, TMEM accumulators)" if dense else "weight-streaming GEMV on CUDA cores",
-                   "resident_weight_gb": round(L * (cfg.n_experts + cfg.n_shared) * cfg.expert_bytes / 1e9, 1)},
-        "clocks": clocks,
-        "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT,
+        "config": workload_config(cfg, batch, world),
+        "path": {"ffn_path": {"decode_token_fused_kernel": "row triples (gate, up, transposed down) streamed by bulk "
+                                                             "copies into shared memory, CUDA-core FMAs, one phase per layer",
+                                "decode_token_kernel": "weight-streaming GEMV on CUDA cores, three phases per layer",
+                                "gate_up_kernel": "weight-streaming GEMV on CUDA cores, per-layer kernels"}.get(
+                                    head["kernel"], "tcgen05 tiles (TMA-fed, TMEM accumulators)"),
+                 "resident_weight_gb": round(L * (cfg.n_experts + cfg.n_shared) * cfg.expert_bytes / 1e9, 1)},
+        "clocks": head["clocks"],
+        "e2e": {"value": tokens / (m["e2e_ms"] * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": batch * H * 4,
                 "d2h_bytes_per_step": batch * H * 4 + L * batch * K * 4},
-        "gpu_launches": run["kernel_launches"],
-        "roofline": {"bound": "hbm",
-                     "kernel": top_kernel,
-                     "achieved": step_gbs if whole_step else achieved, "peak": peak,
-                     "peak_kind": peak_kind, "unit": "GB/s",
-                     "frac": (step_gbs if whole_step else achieved or 0.0) / peak,
-                     "frac_of_8000": (step_gbs if whole_step else achieved or 0.0) / 8000.0,
-                     "traffic": per_layer * L if (whole_step and per_layer) else None,
-                     "algorithmic_bytes_per_launch": statistics.mean(step_bytes) if whole_step else gate_up_bytes,
-                     "us_per_launch": ms / args.steps * 1e3 if whole_step else gu_ms * 1e3,
-                     "per_layer_kernels": {
-                         "note": "second pass over the same steps as per-layer kernels, events around each",
-                         "gate_up": {"achieved": achieved, "us_per_launch": gu_ms * 1e3,
-                                     "algorithmic_bytes_per_launch": gate_up_bytes},
-                         "down": {"achieved": (gate_up_bytes / 2) / (dn_ms * 1e-3) / 1e9 if dn_ms else None,
-                                  "us_per_launch": dn_ms * 1e3},
-                         "router": {"us_per_launch": s2["router_ms"] / max(n_ffn, 1) * 1e3}},
-                     "whole_step": {"bytes_per_token": statistics.mean(step_bytes) / batch,
-                                    "achieved": step_gbs, "frac": step_gbs / peak,
-                                    "frac_of_8000": step_gbs / 8000.0}},
-        "predictor": {"recall": run["hits"] / max(run["routed"], 1),
-                      "precision": run["hits"] / max(run["predicted"], 1),
-                      "mean_predicted": run["predicted"] / max(run["runtime_steps"], 1),
-                      "near_ties": run["near_ties"]},
-        "cache": {"slots": cfg.cache_slots, "hits": run["cache_hits"], "misses": run["cache_misses"],
-                  "hit_rate": run["cache_hits"] / max(run["cache_hits"] + run["cache_misses"], 1),
-                  "prefetch_issued": s1["prefetch_issued"] - s0["prefetch_issued"],
-                  "prefetch_useful": s1["prefetch_useful"] - s0["prefetch_useful"],
-                  "prefetch_wasted": s1["prefetch_wasted"] - s0["prefetch_wasted"],
-                  "h2d_gb": (s1["h2d_bytes_demand"] + s1["h2d_bytes_prefetch"]
-                             - s0["h2d_bytes_demand"] - s0["h2d_bytes_prefetch"]) / 1e9,
-                  "transfer_ms": s1["transfer_ms"] - s0["transfer_ms"],
-                  "exposed_ms": s1["exposed_ms"] - s0["exposed_ms"],
-                  "hidden_frac": 1.0 - (s1["exposed_ms"] - s0["exposed_ms"])
-                  / max(s1["transfer_ms"] - s0["transfer_ms"], 1e-9),
-                  "prefetch_limit": args.prefetch_limit, "prefetch_min_score": args.prefetch_min_score,
-                  "mode": args.mode,
-                  "inter_layer_gap_us": args.inter_layer_gap_us},
+        "gpu_launches": head["gpu_launches"],
+        "roofline": {"bound": "hbm", "kernel": head["kernel"],
+                     "achieved": head["achieved_gbs"], "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": head["frac"], "frac_of_8000": head["frac_of_8000"],
+                     "traffic": traffic, "traffic_source": traffic_src,
+                     "algorithmic_bytes_per_launch": head["algorithmic_bytes_per_step"] if persistent else None,
+                     "us_per_launch": head["ms_per_step"] * 1e3 if persistent else None,
+                     "note": None if persistent else "offloaded stack: whole-step figures; per-layer kernels, time dominated by "
+                                                     "host->HBM expert copies (see cache)"},
+        "predictor": head["predictor"],
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if "cache" in head:
+        out["cache"] = head["cache"]
+    if default_run:
+        # short runs of the other resident benchmark configurations, so that the roofline fractions
+        # of all of them are in this line (same fields each; `kernel` names what ran)
+        sec = []
+        short = argparse.Namespace(**{**vars(args), "steps": 48, "warmup": 4})
+        sec.append(summarise(cfg, 4, measure(cfg, 4, st, short, dev, world, stream, with_e2e=False), short, world, peak))
         st.close()
+        del st
         torch.cuda.empty_cache()
+        c2 = stacks.CONFIGS["C2"]
+        st2 = make_stack(c2, 8, dev, short)
+        for b in (1, 8):
+            sec.append(summarise(c2, b, measure(c2, b, st2, short, dev, world, stream, with_e2e=False), short, world, peak))
+        st2.close()
+        del st2
+        out["secondary"] = sec
+    else:
+        st.close()
+    torch.cuda.empty_cache()
+    if world == 1 and not args.no_cpu_baseline:
         layers = min(L, args.cpu_sample_layers)
         spent, cores = cpu_oracle_sample(cfg, batch, layers, 2, dev)
         per_token = spent[-1] * L / layers

@@ -135,7 +135,8 @@ int stmoe_load_router(stmoe_t *s, int layer, const void *w);
 /* Weights of experts first_expert .. first_expert+count-1 of one layer (is_shared: the
  * always-on experts).  gate, up: [count][I][H]; down: [count][H][I]; row-major in
  * weight_dtype.  scales (fp8 only, else NULL): [count][2I+H] bf16 = gate rows, up rows,
- * down rows.  Pointers may be host or device.  Synchronous. */
+ * down rows.  Pointers may be host or device.  Synchronous: the sources are read during the call
+ * (a device source must be complete: synchronise the stream that produced it first). */
 int stmoe_load_experts(stmoe_t *s, int layer, int first_expert, int count, const void *gate,
                        const void *up, const void *down, const void *scales, int is_shared);
 

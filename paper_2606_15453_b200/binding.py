@@ -151,7 +151,9 @@ class Stack:
         _check(lib().stmoe_load_router(self._h, layer, _ptr(w)), "stmoe_load_router")
 
     def load_experts(self, layer, first_expert, gate, up, down, scales=None, shared=False) -> None:
-        """gate/up [n][I][H], down [n][H][I] (or 2-D for one expert), host or device."""
+        """gate/up [n][I][H], down [n][H][I] (or 2-D for one expert), host or device.  The call copies
+        at once and does not know torch's streams: synchronise the stream that produced a device
+        source before calling."""
         count = 1 if gate.dim() == 2 else gate.shape[0]
         _check(lib().stmoe_load_experts(self._h, layer, first_expert, count, _ptr(gate), _ptr(up),
                                         _ptr(down), _ptr(scales), int(shared)), "stmoe_load_experts")

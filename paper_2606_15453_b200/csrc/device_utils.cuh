@@ -7,30 +7,6 @@
 
 namespace stmoe_dev {
 
-// Debug builds (-DSTMOE_DBG_PHASES) stamp phase boundaries of the persistent kernel with the
-// global timer; normal builds compile the stamps away.
-#ifdef STMOE_DBG_PHASES
-// per CTA 64 stamps of the SM's cycle counter (layers 0..7 x 8 phase boundaries); then CTA 0's
-// sub-phase stamps (2000.. -> 9472+) and the predictor warp's (2010.. -> 9488+)
-__device__ unsigned long long g_dbg_phases[16384];
-__device__ __forceinline__ void dbg_stamp(int idx)
-{
-    if (threadIdx.x == 0) {
-        if (idx < 64) g_dbg_phases[blockIdx.x * 64 + idx] = (unsigned long long)clock64();
-        else if (idx >= 2000 && idx < 2010 && blockIdx.x == 0) g_dbg_phases[9472 + idx - 2000] = (unsigned long long)clock64();
-    }
-}
-__device__ __forceinline__ void dbg_stamp_lane0(int idx)
-{
-    if (threadIdx.x % 32 == 0 && idx >= 2010 && idx < 2030) g_dbg_phases[9488 + idx - 2010] = (unsigned long long)clock64();
-}
-#define DBG_STAMP(i) dbg_stamp(i)
-#define DBG_STAMP_WARP(i) dbg_stamp_lane0(i)
-#else
-#define DBG_STAMP(i)
-#define DBG_STAMP_WARP(i)
-#endif
-
 constexpr int kWarp = 32;
 constexpr unsigned kFull = 0xffffffffu;
 

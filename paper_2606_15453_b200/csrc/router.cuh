@@ -517,12 +517,9 @@ __device__ __forceinline__ void router_finalize(const RouterArgs &a, int *s_ids,
     } else {
         finalize_tokens<kVplMax>(a, s_ids, nw, C);
     }
-    DBG_STAMP(2001);
     if (a.tk.wl.n_groups == nullptr) return;
     __syncthreads();
-    DBG_STAMP(2002);
     if (threadIdx.x < 256) group_tokens(s_ids, s_scan, B, E, a.tk.K, a.tk.n_shared, a.tk.mt, a.tk.wl);
-    DBG_STAMP(2003);
 }
 
 template <int DT>

@@ -1950,11 +1950,3 @@ extern "C" int stmoe_expert_ffn_dense(const float *h, const float *inv_rms, cons
     CU_TRY(cudaGetLastError());
     return STMOE_OK;
 }
-
-#ifdef STMOE_DBG_PHASES
-extern "C" int stmoe_dbg_phases(unsigned long long *out, int n)
-{
-    cudaDeviceSynchronize();
-    return cudaMemcpyFromSymbol(out, g_dbg_phases, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -3;
-}
-#endif

@@ -121,7 +121,6 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         const float *h = l == 0 ? a.h_in : a.hbuf + (size_t)l * B * H;
 
         // ---- F ---------------------------------------------------------------------------------
-        DBG_STAMP(l * 8 + 0);
         if (l == 0) {
             for (int i = gtid; i < B * H; i += gthreads) xb[i] = to_xt(h[i]);
         } else {
@@ -135,7 +134,6 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         }
         fence_async_proxy();
         grid_barrier(a.barrier, a.err, target, &s_dead);
-        DBG_STAMP(l * 8 + 1);
 
         // ---- R ---------------------------------------------------------------------------------
         RouterArgs ra;
@@ -152,7 +150,6 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         tk.wl = wl;
         router_tasks<RDT, false>(ra, warp * gridDim.x + blockIdx.x, NW * gridDim.x, lane);
         grid_barrier(a.barrier, a.err, target, &s_dead);
-        DBG_STAMP(l * 8 + 2);
 
         // ---- T ---------------------------------------------------------------------------------
         router_finalize<RDT>(ra, s_ids, s_scan, NW);
@@ -161,7 +158,6 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
             for (int i = threadIdx.x; i < B * K; i += blockDim.x) a.ids_all[(size_t)l * a.Bmax * K + i] = s_ids[i];
 
         // ---- GU (+ the predictor on one warp of the last CTA) -----------------------------------
-        DBG_STAMP(l * 8 + 3);
         Group8Args g8{};
         GroupArgs &g = g8.g;
         g.wl = wl, g.E = E, g.img_routed0 = l * E, g.img_shared0 = d.img_shared_base + l * a.n_shared;
@@ -201,8 +197,7 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
             constexpr int kFirst = WDT == 1 ? 6 : 14;
             predictor_step_group(a, l, s_ids, s_prev, warp - kFirst, NW - kFirst, lane);
         }
-        grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 4);
-        DBG_STAMP(l * 8 + 5);
+        grid_barrier(a.barrier, a.err, target, &s_dead);
 
         // ---- D ---------------------------------------------------------------------------------
         g.rows = H, g.kd = I, g.splits = d.splits, g.seg = d.seg;
@@ -231,8 +226,7 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
             group8_convert<1>(g, q, cpos8, warp - 6, warp % 4, lane);
         }
         for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
-        grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 6);
-        DBG_STAMP(l * 8 + 7);
+        grid_barrier(a.barrier, a.err, target, &s_dead);
     }
     // the last layer's output
     if (!s_dead) {

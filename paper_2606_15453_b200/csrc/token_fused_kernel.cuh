@@ -414,7 +414,6 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
         const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
 
         // ---- router rows dealt over the units ------------------------------------------------
-        DBG_STAMP(l * 8 + 0);
         for (int jr = unit; jr < E; jr += n_units) {
             const uint8_t *row = a.router + ((size_t)l * E + jr) * H * Fmt<RDT>::kBytes;
             float p = 0.f;
@@ -432,7 +431,6 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
         }
         target += gridDim.x;
         cta_arrive(cb, a.barrier);
-        DBG_STAMP(l * 8 + 1);
 
         // ---- softmax / top-K once the logits have arrived: the CTA's first 256 threads, thread j
         // owns expert j (rank counting: no dependent rounds); the other threads wait at the CTA
@@ -440,7 +438,6 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
         bool routed_known = false;
         auto route = [&]() {
             cta_wait(cb, a.barrier, a.err, target, &s_dead, fa.poll_limit);
-            DBG_STAMP(l * 8 + 2);
             if (threadIdx.x < 256) {
                 auto sync256 = []() { asm volatile("bar.sync 14, 256;" ::: "memory"); };
                 const int j = threadIdx.x, wj = j / kWarp;
@@ -502,7 +499,6 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
                 }
             }
             routed_known = true;
-            DBG_STAMP(l * 8 + 3);
         };
 
         // Keep the ring full (the unit's first thread only).
@@ -603,7 +599,6 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
             cu.next(pl);
         }
         if (!routed_known) route();  // units without a routed block (the service CTA among them)
-        DBG_STAMP(l * 8 + 4);
 
         if (!service) {
             // the CTA's units add up in shared memory, unit by unit, then one exact atomic per column
@@ -640,12 +635,10 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
             if (u.lane < K) s_prev[u.lane] = s_ids[u.lane];
             __syncwarp();
         }
-        DBG_STAMP(l * 8 + 5);
 
         // ---- h' = h + r * y, from the exact sums ----------------------------------------------
         target += gridDim.x;
         cta_arrive(cb, a.barrier);  // (its CTA barrier also orders the reads of ysum before the next layer's writes)
-        DBG_STAMP(l * 8 + 6);
         // the next layer's shared experts start to arrive while the barrier completes (top_up stops at
         // that layer's routed blocks: iss_layer is past l by now)
         if (u.t == 0) top_up();
@@ -662,7 +655,6 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
                 h[j][e + 1] = fmaf(a.residual_scale, __ll2float_rn((long long)v.y) * kFixInv, h[j][e + 1]);
             }
         }
-        DBG_STAMP(l * 8 + 7);
     }
     __syncthreads();  // the service CTA's predictor warp and its other threads meet again here
     if (tables_staged) {
@@ -718,7 +710,7 @@ __global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(unsigned *cou
     __syncthreads();
     if (which == 0) {
         unsigned target = 1;  // one more arrival than there are CTAs
-        grid_barrier(counter, err, target, &s_dead, -1, limit);
+        grid_barrier(counter, err, target, &s_dead, limit);
     } else if (which == 1) {
         const CtaBar cb{0, 64};
         cta_arrive(cb, counter);

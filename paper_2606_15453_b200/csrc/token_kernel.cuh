@@ -77,7 +77,6 @@ __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int lay
     const long long t = *st.t;
     const bool runtime = t >= a.P;
     const bool last_profiling = (!runtime) && t == a.P - 1 && layer == L - 1;
-    DBG_STAMP_WARP(2010);
     if (runtime && __isGlobal(st.cct_id)) {  // (a caller may keep the tables in shared memory: nothing to pull)
         // Every table row this step touches, pulled into L1 in one trip: the rows are then read
         // one after the other (Algorithm 3 is sequential per row), each of which would otherwise
@@ -113,7 +112,6 @@ __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int lay
                 atomicAdd(&st.stats[3], (unsigned long long)nh);
             }
         }
-        DBG_STAMP_WARP(2011);
         if (layer > 0) {
             uint8_t *gid = st.cct_id + (size_t)(layer - 1) * E * K;
             uint8_t *gcf = st.cct_conf + (size_t)(layer - 1) * E * K;
@@ -128,7 +126,6 @@ __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int lay
         }
     }
     __syncwarp();
-    DBG_STAMP_WARP(2012);
 
     const bool predict_now = runtime || last_profiling;
     const int next = (layer + 1) % L;
@@ -198,12 +195,10 @@ __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int lay
         }
         __syncwarp();
     }
-    DBG_STAMP_WARP(2013);
     for (int i = wi * kWarp + lane; i < B * K; i += nw * kWarp) {
         const int b = i / K, k = i % K;
         st.HT[((size_t)b * L + layer) * K + k] = (int16_t)cur[b * K + k];
     }
-    DBG_STAMP_WARP(2014);
     // every warp has read the step counter before one of them advances it
     if (nw > 1) asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(nw * kWarp) : "memory");
     if (wi == 0 && lane == 0 && layer == L - 1) *st.t = t + 1;
@@ -211,11 +206,10 @@ __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int lay
 
 // Bounded grid barrier on a monotonically increasing counter.
 __device__ __forceinline__ void grid_barrier(unsigned *counter, unsigned *err, unsigned &target, volatile int *s_dead,
-                                             int dbg_idx = -1, int spin_limit = kBarrierSpinLimit)
+                                             int spin_limit = kBarrierSpinLimit)
 {
     target += gridDim.x;
     __syncthreads();
-    if (dbg_idx >= 0) DBG_STAMP(dbg_idx);
     if (threadIdx.x == 0 && !*s_dead) {
         // Release at GPU scope: the CTA barrier above orders every thread's writes before this
         // thread's arrival (cumulativity), so no separate fence is needed; the acquiring load below
@@ -322,16 +316,13 @@ __device__ __forceinline__ void decode_token_single(const TokenArgs &a, int *dyn
         tk.flags_out = (lead && a.flags_out) ? a.flags_out + l : nullptr;
         tk.near_tie_counter = lead ? a.pst.stats + 4 : nullptr;
         tk.wl.n_groups = nullptr;  // no work list: the entries are the K routed ids, then the shared experts
-        DBG_STAMP(l * 8 + 0);
         router_tasks<RDT, false>(ra, warp * gridDim.x + blockIdx.x, NW * gridDim.x, lane);  // over the SMs first
-        grid_barrier(a.barrier, a.err, target, s_dead, l * 8 + 1);
-        DBG_STAMP(l * 8 + 2);
+        grid_barrier(a.barrier, a.err, target, s_dead);
 
         // ---- T: softmax / top-K, redundantly per CTA --------------------------------------
         router_finalize<RDT>(ra, s_ids, s_scan, NW);
         __syncthreads();
         if (lead && threadIdx.x < K) a.ids_all[(size_t)l * a.Bmax * K + threadIdx.x] = s_ids[threadIdx.x];
-        DBG_STAMP(l * 8 + 3);
 
         // ---- GU (+ the predictor on one warp of the last CTA) -----------------------------
         SingleCtx cx;
@@ -346,16 +337,14 @@ __device__ __forceinline__ void decode_token_single(const TokenArgs &a, int *dyn
                 if (pred_cta && warp == NW - 1) predictor_step_group(a, l, s_ids, s_prev, 0, 1, lane);
             },
             [&]() { stage_down_slices<DT>(fa, cx, td, 0, K, a.stage_down_bytes, warp, NW, lane); });
-        grid_barrier(a.barrier, a.err, target, s_dead, l * 8 + 4);
-        DBG_STAMP(l * 8 + 5);
+        grid_barrier(a.barrier, a.err, target, s_dead);
 
         // ---- D ---------------------------------------------------------------------------
         down_single<DT>(fa, cx, td, s_next + 1, KS, [&]() {
             if (l + 1 < L) stage_layer_ahead<DT>(a, l + 1, fa, tg, td, warp, NW, lane);
         });
         if (threadIdx.x < K) s_prev[threadIdx.x] = s_ids[threadIdx.x];
-        grid_barrier(a.barrier, a.err, target, s_dead, l * 8 + 6);
-        DBG_STAMP(l * 8 + 7);
+        grid_barrier(a.barrier, a.err, target, s_dead);
     }
 }
 
@@ -403,10 +392,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs 
         tk.flags_out = (lead && a.flags_out) ? a.flags_out + (size_t)l * B : nullptr;
         tk.near_tie_counter = lead ? a.pst.stats + 4 : nullptr;
         tk.wl = wl;
-        DBG_STAMP(l * 8 + 0);
         router_tasks<RDT, false>(ra, warp * gridDim.x + blockIdx.x, NW * gridDim.x, lane);  // over the SMs first
-        grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 1);
-        DBG_STAMP(l * 8 + 2);
+        grid_barrier(a.barrier, a.err, target, &s_dead);
 
         // ---- T: softmax / top-K / grouping, redundantly per CTA ---------------------------
         router_finalize<RDT>(ra, s_ids, s_scan, NW);
@@ -415,7 +402,6 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs 
             for (int i = threadIdx.x; i < B * K; i += blockDim.x)
                 a.ids_all[(size_t)l * a.Bmax * K + i] = s_ids[i];
 
-        DBG_STAMP(l * 8 + 3);
         // ---- GU (+ the predictor on one warp of the last CTA) -----------------------------
         FfnArgs fa;
         fa.h = h, fa.inv_rms = s_inv, fa.wl = wl, fa.blob = a.blob + (size_t)l * (E + a.n_shared);
@@ -426,14 +412,12 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_kernel(TokenArgs 
         gate_up_phase<DT, MTMAX>(fa, s_next, [&]() {
             if (pred_cta && warp == NW - 1) predictor_step_group(a, l, s_ids, s_prev, 0, 1, lane);
         });
-        grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 4);
-        DBG_STAMP(l * 8 + 5);
+        grid_barrier(a.barrier, a.err, target, &s_dead);
 
         // ---- D ---------------------------------------------------------------------------
         down_phase<DT, MTMAX, false>(fa, s_next);
         for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
-        grid_barrier(a.barrier, a.err, target, &s_dead, l * 8 + 6);
-        DBG_STAMP(l * 8 + 7);
+        grid_barrier(a.barrier, a.err, target, &s_dead);
     }
 }
 
