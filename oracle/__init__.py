@@ -55,9 +55,14 @@ def lib():
         L.orc_predict.restype = C.c_int
         L.orc_predict.argtypes = [i32, i32, vp, i32, vp, vp, vp, vp, vp, vp]
         L.orc_update.argtypes = [i32, i32, vp, i32, vp, i32, vp, vp]
+        L.orc_update_rule.argtypes = [i32, i32, vp, i32, vp, i32, vp, vp, vp]
+        L.orc_pred_set_replacement.argtypes = [vp, i32]
         L.orc_pred_create.restype = vp
         L.orc_pred_create.argtypes = [i32] * 6
         L.orc_pred_destroy.argtypes = [vp]
+        L.orc_pred_set_threshold.argtypes = [vp, i32]
+        L.orc_predict_thr.restype = C.c_int
+        L.orc_predict_thr.argtypes = [i32, i32, vp, i32, vp, vp, vp, i32, vp, vp, vp]
         L.orc_pred_max_pred.restype = C.c_int
         L.orc_pred_max_pred.argtypes = [vp]
         L.orc_pred_step.restype = C.c_int
@@ -180,34 +185,43 @@ def cct_build(Co: np.ndarray, K: int):
     return ids, conf
 
 
-def predict(E: int, K: int, Ei, cct_id, cct_conf, ht):
+def predict(E: int, K: int, Ei, cct_id, cct_conf, ht, threshold: int = 2):
     """Returns (score [E] per Eq. 1, literal-listing score [E], set mask [E])."""
     Ei = _i32(Ei)
     score = np.empty(E, dtype=np.int32)
     lit = np.empty(E, dtype=np.int32)
     mask = np.empty(E, dtype=np.uint8)
     htp = None if ht is None else np.ascontiguousarray(np.asarray(ht, dtype=np.int16))
-    rc = lib().orc_predict(E, K, _p(Ei), Ei.size, _p(cct_id), _p(cct_conf), _p(htp), _p(score),
-                           _p(lit), _p(mask))
+    rc = lib().orc_predict_thr(E, K, _p(Ei), Ei.size, _p(cct_id), _p(cct_conf), _p(htp), threshold,
+                               _p(score), _p(lit), _p(mask))
     if rc < 0:
         raise AssertionError("Eq. 1 and the literal listing of Algorithm 2 disagree")
     return score, lit, mask
 
 
-def update(E: int, K: int, Ei, Fj, cct_id: np.ndarray, cct_conf: np.ndarray) -> None:
+def update(E: int, K: int, Ei, Fj, cct_id: np.ndarray, cct_conf: np.ndarray, co: np.ndarray | None = None) -> None:
+    """Algorithm 3 on one layer pair.  co = None: a replaced slot takes the lowest routed id the row
+    does not hold; co = the pair's [E][E] counts (already holding this step's pairs): the routed id
+    with the largest count in the row."""
     Ei, Fj = _i32(Ei), _i32(Fj)
     assert cct_id.dtype == np.uint8 and cct_conf.dtype == np.uint8
-    lib().orc_update(E, K, _p(Ei), Ei.size, _p(Fj), Fj.size, _p(cct_id), _p(cct_conf))
+    if co is None:
+        lib().orc_update(E, K, _p(Ei), Ei.size, _p(Fj), Fj.size, _p(cct_id), _p(cct_conf))
+    else:
+        assert co.dtype == np.uint32 and co.shape == (E, E) and co.flags.c_contiguous
+        lib().orc_update_rule(E, K, _p(Ei), Ei.size, _p(Fj), Fj.size, _p(cct_id), _p(cct_conf), _p(co))
 
 
 class Predictor:
     """Whole-stack predictor state machine (profiling, build, verify/update, predict)."""
 
-    def __init__(self, L, E, K, B=1, P=0, mode="st"):
+    def __init__(self, L, E, K, B=1, P=0, mode="st", threshold=2, live_counts=False):
         self.L, self.E, self.K, self.B, self.P = L, E, K, B, P
         self._h = lib().orc_pred_create(L, E, K, B, P, MODE[mode])
         if not self._h:
             raise ValueError("bad predictor shape")
+        lib().orc_pred_set_threshold(self._h, threshold)
+        lib().orc_pred_set_replacement(self._h, int(live_counts))
         self.max_pred = lib().orc_pred_max_pred(self._h)
 
     def __del__(self):

@@ -258,9 +258,24 @@ void orc_cct_build(const uint32_t *Co, int E, int K, uint8_t *cct_id, uint8_t *c
  * The printed listing overwrites the score of an HT member with 1 and then
  * adds 1; `literal` (optional) receives those scores.  Both give the same
  * set; the function returns -1 if they ever differ, else the set size. */
+int orc_predict_thr(int E, int K, const int32_t *Ei, int ni, const uint8_t *cct_id,
+                    const uint8_t *cct_conf, const int16_t *ht, int threshold, int32_t *score,
+                    int32_t *literal, uint8_t *in_set);
+
 int orc_predict(int E, int K, const int32_t *Ei, int ni, const uint8_t *cct_id,
                 const uint8_t *cct_conf, const int16_t *ht, int32_t *score, int32_t *literal,
                 uint8_t *in_set)
+{
+    return orc_predict_thr(E, K, Ei, ni, cct_id, cct_conf, ht, ORC_THRESHOLD, score, literal, in_set);
+}
+
+/* The same with the set threshold as a parameter (Section 4.2 fixes it at binary 10; other
+ * values are the threshold sweep of the ablation).  The history bonus stays binary 10 (Eq. 1).
+ * The printed listing is only comparable at the paper's threshold: for other values the check
+ * against it is skipped. */
+int orc_predict_thr(int E, int K, const int32_t *Ei, int ni, const uint8_t *cct_id,
+                    const uint8_t *cct_conf, const int16_t *ht, int threshold, int32_t *score,
+                    int32_t *literal, uint8_t *in_set)
 {
     int32_t *lit = literal ? literal : (int32_t *)malloc(sizeof(int32_t) * (size_t)E);
     for (int f = 0; f < E; ++f) score[f] = lit[f] = 0;
@@ -281,8 +296,8 @@ int orc_predict(int E, int K, const int32_t *Ei, int ni, const uint8_t *cct_id,
     }
     int n = 0, same = 1;
     for (int f = 0; f < E; ++f) {
-        in_set[f] = score[f] >= ORC_THRESHOLD;
-        if (in_set[f] != (lit[f] >= ORC_THRESHOLD)) same = 0;
+        in_set[f] = score[f] >= threshold;
+        if (threshold == ORC_THRESHOLD && in_set[f] != (lit[f] >= ORC_THRESHOLD)) same = 0;
         n += in_set[f];
     }
     if (!literal) free(lit);
@@ -296,15 +311,21 @@ int orc_predict(int E, int K, const int32_t *Ei, int ni, const uint8_t *cct_id,
  * candidate of row e in slot order: confirmed by the layer-(i+1) routing ->
  * confidence +1 capped at 3; not confirmed and confidence > 0 -> -1; not
  * confirmed at confidence 0 -> replaced by an expert of F that the row does
- * not hold, confidence binary 10.  "Any expert" is read as the lowest such
- * id, with the row re-read after each replacement so a row never holds an id
- * twice; when every routed expert is already in the row the slot is left. */
-void orc_update(int E, int K, const int32_t *Ei, int ni, const int32_t *Fj, int nf,
-                uint8_t *cct_id, uint8_t *cct_conf)
+ * not hold, confidence binary 10.  The row is re-read after each replacement
+ * so a row never holds an id twice; when every routed expert is already in
+ * the row the slot is left.  The listing leaves the choice among several such
+ * experts open ("any expert"):
+ *   Co == NULL  the lowest id (the default reading);
+ *   Co != NULL  the one with the largest count in row e of Co, the pair's
+ *               co-activation counts kept up to date at run time (the caller
+ *               has already counted this step's pairs); equal counts -> the
+ *               lower id. */
+void orc_update_rule(int E, int K, const int32_t *Ei, int ni, const int32_t *Fj, int nf,
+                     uint8_t *cct_id, uint8_t *cct_conf, const uint32_t *Co)
 {
-    (void)E;
     for (int a = 0; a < ni; ++a) {
         uint8_t *id = cct_id + (size_t)Ei[a] * K, *cf = cct_conf + (size_t)Ei[a] * K;
+        const uint32_t *row = Co ? Co + (size_t)Ei[a] * E : NULL;
         for (int c = 0; c < K; ++c) {
             int hit = 0;
             for (int b = 0; b < nf; ++b) hit |= (Fj[b] == id[c]);
@@ -314,10 +335,13 @@ void orc_update(int E, int K, const int32_t *Ei, int ni, const int32_t *Fj, int 
                 cf[c] -= 1;
             } else {
                 int g = -1;
-                for (int b = 0; b < nf && g < 0; ++b) { /* Fj is ascending */
+                for (int b = 0; b < nf; ++b) { /* Fj is ascending */
                     int held = 0;
                     for (int d = 0; d < K; ++d) held |= (id[d] == Fj[b]);
-                    if (!held) g = Fj[b];
+                    if (held) continue;
+                    if (g < 0) g = Fj[b];
+                    if (!row) break;
+                    if (row[Fj[b]] > row[g]) g = Fj[b];
                 }
                 if (g >= 0) {
                     id[c] = (uint8_t)g;
@@ -328,11 +352,17 @@ void orc_update(int E, int K, const int32_t *Ei, int ni, const int32_t *Fj, int 
     }
 }
 
+void orc_update(int E, int K, const int32_t *Ei, int ni, const int32_t *Fj, int nf,
+                uint8_t *cct_id, uint8_t *cct_conf)
+{
+    orc_update_rule(E, K, Ei, ni, Fj, nf, cct_id, cct_conf, NULL);
+}
+
 /* ------------------------------------------------------------------ */
 /* predictor state machine over a whole stack                          */
 
 typedef struct {
-    int32_t L, E, K, B, P, mode, built, max_pred;
+    int32_t L, E, K, B, P, mode, built, max_pred, threshold, live_counts;
     int64_t t;          /* decode steps completed */
     uint32_t *Co;       /* [L-1][E][E] */
     uint8_t *cct_id;    /* [L-1][E][K] */
@@ -357,7 +387,7 @@ orc_pred_t *orc_pred_create(int L, int E, int K, int B, int P, int mode)
     if (L < 1 || E < 1 || E > 256 || K < 1 || K > E || K > 32 || B < 1 || P < 0) return NULL;
     orc_pred_t *p = (orc_pred_t *)calloc(1, sizeof(*p));
     int pairs = L > 1 ? L - 1 : 0;
-    p->L = L, p->E = E, p->K = K, p->B = B, p->P = P, p->mode = mode;
+    p->L = L, p->E = E, p->K = K, p->B = B, p->P = P, p->mode = mode, p->threshold = ORC_THRESHOLD;
     p->max_pred = (K * K + K < E) ? K * K + K : E;
     p->Co = (uint32_t *)calloc((size_t)pairs * E * E + 1, 4);
     p->cct_id = (uint8_t *)calloc((size_t)pairs * E * K + 1, 1);
@@ -379,6 +409,21 @@ void orc_pred_destroy(orc_pred_t *p)
 }
 
 int orc_pred_max_pred(const orc_pred_t *p) { return p->max_pred; }
+
+/* Set threshold of Algorithm 2 for this predictor (>= 1; default binary 10).  The set still holds
+ * at most K*K + K experts: a member has a stored candidate of non-zero confidence or is in the
+ * history table. */
+void orc_pred_set_threshold(orc_pred_t *p, int threshold)
+{
+    p->threshold = threshold < 1 ? 1 : threshold;
+}
+
+/* Replacement rule of Algorithm 3 for this predictor.  0 (default): the lowest routed id the
+ * row does not hold; the counts stay as profiling left them.  1: counting goes on at run time
+ * (for every sequence, Co[e][f] += 1 for e routed at the previous layer and f at this one,
+ * right before that sequence's table update) and the new candidate is the routed expert with
+ * the largest count in the row. */
+void orc_pred_set_replacement(orc_pred_t *p, int live_counts) { p->live_counts = live_counts != 0; }
 
 /* One layer step for sequences 0..batch-1 (Section 4.3.4: R, then V and P).
  *
@@ -419,10 +464,13 @@ int orc_pred_step(orc_pred_t *p, int layer, int batch, const int32_t *routed, in
             if (p->pred_valid[b])
                 for (int k = 0; k < K; ++k) nh += p->pred[(size_t)b * E + R[k]];
             p->st_steps += 1, p->st_routed += K, p->st_pred += np, p->st_hit += nh;
-            if (layer > 0)
-                orc_update(E, K, p->prev + (size_t)b * K, K, R, K,
-                           p->cct_id + (size_t)(layer - 1) * E * K,
-                           p->cct_conf + (size_t)(layer - 1) * E * K);
+            if (layer > 0) {
+                uint32_t *Co = p->Co + (size_t)(layer - 1) * E * E;
+                if (p->live_counts) orc_co_accumulate(Co, E, p->prev + (size_t)b * K, K, R, K);
+                orc_update_rule(E, K, p->prev + (size_t)b * K, K, R, K,
+                                p->cct_id + (size_t)(layer - 1) * E * K,
+                                p->cct_conf + (size_t)(layer - 1) * E * K, p->live_counts ? Co : NULL);
+            }
         }
     } else if (layer > 0) {
         for (int b = 0; b < batch; ++b)
@@ -444,10 +492,10 @@ int orc_pred_step(orc_pred_t *p, int layer, int batch, const int32_t *routed, in
             const int next = (layer + 1) % L;
             const int spatial = (p->mode & ORC_MODE_SPATIAL) && layer < L - 1;
             const int temporal = (p->mode & ORC_MODE_TEMPORAL) != 0;
-            n = orc_predict(E, K, routed + (size_t)b * K, spatial ? K : 0,
-                            spatial ? p->cct_id + (size_t)layer * E * K : NULL,
-                            spatial ? p->cct_conf + (size_t)layer * E * K : NULL,
-                            temporal ? p->HT + ((size_t)b * L + next) * K : NULL, score, NULL, set);
+            n = orc_predict_thr(E, K, routed + (size_t)b * K, spatial ? K : 0,
+                                spatial ? p->cct_id + (size_t)layer * E * K : NULL,
+                                spatial ? p->cct_conf + (size_t)layer * E * K : NULL,
+                                temporal ? p->HT + ((size_t)b * L + next) * K : NULL, p->threshold, score, NULL, set);
             if (n < 0) rc = -2, n = 0;
             for (int f = 0; f < E; ++f)
                 if (set[f]) total[f] += score[f];

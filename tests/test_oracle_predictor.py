@@ -356,3 +356,179 @@ def test_worked_example_batch_of_two_pins_queue_scores():
         assert p.tables()["cct_conf"][0].tolist() == _rows(next(it)[1])
         ids, sc = queue(next(it)[1])
         assert out1["queue_ids"].tolist() == ids and out1["queue_score"].tolist() == sc
+
+
+def test_set_threshold_of_algorithm_2_follows_the_pinned_scores():
+    """The threshold only cuts the pinned scores of the worked example at another value; the
+    tables evolve identically; the sets are nested."""
+    recs = _load_example()
+    E, K = 4, 2
+    prof = [[list(map(int, s.split())) for s in pair.split("->")] for pair in recs[0][1].split(";")]
+    steps = recs[5:]
+    ref_tables = None
+    for thr in (1, 2, 3, 5, 7):
+        p = O.Predictor(L=2, E=E, K=K, B=1, P=4, mode="st", threshold=thr)
+        for e, f in prof:
+            p.step(0, [e])
+            p.step(1, [f])
+        for i in range(0, len(steps), 5):
+            e, f = (list(map(int, s.split())) for s in steps[i][1].split("->"))
+            score = [int(v) for v in steps[i + 1][1].split()]
+            out = p.step(0, [e])
+            n = out["n_pred"][0]
+            assert out["pred_ids"][0, :n].tolist() == [x for x in range(E) if score[x] >= thr], (thr, i)
+            p.step(1, [f])
+        tables = (p.tables()["cct_id"].tobytes(), p.tables()["cct_conf"].tobytes())
+        assert ref_tables in (None, tables)
+        ref_tables = tables
+    # function level: the same scores, sets nested in the threshold
+    ids, conf = O.cct_build(np.array(_rows(recs[1][1]), dtype=np.uint32), K)
+    prev = None
+    for thr in (1, 2, 3, 4, 6):
+        score, _, mask = O.predict(E, K, [0, 2], ids, conf, [1, 3], threshold=thr)
+        assert score.tolist() == [0, 2, 4, 6]
+        assert np.flatnonzero(mask).tolist() == [f for f in range(E) if score[f] >= thr]
+        assert prev is None or (mask <= prev).all()
+        prev = mask
+
+
+GOLDEN_LIVE = os.path.join(os.path.dirname(__file__), "golden", "cct_live_counts_example.txt")
+
+
+def _load(path):
+    recs = []
+    with open(path) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                key, val = line.split(":", 1)
+                recs.append((key.strip(), val.strip()))
+    return recs
+
+
+def test_live_count_replacement_worked_example():
+    """Replacement by the largest live count (the open choice of Algorithm 3 taken another way):
+    hand-derived counts and rows, through the single functions and through the state machine; the
+    default rule ends with another row 0, so the two rules cannot be confused."""
+    recs = _load(GOLDEN_LIVE)
+    E, K = 4, 2
+    prof = [[list(map(int, s.split())) for s in pair.split("->")] for pair in recs[0][1].split(";")]
+    Co = np.zeros((E, E), dtype=np.uint32)
+    for e, f in prof:
+        O.co_accumulate(Co, e, f)
+    assert Co.tolist() == _rows(recs[1][1])
+    ids, conf = O.cct_build(Co, K)
+    assert ids.tolist() == _rows(recs[2][1]) and conf.tolist() == _rows(recs[3][1])
+    ids_low, conf_low = ids.copy(), conf.copy()
+    p = O.Predictor(L=2, E=E, K=K, B=1, P=len(prof), mode="st", live_counts=True)
+    for e, f in prof:
+        p.step(0, [e]), p.step(1, [f])
+    steps = recs[4:]
+    for i in range(0, len(steps), 4):
+        assert steps[i][0] == "step"
+        e, f = (list(map(int, s.split())) for s in steps[i][1].split("->"))
+        O.co_accumulate(Co, e, f)
+        O.update(E, K, e, f, ids, conf, co=Co)
+        O.update(E, K, e, f, ids_low, conf_low)
+        p.step(0, [e]), p.step(1, [f])
+        tb = p.tables()
+        for got_co, got_id, got_cf in ((Co, ids, conf), (tb["Co"][0], tb["cct_id"][0], tb["cct_conf"][0])):
+            assert got_co.tolist() == _rows(steps[i + 1][1]), i
+            assert got_id.tolist() == _rows(steps[i + 2][1]), i
+            assert got_cf.tolist() == _rows(steps[i + 3][1]), i
+    assert ids_low[0].tolist() == [0, 1] and ids[0].tolist() == [1, 0]
+
+
+def _update_by_counts_replay(E, K, prev, cur, rows, co):
+    """Algorithm 3 with the live-count rule written another way: dictionaries per row, the
+    candidates of a replacement sorted by (count descending, id ascending)."""
+    for e in prev:
+        row = rows[e]
+        for c in range(K):
+            g, cf = row[c]
+            if g in cur:
+                row[c] = (g, min(cf + 1, 3))
+            elif cf > 0:
+                row[c] = (g, cf - 1)
+            else:
+                held = {x for x, _ in row}
+                cand = sorted((f for f in cur if f not in held), key=lambda f: (-int(co[e][f]), f))
+                if cand:
+                    row[c] = (cand[0], 2)
+
+
+@pytest.mark.parametrize("E,K,B", [(6, 2, 1), (8, 3, 2), (16, 4, 3), (60, 4, 1), (128, 8, 2)])
+def test_live_count_rule_against_a_replay_and_its_invariants(E, K, B):
+    L, P, T = 3, 5, 60
+    rng = np.random.default_rng(11 * E + K)
+    p = O.Predictor(L, E, K, B, P, "st", live_counts=True)
+    co = np.zeros((L - 1, E, E), dtype=np.int64)
+    rows = None
+    routed_rows = np.zeros((L - 1, E), dtype=np.int64)
+    for t in range(T):
+        prev = None
+        for l in range(L):
+            # skewed routing, so counts differ and replacements happen
+            w = 1.0 / (1.0 + ((np.arange(E) * 7 + 3 * l + (t % 4)) % E))
+            cur = np.stack([np.sort(rng.choice(E, K, replace=False, p=w / w.sum())) for _ in range(B)])
+            p.step(l, cur)
+            if l > 0:
+                for b in range(B):
+                    for e in prev[b]:
+                        routed_rows[l - 1, e] += 1
+                        for f in cur[b]:
+                            co[l - 1, e, f] += 1
+                    if t >= P:
+                        _update_by_counts_replay(E, K, prev[b].tolist(), cur[b].tolist(), rows[l - 1], co[l - 1])
+            prev = cur
+        if t == P - 1:
+            tb = p.tables()
+            rows = [[[(int(tb["cct_id"][i, e, c]), int(tb["cct_conf"][i, e, c])) for c in range(K)]
+                     for e in range(E)] for i in range(L - 1)]
+    tb = p.tables()
+    # counting never stops: K x K per sequence, pair and decode step; a row's sum = K x (times routed)
+    assert (tb["Co"] == co).all()
+    assert int(tb["Co"].sum()) == T * B * K * K * (L - 1)
+    assert (tb["Co"].sum(axis=2) == K * routed_rows).all()
+    for i in range(L - 1):
+        for e in range(E):
+            assert [g for g, _ in rows[i][e]] == tb["cct_id"][i, e].tolist(), (i, e)
+            assert [c for _, c in rows[i][e]] == tb["cct_conf"][i, e].tolist(), (i, e)
+            assert len(set(tb["cct_id"][i, e].tolist())) == K
+    assert tb["cct_conf"].max() <= 3
+
+
+def test_live_count_rule_with_one_expert_per_token_equals_the_default_rule():
+    """K = 1: a replacement has at most one candidate (the routed expert), so both rules must keep
+    the same tables; only the counts differ (frozen against live)."""
+    L, E, P, T = 4, 8, 6, 80
+    rng = np.random.default_rng(5)
+    a, b = O.Predictor(L, E, 1, 1, P, "st"), O.Predictor(L, E, 1, 1, P, "st", live_counts=True)
+    for t in range(T):
+        for l in range(L):
+            cur = rng.integers(0, E, size=(1, 1))
+            ra, rb = a.step(l, cur), b.step(l, cur)
+            assert (ra["pred_ids"] == rb["pred_ids"]).all()
+    ta, tb = a.tables(), b.tables()
+    assert (ta["cct_id"] == tb["cct_id"]).all() and (ta["cct_conf"] == tb["cct_conf"]).all()
+    assert int(ta["Co"].sum()) == P * (L - 1) and int(tb["Co"].sum()) == T * (L - 1)
+
+
+def test_live_count_rule_batch_is_the_sequences_in_index_order():
+    """Counting and updating go sequence by sequence: a batch of two must equal the same two
+    routings fed as two single steps of a one-sequence table (tables only; the history is per
+    sequence)."""
+    E, K = 8, 2
+    prev = np.array([[0, 1], [0, 2]]); cur = np.array([[3, 5], [4, 5]])
+    p = O.Predictor(2, E, K, 2, 0, "st", live_counts=True)
+    # a predictor built from all-zero counts (P = 0) holds ids 0..K-1 at confidence 2 in every row
+    ids_b, conf_b = np.tile(np.arange(K, dtype=np.uint8), (E, 1)), np.full((E, K), 2, dtype=np.uint8)
+    co_b = np.zeros((E, E), dtype=np.uint32)
+    for _ in range(4):
+        p.step(0, prev), p.step(1, cur)
+        for b in range(2):
+            O.co_accumulate(co_b, prev[b], cur[b])
+            O.update(E, K, prev[b], cur[b], ids_b, conf_b, co=co_b)
+    tb = p.tables()
+    assert (tb["Co"][0] == co_b).all() and (tb["cct_id"][0] == ids_b).all() and (tb["cct_conf"][0] == conf_b).all()
+    assert ids_b[0].tolist() != [0, 1]          # replacements did happen in the shared row
