@@ -318,6 +318,10 @@ def make_stack(cfg, batch, dev, args):
     st = load_stack(cfg, batch, dev, prefetch_limit=args.prefetch_limit, mode=args.mode, flags=flags)
     if args.prefetch_min_score:
         st.set_prefetch_min_score(args.prefetch_min_score)
+    if args.predict_threshold != 2:
+        st.set_predict_threshold(args.predict_threshold)
+    if args.live_counts:
+        st.set_replacement_rule(True)
     if args.dense_min_batch and not args.no_dense:
         st.set_dense_min_batch(args.dense_min_batch)
     if args.stage_known_kb >= 0 or args.stage_pred_mb >= 0:
@@ -326,6 +330,8 @@ def make_stack(cfg, batch, dev, args):
         if args.cache_policy != "default" or args.prefetch_floor >= 0:
             window, by_turn = {"default": (16, True) if cfg.n_layers * min(cfg.n_experts, batch * cfg.top_k) > cfg.cache_slots
                                else (0, False), "lru": (0, False), "counts": (16, False), "turn": (16, True)}[args.cache_policy]
+            if args.prefetch_floor >= 0 and window == 0:
+                window = 16        # the floor is a test on the use counts: it needs a history window
             st.set_cache_policy(window, by_turn, args.prefetch_floor)
         if args.throttle_chunk_kb:
             st.set_copy_throttle(args.throttle_chunk_kb << 10, args.throttle_gap_us)
@@ -356,6 +362,9 @@ def main():
     ap.add_argument("--throttle-chunk-kb", type=int, default=0, help="offloaded stacks: expert copies in chunks of this size ...")
     ap.add_argument("--throttle-gap-us", type=int, default=0, help="... with this much idle time after each (link-speed sweep)")
     ap.add_argument("--mode", default="st", choices=["off", "temporal", "spatial", "st"])
+    ap.add_argument("--live-counts", action="store_true",
+                    help="Algorithm 3 replaces a candidate by the routed expert with the largest live co-activation count")
+    ap.add_argument("--predict-threshold", type=int, default=2, help="set threshold of Algorithm 2 (the paper: 2)")
     ap.add_argument("--inter-layer-gap-us", type=float, default=0.0,
                     help="idle the compute stream this long after every layer: a stand-in for the attention "
                          "block the paper overlaps expert prefetch with (Section 4.3.4); 0 = pure MoE stack")

@@ -185,6 +185,23 @@ int stmoe_set_kernel_timing(stmoe_t *s, int on);
  * Between decode steps; routing, outputs and predictor tables are unaffected. */
 int stmoe_set_prefetch_min_score(stmoe_t *s, int min_score);
 
+/* Set threshold of Algorithm 2: an expert is predicted when its score (sum of the confidences of
+ * its stored candidates in the routed experts' rows, plus binary 10 if it is in the history table,
+ * Eq. 1) reaches `threshold`.  Section 4.2 fixes it at binary 10 = 2 (default); 1 predicts every
+ * stored candidate of non-zero confidence, larger values trade recall for precision (threshold
+ * sweep of the ablation).  Tables evolve identically for every value.  Between decode steps. */
+int stmoe_set_predict_threshold(stmoe_t *s, int threshold);
+
+/* Replacement rule of Algorithm 3.  When a stored candidate misses at confidence 0 the listing
+ * replaces it by "any" routed expert the row does not hold.  live_counts = 0 (default): the
+ * lowest such id; the co-activation counts stay as profiling (Algorithm 1) left them.
+ * live_counts = 1: counting goes on at run time (for every sequence, in index order, the K x K
+ * pairs of (previous layer's routing, this layer's routing) are counted right before that
+ * sequence's table update) and the new candidate is the routed expert with the largest count in
+ * the row, equal counts -> the lower id.  The exported state then carries the live counts.
+ * Between decode steps. */
+int stmoe_set_replacement_rule(stmoe_t *s, int live_counts);
+
 /* Replacement policy of the HBM slot cache (the paper stages predicted experts and fetches
  * misses at once, Section 4.3.4, and names no replacement policy).  Victims are taken in this
  * order among the slots not needed by the step in progress: empty slots; the expert with the
@@ -193,7 +210,8 @@ int stmoe_set_prefetch_min_score(stmoe_t *s, int min_score);
  * cyclic layer walk is furthest away; the least recently used; the lowest slot.  0, 0 is plain
  * LRU.  prefetch_floor >= 0: a prefetch only takes a slot whose expert has at most that many uses
  * in its window (0: only slots without recent use), otherwise the prediction is dropped; -1: no
- * such test (every predicted expert is prefetched, the paper's behaviour).
+ * such test (every predicted expert is prefetched, the paper's behaviour).  A floor needs a
+ * history window (history_window > 0), else STMOE_ERR_BAD_ARG.
  * Default: LRU when a decode step cannot touch more experts than there are slots
  * (n_layers * min(n_experts, max_batch * top_k) <= cache_slots), else a 16-step window with
  * by_turn (LRU has hit rate zero on a cyclic walk that is larger than the cache); floor -1.

@@ -70,6 +70,8 @@ def lib():
         L.stmoe_set_prefetch_min_score.argtypes = [vp, i32]
         L.stmoe_set_onchip_staging.argtypes = [vp, i64, i64]
         L.stmoe_set_cache_policy.argtypes = [vp, i32, i32, i32]
+        L.stmoe_set_predict_threshold.argtypes = [vp, i32]
+        L.stmoe_set_replacement_rule.argtypes = [vp, i32]
         L.stmoe_set_copy_throttle.argtypes = [vp, i64, i32]
         L.stmoe_test_hook.argtypes = [vp, i32, i64]
         L.stmoe_selftest_bounded_wait.argtypes = [vp, i32, i32, vp]
@@ -189,6 +191,12 @@ class Stack:
     def set_onchip_staging(self, known_bytes: int, predicted_bytes: int) -> None:
         _check(lib().stmoe_set_onchip_staging(self._h, int(known_bytes), int(predicted_bytes)),
                "stmoe_set_onchip_staging")
+
+    def set_predict_threshold(self, threshold: int) -> None:
+        _check(lib().stmoe_set_predict_threshold(self._h, int(threshold)), "stmoe_set_predict_threshold")
+
+    def set_replacement_rule(self, live_counts: bool) -> None:
+        _check(lib().stmoe_set_replacement_rule(self._h, int(bool(live_counts))), "stmoe_set_replacement_rule")
 
     def set_cache_policy(self, history_window: int, by_turn: bool, prefetch_floor: int = -1) -> None:
         _check(lib().stmoe_set_cache_policy(self._h, int(history_window), int(by_turn), int(prefetch_floor)),

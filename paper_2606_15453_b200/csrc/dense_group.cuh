@@ -18,8 +18,20 @@
 // to the weight stream); the epilogue keeps the entry's tokens and applies their RMSNorm factors.  The down projection multiplies
 // against the entry's own rows of the activation buffer, which are consecutive.
 // Every wait is bounded; a wait that runs out raises the error word and the kernel drains.
+//
+// Two operand formats (template parameter WDT):
+//   1  bf16 weights x bf16 activations (kind::f16), 64 reduction columns per 128-byte box row;
+//   2  fp8 stacks: e4m3 weights straight from the expert images x activations held as three
+//      e5m2 planes whose sum is the activation (kind::f8f6f4, 128 reduction columns per box row).
+//      e5m2 has the exponent range of f16, so no scaling pass is needed; each plane takes the
+//      rounding residue of the one before (2 mantissa bits each: relative error 2^-9 after three,
+//      the precision of a bf16 operand).  The three planes multiply the same weight tile into the
+//      same accumulator: three times the MMAs, which are free next to the weight stream.  The
+//      per-output-channel weight scales belong to the accumulator lanes and are applied in the
+//      epilogue.
 #pragma once
 #include <cuda.h>
+#include <cuda_fp8.h>
 
 #include "dense_ffn.cuh"
 
@@ -36,24 +48,41 @@ constexpr int kGroupTmemCols = 256;                               // two accumul
 #ifndef STMOE_GROUP_KBOXES_D
 #define STMOE_GROUP_KBOXES_D 4
 #endif
-// 64-column boxes per matrix and stage: consecutive boxes continue the same rows, so a stage asks
-// for boxes * 128 contiguous bytes of every row at once.  Measured on C1 batch 4 / C2 batch 8:
+#ifndef STMOE_GROUP8_KBOXES_GU
+#define STMOE_GROUP8_KBOXES_GU 1
+#endif
+#ifndef STMOE_GROUP8_KBOXES_D
+#define STMOE_GROUP8_KBOXES_D 2
+#endif
+// reduction columns of a box row (128 bytes) and activation planes per operand format
+template <int WDT> __host__ __device__ constexpr int group_box_cols() { return WDT == 1 ? kDenseKStep : 2 * kDenseKStep; }
+template <int WDT> __host__ __device__ constexpr int group_planes() { return WDT == 1 ? 1 : 3; }
+// Boxes per matrix and stage: consecutive boxes continue the same rows, so a stage asks for
+// boxes * 128 contiguous bytes of every row at once.  bf16, measured on C1 batch 4 / C2 batch 8:
 // (gate/up, down) = (1,1) 0.893 / 0.728 of the HBM roofline, (2,2) 0.919 / 0.754, (2,4) 0.927 /
 // 0.762; 4 for gate/up leaves a single stage.
-template <int NMAT> __host__ __device__ constexpr int group_kboxes() { return NMAT == 2 ? STMOE_GROUP_KBOXES_GU : STMOE_GROUP_KBOXES_D; }
-template <int NMAT> __host__ __device__ constexpr int group_kstage() { return group_kboxes<NMAT>() * kDenseKStep; }  // columns per stage
+template <int NMAT, int WDT> __host__ __device__ constexpr int group_kboxes()
+{
+    return WDT == 1 ? (NMAT == 2 ? STMOE_GROUP_KBOXES_GU : STMOE_GROUP_KBOXES_D)
+                    : (NMAT == 2 ? STMOE_GROUP8_KBOXES_GU : STMOE_GROUP8_KBOXES_D);
+}
+template <int NMAT, int WDT> __host__ __device__ constexpr int group_kstage() { return group_kboxes<NMAT, WDT>() * group_box_cols<WDT>(); }  // columns per stage
 constexpr int kGroupMaxStages = 12;
 constexpr int kGroupSmemBytes = 226 * 1024;                       // dynamic shared memory of a CTA (one per SM)
-// A stage holds NMAT weight tiles and np activation rows of 128 bytes (np a multiple of 16, so
-// every tile base stays 1024-byte aligned once rounded up); as many stages as fit.
-__host__ __device__ constexpr int group_act_bytes(int np) { return (np * kDenseKStep * 2 + 1023) / 1024 * 1024; }
-template <int NMAT> __host__ __device__ constexpr int group_stage_bytes(int np)
+// A box holds NMAT weight tiles and, per activation plane, np rows of 128 bytes (np a multiple
+// of 16, so every tile base stays 1024-byte aligned once rounded up); as many stages as fit.
+__host__ __device__ constexpr int group_act_bytes(int np) { return (np * 128 + 1023) / 1024 * 1024; }
+template <int NMAT, int WDT> __host__ __device__ constexpr int group_box_bytes(int np)
 {
-    return group_kboxes<NMAT>() * (NMAT * kGroupTileBytes + group_act_bytes(np));
+    return NMAT * kGroupTileBytes + group_planes<WDT>() * group_act_bytes(np);
 }
-template <int NMAT> __host__ __device__ constexpr int group_stages(int np)
+template <int NMAT, int WDT> __host__ __device__ constexpr int group_stage_bytes(int np)
 {
-    const int n = (kGroupSmemBytes - 1024) / group_stage_bytes<NMAT>(np);
+    return group_kboxes<NMAT, WDT>() * group_box_bytes<NMAT, WDT>(np);
+}
+template <int NMAT, int WDT> __host__ __device__ constexpr int group_stages(int np)
+{
+    const int n = (kGroupSmemBytes - 1024) / group_stage_bytes<NMAT, WDT>(np);
     return n < kGroupMaxStages ? n : kGroupMaxStages;
 }
 
@@ -68,10 +97,47 @@ struct GroupArgs {
     int splits, seg;       // down: splits of the reduction dimension, columns per split (multiple of 64)
     int KS;                // K + n_shared
     const float *inv_rms;  // gate/up: RMSNorm factor per sequence, applied to the accumulators
-    __nv_bfloat16 *act;    // gate/up out, down in: [pairs][I]
+    __nv_bfloat16 *act;    // bf16 weights: gate/up out, down in: [pairs][I]
     float *part;           // down out: [B*KS][splits][H]
     unsigned *err;
+    // fp8 stacks
+    uint8_t *act8;         // gate/up out, down in: three e5m2 planes [3][act_rows][I]
+    int act_rows;          // rows of one plane of act8
+    int x_rows;            // rows of one plane of this projection's activation operand (hidden state: 64)
+    const uint8_t *store;  // first expert image of the stack, for the row scales behind the matrices
+    unsigned long long img_bytes;
+    int scale_off;         // element offset of this projection's scales in the image's scale vector
 };
+
+// e4m3 weights x e5m2 activations -> fp32, both operands K-major, M = 128, N = n
+__host__ __device__ constexpr uint32_t umma_idesc_e4m3_e5m2(int n)
+{
+    return (1u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kDenseRows >> 4) << 24);
+}
+__device__ __forceinline__ void umma_f8(uint32_t tmem_d, uint64_t a, uint64_t b, uint32_t idesc, bool accumulate)
+{
+    asm volatile(
+        "{.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;}"
+        :
+        : "r"(tmem_d), "l"(a), "l"(b), "r"(idesc), "r"((uint32_t)accumulate)
+        : "memory");
+}
+// v = t[0] + t[1] + t[2] up to 2^-9 |v|: each e5m2 term rounds what the terms before it left
+// (an e5m2 value is the upper byte of the f16 with the same value)
+__device__ __forceinline__ float e5m2_to_f32(uint8_t b)
+{
+    return __half2float(__ushort_as_half((unsigned short)((unsigned short)b << 8)));
+}
+__device__ __forceinline__ void split_e5m2x3(float v, uint8_t (&t)[3])
+{
+#pragma unroll
+    for (int p = 0; p < 3; ++p) {
+        t[p] = (uint8_t)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E5M2);
+        v -= e5m2_to_f32(t[p]);
+    }
+}
 
 __device__ __forceinline__ void dmbar_expect_tx(uint64_t *bar, uint32_t bytes)
 {
@@ -92,7 +158,8 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, i
         : "memory");
 }
 // K-major operand tile in the 128-byte swizzled layout (rows of 128 bytes, 8-row groups 1024
-// bytes apart, tile base 1024-byte aligned); kstep = which 16-column slice of the 64.
+// bytes apart, tile base 1024-byte aligned); kstep = which 32-byte slice of the row (one MMA's
+// reduction depth: 16 two-byte or 32 one-byte elements).
 __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr, int kstep)
 {
     return (uint64_t)(((smem_addr + kstep * 32) >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
@@ -145,13 +212,14 @@ __device__ __forceinline__ void group_ring_init(const GroupRing &r)
 
 // One thread: issue the TMA loads of this CTA's tasks.  pos/issued carry on from earlier calls.
 // NMAT = 2: gate and up projections; NMAT = 1: down projection.
-template <int NMAT>
+template <int NMAT, int WDT>
 __device__ __forceinline__ void group_produce(const CUtensorMap *map_w0, const CUtensorMap *map_w1,
                                               const CUtensorMap *map_x, const GroupArgs &a, const GroupRing &r,
                                               RingPos &pos, int &issued)
 {
-    constexpr int KB = group_kboxes<NMAT>(), KSTAGE = group_kstage<NMAT>();
-    const int np = a.np, box = NMAT * kGroupTileBytes + group_act_bytes(np);
+    constexpr int KB = group_kboxes<NMAT, WDT>(), KSTAGE = group_kstage<NMAT, WDT>(), COLS = group_box_cols<WDT>();
+    constexpr int PLANES = group_planes<WDT>();
+    const int np = a.np, act_bytes = group_act_bytes(np), box = group_box_bytes<NMAT, WDT>(np);
     const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
     const int n_tasks = *a.wl.n_groups * tiles * a.splits;
     for (int task = blockIdx.x; task < n_tasks && !*r.dead; task += gridDim.x) {
@@ -163,13 +231,16 @@ __device__ __forceinline__ void group_produce(const CUtensorMap *map_w0, const C
             if (!dmbar_wait(&r.empty[pos.s], pos.ph ^ 1u, r.dead)) return;
             uint8_t *st = r.dsm + (size_t)pos.s * r.slot;
             // boxes past the end of the reduction dimension are zero-filled and still count
-            dmbar_expect_tx(&r.full[pos.s], (uint32_t)(KB * (NMAT * kGroupTileBytes + np * kDenseKStep * 2)));
+            dmbar_expect_tx(&r.full[pos.s], (uint32_t)(KB * (NMAT * kGroupTileBytes + PLANES * np * 128)));
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
                 uint8_t *sb = st + kb * box;
-                tma_load_3d(sb, map_w0, k + kb * kDenseKStep, t.row0, img, &r.full[pos.s]);
-                if (NMAT == 2) tma_load_3d(sb + kGroupTileBytes, map_w1, k + kb * kDenseKStep, t.row0, img, &r.full[pos.s]);
-                tma_load_2d(sb + NMAT * kGroupTileBytes, map_x, k + kb * kDenseKStep, xrow, &r.full[pos.s]);
+                tma_load_3d(sb, map_w0, k + kb * COLS, t.row0, img, &r.full[pos.s]);
+                if (NMAT == 2) tma_load_3d(sb + kGroupTileBytes, map_w1, k + kb * COLS, t.row0, img, &r.full[pos.s]);
+#pragma unroll
+                for (int p = 0; p < PLANES; ++p)
+                    tma_load_2d(sb + NMAT * kGroupTileBytes + p * act_bytes, map_x, k + kb * COLS, p * a.x_rows + xrow,
+                                &r.full[pos.s]);
             }
             ++issued;
             if (++pos.s == r.NS) pos.s = 0, pos.ph ^= 1u;
@@ -189,12 +260,12 @@ __device__ __forceinline__ void group_drain(const GroupRing &r, RingPos pos, int
 
 // One thread: issue the MMAs of this CTA's tasks.  `it` counts the CTA's tasks across calls
 // (accumulator buffer = it & 1).
-template <int NMAT>
+template <int NMAT, int WDT>
 __device__ __forceinline__ void group_mma(const GroupArgs &a, const GroupRing &r, RingPos &pos, int &it)
 {
-    constexpr int KB = group_kboxes<NMAT>(), KSTAGE = group_kstage<NMAT>();
-    const int np = a.np, box = NMAT * kGroupTileBytes + group_act_bytes(np);
-    const uint32_t idesc = umma_idesc_bf16(np);
+    constexpr int KB = group_kboxes<NMAT, WDT>(), KSTAGE = group_kstage<NMAT, WDT>(), PLANES = group_planes<WDT>();
+    const int np = a.np, act_bytes = group_act_bytes(np), box = group_box_bytes<NMAT, WDT>(np);
+    const uint32_t idesc = WDT == 1 ? umma_idesc_bf16(np) : umma_idesc_e4m3_e5m2(np);
     const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
     const int n_tasks = *a.wl.n_groups * tiles * a.splits;
     for (int task = blockIdx.x; task < n_tasks && !*r.dead; task += gridDim.x, ++it) {
@@ -211,12 +282,20 @@ __device__ __forceinline__ void group_mma(const GroupArgs &a, const GroupRing &r
             for (int kb = 0; kb < KB; ++kb) {
                 const uint32_t st = dsmem_u32(r.dsm + (size_t)pos.s * r.slot) + kb * box;
 #pragma unroll
-                for (int j = 0; j < kDenseKStep / 16; ++j) {
-                    const uint64_t bd = umma_desc_sw128(st + NMAT * kGroupTileBytes, j);
+                for (int j = 0; j < 4; ++j) {  // four 32-byte slices of the 128-byte box row
 #pragma unroll
-                    for (int mat = 0; mat < NMAT; ++mat)
-                        umma_bf16(acc + mat * 64, umma_desc_sw128(st + mat * kGroupTileBytes, j), bd, idesc,
-                                  !first || kb > 0 || j > 0);
+                    for (int p = 0; p < PLANES; ++p) {
+                        const uint64_t bd = umma_desc_sw128(st + NMAT * kGroupTileBytes + p * act_bytes, j);
+#pragma unroll
+                        for (int mat = 0; mat < NMAT; ++mat) {
+                            const uint64_t ad = umma_desc_sw128(st + mat * kGroupTileBytes, j);
+                            const bool accumulate = !first || kb > 0 || j > 0 || p > 0;
+                            if constexpr (WDT == 1)
+                                umma_bf16(acc + mat * 64, ad, bd, idesc, accumulate);
+                            else
+                                umma_f8(acc + mat * 64, ad, bd, idesc, accumulate);
+                        }
+                    }
                 }
             }
             first = false;
@@ -229,7 +308,7 @@ __device__ __forceinline__ void group_mma(const GroupArgs &a, const GroupRing &r
 
 // Four warps (lg = the TMEM lane quarter the warp may read = warp index % 4): thread = one
 // weight row.  `it` as in group_mma.
-template <int NMAT>
+template <int NMAT, int WDT>
 __device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRing &r, int &it, int lg, int lane)
 {
     const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
@@ -238,17 +317,37 @@ __device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRi
         const GroupTask t = group_task(a, task);
         const int ab = it & 1;
         const int start = a.wl.g_start[t.g], count = a.wl.g_count[t.g];
+        const int row = t.row0 + lg * kWarp + lane;
+        float s0 = 1.f, s1 = 1.f;
+        if constexpr (WDT == 2) {
+            // bf16 scales per output channel behind the three matrices: [gate I | up I | down H]
+            const int ge = a.wl.g_expert[t.g];
+            const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
+            const uint16_t *sc = reinterpret_cast<const uint16_t *>(a.store + (size_t)img * a.img_bytes +
+                                                                    3 * (size_t)a.rows * a.kd) + a.scale_off;
+            const int srow = min(row, a.rows - 1);
+            s0 = bf16_to_f32(sc[srow]);
+            if (NMAT == 2) s1 = bf16_to_f32(sc[a.rows + srow]);
+        }
         const bool ok = dmbar_wait(&r.tfull[ab], ((uint32_t)it >> 1) & 1u, r.dead);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t acc = r.tmem + ab * 128 + ((uint32_t)(lg * kWarp) << 16);
-        const int row = t.row0 + lg * kWarp + lane;
         if (NMAT == 2) {
             for (int i = 0; i < count; ++i) {
                 const int tok = a.wl.pair_token[start + i];
                 const float inv = a.inv_rms[tok];  // W (inv * h) = inv * (W h)
-                const float g = inv * tmem_ld1(acc + tok), u = inv * tmem_ld1(acc + 64 + tok);
-                if (ok && row < a.rows)
-                    a.act[(size_t)(start + i) * a.rows + row] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
+                const float g = inv * s0 * tmem_ld1(acc + tok), u = inv * s1 * tmem_ld1(acc + 64 + tok);
+                const float v = g / (1.f + expf(-g)) * u;
+                if (ok && row < a.rows) {
+                    if constexpr (WDT == 1) {
+                        a.act[(size_t)(start + i) * a.rows + row] = __float2bfloat16_rn(v);
+                    } else {
+                        uint8_t tp[3];
+                        split_e5m2x3(v, tp);
+#pragma unroll
+                        for (int p = 0; p < 3; ++p) a.act8[((size_t)p * a.act_rows + start + i) * a.rows + row] = tp[p];
+                    }
+                }
             }
         } else {
             for (int i0 = 0; i0 < count; i0 += 8) {
@@ -259,7 +358,7 @@ __device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRi
                     for (int i = 0; i < 8; ++i)
                         if (i0 + i < count) {
                             const int slot = a.wl.pair_slot[start + i0 + i];
-                            a.part[((size_t)slot * a.splits + t.z) * a.rows + row] = y[i];
+                            a.part[((size_t)slot * a.splits + t.z) * a.rows + row] = s0 * y[i];
                         }
                 }
             }
@@ -272,7 +371,7 @@ __device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRi
 }
 
 // One projection as a kernel of its own (per-layer launches).
-template <int NMAT>
+template <int NMAT, int WDT>
 __global__ void __launch_bounds__(kGroupThreads, 1)
 dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
                    const __grid_constant__ CUtensorMap map_x, GroupArgs a)
@@ -285,9 +384,9 @@ dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_cons
     GroupRing r;
     r.dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dsm_raw) + 1023) & ~(uintptr_t)1023);
     r.full = full, r.empty = empty, r.tfull = tfull, r.tempty = tempty, r.dead = &s_dead;
-    r.NS = group_stages<NMAT>(a.np), r.slot = group_stage_bytes<NMAT>(a.np);
+    r.NS = group_stages<NMAT, WDT>(a.np), r.slot = group_stage_bytes<NMAT, WDT>(a.np);
     if (tid == 0) {
-        s_dead = 0;
+        s_dead = r.NS < 1;  // cannot happen with the host's sizing; never run a ring without stages
         group_ring_init(r);
     }
     if (warp == 1) {
@@ -305,18 +404,18 @@ dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_cons
         if (lane == 0) {
             RingPos pos;
             int issued = 0;
-            group_produce<NMAT>(&map_w0, &map_w1, &map_x, a, r, pos, issued);
+            group_produce<NMAT, WDT>(&map_w0, &map_w1, &map_x, a, r, pos, issued);
             group_drain(r, pos, issued);
         }
     } else if (warp == 1) {
         if (lane == 0) {
             RingPos pos;
             int it = 0;
-            group_mma<NMAT>(a, r, pos, it);
+            group_mma<NMAT, WDT>(a, r, pos, it);
         }
     } else {
         int it = 0;
-        group_epilogue<NMAT>(a, r, it, warp % 4, lane);
+        group_epilogue<NMAT, WDT>(a, r, it, warp % 4, lane);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();

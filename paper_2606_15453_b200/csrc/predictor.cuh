@@ -11,7 +11,7 @@ namespace stmoe_dev {
 
 constexpr int kConfInit = 2;   // binary 10
 constexpr int kConfMax = 3;    // binary 11
-constexpr int kThreshold = 2;  // prefetch when score >= binary 10
+constexpr int kThreshold = 2;  // history bonus of Eq. 1 and the paper's set threshold: binary 10
 
 struct PredState {
     uint32_t *Co;        // [L-1][E][E]
@@ -22,6 +22,9 @@ struct PredState {
     uint32_t *pred_mask; // [Bmax][8] set predicted for the layer that runs next
     uint32_t *pred_valid;// [Bmax]
     unsigned long long *stats;  // [0] steps [1] routed [2] predicted [3] hits [4] near ties
+    int threshold;       // an expert is predicted when its score reaches this (Section 4.2: binary 10)
+    int live_counts;     // Algorithm 3's new candidate: 0 lowest routed id, 1 largest count in a Co row
+                         // that keeps counting at run time
 };
 
 struct PredArgs {
@@ -35,13 +38,41 @@ struct PredArgs {
     int32_t *queue;       // optional: [0] n, [1..E] ids, [1+E..2E] scores (priority order)
 };
 
-// Algorithm 3 for one row, executed by one warp: lane c < K owns candidate slot c.
+// Which routed expert a replacing slot takes (Algorithm 3 leaves it open).  Every lane of a group
+// of `width` lanes calls this; lane k < K of the group carries routed expert k.  avail: the group's
+// routed experts the row does not hold; nth (1-based): this lane is the nth replacing slot of its
+// row in slot order.  The nth replacing slot takes the nth candidate, exactly as a slot-by-slot
+// scan that re-reads the row would: candidates in ascending id or, with by_count (cnt = this
+// lane's expert's count in the row), by (count descending, id ascending).  Returns the group lane that carries the
+// chosen expert, or 0xffffffff when there are fewer candidates than replacing slots.
+__device__ __forceinline__ unsigned replacement_source(unsigned avail, int nth, bool by_count, unsigned cnt, int K,
+                                                       int gl, int width)
+{
+    if (!by_count) return __fns(avail, 0, nth);
+    int rank = 0;
+    for (int k = 0; k < K; ++k) {
+        const unsigned ck = __shfl_sync(kFull, cnt, k, width);
+        rank += ((avail >> k) & 1u) && (ck > cnt || (ck == cnt && k < gl));
+    }
+    unsigned pos = 0xffffffffu;
+    for (int k = 0; k < K; ++k) {
+        const int rk = __shfl_sync(kFull, rank, k, width);
+        if (((avail >> k) & 1u) && rk == nth - 1) pos = (unsigned)k;
+    }
+    return pos;
+}
+
+// Algorithm 3 for one row, executed by one warp: lane c < K owns candidate slot c.  co_row: the
+// row of the pair's co-activation counts when counting goes on at run time (this step's K pairs
+// of the row are counted here, before the update), else nullptr.
 __device__ __forceinline__ void update_row(uint8_t *ids, uint8_t *conf, int K, const int32_t *F,
-                                           int lane)
+                                           int lane, uint32_t *co_row = nullptr)
 {
     const bool act = lane < K;
     int id = act ? ids[lane] : -1, cf = act ? conf[lane] : 0;
     const int myf = act ? F[lane] : -2;  // lane k also carries routed expert k (ascending)
+    unsigned cnt = 0;
+    if (co_row && act) cnt = co_row[myf] + 1u, co_row[myf] = cnt;
     bool hit = false, held = false;
     for (int k = 0; k < K; ++k) {
         hit |= (id == __shfl_sync(kFull, myf, k));
@@ -56,11 +87,11 @@ __device__ __forceinline__ void update_row(uint8_t *ids, uint8_t *conf, int K, c
     }
     const unsigned rep = __ballot_sync(kFull, replace);
     if (rep) {
-        // routed experts the row does not hold, lowest id first; the n-th replacing slot
-        // (in slot order) takes the n-th of them, exactly as a slot-by-slot scan would.
+        // routed experts the row does not hold; the n-th replacing slot (in slot order) takes
+        // the n-th of them, exactly as a slot-by-slot scan would.
         const unsigned avail = __ballot_sync(kFull, act && !held);
         const int nth = __popc(rep & ((1u << lane) - 1u)) + 1;
-        const unsigned pos = replace ? __fns(avail, 0, nth) : 0u;
+        const unsigned pos = replacement_source(avail, nth, co_row != nullptr, cnt, K, lane, kWarp);
         const int g = __shfl_sync(kFull, myf, pos & 31u);
         if (replace && pos != 0xffffffffu) id = g, cf = kConfInit;
     }
@@ -70,10 +101,12 @@ __device__ __forceinline__ void update_row(uint8_t *ids, uint8_t *conf, int K, c
 // Algorithm 3 for the rows of one sequence's previous-layer experts, several rows at a time: the
 // warp is cut into groups of G lanes (G = the power of two >= K) and each group updates one row
 // exactly as update_row does.  The rows of one sequence are distinct, so they do not depend on
-// one another.  take(k) says whether row prev[k] belongs to this warp.
+// one another.  take(k) says whether row prev[k] belongs to this warp.  co: the pair's [E][E]
+// counts when counting goes on at run time, else nullptr.
 template <typename Take>
 __device__ __forceinline__ void update_rows_grouped(uint8_t *gid, uint8_t *gcf, int K, const int32_t *prev,
-                                                    const int32_t *F, int lane, Take take)
+                                                    const int32_t *F, int lane, Take take, uint32_t *co = nullptr,
+                                                    int E = 0)
 {
     int G = 1;
     while (G < K) G <<= 1;
@@ -89,6 +122,11 @@ __device__ __forceinline__ void update_rows_grouped(uint8_t *gid, uint8_t *gcf, 
         uint8_t *ids = gid + (size_t)e * K, *conf = gcf + (size_t)e * K;
         const bool act = row_ok && sl < K;
         int id = act ? ids[sl] : -1, cf = act ? conf[sl] : 0;
+        unsigned cnt = 0;
+        if (co && act) {
+            uint32_t *c = co + (size_t)e * E + myf;
+            cnt = *c + 1u, *c = cnt;
+        }
         bool hit = false, held = false;
         for (int k = 0; k < K; ++k) {
             hit |= (id == __shfl_sync(kFull, myf, k, G));
@@ -103,10 +141,11 @@ __device__ __forceinline__ void update_rows_grouped(uint8_t *gid, uint8_t *gcf, 
         }
         const unsigned rep = (__ballot_sync(kFull, replace) >> (sub * G)) & gmask;
         const unsigned avail = (__ballot_sync(kFull, act && !held) >> (sub * G)) & gmask;
-        // routed experts the row does not hold, lowest id first; the n-th replacing slot (in slot
-        // order) takes the n-th of them
+        // routed experts the row does not hold; the n-th replacing slot (in slot order) takes the
+        // n-th of them
         const int nth = __popc(rep & ((1u << sl) - 1u)) + 1;
-        const unsigned pos = replace ? __fns(avail, 0, nth) : 0u;
+        unsigned pos = replacement_source(avail, nth, co != nullptr, cnt, K, sl, G);
+        if (!replace) pos = 0u;
         const int g = __shfl_sync(kFull, myf, pos & (unsigned)(G - 1), G);
         if (replace && pos != 0xffffffffu) id = g, cf = kConfInit;
         if (act) ids[sl] = (uint8_t)id, conf[sl] = (uint8_t)cf;
@@ -155,10 +194,11 @@ __global__ void __launch_bounds__(256) predictor_step_kernel(PredArgs a)
             uint8_t *gcf = a.st.cct_conf + (size_t)(layer - 1) * E * K;
             for (int i = threadIdx.x; i < E * K; i += blockDim.x) s_id[i] = gid[i], s_cf[i] = gcf[i];
             __syncthreads();
+            uint32_t *co = a.st.live_counts ? a.st.Co + (size_t)(layer - 1) * E * E : nullptr;
             for (int b = 0; b < B; ++b) {
                 for (int k = warp; k < K; k += NW) {
                     const int e = a.prev[b * K + k];
-                    update_row(s_id + e * K, s_cf + e * K, K, a.cur + b * K, lane);
+                    update_row(s_id + e * K, s_cf + e * K, K, a.cur + b * K, lane, co ? co + (size_t)e * E : nullptr);
                 }
                 __syncthreads();
             }
@@ -205,7 +245,7 @@ __global__ void __launch_bounds__(256) predictor_step_kernel(PredArgs a)
         int count = 0;
         for (int w = 0; w < kMaxExperts / kWarp; ++w) {
             const int f = w * kWarp + lane;
-            const bool in = f < E && sc[f] >= kThreshold;
+            const bool in = f < E && sc[f] >= a.st.threshold;
             const unsigned msk = __ballot_sync(kFull, in);
             if (lane == 0) a.st.pred_mask[b * 8 + w] = msk;
             if (in) {

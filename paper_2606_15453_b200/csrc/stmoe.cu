@@ -392,9 +392,9 @@ struct stmoe {
     __nv_bfloat16 *d_xb = nullptr, *d_actb = nullptr;
     float *d_part_dense = nullptr;
     int dense_grid = 0;
-    bool dense8 = false;            // fp8 stacks: dense8_group.cuh (per-layer kernels only)
+    bool dense8 = false;            // fp8 stacks: e4m3 weight tiles x three e5m2 activation planes
     CUtensorMap map8_gate{}, map8_up{}, map8_down{}, map8_x[4]{}, map8_act[4]{};
-    __half *d_xb16 = nullptr, *d_act16 = nullptr;
+    uint8_t *d_x8 = nullptr, *d_act8 = nullptr;  // [3][64][H], [3][pairs + 64][I]
     bool dense_persistent = false;  // one cooperative kernel per decode step (token_dense_kernel.cuh)
     int dense_dyn_bytes = 0;
 
@@ -657,8 +657,7 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
 
 // ---- tensor-core path (dense_group.cuh) ---------------------------------------------------
 constexpr int kDenseMinBatch = 2;   // bf16 stacks: measured ahead of the CUDA-core kernels from two sequences on
-constexpr int kDense8PersistentMaxBatch = 4;
-constexpr int kDense8MinBatch = 3;  // fp8 stacks (the conversion costs issue slots): level at two, ahead from three
+constexpr int kDense8MinBatch = 2;  // fp8 stacks
 constexpr int kDenseMaxSplits = 4;
 constexpr int kTokenDenseDynBytes = 220 * 1024;
 
@@ -718,15 +717,15 @@ int dense_setup(stmoe *s)
         ST_TRY(encode_map(enc, &s->map_x[i], s->d_xb, 2, xd, xs, 16 * (i + 1)));
         ST_TRY(encode_map(enc, &s->map_act[i], s->d_actb, 2, ad, as, 16 * (i + 1)));
     }
-    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
-    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
+    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
+    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
     s->dense_grid = sm_count();
     s->dense_min_batch = kDenseMinBatch;
     s->dense = true;
     if (s->persistent) {  // cooperative launches work and the per-layer buffers exist
         void *k = token_dense_kernel(s->rdt, false);
         const int np = (B + 15) / 16 * 16;
-        const int slot = std::max(group_stage_bytes<1>(np), group_stage_bytes<2>(np));
+        const int slot = std::max(group_stage_bytes<1, 1>(np), group_stage_bytes<2, 1>(np));
         const int need = (int)token_smem(B, c.top_k, c.n_shared) + 1024 + slot;  // at least one stage
         int occ = 0;
         if (need <= kTokenDenseDynBytes &&
@@ -745,7 +744,8 @@ int dense_setup(stmoe *s)
 // list (one entry per expert) and inv_rms come from the router kernel launched before
 int dense_down_splits(const stmoe *s, int batch, int *seg);
 
-// fp8 stacks: tensor maps over the e4m3 images (128 x 128-byte boxes) and f16 activation buffers
+// fp8 stacks: tensor maps over the e4m3 images (128 x 128-byte boxes) and over the e5m2 planes of
+// the activations (a plane after the other in the row dimension)
 int dense8_setup(stmoe *s)
 {
     const stmoe_config_t &c = s->cfg;
@@ -761,34 +761,35 @@ int dense8_setup(stmoe *s)
         return STMOE_OK;
     }
     EncodeTiledFn enc = (EncodeTiledFn)sym;
-    const size_t pairs = (size_t)B * s->KS;
-    CU_TRY(cudaMalloc(&s->d_xb16, sizeof(__half) * (size_t)kDenseMaxTokens * H));
-    CU_TRY(cudaMemset(s->d_xb16, 0, sizeof(__half) * (size_t)kDenseMaxTokens * H));
-    CU_TRY(cudaMalloc(&s->d_act16, sizeof(__half) * (pairs + kDenseMaxTokens) * I));
-    CU_TRY(cudaMemset(s->d_act16, 0, sizeof(__half) * (pairs + kDenseMaxTokens) * I));
+    const size_t pairs = (size_t)B * s->KS, act_rows = pairs + kDenseMaxTokens;
+    CU_TRY(cudaMalloc(&s->d_x8, 3 * (size_t)kDenseMaxTokens * H));
+    CU_TRY(cudaMemset(s->d_x8, 0, 3 * (size_t)kDenseMaxTokens * H));
+    CU_TRY(cudaMalloc(&s->d_act8, 3 * act_rows * I));
+    CU_TRY(cudaMemset(s->d_act8, 0, 3 * act_rows * I));
     CU_TRY(cudaMalloc(&s->d_part_dense, sizeof(float) * pairs * kDenseMaxSplits * H));
     const cuuint64_t n_img = (cuuint64_t)L * (E + c.n_shared);
     const cuuint64_t gd[3] = {(cuuint64_t)H, (cuuint64_t)I, n_img}, gs[2] = {(cuuint64_t)H, s->img_bytes};
     const cuuint64_t dd[3] = {(cuuint64_t)I, (cuuint64_t)H, n_img}, ds[2] = {(cuuint64_t)I, s->img_bytes};
-    const CUtensorMapDataType u8 = CU_TENSOR_MAP_DATA_TYPE_UINT8, f16 = CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
-    ST_TRY(encode_map(enc, &s->map8_gate, s->d_resident, 3, gd, gs, kDenseRows, u8, kGroup8BoxCols));
-    ST_TRY(encode_map(enc, &s->map8_up, s->d_resident + (size_t)I * H, 3, gd, gs, kDenseRows, u8, kGroup8BoxCols));
-    ST_TRY(encode_map(enc, &s->map8_down, s->d_resident + 2 * (size_t)I * H, 3, dd, ds, kDenseRows, u8, kGroup8BoxCols));
+    const CUtensorMapDataType u8 = CU_TENSOR_MAP_DATA_TYPE_UINT8;
+    constexpr int kCols = group_box_cols<2>();
+    ST_TRY(encode_map(enc, &s->map8_gate, s->d_resident, 3, gd, gs, kDenseRows, u8, kCols));
+    ST_TRY(encode_map(enc, &s->map8_up, s->d_resident + (size_t)I * H, 3, gd, gs, kDenseRows, u8, kCols));
+    ST_TRY(encode_map(enc, &s->map8_down, s->d_resident + 2 * (size_t)I * H, 3, dd, ds, kDenseRows, u8, kCols));
     for (int i = 0; i < 4; ++i) {
-        const cuuint64_t xd[2] = {(cuuint64_t)H, (cuuint64_t)kDenseMaxTokens}, xs[1] = {(cuuint64_t)H * 2};
-        const cuuint64_t ad[2] = {(cuuint64_t)I, (cuuint64_t)(pairs + kDenseMaxTokens)}, as[1] = {(cuuint64_t)I * 2};
-        ST_TRY(encode_map(enc, &s->map8_x[i], s->d_xb16, 2, xd, xs, 16 * (i + 1), f16));
-        ST_TRY(encode_map(enc, &s->map8_act[i], s->d_act16, 2, ad, as, 16 * (i + 1), f16));
+        const cuuint64_t xd[2] = {(cuuint64_t)H, (cuuint64_t)(3 * kDenseMaxTokens)}, xs[1] = {(cuuint64_t)H};
+        const cuuint64_t ad[2] = {(cuuint64_t)I, (cuuint64_t)(3 * act_rows)}, as[1] = {(cuuint64_t)I};
+        ST_TRY(encode_map(enc, &s->map8_x[i], s->d_x8, 2, xd, xs, 16 * (i + 1), u8, kCols));
+        ST_TRY(encode_map(enc, &s->map8_act[i], s->d_act8, 2, ad, as, 16 * (i + 1), u8, kCols));
     }
-    CU_TRY(cudaFuncSetAttribute(dense8_group_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
-    CU_TRY(cudaFuncSetAttribute(dense8_group_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
+    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
+    CU_TRY(cudaFuncSetAttribute(dense_group_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGroupSmemBytes));
     s->dense_grid = sm_count();
     s->dense_min_batch = kDense8MinBatch;
     s->dense8 = true;
     if (s->persistent) {  // cooperative launches work and the per-layer buffers exist
         void *k = token_dense_kernel(s->rdt, true);
         const int np = (B + 15) / 16 * 16;
-        const int slot = std::max(group8_stage_bytes<1>(np), group8_stage_bytes<2>(np));
+        const int slot = std::max(group_stage_bytes<1, 2>(np), group_stage_bytes<2, 2>(np));
         const int need = (int)token_smem(B, c.top_k, c.n_shared) + 1024 + slot;  // at least one stage
         int occ = 0;
         if (need <= kTokenDenseDynBytes &&
@@ -816,30 +817,31 @@ int dense8_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, 
         CU_TRY(cudaEventRecord(e0, st));
     }
     if (!chained) {
-        dense8_cast_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fa.h, batch * H, s->d_xb16);
+        dense8_cast_kernel<<<std::min(s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fa.h, batch * H, H, s->d_x8);
         s->launches += 1;
     }
-    Group8Args a8{};
-    GroupArgs &g = a8.g;
+    GroupArgs g{};
     g.wl = fa.wl, g.E = E, g.img_routed0 = layer * E, g.img_shared0 = c.n_layers * E + layer * c.n_shared;
     g.np = np, g.KS = s->KS, g.inv_rms = fa.inv_rms, g.part = s->d_part_dense, g.err = s->d_err;
-    a8.store = s->d_resident, a8.img_bytes = s->img_bytes, a8.act16 = s->d_act16;
-    g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + group8_kstage<2>() - 1) / group8_kstage<2>() * group8_kstage<2>();
-    a8.scale_off = 0;
-    dense8_group_kernel<2><<<s->dense_grid, kGroup8Threads, kGroupSmemBytes, st>>>(s->map8_gate, s->map8_up,
-                                                                                   s->map8_x[np / 16 - 1], a8);
+    g.store = s->d_resident, g.img_bytes = s->img_bytes;
+    g.act8 = s->d_act8, g.act_rows = batch * s->KS + kDenseMaxTokens;
+    constexpr int kGu = group_kstage<2, 2>(), kDn = group_kstage<1, 2>();
+    g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kGu - 1) / kGu * kGu;
+    g.scale_off = 0, g.x_rows = kDenseMaxTokens;
+    dense_group_kernel<2, 2><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map8_gate, s->map8_up,
+                                                                                    s->map8_x[np / 16 - 1], g);
     if (timed) CU_TRY(cudaEventRecord(e1, st));
     int seg = 0;
     int splits = dense_down_splits(s, batch, &seg);
-    seg = (seg + group8_kstage<1>() - 1) / group8_kstage<1>() * group8_kstage<1>();
+    seg = (seg + kDn - 1) / kDn * kDn;
     splits = (I + seg - 1) / seg;
     g.rows = H, g.kd = I, g.splits = splits, g.seg = seg;
-    a8.scale_off = 2 * I;
-    dense8_group_kernel<1><<<s->dense_grid, kGroup8Threads, kGroupSmemBytes, st>>>(s->map8_down, s->map8_down,
-                                                                                   s->map8_act[np / 16 - 1], a8);
+    g.scale_off = 2 * I, g.x_rows = g.act_rows;
+    dense_group_kernel<1, 2><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map8_down, s->map8_down,
+                                                                                    s->map8_act[np / 16 - 1], g);
     FfnArgs fc = fa;
     fc.part = s->d_part_dense;
-    dense8_combine_kernel<<<std::min(8 * s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fc, splits, s->d_xb16);
+    dense8_combine_kernel<<<std::min(8 * s->dense_grid, (batch * H + 255) / 256), 256, 0, st>>>(fc, splits, s->d_x8);
     if (timed) {
         CU_TRY(cudaEventRecord(e2, st));
         s->spans.push_back(TimedSpan{e0, e1, 2});
@@ -871,8 +873,8 @@ int dense_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, c
     GroupArgs g{};
     g.wl = fa.wl, g.E = E, g.img_routed0 = layer * E, g.img_shared0 = c.n_layers * E + layer * c.n_shared;
     g.np = np, g.KS = s->KS, g.inv_rms = fa.inv_rms, g.act = s->d_actb, g.part = s->d_part_dense, g.err = s->d_err;
-    g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + group_kstage<2>() - 1) / group_kstage<2>() * group_kstage<2>();
-    dense_group_kernel<2><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_gate, s->map_up,
+    g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + group_kstage<2, 1>() - 1) / group_kstage<2, 1>() * group_kstage<2, 1>();
+    dense_group_kernel<2, 1><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_gate, s->map_up,
                                                                                       s->map_x[np / 16 - 1], g);
     if (timed) CU_TRY(cudaEventRecord(e1, st));
     // down: split the reduction dimension until there are a few tasks per SM
@@ -881,7 +883,7 @@ int dense_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, c
     const int tiles = (H + kDenseRows - 1) / kDenseRows;
     (void)tiles;
     g.rows = H, g.kd = I, g.splits = splits, g.seg = seg;
-    dense_group_kernel<1><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_down, s->map_down,
+    dense_group_kernel<1, 1><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_down, s->map_down,
                                                                                       s->map_act[np / 16 - 1], g);
     FfnArgs fc = fa;
     fc.part = s->d_part_dense;
@@ -1117,7 +1119,7 @@ int dense_down_splits(const stmoe *s, int batch, int *seg)
     const stmoe_config_t &c = s->cfg;
     const int entries = std::min(c.n_experts, batch * c.top_k) + c.n_shared, tiles = (c.hidden + kDenseRows - 1) / kDenseRows;
     int splits = std::max(1, std::min(kDenseMaxSplits, (4 * s->dense_grid + entries * tiles - 1) / (entries * tiles)));
-    *seg = ((c.inter + splits - 1) / splits + group_kstage<1>() - 1) / group_kstage<1>() * group_kstage<1>();
+    *seg = ((c.inter + splits - 1) / splits + group_kstage<1, 1>() - 1) / group_kstage<1, 1>() * group_kstage<1, 1>();
     return (c.inter + *seg - 1) / *seg;  // no empty split
 }
 
@@ -1143,10 +1145,10 @@ int token_dense(stmoe *s, int batch, const float *h_in, float *h_out, int32_t *r
     d.img_shared_base = c.n_layers * c.n_experts;
     d.dyn_bytes = s->dense_dyn_bytes;
     const bool w8 = s->dense8;
-    d.xb = w8 ? (void *)s->d_xb16 : (void *)s->d_xb, d.actb = w8 ? (void *)s->d_act16 : (void *)s->d_actb;
+    d.xb = w8 ? (void *)s->d_x8 : (void *)s->d_xb, d.actb = w8 ? (void *)s->d_act8 : (void *)s->d_actb;
     d.part = s->d_part_dense, d.store = s->d_resident, d.img_bytes = s->img_bytes;
-    if (w8) {  // the fp8 down projection walks two boxes per stage
-        d.seg = (d.seg + group8_kstage<1>() - 1) / group8_kstage<1>() * group8_kstage<1>();
+    if (w8) {  // a split is a whole number of the fp8 format's stages
+        d.seg = (d.seg + group_kstage<1, 2>() - 1) / group_kstage<1, 2>() * group_kstage<1, 2>();
         d.splits = (c.inter + d.seg - 1) / d.seg;
     }
     const int np = (batch + 15) / 16 * 16;
@@ -1212,7 +1214,7 @@ int stmoe_destroy(stmoe_t *s)
                    s->pst.Co, s->pst.cct_id, s->pst.cct_conf, s->pst.HT, s->pst.t, s->pst.pred_mask,
                    s->pst.pred_valid, s->pst.stats, s->d_rpart, s->d_sspart, s->d_arrivals, s->d_tile_done, s->d_hbuf, s->d_rpart_all, s->d_sspart_all,
                    s->d_act_all, s->d_part_all, s->d_tiles_all, s->d_barrier, s->d_err, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
-                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense, s->d_xb16, s->d_act16,
+                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense, s->d_x8, s->d_act8,
                    s->d_down_t, s->d_zpart, s->d_acc};
     if (s->d_shared && s->d_resident && s->d_shared > s->d_resident) dev[2] = nullptr;  // one allocation
     for (void *p : dev)
@@ -1303,6 +1305,8 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
         CR_TRY(cudaMalloc(&s->d_blob_table, sizeof(void *) * tab.size()));
         CR_TRY(cudaMemcpy(s->d_blob_table, tab.data(), sizeof(void *) * tab.size(), cudaMemcpyHostToDevice));
     }
+    s->pst.threshold = kThreshold;
+    s->pst.live_counts = 0;
     CR_TRY(cudaMalloc(&s->pst.Co, std::max<size_t>(pairs * E * E * 4, 4)));
     CR_TRY(cudaMalloc(&s->pst.cct_id, std::max<size_t>(pairs * E * K, 4)));
     CR_TRY(cudaMalloc(&s->pst.cct_conf, std::max<size_t>(pairs * E * K, 4)));
@@ -1437,10 +1441,19 @@ int stmoe_selftest_bounded_wait(stmoe_t *s, int which, int poll_limit, void *cud
     return STMOE_OK;
 }
 
+int stmoe_set_predict_threshold(stmoe_t *s, int threshold)
+{
+    if (!s || threshold < 1 || threshold > 255 || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
+    s->pst.threshold = threshold;
+    if (s->graph_exec) cudaGraphExecDestroy(s->graph_exec), s->graph_exec = nullptr;  // captured kernels hold the old value
+    memset(s->graph_key, 0, sizeof(s->graph_key));
+    return STMOE_OK;
+}
+
 int stmoe_set_cache_policy(stmoe_t *s, int history_window, int by_turn, int prefetch_floor)
 {
     if (!s || !offloaded(s) || history_window < 0 || history_window > 32 || prefetch_floor < -1 || s->next_layer != 0 ||
-        s->cache.clock != 0)
+        s->cache.clock != 0 || (prefetch_floor >= 0 && history_window == 0))
         return STMOE_ERR_BAD_ARG;
     s->cache.W = history_window, s->cache.by_turn = by_turn != 0, s->cache.floor = prefetch_floor;
     return STMOE_OK;
@@ -1486,6 +1499,15 @@ int stmoe_set_onchip_staging(stmoe_t *s, int64_t known_bytes, int64_t predicted_
     s->stage_shared = known_bytes > 0;
     s->stage_down_bytes = known_bytes;
     s->stage_pred_bytes = predicted_bytes;
+    return STMOE_OK;
+}
+
+int stmoe_set_replacement_rule(stmoe_t *s, int live_counts)
+{
+    if (!s || s->next_layer != 0) return STMOE_ERR_BAD_ARG;
+    s->pst.live_counts = live_counts != 0;
+    if (s->graph_exec) cudaGraphExecDestroy(s->graph_exec), s->graph_exec = nullptr;  // captured kernels hold the old value
+    memset(s->graph_key, 0, sizeof(s->graph_key));
     return STMOE_OK;
 }
 
@@ -1565,9 +1587,7 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, i
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const stmoe_config_t &c = s->cfg;
     const bool build_due = !s->built && s->host_t == c.profile_tokens - 1;
-    // fp8: the persistent kernel is ahead only for small batches (measured on the C4 shape: +6 % at 3
-    // sequences, +2 % at 4, -6 % at 8 and 32, where its ring has a stage less and the predictor two warps)
-    if (s->dense_persistent && !s->time_kernels && use_dense(s, batch) && (!s->dense8 || batch <= kDense8PersistentMaxBatch))
+    if (s->dense_persistent && !s->time_kernels && use_dense(s, batch))
         return token_dense(s, batch, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);
     if (s->fused && batch == 1 && !s->time_kernels)
         return token_fused(s, h_in, h_out, routed_ids, routed_w, predicted_ids, n_predicted, flags, st);

@@ -3,13 +3,13 @@
 //
 // One 512-thread CTA per SM, launched cooperatively, walks the layers:
 //   F   weighted sum + residual of the previous layer from its down-projection partial sums
-//       (layer 0: the input), written as fp32 (router, residual) and bf16 / f16 (gate/up operand)
+//       (layer 0: the input), written as fp32 (router, residual) and as the gate/up operand (bf16,
+//       or three e5m2 planes for fp8 stacks)
 //                                                                          -> grid barrier
 //   R   split-K router GEMV tasks over all warps of the grid               -> grid barrier
 //   T   every CTA runs softmax / top-K / grouping (one work-list entry per expert) itself
 //   GU  gate/up tiles on tcgen05: warp 0 feeds TMA, warp 1 issues MMAs, warps 2-5 read the
-//       accumulators (fp8 weights: warps 6-13 widen them into tensor memory); the predictor
-//       (Algorithms 1-3) runs on the remaining warps of the last CTA
+//       accumulators; the predictor (Algorithms 1-3) runs on the remaining warps of the last CTA
 //                                                                          -> grid barrier
 //   D   down-projection tiles the same way                                 -> grid barrier
 // The stage ring, its barriers and the tensor-memory columns are set up once and carried through
@@ -30,8 +30,8 @@ struct TokenDenseArgs {
     int splits, seg;        // down projection: splits of the reduction dimension, columns per split
     int img_shared_base;    // image index of layer 0's first shared expert (= L * E)
     int dyn_bytes;          // dynamic shared memory of the launch
-    void *xb;               // [64][H] bf16 (bf16 weights) or f16 (fp8 weights)
-    void *actb;             // [pairs + 64][I], same type
+    void *xb;               // [64][H] bf16 (bf16 weights) or [3][64][H] e5m2 planes (fp8 weights)
+    void *actb;             // [pairs + 64][I] bf16 or [3][pairs + 64][I] e5m2 planes
     float *part;            // [pairs][splits][H]
     const uint8_t *store;   // fp8: first expert image (for the row scales) and the image pitch
     unsigned long long img_bytes;
@@ -39,8 +39,8 @@ struct TokenDenseArgs {
 
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// RDT: router weight type; WDT: expert weight type, 1 = bf16 (dense_group.cuh), 2 = fp8 e4m3
-// (dense8_group.cuh: warps 6-13 convert, the predictor gets warps 14-15).
+// RDT: router weight type; WDT: expert weight type, 1 = bf16, 2 = fp8 e4m3 (operand formats of
+// dense_group.cuh).
 template <int RDT, int WDT>
 __global__ void __launch_bounds__(kFfnThreads, 1)
 decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __grid_constant__ CUtensorMap map_up,
@@ -52,9 +52,8 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
     extern __shared__ __align__(16) int dyn[];  // work list | ids | prev ids | gate weights | stage ring
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
     __shared__ float s_inv[kMaxBatch];
-    using XT = typename std::conditional<WDT == 1, __nv_bfloat16, __half>::type;  // activation operand type
-    constexpr int kTmemCols = WDT == 1 ? kGroupTmemCols : 512;
-    __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2], afull[2], aempty[2];
+    constexpr int kTmemCols = kGroupTmemCols;
+    __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2];
     __shared__ uint32_t s_tmem;
     __shared__ int s_dead;
     const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
@@ -70,17 +69,14 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
     float *s_w = reinterpret_cast<float *>(s_prev + B * K);
     const int list_bytes = (int)sizeof(int) * (4 + 5 * pairs + 3 * B * K);
 
-    Group8Ring q;
-    GroupRing &r = q.r;
+    GroupRing r;
     r.dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dyn) + list_bytes + 1023) & ~(uintptr_t)1023);
     r.full = full, r.empty = empty, r.tfull = tfull, r.tempty = tempty, r.dead = &s_dead;
-    q.afull = afull, q.aempty = aempty;
-    r.slot = WDT == 1 ? max(group_stage_bytes<1>(np), group_stage_bytes<2>(np))
-                      : max(group8_stage_bytes<1>(np), group8_stage_bytes<2>(np));
+    r.slot = max(group_stage_bytes<1, WDT>(np), group_stage_bytes<2, WDT>(np));
     r.NS = min(kGroupMaxStages, (int)((reinterpret_cast<uint8_t *>(dyn) + d.dyn_bytes - r.dsm) / r.slot));
     if (threadIdx.x == 0) {
         s_dead = r.NS < 1;  // cannot happen with the host's sizing; never run a ring without stages
-        group8_ring_init(q);
+        group_ring_init(r);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dsmem_u32(&s_tmem)),
@@ -96,15 +92,14 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
     unsigned target = 0;
     const bool lead = blockIdx.x == 0;
     const bool pred_cta = blockIdx.x == gridDim.x - 1;
-    RingPos ppos, mpos;              // producer / MMA thread (bf16 weights)
-    Group8Pos ppos8, mpos8, cpos8;   // producer / MMA thread / converter warps (fp8 weights)
+    RingPos ppos, mpos;              // producer / MMA thread
     int issued = 0, mit = 0, eit = 0;  // loads issued (producer); tasks done (MMA thread, epilogue threads)
-    XT *xb = static_cast<XT *>(d.xb), *actb = static_cast<XT *>(d.actb);
-    auto to_xt = [](float v) {
+    const size_t x_plane = (size_t)kDenseMaxTokens * H;
+    auto store_x = [&](int i, float v) {  // the gate/up operand of element i of the hidden state
         if constexpr (WDT == 1)
-            return __float2bfloat16_rn(v);
+            static_cast<__nv_bfloat16 *>(d.xb)[i] = __float2bfloat16_rn(v);
         else
-            return __float2half_rn(v);
+            store_e5m2_planes(static_cast<uint8_t *>(d.xb), x_plane, (size_t)i, v);
     };
     const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gthreads = gridDim.x * blockDim.x;
 
@@ -122,14 +117,14 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
 
         // ---- F ---------------------------------------------------------------------------------
         if (l == 0) {
-            for (int i = gtid; i < B * H; i += gthreads) xb[i] = to_xt(h[i]);
+            for (int i = gtid; i < B * H; i += gthreads) store_x(i, h[i]);
         } else {
             const FfnArgs fp = finish_args(l - 1);
             float *hl = a.hbuf + (size_t)l * B * H;
             for (int i = gtid; i < B * H; i += gthreads) {
                 const float v = finish_value(fp, i / H, i % H, d.splits);
                 hl[i] = v;
-                xb[i] = to_xt(v);
+                store_x(i, v);
             }
         }
         fence_async_proxy();
@@ -158,72 +153,44 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
             for (int i = threadIdx.x; i < B * K; i += blockDim.x) a.ids_all[(size_t)l * a.Bmax * K + i] = s_ids[i];
 
         // ---- GU (+ the predictor on one warp of the last CTA) -----------------------------------
-        Group8Args g8{};
-        GroupArgs &g = g8.g;
+        GroupArgs g{};
         g.wl = wl, g.E = E, g.img_routed0 = l * E, g.img_shared0 = d.img_shared_base + l * a.n_shared;
         g.np = np, g.KS = KS, g.inv_rms = s_inv, g.part = d.part, g.err = a.err;
-        g8.store = d.store, g8.img_bytes = d.img_bytes;
+        g.store = d.store, g.img_bytes = d.img_bytes;
         if constexpr (WDT == 1)
-            g.act = actb;
+            g.act = static_cast<__nv_bfloat16 *>(d.actb);
         else
-            g8.act16 = actb;
-        constexpr int kGuStage = WDT == 1 ? group_kstage<2>() : group8_kstage<2>();
+            g.act8 = static_cast<uint8_t *>(d.actb), g.act_rows = pairs + kDenseMaxTokens;
+        constexpr int kGuStage = group_kstage<2, WDT>();
         g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kGuStage - 1) / kGuStage * kGuStage;
-        g8.scale_off = 0;
+        g.scale_off = 0, g.x_rows = kDenseMaxTokens;
         if (warp == 0) {
             if (lane == 0) {
                 fence_async_proxy();
-                if constexpr (WDT == 1)
-                    group_produce<2>(&map_gate, &map_up, &map_x, g, r, ppos, issued);
-                else
-                    group8_produce<2>(&map_gate, &map_up, &map_x, g, q, ppos8, issued);
+                group_produce<2, WDT>(&map_gate, &map_up, &map_x, g, r, ppos, issued);
             }
         } else if (warp == 1) {
-            if (lane == 0) {
-                if constexpr (WDT == 1)
-                    group_mma<2>(g, r, mpos, mit);
-                else
-                    group8_mma<2>(g, q, mpos8, mit);
-            }
+            if (lane == 0) group_mma<2, WDT>(g, r, mpos, mit);
         } else if (warp < 6) {
-            if constexpr (WDT == 1)
-                group_epilogue<2>(g, r, eit, warp % 4, lane);
-            else
-                group8_epilogue<2>(g8, q, eit, warp % 4, lane);
+            group_epilogue<2, WDT>(g, r, eit, warp % 4, lane);
             fence_async_proxy();  // the gated activations are fetched by TMA in the next phase
-        } else if (WDT == 2 && warp < 14) {
-            group8_convert<2>(g, q, cpos8, warp - 6, warp % 4, lane);
-        } else if (pred_cta) {  // the warps without a role in this phase: ten (bf16) or two (fp8)
-            constexpr int kFirst = WDT == 1 ? 6 : 14;
-            predictor_step_group(a, l, s_ids, s_prev, warp - kFirst, NW - kFirst, lane);
+        } else if (pred_cta) {  // the ten warps without a role in this phase
+            predictor_step_group(a, l, s_ids, s_prev, warp - 6, NW - 6, lane);
         }
         grid_barrier(a.barrier, a.err, target, &s_dead);
 
         // ---- D ---------------------------------------------------------------------------------
         g.rows = H, g.kd = I, g.splits = d.splits, g.seg = d.seg;
-        g8.scale_off = 2 * I;
+        g.scale_off = 2 * I, g.x_rows = pairs + kDenseMaxTokens;
         if (warp == 0) {
             if (lane == 0) {
                 fence_async_proxy();
-                if constexpr (WDT == 1)
-                    group_produce<1>(&map_down, &map_down, &map_act, g, r, ppos, issued);
-                else
-                    group8_produce<1>(&map_down, &map_down, &map_act, g, q, ppos8, issued);
+                group_produce<1, WDT>(&map_down, &map_down, &map_act, g, r, ppos, issued);
             }
         } else if (warp == 1) {
-            if (lane == 0) {
-                if constexpr (WDT == 1)
-                    group_mma<1>(g, r, mpos, mit);
-                else
-                    group8_mma<1>(g, q, mpos8, mit);
-            }
+            if (lane == 0) group_mma<1, WDT>(g, r, mpos, mit);
         } else if (warp < 6) {
-            if constexpr (WDT == 1)
-                group_epilogue<1>(g, r, eit, warp % 4, lane);
-            else
-                group8_epilogue<1>(g8, q, eit, warp % 4, lane);
-        } else if (WDT == 2 && warp < 14) {
-            group8_convert<1>(g, q, cpos8, warp - 6, warp % 4, lane);
+            group_epilogue<1, WDT>(g, r, eit, warp % 4, lane);
         }
         for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
         grid_barrier(a.barrier, a.err, target, &s_dead);
@@ -233,10 +200,7 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         const FfnArgs fl = finish_args(L - 1);
         for (int i = gtid; i < B * H; i += gthreads) a.h_out[i] = finish_value(fl, i / H, i % H, d.splits);
     }
-    if (warp == 0 && lane == 0) {
-        if (WDT == 2) ppos.s = ppos8.s, ppos.ph = ppos8.ph;
-        group_drain(r, ppos, issued);
-    }
+    if (warp == 0 && lane == 0) group_drain(r, ppos, issued);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (threadIdx.x == 0 && s_dead) *a.err = 1u;

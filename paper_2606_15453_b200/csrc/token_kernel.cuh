@@ -115,8 +115,10 @@ __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int lay
         if (layer > 0) {
             uint8_t *gid = st.cct_id + (size_t)(layer - 1) * E * K;
             uint8_t *gcf = st.cct_conf + (size_t)(layer - 1) * E * K;
+            uint32_t *co = st.live_counts ? st.Co + (size_t)(layer - 1) * E * E : nullptr;
             for (int b = 0; b < B; ++b)
-                update_rows_grouped(gid, gcf, K, prev + b * K, cur + b * K, lane, [&](int e) { return e % nw == wi; });
+                update_rows_grouped(gid, gcf, K, prev + b * K, cur + b * K, lane, [&](int e) { return e % nw == wi; },
+                                    co, E);
         }
     } else if (layer > 0) {
         uint32_t *Co = st.Co + (size_t)(layer - 1) * E * E;
@@ -178,7 +180,7 @@ __device__ __forceinline__ void predictor_step_group(const TokenArgs &a, int lay
         for (int w = 0; w < kMaxExperts / kWarp; ++w) {
             const int f = w * kWarp + lane;
             const int score = (int)(((w < 4 ? lo : hi) >> ((w & 3) * 8)) & 0xffu);
-            const bool in = f < E && score >= kThreshold;
+            const bool in = f < E && score >= st.threshold;
             const unsigned msk = __ballot_sync(kFull, in);
             if (lane == 0) st.pred_mask[b * 8 + w] = msk;
             if (in) {

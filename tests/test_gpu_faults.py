@@ -133,6 +133,8 @@ def test_cache_policy_setter_matches_the_oracle_model_and_throttle_slows_the_lin
     for name, policy, throttle in (("lru", (0, False, -1), None), ("counts", (8, True, 0), None),
                                    ("throttled", (0, False, -1), (4096, 50))):
         pr = Pair(cfg, Bt, oracle=False, prefetch_limit=2)
+        with pytest.raises(P.StmoeError):
+            pr.stack.set_cache_policy(0, False, 0)     # a floor is a test on use counts: it needs a window
         pr.stack.set_cache_policy(*policy)
         if throttle:
             pr.stack.set_copy_throttle(*throttle)

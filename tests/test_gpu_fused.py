@@ -77,3 +77,36 @@ def test_shapes_outside_the_fused_kernel_use_the_three_phase_kernel():
                                       n_shared=1, dtype="bf16")    # 272 columns: not a whole number of warps per row
     st = decode_tokens_vs_oracle(cfg, 1, 3, min_checked=2)
     assert st["kernel_launches"] <= 3 + 1
+
+
+@pytest.mark.parametrize("flags,B,threshold,live", [(0, 1, 3, False), (P.FLAG_NO_FUSED, 1, 3, False), (0, 1, 2, True),
+                                                    (P.FLAG_NO_FUSED, 1, 2, True), (0, 4, 1, True),
+                                                    (P.FLAG_NO_DENSE, 3, 2, True)])
+def test_in_kernel_predictors_honour_threshold_and_replacement_rule(flags, B, threshold, live):
+    """The persistent kernels run Algorithms 2 and 3 inside the kernel (single-sequence row-triple
+    kernel, three-phase kernel, tensor-core kernel for batches): with another set threshold, or with
+    replacement by live counts, their predictions and tables equal the oracle predictor's,
+    replayed on the GPU's routing."""
+    import oracle as O
+    cfg = stacks.CONFIGS["C2"].scaled(n_layers=4, profile_tokens=3, cache_slots=0, **SHAPES[1])
+    pr = Pair(cfg, B, oracle=False, flags=flags)
+    pr.stack.set_predict_threshold(threshold)
+    pr.stack.set_replacement_rule(live)
+    L, K, T = cfg.n_layers, cfg.top_k, 24
+    ids = torch.empty(L, B, K, dtype=torch.int32, device=DEV)
+    pred = torch.empty(L, B, pr.stack.max_pred, dtype=torch.int32, device=DEV)
+    npred = torch.empty(L, B, dtype=torch.int32, device=DEV)
+    ho = torch.empty(B, cfg.hidden, device=DEV)
+    x = stacks.token_inputs(cfg, B, T).to(DEV)
+    replay = O.Predictor(L, cfg.n_experts, K, B, cfg.profile_tokens, "st", threshold=threshold, live_counts=live)
+    for t in range(T):
+        pr.stack.decode_token(x[t].clone(), ho, ids, None, pred, npred)
+        torch.cuda.synchronize()
+        for l in range(L):
+            rp = replay.step(l, ids[l].cpu().numpy())
+            assert npred[l].cpu().tolist() == rp["n_pred"].tolist(), (t, l)
+            assert (pred[l].cpu().numpy() == rp["pred_ids"]).all(), (t, l)
+    assert pr.stack.export_state() == replay.export()
+    if live:
+        assert int(O.parse_state(replay.export())["Co"].sum()) == T * B * K * K * (L - 1)
+    pr.close()

@@ -12,10 +12,14 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def _replay(L, E, K, B, P_tok, mode, trace, check_every=7):
+def _replay(L, E, K, B, P_tok, mode, trace, check_every=7, threshold=2, live_counts=False):
     """trace: int32 [T][L][B][K].  Runs both sides step by step."""
     st = P.Stack(L, E, K, 64, 64, max_batch=B, dtype="f32", profile_tokens=P_tok, mode=mode)
-    orc = O.Predictor(L, E, K, B, P_tok, mode)
+    if threshold != 2:
+        st.set_predict_threshold(threshold)
+    if live_counts:
+        st.set_replacement_rule(True)
+    orc = O.Predictor(L, E, K, B, P_tok, mode, threshold=threshold, live_counts=live_counts)
     pred = torch.empty(B, st.max_pred, dtype=torch.int32, device=DEV)
     npred = torch.empty(B, dtype=torch.int32, device=DEV)
     tr = torch.from_numpy(trace).to(DEV)
@@ -46,6 +50,37 @@ def test_predictor_replay_random_traces(E, K, B, L, mode):
     T, P_tok = 36, 9
     trace = stacks.random_topk_trace(E, K, T, L, B, stream=E * 7 + K).numpy()
     _replay(L, E, K, B, P_tok, mode, trace)
+
+
+@pytest.mark.parametrize("threshold", [1, 3, 5])
+def test_predictor_replay_with_another_set_threshold(threshold):
+    """The threshold sweep of the ablation: Algorithm 2's set at a threshold other than binary 10,
+    stand-alone predictor kernel, bit-exact against the oracle."""
+    E, K, B, L = 64, 6, 4, 3
+    trace = stacks.random_topk_trace(E, K, 30, L, B, stream=77).numpy()
+    so = _replay(L, E, K, B, 8, "st", trace, check_every=3, threshold=threshold)
+    assert so["predicted"] > 0
+
+
+@pytest.mark.parametrize("E,K,B,L", [(8, 2, 1, 4), (60, 4, 3, 3), (64, 6, 8, 3), (128, 8, 16, 3), (256, 8, 4, 2),
+                                     (12, 12, 2, 2), (40, 1, 5, 2), (32, 16, 3, 2)])
+def test_predictor_replay_with_live_count_replacement(E, K, B, L):
+    """Algorithm 3 with the new candidate taken by the largest live co-activation count: counts
+    (they keep growing at run time), tables and predictions bit-exact against the oracle.  Skewed
+    traces, so that counts differ and confidences reach zero."""
+    T = 40
+    base = stacks.random_topk_trace(E, K, T, L, B, stream=E + 3 * K).numpy()
+    hot = stacks.random_topk_trace(min(E, max(K + 2, E // 4)), K, T, L, B, stream=9).numpy()
+    trace = np.where((np.arange(T) % 3 != 2)[:, None, None, None], hot, base).astype(np.int32)
+    assert trace.max() < E
+    _replay(L, E, K, B, 6, "st", trace, check_every=2, live_counts=True)
+    # the rule is live: the default rule ends with other tables on the same trace (K > 1)
+    if 1 < K < E:
+        a = O.Predictor(L, E, K, B, 6, "st"); b = O.Predictor(L, E, K, B, 6, "st", live_counts=True)
+        for t in range(T):
+            for l in range(L):
+                a.step(l, trace[t, l]), b.step(l, trace[t, l])
+        assert (a.tables()["cct_id"] != b.tables()["cct_id"]).any()
 
 
 def test_predictor_replay_correlated_trace_and_recall():
