@@ -191,10 +191,9 @@ def top_kernel_name(cfg, batch, args):
     """The kernel that dominates a decode step of this workload (one launch per step for resident stacks)."""
     if cfg.cache_slots:
         return "gate_up_kernel"
-    dense = not args.no_dense and ((cfg.dtype == "bf16" and batch >= (args.dense_min_batch or 2)) or
-                                   (cfg.dtype == "fp8" and batch >= (args.dense_min_batch or 3)))
+    dense = not args.no_dense and cfg.dtype in ("bf16", "fp8") and batch >= (args.dense_min_batch or 2)
     if dense:
-        return "dense8_group_kernel<2>" if cfg.dtype == "fp8" and batch > 4 else "decode_token_dense_kernel"
+        return "dense_group_kernel (gate/up)" if args.no_persistent else "decode_token_dense_kernel"
     epl = {"f32": 4, "bf16": 8, "fp8": 16}[cfg.dtype]
     fused = batch == 1 and not args.no_fused and cfg.hidden % epl == 0 and cfg.hidden <= 4096 and \
         cfg.hidden // epl in (64, 128, 256, 512)
@@ -263,12 +262,8 @@ def measure(cfg, batch, st, args, dev, world, stream, with_e2e):
         ids_host = torch.empty(L, batch, K, dtype=torch.int32).pin_memory()
         barrier()
         w0 = time.perf_counter()
-        for i in range(steps):
-            h_in.copy_(x_host[t + i], non_blocking=True)
-            st.decode_token(h_in, h_out, ids, None, pred, npred)
-            out_host.copy_(h_out, non_blocking=True)
-            ids_host.copy_(ids, non_blocking=True)
-            torch.cuda.synchronize()
+        for i in range(steps):      # one library call per step: pinned input in, output and routing back
+            st.decode_token_host(x_host[t + i], out_host, ids_host)
         e2e_ms = (time.perf_counter() - w0) * 1e3
         barrier()
     times = torch.tensor([ms, e2e_ms or 0.0], dtype=torch.float64, device=dev)
@@ -314,7 +309,8 @@ def summarise(cfg, batch, m, args, world, peak):
 
 def make_stack(cfg, batch, dev, args):
     import paper_2606_15453_b200 as P
-    flags = (P.FLAG_NO_DENSE if args.no_dense else 0) | (P.FLAG_NO_FUSED if args.no_fused else 0)
+    flags = ((P.FLAG_NO_DENSE if args.no_dense else 0) | (P.FLAG_NO_FUSED if args.no_fused else 0) |
+             (P.FLAG_NO_PERSISTENT if args.no_persistent else 0))
     st = load_stack(cfg, batch, dev, prefetch_limit=args.prefetch_limit, mode=args.mode, flags=flags)
     if args.prefetch_min_score:
         st.set_prefetch_min_score(args.prefetch_min_score)
@@ -379,6 +375,8 @@ def main():
                          "ahead of the router (-1: the library's default)")
     ap.add_argument("--no-dense", action="store_true",
                     help="batched steps of resident bf16 stacks on the CUDA-core kernels instead of the tcgen05 ones")
+    ap.add_argument("--no-persistent", action="store_true",
+                    help="resident stacks: per-layer kernels (replayed as a CUDA graph) instead of one persistent kernel per step")
     ap.add_argument("--no-fused", action="store_true",
                     help="single-sequence resident steps on the three-phase kernel instead of the one-phase one")
     args = ap.parse_args()
@@ -422,7 +420,7 @@ def main():
     peak, peak_kind = measured_peaks()
     head = summarise(cfg, batch, m, args, world, peak)
     tokens = args.steps * batch * world
-    persistent = cfg.cache_slots == 0          # resident stacks: one kernel launch per decode step
+    persistent = cfg.cache_slots == 0 and not args.no_persistent   # resident stacks: one kernel launch per decode step
     whole_step = head["kernel"].startswith("decode_token")
     traffic, traffic_src = (None, None)
     if whole_step and batch == 1 and args.workload == "C1" and not args.no_fused:

@@ -171,6 +171,14 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out,
                        int32_t *routed_ids, float *routed_w, int32_t *predicted_ids,
                        int32_t *n_predicted, uint32_t *flags, void *cuda_stream);
 
+/* stmoe_decode_token for callers whose buffers are in HOST memory (pinned for the copies to run
+ * at link speed; pageable works): copies h_in_host [batch][H] to the device, runs the decode step,
+ * copies h_out_host [batch][H] and, if not NULL, routed_ids_host [n_layers][batch][K] back, and
+ * waits for cuda_stream.  The device staging buffers belong to the stack (allocated at the first
+ * call).  Errors as stmoe_decode_token; a failed copy or wait returns STMOE_ERR_CUDA. */
+int stmoe_decode_token_host(stmoe_t *s, int batch, const float *h_in_host, float *h_out_host,
+                            int32_t *routed_ids_host, void *cuda_stream);
+
 int stmoe_max_predicted(const stmoe_t *s); /* min(E, K*K+K) */
 
 /* on != 0: bracket the expert-FFN kernels of every following layer step with CUDA events

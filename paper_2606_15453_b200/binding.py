@@ -64,6 +64,7 @@ def lib():
         L.stmoe_load_experts.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, i32]
         L.stmoe_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.stmoe_decode_token.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.stmoe_decode_token_host.argtypes = [vp, i32, vp, vp, vp, vp]
         L.stmoe_max_predicted.argtypes = [vp]
         L.stmoe_set_kernel_timing.argtypes = [vp, i32]
         L.stmoe_set_dense_min_batch.argtypes = [vp, i32]
@@ -175,6 +176,14 @@ class Stack:
                                         _dev(h_out, torch.float32), _ptr(routed_ids), _ptr(routed_w),
                                         _ptr(predicted_ids), _ptr(n_predicted), _ptr(flags),
                                         _stream(stream)), "stmoe_decode_token")
+
+    def decode_token_host(self, h_in, h_out, routed_ids=None, stream=None) -> None:
+        """h_in / h_out / routed_ids: CPU tensors (pinned for full copy speed); returns when done."""
+        assert not h_in.is_cuda and not h_out.is_cuda and h_in.is_contiguous() and h_out.is_contiguous()
+        assert h_in.dtype == torch.float32 and h_out.dtype == torch.float32
+        assert routed_ids is None or (not routed_ids.is_cuda and routed_ids.dtype == torch.int32)
+        _check(lib().stmoe_decode_token_host(self._h, h_in.shape[0], h_in.data_ptr(), h_out.data_ptr(),
+                                             _ptr(routed_ids), _stream(stream)), "stmoe_decode_token_host")
 
     def predictor_step(self, layer, routed_ids, predicted_ids=None, n_predicted=None,
                        stream=None) -> None:

@@ -25,8 +25,12 @@
 //      e5m2 planes whose sum is the activation (kind::f8f6f4, 128 reduction columns per box row).
 //      e5m2 has the exponent range of f16, so no scaling pass is needed; each plane takes the
 //      rounding residue of the one before (2 mantissa bits each: relative error 2^-9 after three,
-//      the precision of a bf16 operand).  The three planes multiply the same weight tile into the
-//      same accumulator: three times the MMAs, which are free next to the weight stream.  The
+//      the precision of a bf16 operand).  The planes' tiles lie one after the other in shared
+//      memory and form ONE B operand of 3 x np rows: one MMA per weight tile and reduction slice
+//      (an MMA's cost here is reading its 128 x 32-byte A tile from shared memory: one MMA per
+//      plane into shared columns measured slower than widening the weights), three accumulator
+//      columns per token that the epilogue adds.  Gate and up accumulators of more than 32 tokens
+//      fit tensor memory only once, so those tasks run with a single accumulator buffer.  The
 //      per-output-channel weight scales belong to the accumulator lanes and are applied in the
 //      epilogue.
 #pragma once
@@ -41,6 +45,25 @@ constexpr int kGroupThreads = 192;
 constexpr int kGroupTileBytes = kDenseRows * kDenseKStep * 2;     // 16 KB weight tile of a stage
 constexpr int kGroupActBytes = kDenseMaxTokens * kDenseKStep * 2; // 8 KB activation tile (64 tokens)
 constexpr int kGroupTmemCols = 256;                               // two accumulator buffers of 128 columns
+constexpr int kGroup8TmemCols = 512;                              // fp8 format: two buffers of 192 columns (power of two)
+// Accumulator layout in tensor memory.  bf16: two buffers of 128 columns, gate at +0 and up at +64.
+// fp8 (three columns per token, np apart): buffers 192 columns apart; gate/up of up to 32 tokens at
+// +0 / +96 in each of two buffers, of more tokens at +0 / +192 in a single buffer.
+__host__ __device__ constexpr int group_acc_bufs(int nmat, int wdt, int np) { return wdt == 2 && nmat == 2 && np > 32 ? 1 : 2; }
+__host__ __device__ constexpr int group_acc_stride(int wdt) { return wdt == 2 ? 192 : 128; }
+__host__ __device__ constexpr int group_mat_stride(int wdt, int np) { return wdt == 1 ? 64 : (np > 32 ? 192 : 96); }
+// which accumulator buffer the next task takes and how often each was used (its barriers' phase);
+// the MMA thread and the epilogue threads each keep one and walk the same task sequence
+struct AccPos {
+    int use[2] = {0, 0};
+    int next = 0;
+    __device__ __forceinline__ int take(int bufs)
+    {
+        const int ab = bufs == 1 ? 0 : next;
+        if (bufs == 2) next ^= 1;
+        return ab;
+    }
+};
 
 #ifndef STMOE_GROUP_KBOXES_GU
 #define STMOE_GROUP_KBOXES_GU 2
@@ -198,9 +221,20 @@ struct GroupRing {
     uint32_t tmem;                          // base of the 256 accumulator columns
     volatile int *dead;
 };
+// A role's place in the ring: the stage it handles next and, per stage, the parity of the barrier
+// phase it waits for next (bit s toggles each time the role has used stage s).  Per-stage bits,
+// not one wrap-around bit, so that a caller may restart at stage 0 with another stage count at a
+// moment when every stage is empty (the persistent kernel does between its phases) without
+// touching the barriers.
 struct RingPos {
     int s = 0;
-    uint32_t ph = 0;
+    uint32_t par = 0;
+    __device__ __forceinline__ uint32_t parity() const { return (par >> s) & 1u; }
+    __device__ __forceinline__ void advance(int NS)
+    {
+        par ^= 1u << s;
+        if (++s == NS) s = 0;
+    }
 };
 
 __device__ __forceinline__ void group_ring_init(const GroupRing &r)
@@ -228,7 +262,7 @@ __device__ __forceinline__ void group_produce(const CUtensorMap *map_w0, const C
         const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
         const int xrow = NMAT == 2 ? 0 : a.wl.g_start[t.g];
         for (int k = t.k0; k < t.k1; k += KSTAGE) {
-            if (!dmbar_wait(&r.empty[pos.s], pos.ph ^ 1u, r.dead)) return;
+            if (!dmbar_wait(&r.empty[pos.s], pos.parity() ^ 1u, r.dead)) return;
             uint8_t *st = r.dsm + (size_t)pos.s * r.slot;
             // boxes past the end of the reduction dimension are zero-filled and still count
             dmbar_expect_tx(&r.full[pos.s], (uint32_t)(KB * (NMAT * kGroupTileBytes + PLANES * np * 128)));
@@ -243,7 +277,7 @@ __device__ __forceinline__ void group_produce(const CUtensorMap *map_w0, const C
                                 &r.full[pos.s]);
             }
             ++issued;
-            if (++pos.s == r.NS) pos.s = 0, pos.ph ^= 1u;
+            pos.advance(r.NS);
         }
     }
 }
@@ -251,71 +285,72 @@ __device__ __forceinline__ void group_produce(const CUtensorMap *map_w0, const C
 // Every load that was issued has to land before the CTA may exit.
 __device__ __forceinline__ void group_drain(const GroupRing &r, RingPos pos, int issued)
 {
-    for (int i = 0; i < min(issued, r.NS); ++i) {
-        if (pos.s == 0) pos.s = r.NS, pos.ph ^= 1u;
+    for (int i = 0; i < min(issued, r.NS); ++i) {  // the last loads, newest first: one per stage at most
+        if (pos.s == 0) pos.s = r.NS;
         --pos.s;
-        dmbar_wait(&r.full[pos.s], pos.ph, r.dead);
+        dmbar_wait(&r.full[pos.s], pos.parity() ^ 1u, r.dead);  // the phase before the producer's last toggle
     }
 }
 
-// One thread: issue the MMAs of this CTA's tasks.  `it` counts the CTA's tasks across calls
-// (accumulator buffer = it & 1).
+// One thread: issue the MMAs of this CTA's tasks.  `ap` carries the accumulator hand-off state
+// across calls.
 template <int NMAT, int WDT>
-__device__ __forceinline__ void group_mma(const GroupArgs &a, const GroupRing &r, RingPos &pos, int &it)
+__device__ __forceinline__ void group_mma(const GroupArgs &a, const GroupRing &r, RingPos &pos, AccPos &ap)
 {
-    constexpr int KB = group_kboxes<NMAT, WDT>(), KSTAGE = group_kstage<NMAT, WDT>(), PLANES = group_planes<WDT>();
-    const int np = a.np, act_bytes = group_act_bytes(np), box = group_box_bytes<NMAT, WDT>(np);
-    const uint32_t idesc = WDT == 1 ? umma_idesc_bf16(np) : umma_idesc_e4m3_e5m2(np);
+    constexpr int KB = group_kboxes<NMAT, WDT>(), KSTAGE = group_kstage<NMAT, WDT>();
+    const int np = a.np, box = group_box_bytes<NMAT, WDT>(np);
+    const uint32_t idesc = WDT == 1 ? umma_idesc_bf16(np) : umma_idesc_e4m3_e5m2(3 * np);
+    const int mat_stride = group_mat_stride(WDT, np), bufs = group_acc_bufs(NMAT, WDT, np);
     const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
     const int n_tasks = *a.wl.n_groups * tiles * a.splits;
-    for (int task = blockIdx.x; task < n_tasks && !*r.dead; task += gridDim.x, ++it) {
+    for (int task = blockIdx.x; task < n_tasks && !*r.dead; task += gridDim.x) {
         const GroupTask t = group_task(a, task);
-        const int ab = it & 1;
-        if (!dmbar_wait(&r.tempty[ab], (((uint32_t)it >> 1) & 1u) ^ 1u, r.dead)) return;
+        const int ab = ap.take(bufs);
+        if (!dmbar_wait(&r.tempty[ab], ((uint32_t)ap.use[ab] & 1u) ^ 1u, r.dead)) return;
+        ap.use[ab] += 1;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t acc = r.tmem + ab * 128;
+        const uint32_t acc = r.tmem + ab * group_acc_stride(WDT);
         bool first = true;
         for (int k = t.k0; k < t.k1; k += KSTAGE) {
-            if (!dmbar_wait(&r.full[pos.s], pos.ph, r.dead)) return;
+            if (!dmbar_wait(&r.full[pos.s], pos.parity(), r.dead)) return;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
                 const uint32_t st = dsmem_u32(r.dsm + (size_t)pos.s * r.slot) + kb * box;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {  // four 32-byte slices of the 128-byte box row
+                    // fp8: the planes' tiles follow one another and are the rows np.. of one operand
+                    const uint64_t bd = umma_desc_sw128(st + NMAT * kGroupTileBytes, j);
 #pragma unroll
-                    for (int p = 0; p < PLANES; ++p) {
-                        const uint64_t bd = umma_desc_sw128(st + NMAT * kGroupTileBytes + p * act_bytes, j);
-#pragma unroll
-                        for (int mat = 0; mat < NMAT; ++mat) {
-                            const uint64_t ad = umma_desc_sw128(st + mat * kGroupTileBytes, j);
-                            const bool accumulate = !first || kb > 0 || j > 0 || p > 0;
-                            if constexpr (WDT == 1)
-                                umma_bf16(acc + mat * 64, ad, bd, idesc, accumulate);
-                            else
-                                umma_f8(acc + mat * 64, ad, bd, idesc, accumulate);
-                        }
+                    for (int mat = 0; mat < NMAT; ++mat) {
+                        const uint64_t ad = umma_desc_sw128(st + mat * kGroupTileBytes, j);
+                        const bool accumulate = !first || kb > 0 || j > 0;
+                        if constexpr (WDT == 1)
+                            umma_bf16(acc + mat * mat_stride, ad, bd, idesc, accumulate);
+                        else
+                            umma_f8(acc + mat * mat_stride, ad, bd, idesc, accumulate);
                     }
                 }
             }
             first = false;
             umma_commit(&r.empty[pos.s]);
-            if (++pos.s == r.NS) pos.s = 0, pos.ph ^= 1u;
+            pos.advance(r.NS);
         }
         umma_commit(&r.tfull[ab]);
     }
 }
 
 // Four warps (lg = the TMEM lane quarter the warp may read = warp index % 4): thread = one
-// weight row.  `it` as in group_mma.
+// weight row.  `ap` as in group_mma.
 template <int NMAT, int WDT>
-__device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRing &r, int &it, int lg, int lane)
+__device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRing &r, AccPos &ap, int lg, int lane)
 {
     const int tiles = (a.rows + kDenseRows - 1) / kDenseRows;
     const int n_tasks = *a.wl.n_groups * tiles * a.splits;
-    for (int task = blockIdx.x; task < n_tasks; task += gridDim.x, ++it) {
+    const int bufs = group_acc_bufs(NMAT, WDT, a.np);
+    for (int task = blockIdx.x; task < n_tasks; task += gridDim.x) {
         const GroupTask t = group_task(a, task);
-        const int ab = it & 1;
+        const int ab = ap.take(bufs);
         const int start = a.wl.g_start[t.g], count = a.wl.g_count[t.g];
         const int row = t.row0 + lg * kWarp + lane;
         float s0 = 1.f, s1 = 1.f;
@@ -329,14 +364,22 @@ __device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRi
             s0 = bf16_to_f32(sc[srow]);
             if (NMAT == 2) s1 = bf16_to_f32(sc[a.rows + srow]);
         }
-        const bool ok = dmbar_wait(&r.tfull[ab], ((uint32_t)it >> 1) & 1u, r.dead);
+        const bool ok = dmbar_wait(&r.tfull[ab], (uint32_t)ap.use[ab] & 1u, r.dead);
+        ap.use[ab] += 1;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t acc = r.tmem + ab * 128 + ((uint32_t)(lg * kWarp) << 16);
+        const uint32_t acc = r.tmem + ab * group_acc_stride(WDT) + ((uint32_t)(lg * kWarp) << 16);
+        constexpr bool stacked = WDT == 2;  // three columns per token, np apart: add them
+        const int mat_stride = group_mat_stride(WDT, a.np);
         if (NMAT == 2) {
             for (int i = 0; i < count; ++i) {
                 const int tok = a.wl.pair_token[start + i];
                 const float inv = a.inv_rms[tok];  // W (inv * h) = inv * (W h)
-                const float g = inv * s0 * tmem_ld1(acc + tok), u = inv * s1 * tmem_ld1(acc + 64 + tok);
+                float ga = tmem_ld1(acc + tok), ua = tmem_ld1(acc + mat_stride + tok);
+                if (stacked) {
+                    ga = (ga + tmem_ld1(acc + a.np + tok)) + tmem_ld1(acc + 2 * a.np + tok);
+                    ua = (ua + tmem_ld1(acc + mat_stride + a.np + tok)) + tmem_ld1(acc + mat_stride + 2 * a.np + tok);
+                }
+                const float g = inv * s0 * ga, u = inv * s1 * ua;
                 const float v = g / (1.f + expf(-g)) * u;
                 if (ok && row < a.rows) {
                     if constexpr (WDT == 1) {
@@ -353,6 +396,13 @@ __device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRi
             for (int i0 = 0; i0 < count; i0 += 8) {
                 float y[8];
                 tmem_ld8(acc + i0, y);
+                if (stacked) {
+                    float y1[8], y2[8];
+                    tmem_ld8(acc + a.np + i0, y1);
+                    tmem_ld8(acc + 2 * a.np + i0, y2);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) y[i] = (y[i] + y1[i]) + y2[i];
+                }
                 if (ok && row < a.rows) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
@@ -376,6 +426,7 @@ __global__ void __launch_bounds__(kGroupThreads, 1)
 dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_constant__ CUtensorMap map_w1,
                    const __grid_constant__ CUtensorMap map_x, GroupArgs a)
 {
+    constexpr int kTmemCols = WDT == 1 ? kGroupTmemCols : kGroup8TmemCols;
     extern __shared__ uint8_t dsm_raw[];
     __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2];
     __shared__ uint32_t s_tmem;
@@ -391,7 +442,7 @@ dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_cons
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dsmem_u32(&s_tmem)),
-                     "r"(kGroupTmemCols)
+                     "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -410,17 +461,17 @@ dense_group_kernel(const __grid_constant__ CUtensorMap map_w0, const __grid_cons
     } else if (warp == 1) {
         if (lane == 0) {
             RingPos pos;
-            int it = 0;
-            group_mma<NMAT, WDT>(a, r, pos, it);
+            AccPos ap;
+            group_mma<NMAT, WDT>(a, r, pos, ap);
         }
     } else {
-        int it = 0;
-        group_epilogue<NMAT, WDT>(a, r, it, warp % 4, lane);
+        AccPos ap;
+        group_epilogue<NMAT, WDT>(a, r, ap, warp % 4, lane);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(r.tmem), "r"(kGroupTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(r.tmem), "r"(kTmemCols) : "memory");
     }
     if (tid == 0 && s_dead) *a.err = 1u;
 }

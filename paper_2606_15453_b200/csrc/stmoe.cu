@@ -395,6 +395,8 @@ struct stmoe {
     bool dense8 = false;            // fp8 stacks: e4m3 weight tiles x three e5m2 activation planes
     CUtensorMap map8_gate{}, map8_up{}, map8_down{}, map8_x[4]{}, map8_act[4]{};
     uint8_t *d_x8 = nullptr, *d_act8 = nullptr;  // [3][64][H], [3][pairs + 64][I]
+    float *d_host_io = nullptr;     // stmoe_decode_token_host: [2][max_batch][H] staging of h_in / h_out
+    int32_t *d_host_ids = nullptr;  // and [L][max_batch][K] of the routed ids
     bool dense_persistent = false;  // one cooperative kernel per decode step (token_dense_kernel.cuh)
     int dense_dyn_bytes = 0;
 
@@ -1214,7 +1216,7 @@ int stmoe_destroy(stmoe_t *s)
                    s->pst.Co, s->pst.cct_id, s->pst.cct_conf, s->pst.HT, s->pst.t, s->pst.pred_mask,
                    s->pst.pred_valid, s->pst.stats, s->d_rpart, s->d_sspart, s->d_arrivals, s->d_tile_done, s->d_hbuf, s->d_rpart_all, s->d_sspart_all,
                    s->d_act_all, s->d_part_all, s->d_tiles_all, s->d_barrier, s->d_err, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
-                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense, s->d_x8, s->d_act8,
+                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense, s->d_x8, s->d_act8, s->d_host_io, s->d_host_ids,
                    s->d_down_t, s->d_zpart, s->d_acc};
     if (s->d_shared && s->d_resident && s->d_shared > s->d_resident) dev[2] = nullptr;  // one allocation
     for (void *p : dev)
@@ -1638,6 +1640,30 @@ int stmoe_decode_token(stmoe_t *s, int batch, const float *h_in, float *h_out, i
     s->graph_launches = s->launches - before;
     s->graph_captures += 1;
     CU_TRY(cudaGraphLaunch(s->graph_exec, st));
+    return STMOE_OK;
+}
+
+int stmoe_decode_token_host(stmoe_t *s, int batch, const float *h_in_host, float *h_out_host,
+                            int32_t *routed_ids_host, void *cuda_stream)
+{
+    if (!s || !h_in_host || !h_out_host || batch < 1 || batch > s->cfg.max_batch) return STMOE_ERR_BAD_ARG;
+    const stmoe_config_t &c = s->cfg;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t hb = sizeof(float) * (size_t)batch * c.hidden, plane = (size_t)c.max_batch * c.hidden;
+    if (!s->d_host_io) {
+        CU_TRY(cudaMalloc(&s->d_host_io, sizeof(float) * 2 * plane));
+        CU_TRY(cudaMalloc(&s->d_host_ids, sizeof(int32_t) * (size_t)c.n_layers * c.max_batch * c.top_k));
+    }
+    float *d_in = s->d_host_io, *d_out = s->d_host_io + plane;
+    CU_TRY(cudaMemcpyAsync(d_in, h_in_host, hb, cudaMemcpyHostToDevice, st));
+    const int rc = stmoe_decode_token(s, batch, d_in, d_out, routed_ids_host ? s->d_host_ids : nullptr, nullptr, nullptr,
+                                      nullptr, nullptr, cuda_stream);
+    if (rc != STMOE_OK) return rc;
+    CU_TRY(cudaMemcpyAsync(h_out_host, d_out, hb, cudaMemcpyDeviceToHost, st));
+    if (routed_ids_host)
+        CU_TRY(cudaMemcpyAsync(routed_ids_host, s->d_host_ids, sizeof(int32_t) * (size_t)c.n_layers * batch * c.top_k,
+                               cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
     return STMOE_OK;
 }
 

@@ -12,8 +12,9 @@
 //       accumulators; the predictor (Algorithms 1-3) runs on the remaining warps of the last CTA
 //                                                                          -> grid barrier
 //   D   down-projection tiles the same way                                 -> grid barrier
-// The stage ring, its barriers and the tensor-memory columns are set up once and carried through
-// all phases and layers.  Data written with ordinary stores and then fetched by TMA from another
+// The tensor-memory columns and the accumulator hand-off barriers are set up once and carried
+// through all phases and layers; the stage ring is laid out anew for every GU and D phase (its
+// stage size differs between the two, and every stage is empty at a phase boundary).  Data written with ordinary stores and then fetched by TMA from another
 // SM (the bf16 hidden state, the gated activations) is fenced for the async proxy on both sides
 // of the grid barrier in between.
 #pragma once
@@ -52,7 +53,7 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
     extern __shared__ __align__(16) int dyn[];  // work list | ids | prev ids | gate weights | stage ring
     __shared__ int s_scan[2 * (kMaxExperts + 1)];
     __shared__ float s_inv[kMaxBatch];
-    constexpr int kTmemCols = kGroupTmemCols;
+    constexpr int kTmemCols = WDT == 1 ? kGroupTmemCols : kGroup8TmemCols;
     __shared__ uint64_t full[kGroupMaxStages], empty[kGroupMaxStages], tfull[2], tempty[2];
     __shared__ uint32_t s_tmem;
     __shared__ int s_dead;
@@ -72,11 +73,19 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
     GroupRing r;
     r.dsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(dyn) + list_bytes + 1023) & ~(uintptr_t)1023);
     r.full = full, r.empty = empty, r.tfull = tfull, r.tempty = tempty, r.dead = &s_dead;
-    r.slot = max(group_stage_bytes<1, WDT>(np), group_stage_bytes<2, WDT>(np));
-    r.NS = min(kGroupMaxStages, (int)((reinterpret_cast<uint8_t *>(dyn) + d.dyn_bytes - r.dsm) / r.slot));
+    const int ring_bytes = (int)(reinterpret_cast<uint8_t *>(dyn) + d.dyn_bytes - r.dsm);
+    // the ring of one phase: as many stages of that projection's size as fit (the host checked that
+    // one of the larger kind fits)
+    auto ring_for = [&](int stage_bytes) {
+        r.slot = stage_bytes;
+        r.NS = min(kGroupMaxStages, ring_bytes / stage_bytes);
+    };
+    ring_for(max(group_stage_bytes<1, WDT>(np), group_stage_bytes<2, WDT>(np)));
     if (threadIdx.x == 0) {
         s_dead = r.NS < 1;  // cannot happen with the host's sizing; never run a ring without stages
-        group_ring_init(r);
+        GroupRing all = r;
+        all.NS = kGroupMaxStages;  // the barriers of every stage any phase's layout can have
+        group_ring_init(all);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dsmem_u32(&s_tmem)),
@@ -93,7 +102,15 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
     const bool lead = blockIdx.x == 0;
     const bool pred_cta = blockIdx.x == gridDim.x - 1;
     RingPos ppos, mpos;              // producer / MMA thread
-    int issued = 0, mit = 0, eit = 0;  // loads issued (producer); tasks done (MMA thread, epilogue threads)
+    AccPos macc, eacc;               // accumulator hand-off state of the MMA thread / the epilogue threads
+    int issued = 0;                  // loads issued in the current phase (producer)
+    // Start of a GU or D phase: every stage of the ring is empty (the MMA thread consumed every
+    // load), so the ring is laid out for this phase's stage size and both roles restart at stage 0;
+    // the barriers keep their state, the roles their per-stage parities.
+    auto ring_restart = [&](int stage_bytes) {
+        ring_for(stage_bytes);
+        ppos.s = 0, mpos.s = 0, issued = 0;
+    };
     const size_t x_plane = (size_t)kDenseMaxTokens * H;
     auto store_x = [&](int i, float v) {  // the gate/up operand of element i of the hidden state
         if constexpr (WDT == 1)
@@ -164,15 +181,16 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         constexpr int kGuStage = group_kstage<2, WDT>();
         g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kGuStage - 1) / kGuStage * kGuStage;
         g.scale_off = 0, g.x_rows = kDenseMaxTokens;
+        ring_restart(group_stage_bytes<2, WDT>(np));
         if (warp == 0) {
             if (lane == 0) {
                 fence_async_proxy();
                 group_produce<2, WDT>(&map_gate, &map_up, &map_x, g, r, ppos, issued);
             }
         } else if (warp == 1) {
-            if (lane == 0) group_mma<2, WDT>(g, r, mpos, mit);
+            if (lane == 0) group_mma<2, WDT>(g, r, mpos, macc);
         } else if (warp < 6) {
-            group_epilogue<2, WDT>(g, r, eit, warp % 4, lane);
+            group_epilogue<2, WDT>(g, r, eacc, warp % 4, lane);
             fence_async_proxy();  // the gated activations are fetched by TMA in the next phase
         } else if (pred_cta) {  // the ten warps without a role in this phase
             predictor_step_group(a, l, s_ids, s_prev, warp - 6, NW - 6, lane);
@@ -182,15 +200,16 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         // ---- D ---------------------------------------------------------------------------------
         g.rows = H, g.kd = I, g.splits = d.splits, g.seg = d.seg;
         g.scale_off = 2 * I, g.x_rows = pairs + kDenseMaxTokens;
+        ring_restart(group_stage_bytes<1, WDT>(np));
         if (warp == 0) {
             if (lane == 0) {
                 fence_async_proxy();
                 group_produce<1, WDT>(&map_down, &map_down, &map_act, g, r, ppos, issued);
             }
         } else if (warp == 1) {
-            if (lane == 0) group_mma<1, WDT>(g, r, mpos, mit);
+            if (lane == 0) group_mma<1, WDT>(g, r, mpos, macc);
         } else if (warp < 6) {
-            group_epilogue<1, WDT>(g, r, eit, warp % 4, lane);
+            group_epilogue<1, WDT>(g, r, eacc, warp % 4, lane);
         }
         for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
         grid_barrier(a.barrier, a.err, target, &s_dead);

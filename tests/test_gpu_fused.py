@@ -110,3 +110,26 @@ def test_in_kernel_predictors_honour_threshold_and_replacement_rule(flags, B, th
     if live:
         assert int(O.parse_state(replay.export())["Co"].sum()) == T * B * K * K * (L - 1)
     pr.close()
+
+
+@pytest.mark.parametrize("B", [1, 3])
+def test_decode_token_host_equals_the_device_call(B):
+    """The host-buffer entry point (copies in, decode step, copies out, wait) against the
+    device-pointer call on a second stack: outputs and routing bit-identical, pinned or pageable."""
+    cfg = stacks.CONFIGS["C2"].scaled(n_layers=3, profile_tokens=2, cache_slots=0, **SHAPES[1])
+    a, b = Pair(cfg, B, oracle=False), Pair(cfg, B, oracle=False)
+    L, K, T = cfg.n_layers, cfg.top_k, 6
+    ids = torch.empty(L, B, K, dtype=torch.int32, device=DEV)
+    ho = torch.empty(B, cfg.hidden, device=DEV)
+    x = stacks.token_inputs(cfg, B, T)
+    out_host = torch.empty(B, cfg.hidden).pin_memory()
+    ids_host = torch.empty(L, B, K, dtype=torch.int32)
+    for t in range(T):
+        a.stack.decode_token(x[t].to(DEV), ho, ids)
+        b.stack.decode_token_host(x[t].contiguous(), out_host, ids_host if t % 2 == 0 else None)
+        torch.cuda.synchronize()
+        assert torch.equal(ho.cpu(), out_host), t
+        if t % 2 == 0:
+            assert torch.equal(ids.cpu(), ids_host), t
+    assert a.stack.export_state() == b.stack.export_state()
+    a.close(), b.close()
