@@ -55,13 +55,21 @@ __host__ __device__ constexpr int group_mat_stride(int wdt, int np) { return wdt
 // which accumulator buffer the next task takes and how often each was used (its barriers' phase);
 // the MMA thread and the epilogue threads each keep one and walk the same task sequence
 struct AccPos {
-    int use[2] = {0, 0};
+    int use0 = 0, use1 = 0;  // scalars (an indexed array would live in local memory)
     int next = 0;
     __device__ __forceinline__ int take(int bufs)
     {
         const int ab = bufs == 1 ? 0 : next;
         if (bufs == 2) next ^= 1;
         return ab;
+    }
+    __device__ __forceinline__ uint32_t parity(int ab) const { return (uint32_t)(ab ? use1 : use0) & 1u; }
+    __device__ __forceinline__ void used(int ab)
+    {
+        if (ab)
+            ++use1;
+        else
+            ++use0;
     }
 };
 
@@ -306,8 +314,8 @@ __device__ __forceinline__ void group_mma(const GroupArgs &a, const GroupRing &r
     for (int task = blockIdx.x; task < n_tasks && !*r.dead; task += gridDim.x) {
         const GroupTask t = group_task(a, task);
         const int ab = ap.take(bufs);
-        if (!dmbar_wait(&r.tempty[ab], ((uint32_t)ap.use[ab] & 1u) ^ 1u, r.dead)) return;
-        ap.use[ab] += 1;
+        if (!dmbar_wait(&r.tempty[ab], ap.parity(ab) ^ 1u, r.dead)) return;
+        ap.used(ab);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t acc = r.tmem + ab * group_acc_stride(WDT);
         bool first = true;
@@ -364,8 +372,8 @@ __device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRi
             s0 = bf16_to_f32(sc[srow]);
             if (NMAT == 2) s1 = bf16_to_f32(sc[a.rows + srow]);
         }
-        const bool ok = dmbar_wait(&r.tfull[ab], (uint32_t)ap.use[ab] & 1u, r.dead);
-        ap.use[ab] += 1;
+        const bool ok = dmbar_wait(&r.tfull[ab], ap.parity(ab), r.dead);
+        ap.used(ab);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t acc = r.tmem + ab * group_acc_stride(WDT) + ((uint32_t)(lg * kWarp) << 16);
         constexpr bool stacked = WDT == 2;  // three columns per token, np apart: add them

@@ -139,15 +139,18 @@ __device__ __forceinline__ void update_rows_grouped(uint8_t *gid, uint8_t *gcf, 
             else if (cf > 0)
                 cf -= 1;
         }
-        const unsigned rep = (__ballot_sync(kFull, replace) >> (sub * G)) & gmask;
-        const unsigned avail = (__ballot_sync(kFull, act && !held) >> (sub * G)) & gmask;
-        // routed experts the row does not hold; the n-th replacing slot (in slot order) takes the
-        // n-th of them
-        const int nth = __popc(rep & ((1u << sl) - 1u)) + 1;
-        unsigned pos = replacement_source(avail, nth, co != nullptr, cnt, K, sl, G);
-        if (!replace) pos = 0u;
-        const int g = __shfl_sync(kFull, myf, pos & (unsigned)(G - 1), G);
-        if (replace && pos != 0xffffffffu) id = g, cf = kConfInit;
+        const unsigned rep_all = __ballot_sync(kFull, replace);
+        if (rep_all) {  // rare; the whole warp takes the branch
+            const unsigned rep = (rep_all >> (sub * G)) & gmask;
+            const unsigned avail = (__ballot_sync(kFull, act && !held) >> (sub * G)) & gmask;
+            // routed experts the row does not hold; the n-th replacing slot (in slot order) takes
+            // the n-th of them
+            const int nth = __popc(rep & ((1u << sl) - 1u)) + 1;
+            unsigned pos = replacement_source(avail, nth, co != nullptr, cnt, K, sl, G);
+            if (!replace) pos = 0u;
+            const int g = __shfl_sync(kFull, myf, pos & (unsigned)(G - 1), G);
+            if (replace && pos != 0xffffffffu) id = g, cf = kConfInit;
+        }
         if (act) ids[sl] = (uint8_t)id, conf[sl] = (uint8_t)cf;
         __syncwarp();
     }
