@@ -201,7 +201,7 @@ int stmoe_set_prefetch_min_score(stmoe_t *s, int min_score);
 int stmoe_set_predict_threshold(stmoe_t *s, int threshold);
 
 /* Replacement rule of Algorithm 3.  When a stored candidate misses at confidence 0 the listing
- * replaces it by "any" routed expert the row does not hold.  live_counts = 0 (default): the
+ * replaces it by a routed expert the row does not hold and leaves open which.  live_counts = 0 (default): the
  * lowest such id; the co-activation counts stay as profiling (Algorithm 1) left them.
  * live_counts = 1: counting goes on at run time (for every sequence, in index order, the K x K
  * pairs of (previous layer's routing, this layer's routing) are counted right before that

@@ -314,7 +314,7 @@ int orc_predict_thr(int E, int K, const int32_t *Ei, int ni, const uint8_t *cct_
  * not hold, confidence binary 10.  The row is re-read after each replacement
  * so a row never holds an id twice; when every routed expert is already in
  * the row the slot is left.  The listing leaves the choice among several such
- * experts open ("any expert"):
+ * experts open:
  *   Co == NULL  the lowest id (the default reading);
  *   Co != NULL  the one with the largest count in row e of Co, the pair's
  *               co-activation counts kept up to date at run time (the caller
