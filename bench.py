@@ -366,7 +366,7 @@ def main():
                          "block the paper overlaps expert prefetch with (Section 4.3.4); 0 = pure MoE stack")
     ap.add_argument("--resident", action="store_true", help="keep every expert in HBM (cache_slots = 0)")
     ap.add_argument("--dense-min-batch", type=int, default=0,
-                    help="smallest batch that takes the tcgen05 path (0: the library's default, 2 for bf16, 3 for fp8)")
+                    help="smallest batch that takes the tcgen05 path (0: the library's default, 2)")
     ap.add_argument("--stage-known-kb", type=int, default=-1,
                     help="three-phase single-sequence kernel: L2 staging of known weights, KiB per expert and SM "
                          "(-1: the library's default, 0: off)")

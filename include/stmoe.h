@@ -59,9 +59,10 @@ extern "C" {
 
 #define STMOE_FLAG_NO_DENSE 4 /* never use the tensor-core FFN kernels: by default resident bf16 and fp8
                                 stacks run decode steps of at least stmoe_set_dense_min_batch() sequences
-                                (default 2 for bf16, 3 for fp8) with one work-list entry per expert on
-                                tcgen05 tiles, rounding the hidden state and the gated activations to
-                                bf16 (bf16 stacks) or f16 (fp8 stacks, whose weights are widened to f16) */
+                                (default 2) with one work-list entry per expert on tcgen05 tiles,
+                                rounding the hidden state and the gated activations to bf16 (bf16
+                                stacks) or to the sum of three e5m2 values (fp8 stacks, whose e4m3
+                                weights are multiplied as stored): relative 2^-9 either way */
 
 #define STMOE_FLAG_NO_FUSED 8 /* resident stacks, one sequence: by default stmoe_decode_token runs a kernel
                                 that streams each expert's gate, up and (from a transposed copy made at
