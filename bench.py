@@ -189,9 +189,9 @@ def profile_value(name):
 
 def top_kernel_name(cfg, batch, args):
     """The kernel that dominates a decode step of this workload (one launch per step for resident stacks)."""
-    if cfg.cache_slots:
-        return "gate_up_kernel"
     dense = not args.no_dense and cfg.dtype in ("bf16", "fp8") and batch >= (args.dense_min_batch or 2)
+    if cfg.cache_slots:   # per-layer kernels; the tensor-core ones read the slot store (no shared experts there)
+        return "dense_group_kernel (gate/up)" if dense and cfg.n_shared == 0 else "gate_up_kernel"
     if dense:
         return "dense_group_kernel (gate/up)" if args.no_persistent else "decode_token_dense_kernel"
     epl = {"f32": 4, "bf16": 8, "fp8": 16}[cfg.dtype]

@@ -122,6 +122,8 @@ struct GroupArgs {
     int E;                 // routed experts (entries with g_expert >= E are shared experts)
     int img_routed0;       // image index of this layer's expert 0 in the store
     int img_shared0;       // image index of this layer's shared expert 0
+    const uint8_t *const *blob;  // offloaded stacks: this step's image pointer of every expert (into the slot
+                                 // store the tensor maps cover); nullptr: images in layer order
     int rows;              // weight rows: I (gate/up) or H (down)
     int kd;                // reduction length: H (gate/up) or I (down)
     int np;                // batch padded to a multiple of 16 (MMA N and activation box rows)
@@ -135,10 +137,18 @@ struct GroupArgs {
     uint8_t *act8;         // gate/up out, down in: three e5m2 planes [3][act_rows][I]
     int act_rows;          // rows of one plane of act8
     int x_rows;            // rows of one plane of this projection's activation operand (hidden state: 64)
-    const uint8_t *store;  // first expert image of the stack, for the row scales behind the matrices
+    const uint8_t *store;  // first expert image the tensor maps cover (stack or slot store); fp8: the row scales
+                           // sit behind the matrices of an image
     unsigned long long img_bytes;
     int scale_off;         // element offset of this projection's scales in the image's scale vector
 };
+
+// image index (third tensor-map coordinate) of work-list expert ge
+__device__ __forceinline__ int group_image(const GroupArgs &a, int ge)
+{
+    if (a.blob) return (int)((size_t)(a.blob[ge] - a.store) / a.img_bytes);
+    return ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
+}
 
 // e4m3 weights x e5m2 activations -> fp32, both operands K-major, M = 128, N = n
 __host__ __device__ constexpr uint32_t umma_idesc_e4m3_e5m2(int n)
@@ -267,7 +277,7 @@ __device__ __forceinline__ void group_produce(const CUtensorMap *map_w0, const C
     for (int task = blockIdx.x; task < n_tasks && !*r.dead; task += gridDim.x) {
         const GroupTask t = group_task(a, task);
         const int ge = a.wl.g_expert[t.g];
-        const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
+        const int img = group_image(a, ge);
         const int xrow = NMAT == 2 ? 0 : a.wl.g_start[t.g];
         for (int k = t.k0; k < t.k1; k += KSTAGE) {
             if (!dmbar_wait(&r.empty[pos.s], pos.parity() ^ 1u, r.dead)) return;
@@ -365,7 +375,7 @@ __device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRi
         if constexpr (WDT == 2) {
             // bf16 scales per output channel behind the three matrices: [gate I | up I | down H]
             const int ge = a.wl.g_expert[t.g];
-            const int img = ge < a.E ? a.img_routed0 + ge : a.img_shared0 + (ge - a.E);
+            const int img = group_image(a, ge);
             const uint16_t *sc = reinterpret_cast<const uint16_t *>(a.store + (size_t)img * a.img_bytes +
                                                                     3 * (size_t)a.rows * a.kd) + a.scale_off;
             const int srow = min(row, a.rows - 1);

@@ -685,6 +685,8 @@ int encode_map(EncodeTiledFn fn, CUtensorMap *m, void *base, int rank, const cuu
 }
 
 void *token_dense_kernel(int rdt, bool w8);
+// first image the tensor maps of the tensor-core path cover
+uint8_t *dense_store(const stmoe *s) { return offloaded(s) ? s->d_slots : s->d_resident; }
 
 int dense_setup(stmoe *s)
 {
@@ -707,12 +709,14 @@ int dense_setup(stmoe *s)
     CU_TRY(cudaMalloc(&s->d_actb, sizeof(__nv_bfloat16) * (pairs + kDenseMaxTokens) * I));
     CU_TRY(cudaMemset(s->d_actb, 0, sizeof(__nv_bfloat16) * (pairs + kDenseMaxTokens) * I));
     CU_TRY(cudaMalloc(&s->d_part_dense, sizeof(float) * pairs * kDenseMaxSplits * H));
-    const cuuint64_t n_img = (cuuint64_t)L * (E + c.n_shared);
+    // the images the maps cover: the whole resident stack, or the slot store of an offloaded one
+    uint8_t *store = dense_store(s);
+    const cuuint64_t n_img = offloaded(s) ? (cuuint64_t)c.cache_slots : (cuuint64_t)L * (E + c.n_shared);
     const cuuint64_t gd[3] = {(cuuint64_t)H, (cuuint64_t)I, n_img}, gs[2] = {(cuuint64_t)H * 2, s->img_bytes};
     const cuuint64_t dd[3] = {(cuuint64_t)I, (cuuint64_t)H, n_img}, ds[2] = {(cuuint64_t)I * 2, s->img_bytes};
-    ST_TRY(encode_map(enc, &s->map_gate, s->d_resident, 3, gd, gs, kDenseRows));
-    ST_TRY(encode_map(enc, &s->map_up, s->d_resident + (size_t)I * H * 2, 3, gd, gs, kDenseRows));
-    ST_TRY(encode_map(enc, &s->map_down, s->d_resident + 2 * (size_t)I * H * 2, 3, dd, ds, kDenseRows));
+    ST_TRY(encode_map(enc, &s->map_gate, store, 3, gd, gs, kDenseRows));
+    ST_TRY(encode_map(enc, &s->map_up, store + (size_t)I * H * 2, 3, gd, gs, kDenseRows));
+    ST_TRY(encode_map(enc, &s->map_down, store + 2 * (size_t)I * H * 2, 3, dd, ds, kDenseRows));
     for (int i = 0; i < 4; ++i) {
         const cuuint64_t xd[2] = {(cuuint64_t)H, (cuuint64_t)kDenseMaxTokens}, xs[1] = {(cuuint64_t)H * 2};
         const cuuint64_t ad[2] = {(cuuint64_t)I, (cuuint64_t)(pairs + kDenseMaxTokens)}, as[1] = {(cuuint64_t)I * 2};
@@ -769,14 +773,15 @@ int dense8_setup(stmoe *s)
     CU_TRY(cudaMalloc(&s->d_act8, 3 * act_rows * I));
     CU_TRY(cudaMemset(s->d_act8, 0, 3 * act_rows * I));
     CU_TRY(cudaMalloc(&s->d_part_dense, sizeof(float) * pairs * kDenseMaxSplits * H));
-    const cuuint64_t n_img = (cuuint64_t)L * (E + c.n_shared);
+    uint8_t *store = dense_store(s);
+    const cuuint64_t n_img = offloaded(s) ? (cuuint64_t)c.cache_slots : (cuuint64_t)L * (E + c.n_shared);
     const cuuint64_t gd[3] = {(cuuint64_t)H, (cuuint64_t)I, n_img}, gs[2] = {(cuuint64_t)H, s->img_bytes};
     const cuuint64_t dd[3] = {(cuuint64_t)I, (cuuint64_t)H, n_img}, ds[2] = {(cuuint64_t)I, s->img_bytes};
     const CUtensorMapDataType u8 = CU_TENSOR_MAP_DATA_TYPE_UINT8;
     constexpr int kCols = group_box_cols<2>();
-    ST_TRY(encode_map(enc, &s->map8_gate, s->d_resident, 3, gd, gs, kDenseRows, u8, kCols));
-    ST_TRY(encode_map(enc, &s->map8_up, s->d_resident + (size_t)I * H, 3, gd, gs, kDenseRows, u8, kCols));
-    ST_TRY(encode_map(enc, &s->map8_down, s->d_resident + 2 * (size_t)I * H, 3, dd, ds, kDenseRows, u8, kCols));
+    ST_TRY(encode_map(enc, &s->map8_gate, store, 3, gd, gs, kDenseRows, u8, kCols));
+    ST_TRY(encode_map(enc, &s->map8_up, store + (size_t)I * H, 3, gd, gs, kDenseRows, u8, kCols));
+    ST_TRY(encode_map(enc, &s->map8_down, store + 2 * (size_t)I * H, 3, dd, ds, kDenseRows, u8, kCols));
     for (int i = 0; i < 4; ++i) {
         const cuuint64_t xd[2] = {(cuuint64_t)H, (cuuint64_t)(3 * kDenseMaxTokens)}, xs[1] = {(cuuint64_t)H};
         const cuuint64_t ad[2] = {(cuuint64_t)I, (cuuint64_t)(3 * act_rows)}, as[1] = {(cuuint64_t)I};
@@ -825,7 +830,7 @@ int dense8_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, 
     GroupArgs g{};
     g.wl = fa.wl, g.E = E, g.img_routed0 = layer * E, g.img_shared0 = c.n_layers * E + layer * c.n_shared;
     g.np = np, g.KS = s->KS, g.inv_rms = fa.inv_rms, g.part = s->d_part_dense, g.err = s->d_err;
-    g.store = s->d_resident, g.img_bytes = s->img_bytes;
+    g.store = dense_store(s), g.img_bytes = s->img_bytes, g.blob = offloaded(s) ? fa.blob : nullptr;
     g.act8 = s->d_act8, g.act_rows = batch * s->KS + kDenseMaxTokens;
     constexpr int kGu = group_kstage<2, 2>(), kDn = group_kstage<1, 2>();
     g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kGu - 1) / kGu * kGu;
@@ -875,6 +880,7 @@ int dense_ffn(stmoe *s, int layer, int batch, bool chained, const FfnArgs &fa, c
     GroupArgs g{};
     g.wl = fa.wl, g.E = E, g.img_routed0 = layer * E, g.img_shared0 = c.n_layers * E + layer * c.n_shared;
     g.np = np, g.KS = s->KS, g.inv_rms = fa.inv_rms, g.act = s->d_actb, g.part = s->d_part_dense, g.err = s->d_err;
+    g.store = dense_store(s), g.img_bytes = s->img_bytes, g.blob = offloaded(s) ? fa.blob : nullptr;
     g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + group_kstage<2, 1>() - 1) / group_kstage<2, 1>() * group_kstage<2, 1>();
     dense_group_kernel<2, 1><<<s->dense_grid, kGroupThreads, kGroupSmemBytes, st>>>(s->map_gate, s->map_up,
                                                                                       s->map_x[np / 16 - 1], g);
@@ -1396,11 +1402,14 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
             s->d_down_t = nullptr, s->d_zpart = nullptr, s->d_acc = nullptr;
         }
     }
-    if (c.cache_slots == 0 && c.weight_dtype == STMOE_BF16 && !(c.flags & STMOE_FLAG_NO_DENSE) && B >= 2) {
+    // tensor-core FFN: resident stacks, and offloaded ones whose images all live in the slot store
+    // (shared experts of an offloaded stack sit in an allocation of their own, outside the maps)
+    const bool dense_ok = (c.cache_slots == 0 || c.n_shared == 0) && !(c.flags & STMOE_FLAG_NO_DENSE) && B >= 2;
+    if (dense_ok && c.weight_dtype == STMOE_BF16) {
         const int rc = dense_setup(s);
         if (rc != STMOE_OK) return fail(rc);
     }
-    if (c.cache_slots == 0 && c.weight_dtype == STMOE_FP8_E4M3 && !(c.flags & STMOE_FLAG_NO_DENSE) && B >= 2) {
+    if (dense_ok && c.weight_dtype == STMOE_FP8_E4M3) {
         const int rc = dense8_setup(s);
         if (rc != STMOE_OK) return fail(rc);
     }
