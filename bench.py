@@ -271,7 +271,18 @@ def measure(cfg, batch, st, args, dev, world, stream, with_e2e):
         dist.all_reduce(times, op=dist.ReduceOp.MAX)
     ms, e2e_ms = (float(v) for v in times.cpu())
     step_bytes = [algorithmic_bytes(cfg, a) for a in ids_seen]
-    return dict(ms=ms, e2e_ms=e2e_ms, clocks=clocks, s0=s0, s1=s1, step_bytes=step_bytes, steps=steps)
+    return dict(ms=ms, e2e_ms=e2e_ms, clocks=clocks, s0=s0, s1=s1, step_bytes=step_bytes, steps=steps,
+                overlap=routing_overlap(ids_seen))
+
+
+def routing_overlap(ids_seen):
+    """Mean number of experts two routings share: the same layer at consecutive decode steps of a
+    sequence (temporal) and adjacent layers of one step (spatial); ids_seen: [T] arrays [L][B][K].
+    Independent uniform routings would share K*K/N (the paper's random baseline, Section 3.2)."""
+    a = np.stack(ids_seen)                                    # [T][L][B][K]
+    def shared(u, v):                                         # [...][K] x [...][K] -> mean |u & v|
+        return float((u[..., :, None] == v[..., None, :]).sum(axis=(-1, -2)).mean()) if u.size and v.size else None
+    return {"temporal": shared(a[1:], a[:-1]), "spatial": shared(a[:, 1:], a[:, :-1])}
 
 
 def summarise(cfg, batch, m, args, world, peak):
@@ -288,7 +299,8 @@ def summarise(cfg, batch, m, args, world, peak):
            "frac": step_gbs / peak, "frac_of_8000": step_gbs / 8000.0, "kernel": top_kernel_name(cfg, batch, args),
            "clocks": m["clocks"], "gpu_launches": run["kernel_launches"],
            "predictor": {"recall": run["hits"] / max(run["routed"], 1), "precision": run["hits"] / max(run["predicted"], 1),
-                         "mean_predicted": run["predicted"] / max(run["runtime_steps"], 1), "near_ties": run["near_ties"]}}
+                         "mean_predicted": run["predicted"] / max(run["runtime_steps"], 1), "near_ties": run["near_ties"],
+                         "routing_overlap": dict(m["overlap"], random=cfg.top_k * cfg.top_k / cfg.n_experts)}}
     if cfg.cache_slots:
         h2d = (s1["h2d_bytes_demand"] + s1["h2d_bytes_prefetch"] - s0["h2d_bytes_demand"] - s0["h2d_bytes_prefetch"])
         transfer, exposed = run["transfer_ms"], run["exposed_ms"]
