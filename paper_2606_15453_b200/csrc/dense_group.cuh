@@ -5,18 +5,21 @@
 // one tile of 128 weight rows (x one split of the reduction dimension for the down
 // projection); tasks are dealt round-robin over a persistent grid of one CTA per SM.  Weights
 // stay the streamed operand: the 128 weight rows are the MMA's M, the tokens its N (the batch
-// padded to a multiple of 16), and the CTA walks the reduction dimension 64 columns per stage.
-//   warp 0      one thread issues the TMA loads of a stage: the 128x64 weight tile(s) through a
-//               3-D tensor map over the expert store (column, row, image) and the Nx64
-//               activation tile, all in the 128-byte swizzled layout the MMA reads
-//   warp 1      one thread issues four K=16 tcgen05.mma per stage and matrix, frees the stage
-//               with tcgen05.commit and hands a finished accumulator to the epilogue; the warp
-//               also owns the tensor-memory allocation
+// padded to a multiple of 16), and the CTA walks the reduction dimension in boxes of 128 bytes
+// per row (64 bf16 or 128 fp8 columns), one or more boxes per stage.
+//   warp 0      one thread issues the TMA loads of a stage: the 128-row weight tile(s) through a
+//               3-D tensor map over the expert store (column, row, image; for offloaded stacks
+//               the slot store, the image index taken from the step's pointer table) and the
+//               activation tile(s), all in the 128-byte swizzled layout the MMA reads
+//   warp 1      one thread issues four tcgen05.mma per box and matrix (one per 32-byte slice),
+//               frees the stage with tcgen05.commit and hands a finished accumulator to the
+//               epilogue; the warp also owns the tensor-memory allocation
 //   warps 2-5   epilogue: read the accumulator (two buffers, so the next task's MMAs overlap),
 //               apply SiLU(gate)*up or nothing, store the rows of the entry's tokens
-// Gate/up multiplies against the whole batch's hidden state in bf16 (tensor work is free next
-// to the weight stream); the epilogue keeps the entry's tokens and applies their RMSNorm factors.  The down projection multiplies
-// against the entry's own rows of the activation buffer, which are consecutive.
+// Gate/up multiplies against the whole batch's hidden state (tensor work is free next to the
+// weight stream); the epilogue keeps the entry's tokens and applies their RMSNorm factors.  The
+// down projection multiplies against the entry's own rows of the activation buffer, which are
+// consecutive.
 // Every wait is bounded; a wait that runs out raises the error word and the kernel drains.
 //
 // Two operand formats (template parameter WDT):

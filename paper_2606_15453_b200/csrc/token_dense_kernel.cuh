@@ -14,12 +14,11 @@
 //   D   down-projection tiles the same way                                 -> grid barrier
 // The tensor-memory columns and the accumulator hand-off barriers are set up once and carried
 // through all phases and layers; the stage ring is laid out anew for every GU and D phase (its
-// stage size differs between the two, and every stage is empty at a phase boundary).  Data written with ordinary stores and then fetched by TMA from another
-// SM (the bf16 hidden state, the gated activations) is fenced for the async proxy on both sides
-// of the grid barrier in between.
+// stage size differs between the two, and every stage is empty at a phase boundary).  Data
+// written with ordinary stores and then fetched by TMA from another SM (the gate/up operand of
+// the hidden state, the gated activations) is fenced for the async proxy on both sides of the
+// grid barrier in between.
 #pragma once
-#include <type_traits>
-
 #include "dense8_group.cuh"
 #include "dense_group.cuh"
 #include "token_kernel.cuh"
