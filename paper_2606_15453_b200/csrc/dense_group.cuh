@@ -127,6 +127,11 @@ struct GroupArgs {
     int img_shared0;       // image index of this layer's shared expert 0
     const uint8_t *const *blob;  // offloaded stacks: this step's image pointer of every expert (into the slot
                                  // store the tensor maps cover); nullptr: images in layer order
+    // Hand-over of the gated activations between the two projections of a layer inside one kernel,
+    // entry by entry instead of by a grid barrier (nullptr: the caller separates the projections):
+    unsigned *signal;            // gate/up: every epilogue warp adds 1 to signal[entry] per finished tile
+    const unsigned *ready;       // down: an entry's tasks are loaded once ready[entry] >= ready_target
+    unsigned ready_target;       // = epilogue warps x gate/up row tiles
     int rows;              // weight rows: I (gate/up) or H (down)
     int kd;                // reduction length: H (gate/up) or I (down)
     int np;                // batch padded to a multiple of 16 (MMA N and activation box rows)
@@ -145,6 +150,8 @@ struct GroupArgs {
     unsigned long long img_bytes;
     int scale_off;         // element offset of this projection's scales in the image's scale vector
 };
+
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // image index (third tensor-map coordinate) of work-list expert ge
 __device__ __forceinline__ int group_image(const GroupArgs &a, int ge)
@@ -282,6 +289,21 @@ __device__ __forceinline__ void group_produce(const CUtensorMap *map_w0, const C
         const int ge = a.wl.g_expert[t.g];
         const int img = group_image(a, ge);
         const int xrow = NMAT == 2 ? 0 : a.wl.g_start[t.g];
+        if (NMAT == 1 && a.ready) {
+            // the entry's gated activations: every gate/up tile of it has been stored and fenced
+            int spins = 0;
+            for (;;) {
+                unsigned seen;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.ready + t.g) : "memory");
+                if (seen >= a.ready_target) break;
+                if (++spins > kDenseSpinLimit || *r.dead) {
+                    *r.dead = 1;
+                    return;
+                }
+                __nanosleep(64);
+            }
+            fence_async_proxy();  // they were written through the generic proxy, TMA reads them
+        }
         for (int k = t.k0; k < t.k1; k += KSTAGE) {
             if (!dmbar_wait(&r.empty[pos.s], pos.parity() ^ 1u, r.dead)) return;
             uint8_t *st = r.dsm + (size_t)pos.s * r.slot;
@@ -311,6 +333,15 @@ __device__ __forceinline__ void group_drain(const GroupRing &r, RingPos pos, int
         --pos.s;
         dmbar_wait(&r.full[pos.s], pos.parity() ^ 1u, r.dead);  // the phase before the producer's last toggle
     }
+}
+
+// The producer thread, before the ring is laid out anew: every stage it filled has been read by
+// the MMAs (the waits it would do before refilling each stage; they change no state).
+__device__ __forceinline__ bool group_wait_stages_free(const GroupRing &r, const RingPos &pos)
+{
+    for (int s = 0; s < r.NS; ++s)
+        if (!dmbar_wait(&r.empty[s], ((pos.par >> s) & 1u) ^ 1u, r.dead)) return false;
+    return true;
 }
 
 // One thread: issue the MMAs of this CTA's tasks.  `ap` carries the accumulator hand-off state
@@ -435,8 +466,13 @@ __device__ __forceinline__ void group_epilogue(const GroupArgs &a, const GroupRi
             }
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        if (NMAT == 2 && a.signal) fence_async_proxy();  // this thread's activation stores, for the TMA of another SM
         __syncwarp();
-        if (lane == 0) dmbar_arrive(&r.tempty[ab]);
+        if (lane == 0) {
+            dmbar_arrive(&r.tempty[ab]);
+            if (NMAT == 2 && a.signal && ok)
+                asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(a.signal + t.g), "r"(1u) : "memory");
+        }
         if (!ok) return;
     }
 }

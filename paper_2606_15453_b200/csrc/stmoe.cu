@@ -398,6 +398,7 @@ struct stmoe {
     float *d_host_io = nullptr;     // stmoe_decode_token_host: [2][max_batch][H] staging of h_in / h_out
     int32_t *d_host_ids = nullptr;  // and [L][max_batch][K] of the routed ids
     bool dense_persistent = false;  // one cooperative kernel per decode step (token_dense_kernel.cuh)
+    unsigned *d_gu_done = nullptr;  // its per-entry gate/up completion counters, [L][E + n_shared]
     int dense_dyn_bytes = 0;
 
     // on-chip staging of the single-sequence persistent kernel (see ffn.cuh)
@@ -737,7 +738,8 @@ int dense_setup(stmoe *s)
         if (need <= kTokenDenseDynBytes &&
             cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokenDenseDynBytes) == cudaSuccess &&
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kFfnThreads, kTokenDenseDynBytes) == cudaSuccess &&
-            occ >= 1) {
+            occ >= 1 &&
+            cudaMalloc(&s->d_gu_done, sizeof(unsigned) * (size_t)L * (E + c.n_shared)) == cudaSuccess) {
             s->dense_persistent = true;
             s->dense_dyn_bytes = kTokenDenseDynBytes;
         }
@@ -802,7 +804,8 @@ int dense8_setup(stmoe *s)
         if (need <= kTokenDenseDynBytes &&
             cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokenDenseDynBytes) == cudaSuccess &&
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k, kFfnThreads, kTokenDenseDynBytes) == cudaSuccess &&
-            occ >= 1) {
+            occ >= 1 &&
+            cudaMalloc(&s->d_gu_done, sizeof(unsigned) * (size_t)L * (E + c.n_shared)) == cudaSuccess) {
             s->dense_persistent = true;
             s->dense_dyn_bytes = kTokenDenseDynBytes;
         }
@@ -1154,7 +1157,7 @@ int token_dense(stmoe *s, int batch, const float *h_in, float *h_out, int32_t *r
     d.dyn_bytes = s->dense_dyn_bytes;
     const bool w8 = s->dense8;
     d.xb = w8 ? (void *)s->d_x8 : (void *)s->d_xb, d.actb = w8 ? (void *)s->d_act8 : (void *)s->d_actb;
-    d.part = s->d_part_dense, d.store = s->d_resident, d.img_bytes = s->img_bytes;
+    d.part = s->d_part_dense, d.store = s->d_resident, d.img_bytes = s->img_bytes, d.gu_done = s->d_gu_done;
     if (w8) {  // a split is a whole number of the fp8 format's stages
         d.seg = (d.seg + group_kstage<1, 2>() - 1) / group_kstage<1, 2>() * group_kstage<1, 2>();
         d.splits = (c.inter + d.seg - 1) / d.seg;
@@ -1222,7 +1225,7 @@ int stmoe_destroy(stmoe_t *s)
                    s->pst.Co, s->pst.cct_id, s->pst.cct_conf, s->pst.HT, s->pst.t, s->pst.pred_mask,
                    s->pst.pred_valid, s->pst.stats, s->d_rpart, s->d_sspart, s->d_arrivals, s->d_tile_done, s->d_hbuf, s->d_rpart_all, s->d_sspart_all,
                    s->d_act_all, s->d_part_all, s->d_tiles_all, s->d_barrier, s->d_err, s->d_inv, s->d_logits, s->d_w, s->d_act, s->d_part,
-                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense, s->d_x8, s->d_act8, s->d_host_io, s->d_host_ids,
+                   s->d_ids, s->d_queue, s->d_xb, s->d_actb, s->d_part_dense, s->d_x8, s->d_act8, s->d_host_io, s->d_host_ids, s->d_gu_done,
                    s->d_down_t, s->d_zpart, s->d_acc};
     if (s->d_shared && s->d_resident && s->d_shared > s->d_resident) dev[2] = nullptr;  // one allocation
     for (void *p : dev)

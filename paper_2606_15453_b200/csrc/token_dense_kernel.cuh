@@ -10,8 +10,10 @@
 //   T   every CTA runs softmax / top-K / grouping (one work-list entry per expert) itself
 //   GU  gate/up tiles on tcgen05: warp 0 feeds TMA, warp 1 issues MMAs, warps 2-5 read the
 //       accumulators; the predictor (Algorithms 1-3) runs on the remaining warps of the last CTA
-//                                                                          -> grid barrier
-//   D   down-projection tiles the same way                                 -> grid barrier
+//   D   down-projection tiles the same way, with no grid barrier before them: a CTA that has
+//       finished its gate/up tiles goes on, and the loads of an entry's down tiles wait for that
+//       entry's gate/up tiles only (a counter per entry; gate/up tiles wait for nothing, so
+//       every counter fills)                                                -> grid barrier
 // The tensor-memory columns and the accumulator hand-off barriers are set up once and carried
 // through all phases and layers; the stage ring is laid out anew for every GU and D phase (its
 // stage size differs between the two, and every stage is empty at a phase boundary).  Data
@@ -35,9 +37,8 @@ struct TokenDenseArgs {
     float *part;            // [pairs][splits][H]
     const uint8_t *store;   // fp8: first expert image (for the row scales) and the image pitch
     unsigned long long img_bytes;
+    unsigned *gu_done;      // [L][E + n_shared]: finished gate/up tiles x epilogue warps per work-list entry
 };
-
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // RDT: router weight type; WDT: expert weight type, 1 = bf16, 2 = fp8 e4m3 (operand formats of
 // dense_group.cuh).
@@ -134,6 +135,7 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         // ---- F ---------------------------------------------------------------------------------
         if (l == 0) {
             for (int i = gtid; i < B * H; i += gthreads) store_x(i, h[i]);
+            for (int i = gtid; i < L * (E + a.n_shared); i += gthreads) d.gu_done[i] = 0u;  // read after later barriers
         } else {
             const FfnArgs fp = finish_args(l - 1);
             float *hl = a.hbuf + (size_t)l * B * H;
@@ -180,6 +182,7 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         constexpr int kGuStage = group_kstage<2, WDT>();
         g.rows = I, g.kd = H, g.splits = 1, g.seg = (H + kGuStage - 1) / kGuStage * kGuStage;
         g.scale_off = 0, g.x_rows = kDenseMaxTokens;
+        g.signal = d.gu_done + (size_t)l * (E + a.n_shared), g.ready = nullptr;
         ring_restart(group_stage_bytes<2, WDT>(np));
         if (warp == 0) {
             if (lane == 0) {
@@ -190,15 +193,16 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
             if (lane == 0) group_mma<2, WDT>(g, r, mpos, macc);
         } else if (warp < 6) {
             group_epilogue<2, WDT>(g, r, eacc, warp % 4, lane);
-            fence_async_proxy();  // the gated activations are fetched by TMA in the next phase
         } else if (pred_cta) {  // the ten warps without a role in this phase
             predictor_step_group(a, l, s_ids, s_prev, warp - 6, NW - 6, lane);
         }
-        grid_barrier(a.barrier, a.err, target, &s_dead);
 
-        // ---- D ---------------------------------------------------------------------------------
+        // ---- D (every role moves on by itself) ----------------------------------------------------
         g.rows = H, g.kd = I, g.splits = d.splits, g.seg = d.seg;
         g.scale_off = 2 * I, g.x_rows = pairs + kDenseMaxTokens;
+        g.ready = g.signal, g.signal = nullptr, g.ready_target = 4u * (unsigned)((I + kDenseRows - 1) / kDenseRows);
+        // the MMAs have read every gate/up stage before the producer lays the ring out for this phase
+        if (warp == 0 && lane == 0) group_wait_stages_free(r, ppos);
         ring_restart(group_stage_bytes<1, WDT>(np));
         if (warp == 0) {
             if (lane == 0) {
@@ -210,8 +214,9 @@ decode_token_dense_kernel(const __grid_constant__ CUtensorMap map_gate, const __
         } else if (warp < 6) {
             group_epilogue<1, WDT>(g, r, eacc, warp % 4, lane);
         }
-        for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
         grid_barrier(a.barrier, a.err, target, &s_dead);
+        // (after the barrier: the predictor warps of the last CTA read s_prev until they reach it)
+        for (int i = threadIdx.x; i < B * K; i += blockDim.x) s_prev[i] = s_ids[i];
     }
     // the last layer's output
     if (!s_dead) {
