@@ -266,13 +266,20 @@ def measure(cfg, batch, st, args, dev, world, stream, with_e2e):
             st.decode_token_host(x_host[t + i], out_host, ids_host)
         e2e_ms = (time.perf_counter() - w0) * 1e3
         barrier()
-    times = torch.tensor([ms, e2e_ms or 0.0], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = (float(v) for v in times.cpu())
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms or 0.0], world, dev)
     step_bytes = [algorithmic_bytes(cfg, a) for a in ids_seen]
     return dict(ms=ms, e2e_ms=e2e_ms, clocks=clocks, s0=s0, s1=s1, step_bytes=step_bytes, steps=steps,
                 overlap=routing_overlap(ids_seen))
+
+
+def max_over_ranks(values, world, device):
+    """The slowest rank's figures: replicas run the same steps side by side, the job's time per step is
+    the maximum over ranks (value = the tokens of all ranks over that time)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
 
 
 def routing_overlap(ids_seen):

@@ -30,3 +30,36 @@ def test_reference_arm_prints_the_contract_line():
 def test_reference_arm_other_ranks_exit_quietly():
     r = _run({"RANK": "1", "WORLD_SIZE": "2", "LOCAL_RANK": "1", "CUDA_VISIBLE_DEVICES": ""})
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def _rank_main(rank, world, port, out):
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    # rank r measured (10 + r) ms device-timed and (20 - r) ms end to end: the job's figures are the maxima
+    ms, e2e = bench.max_over_ranks([10.0 + rank, 20.0 - rank], world, torch.device("cpu"))
+    dist.barrier()
+    dist.destroy_process_group()
+    out.put((rank, ms, e2e))
+
+
+def test_replica_timing_is_the_maximum_over_ranks_gloo_world_2():
+    """The N > 1 path of the main arm (replicas only: no data-path collective): every rank gets the
+    slowest rank's times, from which rank 0 reports tokens of all ranks over that time."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_rank_main, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert got == [(0, 11.0, 20.0), (1, 11.0, 20.0)]
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks([3.0, 4.0], 1, "cpu") == [3.0, 4.0]      # a single rank: no collective
