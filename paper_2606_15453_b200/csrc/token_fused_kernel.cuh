@@ -269,6 +269,29 @@ __device__ __forceinline__ bool fused_wait(uint64_t *bar, uint32_t parity, volat
     return false;
 }
 
+// Sixteen e4m3 weights (one 16-byte chunk) times sixteen f16 activations held as eight pairs:
+// exact e4m3 -> f16 conversions two at a time, f16 pair FMAs on two independent accumulators, the
+// four partial sums added in fp32.
+__device__ __forceinline__ float dot_e4m3_f16(const uint4 &w4, const uint32_t (&hx)[8])
+{
+    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+    __half2 acc0 = __float2half2_rn(0.f), acc1 = acc0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint32_t lo, hi;  // weights 4i, 4i+1 and 4i+2, 4i+3 as f16 pairs
+        asm("{.reg .b16 a, b;\n\t"
+            "mov.b32 {a, b}, %2;\n\t"
+            "cvt.rn.f16x2.e4m3x2 %0, a;\n\t"
+            "cvt.rn.f16x2.e4m3x2 %1, b;}"
+            : "=r"(lo), "=r"(hi)
+            : "r"(w[i]));
+        acc0 = __hfma2(*reinterpret_cast<const __half2 *>(&lo), *reinterpret_cast<const __half2 *>(&hx[2 * i]), acc0);
+        acc1 = __hfma2(*reinterpret_cast<const __half2 *>(&hi), *reinterpret_cast<const __half2 *>(&hx[2 * i + 1]), acc1);
+    }
+    const float2 a = __half22float2(acc0), b = __half22float2(acc1);
+    return (a.x + a.y) + (b.x + b.y);
+}
+
 // CH: 16-byte chunks of a row a thread owns (chunk j = columns [(t + j*TPR)*EPL, +EPL)).  Two
 // chunks halve the per-block bookkeeping (waits, reductions, barriers) per byte, which is what
 // bounds the kernel once the copies keep HBM busy; they need twice the registers for the
@@ -412,6 +435,19 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
             for (int e = 0; e < EPL; ++e) ss = fmaf(h[j][e], h[j][e], ss);
         ss = unit_sum(u, ss);
         const float inv = 1.0f / sqrtf(ss / (float)H + a.eps);
+        // fp8 stacks: the gate/up dot products run on f16 pairs (an e4m3 weight is exact in f16, and
+        // converting it on to fp32 costs more issue slots than the FMA it feeds).  The normalised
+        // hidden state is at most sqrt(H) <= 64 in magnitude, so x / 8 times a weight (<= 448), summed
+        // over the eight products a lane adds up in f16, stays below 28672: no overflow; the partial
+        // sums go to fp32 before they are added across lanes.
+        uint32_t hx[DT == 2 ? EPL / 2 : 1];
+        if (DT == 2) {
+#pragma unroll
+            for (int e2 = 0; e2 < EPL / 2; ++e2) {
+                const __half2 p = __floats2half2_rn(h[0][2 * e2] * inv * 0.125f, h[0][2 * e2 + 1] * inv * 0.125f);
+                hx[e2] = *reinterpret_cast<const uint32_t *>(&p);
+            }
+        }
 
         // ---- router rows dealt over the units ------------------------------------------------
         for (int jr = unit; jr < E; jr += n_units) {
@@ -547,13 +583,18 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
                         wu4 = *reinterpret_cast<const uint4 *>(stage + R * row_bytes + off);
                         wd[r][j] = *reinterpret_cast<const uint4 *>(stage + 2 * R * row_bytes + off);
                     }
-                    float wg[EPL], wu[EPL];
-                    Fmt<DT>::unpack(wg4, wg);
-                    Fmt<DT>::unpack(wu4, wu);
+                    if constexpr (DT == 2) {
+                        v[2 * r] += dot_e4m3_f16(wg4, hx);
+                        v[2 * r + 1] += dot_e4m3_f16(wu4, hx);
+                    } else {
+                        float wg[EPL], wu[EPL];
+                        Fmt<DT>::unpack(wg4, wg);
+                        Fmt<DT>::unpack(wu4, wu);
 #pragma unroll
-                    for (int e = 0; e < EPL; ++e) {
-                        v[2 * r] = fmaf(wg[e], h[j][e], v[2 * r]);
-                        v[2 * r + 1] = fmaf(wu[e], h[j][e], v[2 * r + 1]);
+                        for (int e = 0; e < EPL; ++e) {
+                            v[2 * r] = fmaf(wg[e], h[j][e], v[2 * r]);
+                            v[2 * r + 1] = fmaf(wu[e], h[j][e], v[2 * r + 1]);
+                        }
                     }
                 }
             unit_sum4(u, v);  // past its barrier every thread has read the stage: it may be refilled
@@ -565,7 +606,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
                                                         image_scales(H, I, BYTES));
             // odd lanes evaluate row 1, even lanes row 0; one exchange gives every lane both
             const int r_mine = u.lane & 1;
-            float gv = (r_mine ? v[2] : v[0]) * inv, uv = (r_mine ? v[3] : v[1]) * inv;
+            const float vs = DT == 2 ? 8.f : inv;  // fp8: the f16 pairs carry inv / 8 already
+            float gv = (r_mine ? v[2] : v[0]) * vs, uv = (r_mine ? v[3] : v[1]) * vs;
             if (DT == 2 && i0 + r_mine < I) {
                 gv *= bf16_to_f32(sc[i0 + r_mine]);
                 uv *= bf16_to_f32(sc[I + i0 + r_mine]);

@@ -65,8 +65,11 @@ def test_fused_step_is_reproducible_and_agrees_with_three_phase_kernel(shape):
         if not torch.equal(u[1], v[1]):   # routing parted: only at a flagged near tie
             assert int(u[4].sum()) + int(v[4].sum()) > 0, t
             break
-        assert rel_err(u[0].numpy(), v[0].numpy()) <= 1e-4, t
-        assert np.abs(u[2].numpy() - v[2].numpy()).max() < 2e-6
+        # fp8 stacks: the one-phase kernel forms its gate/up dot products from f16 pairs (exact weights,
+        # activations and eight-term partial sums rounded to f16): a rounding-level difference
+        fp8 = cfg.dtype == "fp8"
+        assert rel_err(u[0].numpy(), v[0].numpy()) <= (2e-3 if fp8 else 1e-4), t
+        assert np.abs(u[2].numpy() - v[2].numpy()).max() < (2e-5 if fp8 else 2e-6)   # (later layers see that h)
         assert torch.equal(u[3], v[3])
     else:
         assert a[1] == three[1]           # same routing all the way: same predictor tables
