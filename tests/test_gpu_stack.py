@@ -191,3 +191,39 @@ def test_argument_and_state_errors():
     with pytest.raises(P.StmoeError):
         s.decode_step(0, torch.zeros(2, 64, device=DEV), torch.zeros(2, 64, device=DEV))  # batch > max
     s.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_offloaded_batches_take_the_tensor_core_tiles(dtype):
+    """An offloaded stack without shared experts runs batched steps on the tcgen05 kernels, whose tensor
+    maps cover the slot store: more launches per layer than the CUDA-core tiles (operand cast, weighted
+    sum), the same routing and cache traffic while the routing agrees, outputs within the tolerance."""
+    cfg = stacks.CONFIGS["C3"].scaled(n_layers=3, profile_tokens=1, cache_slots=64, hidden=512, inter=384,
+                                      n_experts=32, top_k=4, dtype=dtype)
+    B, T = 8, 4
+    L, K = cfg.n_layers, cfg.top_k
+    x = stacks.token_inputs(cfg, B, T).to(DEV)
+    runs = []
+    for flags in (0, P.FLAG_NO_DENSE):
+        pr = Pair(cfg, B, oracle=False, flags=flags, prefetch_limit=2)
+        ids = torch.empty(L, B, K, dtype=torch.int32, device=DEV)
+        ho = torch.empty(B, cfg.hidden, device=DEV)
+        outs = []
+        for t in range(T):
+            pr.stack.decode_token(x[t].clone(), ho, ids)
+            torch.cuda.synchronize()
+            outs.append((ho.cpu().clone(), ids.cpu().clone()))
+        runs.append((outs, pr.stack.stats()))
+        pr.close()
+    (dense, sd), (core, sc) = runs
+    assert sd["kernel_launches"] > sc["kernel_launches"]
+    same = True
+    for t, ((hd, idd), (hc, idc)) in enumerate(zip(dense, core)):
+        if t == 0:
+            assert torch.equal(idd[0], idc[0])                      # layer 0 sees identical inputs
+        same = same and torch.equal(idd, idc)
+        if same:
+            assert (hd - hc).abs().max().item() <= 2e-2 * hc.abs().max().item(), t
+    if same:
+        assert (sd["cache_hits"], sd["cache_misses"], sd["prefetch_issued"]) == \
+            (sc["cache_hits"], sc["cache_misses"], sc["prefetch_issued"])
