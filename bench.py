@@ -383,6 +383,9 @@ def main():
     ap.add_argument("--inter-layer-gap-us", type=float, default=0.0,
                     help="idle the compute stream this long after every layer: a stand-in for the attention "
                          "block the paper overlaps expert prefetch with (Section 4.3.4); 0 = pure MoE stack")
+    ap.add_argument("--cache-slots", type=int, default=0,
+                    help="offloaded stacks: override the number of HBM slots (a few times top_k: the paper's setting, "
+                         "a buffer for one layer's experts and no cache)")
     ap.add_argument("--resident", action="store_true", help="keep every expert in HBM (cache_slots = 0)")
     ap.add_argument("--dense-min-batch", type=int, default=0,
                     help="smallest batch that takes the tcgen05 path (0: the library's default, 2)")
@@ -406,6 +409,8 @@ def main():
                          cache_slots=min(cfg.cache_slots, args.layers * cfg.n_experts))
     if args.resident:
         cfg = cfg.scaled(cache_slots=0, name=cfg.name + "-resident")
+    if args.cache_slots:
+        cfg = cfg.scaled(cache_slots=args.cache_slots, name=cfg.name + f"-slots{args.cache_slots}")
     batch = args.batch
     if args.impl == "reference":
         return run_reference(args, cfg, batch)
