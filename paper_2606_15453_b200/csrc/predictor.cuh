@@ -36,6 +36,10 @@ struct PredArgs {
     int32_t *n_pred;      // optional [B]
     int max_pred;
     int32_t *queue;       // optional: [0] n, [1..E] ids, [1+E..2E] scores (priority order)
+    // optional, with queue: host memory mapped into the device's address space that the host polls
+    // instead of copying: [0] <- host_seq last, [1..1+Bmax*K) this layer's routing, then the queue
+    int32_t *host_out;
+    int32_t host_seq, host_queue_off;
 };
 
 // Which routed expert a replacing slot takes (Algorithm 3 leaves it open).  Every lane of a group
@@ -281,10 +285,25 @@ __global__ void __launch_bounds__(256) predictor_step_kernel(PredArgs a)
             }
             a.queue[1 + rank] = f;
             a.queue[1 + E + rank] = mine;
+            if (a.host_out) {
+                a.host_out[a.host_queue_off + 1 + rank] = f;
+                a.host_out[a.host_queue_off + 1 + E + rank] = mine;
+            }
             atomicAdd(&s_nq, 1);
         }
         __syncthreads();
-        if (threadIdx.x == 0) a.queue[0] = s_nq;
+        if (threadIdx.x == 0) {
+            a.queue[0] = s_nq;
+            if (a.host_out) a.host_out[a.host_queue_off] = s_nq;
+        }
+    }
+    if (a.queue && a.host_out) {
+        // hand the routing and the queue to the host without a copy: every writer fences its stores
+        // to system scope, the stamp goes last
+        for (int i = threadIdx.x; i < B * K; i += blockDim.x) a.host_out[1 + i] = a.cur[i];
+        __threadfence_system();
+        __syncthreads();
+        if (threadIdx.x == 0) *reinterpret_cast<volatile int32_t *>(a.host_out) = a.host_seq;
     }
 
     // HT[layer] <- routing; advance the step counter after the last layer

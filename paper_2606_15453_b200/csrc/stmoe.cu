@@ -2,6 +2,7 @@
 // tables, the HBM slot cache with its copy stream and event fences, kernel launches.
 #include "../../include/stmoe.h"
 
+#include <atomic>
 #include <chrono>
 #include <cstdio>
 #include <cstring>
@@ -356,7 +357,10 @@ struct stmoe {
     float *d_inv = nullptr, *d_logits = nullptr, *d_w = nullptr, *d_act = nullptr, *d_part = nullptr;
     int32_t *d_ids = nullptr;   // [L][B][K] routing of the current decode step
     int32_t *d_queue = nullptr; // [1 + 2E]
-    int32_t *h_ids = nullptr, *h_queue = nullptr;  // pinned mirrors
+    // the routing and the prefetch queue of a layer step, written by the predictor kernel into pinned host
+    // memory mapped on the device: [0] stamp of the step | ids | queue; h_ids / h_queue point into it
+    int32_t *h_route = nullptr, *d_route = nullptr, *h_ids = nullptr, *h_queue = nullptr;
+    int32_t route_seq = 0;
     WorkListMem wlm;
     FfnPlan plan1, plan4;
 
@@ -476,6 +480,10 @@ int launch_predictor(stmoe *s, int layer, int batch, const int32_t *cur, const i
     a.cur = cur, a.prev = prev;
     a.pred_ids = pred_ids, a.n_pred = n_pred, a.max_pred = s->max_pred;
     a.queue = want_queue ? s->d_queue : nullptr;
+    if (want_queue && s->d_route) {
+        a.host_out = s->d_route, a.host_seq = ++s->route_seq;
+        a.host_queue_off = (int)(s->h_queue - s->h_route);
+    }
     predictor_step_kernel<<<1, 256, 0, st>>>(a);
     s->launches += 1;
     if (layer == c.n_layers - 1) {
@@ -535,20 +543,23 @@ int cache_step(stmoe *s, int layer, int batch, cudaStream_t st)
     const int next = (layer + 1) % L;
     SlotCache &ch = s->cache;
 
-    // this layer's routing and the prefetch queue, on the host (bounded wait)
-    CU_TRY(cudaMemcpyAsync(s->h_ids, s->d_ids + (size_t)layer * c.max_batch * K, sizeof(int32_t) * batch * K,
-                           cudaMemcpyDeviceToHost, st));
-    CU_TRY(cudaMemcpyAsync(s->h_queue, s->d_queue, sizeof(int32_t) * (1 + 2 * E), cudaMemcpyDeviceToHost, st));
-    CU_TRY(cudaEventRecord(s->ev_route, st));
-    const auto t0 = std::chrono::steady_clock::now();
-    for (;;) {
-        const cudaError_t q = cudaEventQuery(s->ev_route);
-        if (q == cudaSuccess) break;
-        if (q != cudaErrorNotReady) {
-            (void)cudaGetLastError();
-            return STMOE_ERR_CUDA;
+    // this layer's routing and the prefetch queue: the predictor kernel has been enqueued and stamps
+    // the mapped host block when they are there (bounded wait; no copy, no event)
+    {
+        const auto t0 = std::chrono::steady_clock::now();
+        volatile int32_t *stamp = s->h_route;
+        for (unsigned spins = 0; *stamp != s->route_seq; ++spins) {
+            if ((spins & 1023u) == 1023u) {
+                const cudaError_t q = cudaStreamQuery(st);
+                if (q != cudaSuccess && q != cudaErrorNotReady) {
+                    (void)cudaGetLastError();
+                    return STMOE_ERR_CUDA;
+                }
+                if (std::chrono::steady_clock::now() - t0 > std::chrono::milliseconds(s->host_wait_ms))
+                    return STMOE_ERR_TIMEOUT;
+            }
         }
-        if (std::chrono::steady_clock::now() - t0 > std::chrono::milliseconds(s->host_wait_ms)) return STMOE_ERR_TIMEOUT;
+        std::atomic_thread_fence(std::memory_order_acquire);
     }
     harvest_spans(s, false);
 
@@ -1231,7 +1242,7 @@ int stmoe_destroy(stmoe_t *s)
     for (void *p : dev)
         if (p) cudaFree(p);
     s->wlm.release();
-    void *host[] = {s->h_store, (void *)s->h_blob_table, s->h_ids, s->h_queue};
+    void *host[] = {s->h_store, (void *)s->h_blob_table, s->h_route};
     for (void *p : host)
         if (p) cudaFreeHost(p);
     (void)cudaGetLastError();
@@ -1292,8 +1303,10 @@ int stmoe_create(const stmoe_config_t *cfg, stmoe_t **out)
         CR_TRY(cudaMalloc(&s->d_slots, (size_t)c.cache_slots * s->img_bytes));
         CR_TRY(cudaMalloc(&s->d_blob_table, sizeof(void *) * (E + c.n_shared)));
         CR_TRY(cudaHostAlloc(&s->h_blob_table, sizeof(void *) * (E + c.n_shared), cudaHostAllocDefault));
-        CR_TRY(cudaHostAlloc(&s->h_ids, sizeof(int32_t) * B * K, cudaHostAllocDefault));
-        CR_TRY(cudaHostAlloc(&s->h_queue, sizeof(int32_t) * (1 + 2 * E), cudaHostAllocDefault));
+        CR_TRY(cudaHostAlloc(&s->h_route, sizeof(int32_t) * (1 + (size_t)B * K + 1 + 2 * E), cudaHostAllocMapped));
+        memset(s->h_route, 0, sizeof(int32_t) * (1 + (size_t)B * K + 1 + 2 * E));
+        CR_TRY(cudaHostGetDevicePointer((void **)&s->d_route, s->h_route, 0));
+        s->h_ids = s->h_route + 1, s->h_queue = s->h_route + 1 + (size_t)B * K;
         CR_TRY(cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking));
         CR_TRY(cudaEventCreateWithFlags(&s->ev_route, cudaEventDisableTiming));
         s->cache.init(c.cache_slots, L, E);
