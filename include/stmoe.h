@@ -258,7 +258,8 @@ int stmoe_test_hook(stmoe_t *s, int what, int64_t value);
 /* Runs the bounded waits of the persistent kernels on barriers that nobody completes, with a poll
  * limit of a few thousand: which = 0 the grid barrier of the three-phase kernel, 1 the grid barrier
  * of the single-sequence kernel, 2 an mbarrier wait of the tensor-core kernels, 3 the mbarrier wait
- * of the single-sequence kernel's copy ring.  Each wait gives up, the stack's error word is set
+ * of the single-sequence kernel's copy ring, 4 the wait of the tensor-core kernel's down-projection
+ * loads for an entry's gate/up tiles.  Each wait gives up, the stack's error word is set
  * and stmoe_stats returns STMOE_ERR_TIMEOUT from then on (destroy the stack afterwards); the
  * kernel itself ends normally.  Asynchronous on cuda_stream. */
 int stmoe_selftest_bounded_wait(stmoe_t *s, int which, int poll_limit, void *cuda_stream);

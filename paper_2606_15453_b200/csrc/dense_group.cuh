@@ -153,6 +153,22 @@ struct GroupArgs {
 
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
+// Bounded wait (one thread) until a counter that other CTAs raise with release semantics reaches
+// `target`; false when the limit ran out or another thread of the CTA gave up.
+__device__ __forceinline__ bool group_wait_counter(const unsigned *counter, unsigned target, volatile int *dead,
+                                                   int spin_limit = kDenseSpinLimit)
+{
+    for (int spins = 0; spins < spin_limit; ++spins) {
+        unsigned seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+        if (seen >= target) return true;
+        if (*dead) return false;
+        __nanosleep(64);
+    }
+    *dead = 1;
+    return false;
+}
+
 // image index (third tensor-map coordinate) of work-list expert ge
 __device__ __forceinline__ int group_image(const GroupArgs &a, int ge)
 {
@@ -291,17 +307,7 @@ __device__ __forceinline__ void group_produce(const CUtensorMap *map_w0, const C
         const int xrow = NMAT == 2 ? 0 : a.wl.g_start[t.g];
         if (NMAT == 1 && a.ready) {
             // the entry's gated activations: every gate/up tile of it has been stored and fenced
-            int spins = 0;
-            for (;;) {
-                unsigned seen;
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.ready + t.g) : "memory");
-                if (seen >= a.ready_target) break;
-                if (++spins > kDenseSpinLimit || *r.dead) {
-                    *r.dead = 1;
-                    return;
-                }
-                __nanosleep(64);
-            }
+            if (!group_wait_counter(a.ready + t.g, a.ready_target, r.dead)) return;
             fence_async_proxy();  // they were written through the generic proxy, TMA reads them
         }
         for (int k = t.k0; k < t.k1; k += KSTAGE) {

@@ -1459,7 +1459,7 @@ int stmoe_set_prefetch_min_score(stmoe_t *s, int min_score)
 
 int stmoe_selftest_bounded_wait(stmoe_t *s, int which, int poll_limit, void *cuda_stream)
 {
-    if (!s || which < 0 || which > 3 || poll_limit < 1 || poll_limit > (1 << 16)) return STMOE_ERR_BAD_ARG;
+    if (!s || which < 0 || which > 4 || poll_limit < 1 || poll_limit > (1 << 16)) return STMOE_ERR_BAD_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (!s->d_barrier) CU_TRY(cudaMalloc(&s->d_barrier, 16));
     CU_TRY(cudaMemsetAsync(s->d_barrier, 0, 4, st));

@@ -739,7 +739,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
 // The bounded waits of the persistent kernels, run on barriers that nobody completes: two CTAs of
 // 64 threads call the same helpers the kernels use, with a small poll limit; every wait gives up,
 // raises the error word and returns.  which: 0 grid_barrier (token_kernel.cuh), 1 cta_wait
-// (this file), 2 dmbar_wait (tensor-core kernels), 3 fused_wait (this file's copy ring).
+// (this file), 2 dmbar_wait (tensor-core kernels), 3 fused_wait (this file's copy ring), 4
+// group_wait_counter (the tensor-core kernel's hand-over between its projections).
 __global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(unsigned *counter, unsigned *err, int which, int limit)
 {
     __shared__ int s_dead;
@@ -759,8 +760,11 @@ __global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(unsigned *cou
         cta_wait(cb, counter, err, gridDim.x + 1, &s_dead, limit);
     } else if (which == 2) {
         if (!dmbar_wait(&s_bar, 0u, &s_dead, limit) && threadIdx.x == 0) *err = 1u;
-    } else {
+    } else if (which == 3) {
         if (!fused_wait(&s_bar, 0u, &s_dead, limit) && threadIdx.x == 0) *err = 1u;
+    } else {
+        // a completion counter that stays one short (the grid barrier's counter: zero, nobody adds)
+        if (threadIdx.x == 0 && !group_wait_counter(counter, 1u, &s_dead, limit)) *err = 1u;
     }
 }
 

@@ -16,10 +16,11 @@ DEV = "cuda:0"
 B = P.binding
 
 
-@pytest.mark.parametrize("which", [0, 1, 2, 3])
+@pytest.mark.parametrize("which", [0, 1, 2, 3, 4])
 def test_bounded_waits_run_out_and_report_a_timeout(which):
-    """The wait helpers of the persistent kernels on a barrier that is one arrival short (or an
-    mbarrier nobody arrives at), poll limit 4096: the kernel ends, the error word is set."""
+    """The wait helpers of the persistent kernels on a barrier that is one arrival short (an mbarrier
+    nobody arrives at, a completion counter nobody raises), poll limit 4096: the kernel ends, the error
+    word is set."""
     cfg = stacks.CONFIGS["C0"].scaled(n_layers=2)
     pr = Pair(cfg, 1, oracle=False)
     assert pr.stack.stats()["decode_steps"] == 0           # healthy before
