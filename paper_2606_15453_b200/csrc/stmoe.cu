@@ -1090,7 +1090,8 @@ void *token_fused_kernel(const stmoe_config_t &c)
     const int ch = fused_chunks(c.hidden, 16 / dtype_bytes(dt), c.inter, c.top_k, sm_count());
     if (dt == STMOE_F32) return ch == 2 ? (void *)decode_token_fused_kernel<0, 0, 2> : (void *)decode_token_fused_kernel<0, 0, 1>;
     if (dt == STMOE_BF16) return ch == 2 ? (void *)decode_token_fused_kernel<1, 1, 2> : (void *)decode_token_fused_kernel<1, 1, 1>;
-    return (void *)decode_token_fused_kernel<2, 1, 1>;
+    const int rows = fused_rows(c.hidden, 16 / dtype_bytes(dt), c.inter, c.top_k, sm_count(), ch);
+    return rows == 4 ? (void *)decode_token_fused_kernel<2, 1, 1, 4> : (void *)decode_token_fused_kernel<2, 1, 1, 2>;
 }
 
 int token_fused(stmoe *s, const float *h_in, float *h_out, int32_t *routed_ids, float *routed_w,

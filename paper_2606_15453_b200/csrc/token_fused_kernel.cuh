@@ -52,7 +52,7 @@ struct FusedArgs {
     int poll_limit;             // polls before a grid-barrier wait gives up
 };
 
-constexpr int kFusedRows = 2;          // rows per block
+constexpr int kFusedRows = 2;          // rows per block (four for some fp8 shapes, see fused_rows)
 constexpr int kFusedStages = 4;        // ring stages per unit (blocks in flight) with one chunk per thread
 // ring bytes: units * stages * 3 matrices * rows * (H * element bytes) = 512 threads * 16 B * 24
 constexpr int kFusedRingBytes = kFfnThreads * 16 * 3 * kFusedRows * kFusedStages;
@@ -85,9 +85,22 @@ __host__ __device__ inline int fused_chunks(int H, int epl, int I, int K, int n_
     return blocks >= 6 * units ? 2 : 1;
 }
 
+// Rows per block: four for fp8 stacks with enough row blocks per unit (the same test as for a second
+// chunk, which their 16-column layout has no registers for).  A block's cost beside its bytes is a
+// serial chain (shared-memory reads, the unit's reduction with its barrier, the exponential, the
+// exchange of the activations); with four rows the chain is paid once per 48 KB instead of 24 KB.
+__host__ __device__ inline int fused_rows(int H, int epl, int I, int K, int n_ctas, int chunks)
+{
+    if (epl < 16 || chunks != 1) return kFusedRows;
+    const long long units = (long long)(n_ctas - 1) * (kFfnThreads / (H / epl));
+    const long long blocks = (long long)K * ((I + 3) / 4);
+    return blocks >= 6 * units ? 4 : kFusedRows;
+}
+
+constexpr int kRedStride = 128;  // floats of one exchange buffer of a unit: up to 16 warps x 8 values
 struct UnitCtx {
     int tpr, grp, t, wig, nwg, lane, bar_id;
-    float *red;      // [2][16][4] this unit's exchange buffers
+    float *red;      // [2][kRedStride] this unit's exchange buffers
     int par;         // which of the two is written next
 };
 
@@ -101,7 +114,7 @@ __device__ __forceinline__ void unit_sync(const UnitCtx &u)
 __device__ __forceinline__ float unit_sum(UnitCtx &u, float v)
 {
     v = warp_sum(v);
-    float *buf = u.red + u.par * 64;
+    float *buf = u.red + u.par * kRedStride;
     u.par ^= 1;
     if (u.lane == 0) buf[u.wig * 4] = v;
     unit_sync(u);
@@ -113,7 +126,7 @@ __device__ __forceinline__ float unit_sum(UnitCtx &u, float v)
 __device__ __forceinline__ float unit_max(UnitCtx &u, float v)
 {
     v = warp_max(v);
-    float *buf = u.red + u.par * 64;
+    float *buf = u.red + u.par * kRedStride;
     u.par ^= 1;
     if (u.lane == 0) buf[u.wig * 4] = v;
     unit_sync(u);
@@ -139,7 +152,7 @@ __device__ __forceinline__ void unit_sum4(UnitCtx &u, float (&v)[4])
     k += __shfl_xor_sync(kFull, k, 4);
     k += __shfl_xor_sync(kFull, k, 2);
     k += __shfl_xor_sync(kFull, k, 1);
-    float *buf = u.red + u.par * 64;
+    float *buf = u.red + u.par * kRedStride;
     u.par ^= 1;
     if ((u.lane & 7) == 0) buf[u.wig * 4 + (u.lane >> 3)] = k;
     unit_sync(u);
@@ -152,6 +165,43 @@ __device__ __forceinline__ void unit_sum4(UnitCtx &u, float (&v)[4])
     t += __shfl_xor_sync(kFull, t, 16);
 #pragma unroll
     for (int i = 0; i < 4; ++i) v[i] = __shfl_sync(kFull, t, i);
+}
+
+// Sums of eight values over the unit, the same way: three folding exchanges leave every lane with
+// one value's sum over eight lanes, two more finish the warp (9 shuffles); lane 4 i holds value i.
+__device__ __forceinline__ void unit_sum8(UnitCtx &u, float (&v)[8])
+{
+    const bool b16 = u.lane & 16, b8 = u.lane & 8, b4 = u.lane & 4;
+    float k[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        k[i] = b16 ? v[4 + i] : v[i];
+        const float s = b16 ? v[i] : v[4 + i];
+        k[i] += __shfl_xor_sync(kFull, s, 16);
+    }
+    float k2[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        k2[i] = b8 ? k[2 + i] : k[i];
+        const float s = b8 ? k[i] : k[2 + i];
+        k2[i] += __shfl_xor_sync(kFull, s, 8);
+    }
+    float kk = b4 ? k2[1] : k2[0];
+    kk += __shfl_xor_sync(kFull, b4 ? k2[0] : k2[1], 4);
+    kk += __shfl_xor_sync(kFull, kk, 2);
+    kk += __shfl_xor_sync(kFull, kk, 1);
+    float *buf = u.red + u.par * kRedStride;
+    u.par ^= 1;
+    if ((u.lane & 3) == 0) buf[u.wig * 8 + (u.lane >> 2)] = kk;
+    unit_sync(u);
+    // slot = warp * 8 + value: lane i adds the slots i, i + 32, ..., lanes of equal i % 8 are folded
+    const int n = u.nwg * 8;
+    float t = 0.f;
+    for (int i = u.lane; i < n; i += kWarp) t += buf[i];
+    t += __shfl_xor_sync(kFull, t, 8);
+    t += __shfl_xor_sync(kFull, t, 16);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __shfl_sync(kFull, t, i);
 }
 
 // Grid barrier with one arrival and one poller per CTA (the units of a CTA meet at a CTA barrier
@@ -195,9 +245,9 @@ __device__ __forceinline__ void cta_wait(const CtaBar &cb, unsigned *counter, un
 // experts, the others are global block first_r + q - nq_s of the routed ones; global block g is
 // rows [bi*R, bi*R + nrows) of entry g / bpe, bi = g % bpe.
 struct FusedPlan {
-    int rows, bpe, first_s, nq_s, first_r, nq_r;
+    int rows, R, bpe, first_s, nq_s, first_r, nq_r;  // R: rows per block
     __device__ __forceinline__ int nq() const { return nq_s + nq_r; }
-    __device__ __forceinline__ int nrows(int bi) const { return min(kFusedRows, rows - bi * kFusedRows); }
+    __device__ __forceinline__ int nrows(int bi) const { return min(R, rows - bi * R); }
 };
 
 // Walks the blocks of a unit's layer sequence without a division: next rows of the entry, next
@@ -224,10 +274,10 @@ __device__ __forceinline__ size_t fused_image_index(const TokenArgs &a, int laye
 
 // The unit's first thread: bulk copies of one block (rows [i0, i0+nrows) of the three matrices of
 // image idx) into a ring stage.
-template <int DT>
+template <int DT, int R>
 __device__ __forceinline__ void fused_issue(const FusedArgs &fa, size_t idx, int i0, int nrows, uint8_t *stage, uint64_t *full)
 {
-    constexpr int BYTES = Fmt<DT>::kBytes, R = kFusedRows;
+    constexpr int BYTES = Fmt<DT>::kBytes;
     const TokenArgs &a = fa.t;
     const size_t row_bytes = (size_t)a.H * BYTES;
     const uint8_t *img = a.store + idx * a.img_bytes;
@@ -296,18 +346,18 @@ __device__ __forceinline__ float dot_e4m3_f16(const uint4 &w4, const uint32_t (&
 // chunks halve the per-block bookkeeping (waits, reductions, barriers) per byte, which is what
 // bounds the kernel once the copies keep HBM busy; they need twice the registers for the
 // thread's columns of h and of the output, which the 16-column fp8 layout does not have.
-template <int DT, int RDT, int CH>
+template <int DT, int RDT, int CH, int R = kFusedRows>
 __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(FusedArgs fa)
 {
-    constexpr int EPL = Fmt<DT>::kEpl, BYTES = Fmt<DT>::kBytes, R = kFusedRows;
+    constexpr int EPL = Fmt<DT>::kEpl, BYTES = Fmt<DT>::kBytes;
     // The ring is 192 KB per CTA whatever the unit size: a CTA of two-chunk threads has twice the
     // units, each with half the stages (the bytes in flight per SM are the same).
-    constexpr int NS = kFusedStages / CH;
+    constexpr int NS = kFusedStages * kFusedRows / (CH * R);
     constexpr int EPLR = Fmt<RDT>::kEpl, NRL = EPL / EPLR;  // router loads per chunk and row
-    static_assert(R == 2, "unit_sum4 reduces the two dot products of two rows");
+    static_assert((R == 2 || R == 4) && CH * R <= 4, "the ring holds at least two stages per unit");
     const TokenArgs &a = fa.t;
     const int L = a.L, E = a.E, K = a.K, H = a.H, I = a.I;
-    __shared__ __align__(16) float s_red[kFusedMaxUnits][2 * 64];
+    __shared__ __align__(16) float s_red[kFusedMaxUnits][2 * kRedStride];
     __shared__ uint32_t s_key[kMaxExperts];
     __shared__ float s_tk[3][8];   // top-K: per-warp maxima, sums, selected sums
     __shared__ int s_cnt[8];       // top-K: selected experts per warp
@@ -408,13 +458,23 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
     const bool in_loop = !(async_pred && threadIdx.x >= 256);
 
     FusedPlan pl;
-    pl.rows = I, pl.bpe = (I + R - 1) / R;
+    pl.rows = I, pl.R = R, pl.bpe = (I + R - 1) / R;
     {
         const long long all_s = (long long)a.n_shared * pl.bpe, all_r = (long long)K * pl.bpe;
         pl.first_s = service ? 0 : (int)(all_s * unit / n_stream);
         pl.nq_s = service ? 0 : (int)(all_s * (unit + 1) / n_stream) - pl.first_s;
-        pl.first_r = service ? 0 : (int)(all_r * unit / n_stream);
-        pl.nq_r = service ? 0 : (int)(all_r * (unit + 1) / n_stream) - pl.first_r;
+        if (all_s > 0 && all_r >= n_stream) {
+            // both kinds together are dealt evenly (to within one block per unit, not one of each
+            // kind): a unit with one shared block more takes one routed block less.  The routed
+            // ranges stay contiguous: unit u starts where the units before it end.
+            const long long all = all_s + all_r;
+            const long long t0 = all * unit / n_stream, t1 = all * (unit + 1) / n_stream;
+            pl.first_r = service ? 0 : (int)(t0 - pl.first_s);
+            pl.nq_r = service ? 0 : (int)(t1 - t0) - pl.nq_s;
+        } else {
+            pl.first_r = service ? 0 : (int)(all_r * unit / n_stream);
+            pl.nq_r = service ? 0 : (int)(all_r * (unit + 1) / n_stream) - pl.first_r;
+        }
     }
     const int nq = pl.nq();
     // Ring position: `done` = blocks the unit has consumed since the start of the launch (stage =
@@ -543,7 +603,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
                 // a routed block of a later layer, or of this one before its top-K: not known yet
                 if (!iss.sh && (iss_layer != l || !routed_known)) break;
                 const unsigned st = issued % NS;
-                fused_issue<DT>(fa, fused_image_index(a, iss_layer, iss.sh, iss.entry, s_ids), iss.bi * R,
+                fused_issue<DT, R>(fa, fused_image_index(a, iss_layer, iss.sh, iss.entry, s_ids), iss.bi * R,
                                 pl.nrows(iss.bi), my_ring + st * stage_bytes, my_full + st);
                 ++issued, ++iss_seq;
                 iss.next(pl);
@@ -569,7 +629,9 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
             if (q == pl.nq_s && q > 0) cu.start(pl, false);
             const int i0 = cu.bi * R, nrows = pl.nrows(cu.bi);
             const uint8_t *stage = my_ring + st * stage_bytes;
-            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            float v[2 * R];
+#pragma unroll
+            for (int i = 0; i < 2 * R; ++i) v[i] = 0.f;
             uint4 wd[R][CH];
 #pragma unroll
             for (int r = 0; r < R; ++r)
@@ -597,26 +659,41 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
                         }
                     }
                 }
-            unit_sum4(u, v);  // past its barrier every thread has read the stage: it may be refilled
+            // past the reduction's barrier every thread has read the stage: it may be refilled
+            if constexpr (R == 2)
+                unit_sum4(u, v);
+            else
+                unit_sum8(u, v);
             ++done;
             const float wgt = cu.sh ? 1.f : s_w[cu.entry];
             const uint16_t *sc = nullptr;
             if (DT == 2)
                 sc = reinterpret_cast<const uint16_t *>(a.store + fused_image_index(a, l, cu.sh, cu.entry, s_ids) * a.img_bytes +
                                                         image_scales(H, I, BYTES));
-            // odd lanes evaluate row 1, even lanes row 0; one exchange gives every lane both
-            const int r_mine = u.lane & 1;
+            // lane i evaluates row i % R; an exchange inside each group of R lanes gives every lane all
+            const int r_mine = u.lane & (R - 1);
             const float vs = DT == 2 ? 8.f : inv;  // fp8: the f16 pairs carry inv / 8 already
-            float gv = (r_mine ? v[2] : v[0]) * vs, uv = (r_mine ? v[3] : v[1]) * vs;
+            float gsel = v[0], usel = v[1];
+#pragma unroll
+            for (int r = 1; r < R; ++r)
+                if (r_mine == r) gsel = v[2 * r], usel = v[2 * r + 1];
+            float gv = gsel * vs, uv = usel * vs;
             if (DT == 2 && i0 + r_mine < I) {
                 gv *= bf16_to_f32(sc[i0 + r_mine]);
                 uv *= bf16_to_f32(sc[I + i0 + r_mine]);
             }
             const float act_mine = gv / (1.f + expf(-gv)) * uv;  // rows past the end: zero weights, act = 0
-            const float act_other = __shfl_xor_sync(kFull, act_mine, 1);
+            float acts[R];
+            if constexpr (R == 2) {
+                const float act_other = __shfl_xor_sync(kFull, act_mine, 1);
+                acts[0] = r_mine ? act_other : act_mine, acts[1] = r_mine ? act_mine : act_other;
+            } else {
+#pragma unroll
+                for (int r = 0; r < R; ++r) acts[r] = __shfl_sync(kFull, act_mine, (u.lane & ~(R - 1)) | r);
+            }
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                float act = (r == r_mine) ? act_mine : act_other;
+                float act = acts[r];
                 if (DT != 2) act *= wgt;
 #pragma unroll
                 for (int j = 0; j < CH; ++j) {

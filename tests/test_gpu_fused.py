@@ -21,6 +21,8 @@ SHAPES = [
     dict(dtype="fp8", hidden=4096, inter=768, n_experts=32, top_k=8, n_shared=0),      # fp8, 256 threads, row and column scales
     dict(dtype="fp8", hidden=1024, inter=320, n_experts=256, top_k=8, n_shared=1),     # maximum expert count, 4 experts per thread
     dict(dtype="bf16", hidden=512, inter=64, n_experts=4, top_k=4, n_shared=0),        # K = E: everything routed
+    dict(dtype="fp8", hidden=4096, inter=1008, n_experts=16, top_k=8, n_shared=0),     # fp8 with enough row blocks per unit: blocks of four rows
+    dict(dtype="fp8", hidden=1024, inter=3536, n_experts=12, top_k=8, n_shared=1),     # four-row blocks, units of two warps
 ]
 
 
@@ -51,7 +53,7 @@ def _run(cfg, T, flags=0):
     return out
 
 
-@pytest.mark.parametrize("shape", [SHAPES[1], SHAPES[3], SHAPES[5]])
+@pytest.mark.parametrize("shape", [SHAPES[1], SHAPES[3], SHAPES[5], SHAPES[8]])
 def test_fused_step_is_reproducible_and_agrees_with_three_phase_kernel(shape):
     cfg = stacks.CONFIGS["C2"].scaled(n_layers=4, profile_tokens=2, cache_slots=0, **shape)
     T = 8
