@@ -19,7 +19,7 @@
 // of the last CTA stream an equal slice of the rows of every expert.  The two dot products of a
 // row are reduced over the unit (a transposed warp butterfly, then one shared-memory exchange and
 // a named barrier per block of two rows).  The rows reach the SM by bulk asynchronous copies
-// (cp.async.bulk, completion counted on an mbarrier; no multicast) into a shared-memory ring of
+// (cp.async.bulk, one destination CTA, completion counted on an mbarrier) into a shared-memory ring of
 // four blocks per unit, issued by the unit's first thread three blocks ahead of the arithmetic:
 // 192 KB in flight per SM without holding a register, which the column-owner layout needs for its
 // state.  A stage is free again once the unit has passed the barrier of the block that read it.
