@@ -483,28 +483,34 @@ def main():
         # of all of them are in this line (same fields each; `kernel` names what ran)
         sec = []
         short = argparse.Namespace(**{**vars(args), "steps": 48, "warmup": 4})
-        sec.append(summarise(cfg, 4, measure(cfg, 4, st, short, dev, world, stream, with_e2e=False), short, world, peak))
-        st.close()
-        del st
-        torch.cuda.empty_cache()
-        c2 = stacks.CONFIGS["C2"]
-        st2 = make_stack(c2, 8, dev, short)
-        for b in (1, 8):
-            sec.append(summarise(c2, b, measure(c2, b, st2, short, dev, world, stream, with_e2e=False), short, world, peak))
-        st2.close()
-        del st2
+        try:    # a failure here must not cost the headline line
+            sec.append(summarise(cfg, 4, measure(cfg, 4, st, short, dev, world, stream, with_e2e=False), short, world, peak))
+            st.close()
+            del st
+            torch.cuda.empty_cache()
+            c2 = stacks.CONFIGS["C2"]
+            st2 = make_stack(c2, 8, dev, short)
+            for b in (1, 8):
+                sec.append(summarise(c2, b, measure(c2, b, st2, short, dev, world, stream, with_e2e=False), short, world, peak))
+            st2.close()
+            del st2
+        except Exception as e:  # noqa: BLE001
+            sec.append({"error": repr(e)})
         out["secondary"] = sec
     else:
         st.close()
     torch.cuda.empty_cache()
     if world == 1 and not args.no_cpu_baseline:
         layers = min(L, args.cpu_sample_layers)
-        spent, cores = cpu_oracle_sample(cfg, batch, layers, 2, dev)
-        per_token = spent[-1] * L / layers
-        out["cpu_baseline"] = {
-            "value": batch / per_token, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"second decode step, first {layers} of {L} layers, batch {batch}, "
-                      f"scaled to the full depth"}
+        try:
+            spent, cores = cpu_oracle_sample(cfg, batch, layers, 2, dev)
+            per_token = spent[-1] * L / layers
+            out["cpu_baseline"] = {
+                "value": batch / per_token, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"second decode step, first {layers} of {L} layers, batch {batch}, "
+                          f"scaled to the full depth"}
+        except Exception as e:  # noqa: BLE001
+            out["cpu_baseline"] = {"value": None, "unit": UNIT, "cores": 0, "kind": "oracle", "sample": "failed: " + repr(e)}
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
