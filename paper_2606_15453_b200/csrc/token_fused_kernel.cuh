@@ -691,18 +691,48 @@ __global__ void __launch_bounds__(kFfnThreads, 1) decode_token_fused_kernel(Fuse
 #pragma unroll
                 for (int r = 0; r < R; ++r) acts[r] = __shfl_sync(kFull, act_mine, (u.lane & ~(R - 1)) | r);
             }
+            if constexpr (DT == 2) {
+                // fp8: the block's rows are combined in f16 pairs before they meet the fp32 sums.  The
+                // activations are scaled by the block's largest magnitude, so a product is at most 448
+                // and a column's sum over the block's rows at most 448 R: no overflow whatever the
+                // activations are; the scale goes back in with the one fp32 FMA per column.
+                float amax = fabsf(acts[0]);
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                float act = acts[r];
-                if (DT != 2) act *= wgt;
+                for (int r = 1; r < R; ++r) amax = fmaxf(amax, fabsf(acts[r]));
+                const float rs = amax > 0.f ? 1.f / amax : 0.f;
+                __half2 a2[R];
 #pragma unroll
-                for (int j = 0; j < CH; ++j) {
-                    float wf[EPL];
-                    Fmt<DT>::unpack(wd[r][j], wf);
-                    if (DT == 2) {
+                for (int r = 0; r < R; ++r) a2[r] = __float2half2_rn(acts[r] * rs);
 #pragma unroll
-                        for (int e = 0; e < EPL; ++e) ye[e] = fmaf(act, wf[e], ye[e]);
-                    } else {
+                for (int i = 0; i < 4; ++i) {
+                    __half2 plo = __float2half2_rn(0.f), phi = plo;
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        const uint32_t w = i == 0 ? wd[r][0].x : i == 1 ? wd[r][0].y : i == 2 ? wd[r][0].z : wd[r][0].w;
+                        uint32_t lo, hi;  // weights 4i, 4i+1 and 4i+2, 4i+3 of the row as f16 pairs
+                        asm("{.reg .b16 a, b;\n\t"
+                            "mov.b32 {a, b}, %2;\n\t"
+                            "cvt.rn.f16x2.e4m3x2 %0, a;\n\t"
+                            "cvt.rn.f16x2.e4m3x2 %1, b;}"
+                            : "=r"(lo), "=r"(hi)
+                            : "r"(w));
+                        plo = __hfma2(*reinterpret_cast<const __half2 *>(&lo), a2[r], plo);
+                        phi = __hfma2(*reinterpret_cast<const __half2 *>(&hi), a2[r], phi);
+                    }
+                    const float2 fl = __half22float2(plo), fh = __half22float2(phi);
+                    ye[4 * i] = fmaf(amax, fl.x, ye[4 * i]);
+                    ye[4 * i + 1] = fmaf(amax, fl.y, ye[4 * i + 1]);
+                    ye[4 * i + 2] = fmaf(amax, fh.x, ye[4 * i + 2]);
+                    ye[4 * i + 3] = fmaf(amax, fh.y, ye[4 * i + 3]);
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const float act = acts[r] * wgt;
+#pragma unroll
+                    for (int j = 0; j < CH; ++j) {
+                        float wf[EPL];
+                        Fmt<DT>::unpack(wd[r][j], wf);
 #pragma unroll
                         for (int e = 0; e < EPL; ++e) y[j][e] = fmaf(act, wf[e], y[j][e]);
                     }
