@@ -308,6 +308,13 @@ def summarise(cfg, batch, m, args, world, peak):
            "predictor": {"recall": run["hits"] / max(run["routed"], 1), "precision": run["hits"] / max(run["predicted"], 1),
                          "mean_predicted": run["predicted"] / max(run["runtime_steps"], 1), "near_ties": run["near_ties"],
                          "routing_overlap": dict(m["overlap"], random=cfg.top_k * cfg.top_k / cfg.n_experts)}}
+    if batch == 1 and out["kernel"] == "decode_token_fused_kernel" and cfg.name.startswith(("C1", "C2")) and \
+            cfg.n_layers == stacks.CONFIGS[cfg.name[:2]].n_layers:
+        # DRAM traffic of one launch from the ncu summary of a short cut of this workload (a single
+        # sequence streams the same number of experts in every layer, so traffic grows with the depth)
+        per_layer, src = profile_value(f"dram_bytes_per_layer_{cfg.name[:2].lower()}_batch1_decode_token_fused_kernel")
+        out["traffic"] = per_layer * cfg.n_layers if per_layer else None
+        out["traffic_source"] = src
     if cfg.cache_slots:
         h2d = (s1["h2d_bytes_demand"] + s1["h2d_bytes_prefetch"] - s0["h2d_bytes_demand"] - s0["h2d_bytes_prefetch"])
         transfer, exposed = run["transfer_ms"], run["exposed_ms"]
@@ -446,10 +453,7 @@ def main():
     tokens = args.steps * batch * world
     persistent = cfg.cache_slots == 0 and not args.no_persistent   # resident stacks: one kernel launch per decode step
     whole_step = head["kernel"].startswith("decode_token")
-    traffic, traffic_src = (None, None)
-    if whole_step and batch == 1 and args.workload == "C1" and not args.no_fused:
-        per_layer, traffic_src = profile_value("dram_bytes_per_layer_c1_batch1_" + head["kernel"])
-        traffic = per_layer * L if per_layer else None
+    traffic, traffic_src = head.get("traffic"), head.get("traffic_source")
     out = {
         "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True,
