@@ -63,3 +63,15 @@ def test_replica_timing_is_the_maximum_over_ranks_gloo_world_2():
     sys.path.insert(0, ROOT)
     import bench
     assert bench.max_over_ranks([3.0, 4.0], 1, "cpu") == [3.0, 4.0]      # a single rank: no collective
+
+
+def test_routing_overlap_statistics_by_hand():
+    """Temporal overlap = experts shared by the same layer at consecutive steps, spatial = by adjacent
+    layers of one step; two layers, one sequence, top-2, three steps, counted by hand."""
+    import numpy as np
+    sys.path.insert(0, ROOT)
+    import bench
+    ids = [np.array([[[0, 1]], [[1, 2]]]), np.array([[[0, 1]], [[2, 3]]]), np.array([[[1, 5]], [[0, 1]]])]
+    ov = bench.routing_overlap(ids)
+    assert ov["temporal"] == (2 + 1 + 1 + 0) / 4          # (t1,t0): layers 0,1; (t2,t1): layers 0,1
+    assert abs(ov["spatial"] - (1 + 0 + 1) / 3) < 1e-12   # steps 0,1,2: layer 1 against layer 0
