@@ -117,11 +117,12 @@ def test_in_kernel_predictors_honour_threshold_and_replacement_rule(flags, B, th
     pr.close()
 
 
-@pytest.mark.parametrize("B", [1, 3])
-def test_decode_token_host_equals_the_device_call(B):
+@pytest.mark.parametrize("B,slots", [(1, 0), (3, 0), (2, 24)])
+def test_decode_token_host_equals_the_device_call(B, slots):
     """The host-buffer entry point (copies in, decode step, copies out, wait) against the
-    device-pointer call on a second stack: outputs and routing bit-identical, pinned or pageable."""
-    cfg = stacks.CONFIGS["C2"].scaled(n_layers=3, profile_tokens=2, cache_slots=0, **SHAPES[1])
+    device-pointer call on a second stack: outputs and routing bit-identical, pinned or pageable;
+    resident stacks and an offloaded one."""
+    cfg = stacks.CONFIGS["C2"].scaled(n_layers=3, profile_tokens=2, cache_slots=slots, **SHAPES[1])
     a, b = Pair(cfg, B, oracle=False), Pair(cfg, B, oracle=False)
     L, K, T = cfg.n_layers, cfg.top_k, 6
     ids = torch.empty(L, B, K, dtype=torch.int32, device=DEV)
